@@ -1,0 +1,665 @@
+/*
+ * CPU oracle for the MaxScore router (arXiv 2508.12801).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is a plain, slow, deliberately
+ * unoptimised restatement of what the router computes, written from the
+ * paper's definitions.  It shares no code with the CUDA library and must
+ * never be called from the product path; only tests, the smoke check and
+ * the CPU-baseline leg of the benchmark use it.
+ *
+ * Arithmetic: double precision for floating point, int64 keys (with
+ * __int128 totals) for the assignment problem.
+ *
+ * Stages (paper passage each follows):
+ *   mso_capacity            Sec. 2.3, c = cf * k * n / e ; Algorithm 1 step 1
+ *   mso_gate                Eq. 2, x . W_g  (plus the optional expert bias)
+ *   mso_softtopk_fwd/bwd    Eq. 6 (reading "ITERMASK", see below) and its derivative
+ *   mso_keys_from_scores    fixed-point keys of the affinities A (Eq. 8 objective)
+ *   mso_keys_from_logits    int16-quantised logits with a hashed tie-break
+ *   mso_flow_ssp            Eq. 7-8 on the network of Table 1, solved by
+ *                           successive shortest augmenting paths (SPFA), Sec. 3.2
+ *   mso_flow_condensed      the same method with the path search done on the
+ *                           expert-level residual graph (for the large configs)
+ *   mso_flow_bruteforce     Eq. 7-8 by enumeration (tiny inputs)
+ *   mso_flow_certificate    optimality / uniqueness check of a given P
+ *   mso_index_build, mso_dispatch, mso_combine      Eq. 1 through E x C buffers
+ *   mso_combine_bwd, mso_gate_bwd                   derivatives of Eq. 1 and Eq. 2
+ *   mso_aux_loss            Eq. 9
+ *
+ * Reading of Eq. 6 ("ITERMASK"): SoftTopk^(0) = 0; level j (1-based) adds a
+ * softmax with temperature t over the entries that are NOT among the j-1
+ * largest; ties go to the lowest expert index.
+ *
+ * Every function here is pinned by tests/test_oracle_*.py against closed
+ * forms, library routines, brute force or invariants; none is "parity
+ * unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+typedef __int128 i128;
+
+#define MSO_OK 0
+#define MSO_ERR_ARG 1
+#define MSO_ERR_INFEASIBLE 2
+#define MSO_ERR_ALLOC 3
+
+/* ------------------------------------------------------------------ */
+/* Capacity: C = ceil(cf * T * k / E)  (Sec. 2.3; Algorithm 1 step 1). */
+/* cf is given as a rational cf_num / cf_den so the ceiling is exact.   */
+int64_t mso_capacity(int64_t T, int64_t k, int64_t E, int64_t cf_num, int64_t cf_den) {
+  i128 num = (i128)cf_num * T * k;
+  i128 den = (i128)cf_den * E;
+  return (int64_t)((num + den - 1) / den);
+}
+
+/* Feasible iff every token can get k distinct experts under capacity C. */
+int mso_feasible(int64_t T, int64_t k, int64_t E, int64_t C) {
+  if (k > E) return 0;
+  int64_t cap = C < T ? C : T;
+  return (i128)E * cap >= (i128)T * k;
+}
+
+/* ------------------------------------------------------------------ */
+/* Gate, Eq. 2:  L[i][j] = sum_m H[i][m] * W[m][j] (+ bias[j]).         */
+/* H is [T,d], W is [d,E] as the paper writes x . W_g, both row-major.  */
+void mso_gate(int64_t T, int64_t d, int64_t E, const double *H, const double *W,
+              const double *bias, double *L) {
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < T; ++i) {
+    for (int64_t j = 0; j < E; ++j) {
+      double acc = 0.0;
+      for (int64_t m = 0; m < d; ++m) acc += H[i * d + m] * W[m * E + j];
+      if (bias) acc += bias[j];
+      L[i * E + j] = acc;
+    }
+  }
+}
+
+/* ------------------------------------------------------------------ */
+/* SoftTopk forward, Eq. 6, one token at a time.                        */
+static void softtopk_row(int64_t E, int64_t k, double t, const double *a, double *y,
+                         char *sel) {
+  for (int64_t i = 0; i < E; ++i) { y[i] = 0.0; sel[i] = 0; }
+  for (int64_t level = 0; level < k; ++level) {
+    /* largest unmasked entry, lowest index on ties */
+    int64_t arg = -1;
+    for (int64_t i = 0; i < E; ++i)
+      if (!sel[i] && (arg < 0 || a[i] > a[arg])) arg = i;
+    if (arg < 0) return;
+    double m = a[arg];
+    double Z = 0.0;
+    for (int64_t i = 0; i < E; ++i)
+      if (!sel[i]) Z += exp((a[i] - m) / t);
+    for (int64_t i = 0; i < E; ++i)
+      if (!sel[i]) y[i] += exp((a[i] - m) / t) / Z;
+    sel[arg] = 1; /* masked from the next level on */
+  }
+}
+
+int mso_softtopk_fwd(int64_t T, int64_t E, int64_t k, double t, const double *L, double *A) {
+  if (k < 1 || k > E || !(t > 0.0)) return MSO_ERR_ARG;
+#pragma omp parallel
+  {
+    char *sel = (char *)malloc((size_t)E);
+#pragma omp for schedule(static)
+    for (int64_t i = 0; i < T; ++i) softtopk_row(E, k, t, L + i * E, A + i * E, sel);
+    free(sel);
+  }
+  return MSO_OK;
+}
+
+/* SoftTopk backward: the masks are held constant; level j is a softmax  */
+/* q over its unmasked set U_j, so                                       */
+/*   da_l = (1/t) * sum_{j : l in U_j} q_l * (g_l - sum_{i in U_j} g_i q_i). */
+int mso_softtopk_bwd(int64_t T, int64_t E, int64_t k, double t, const double *L,
+                     const double *G, double *dL) {
+  if (k < 1 || k > E || !(t > 0.0)) return MSO_ERR_ARG;
+#pragma omp parallel
+  {
+    char *sel = (char *)malloc((size_t)E);
+    double *q = (double *)malloc(sizeof(double) * (size_t)E);
+#pragma omp for schedule(static)
+    for (int64_t r = 0; r < T; ++r) {
+      const double *a = L + r * E, *g = G + r * E;
+      double *da = dL + r * E;
+      for (int64_t i = 0; i < E; ++i) { da[i] = 0.0; sel[i] = 0; }
+      for (int64_t level = 0; level < k; ++level) {
+        int64_t arg = -1;
+        for (int64_t i = 0; i < E; ++i)
+          if (!sel[i] && (arg < 0 || a[i] > a[arg])) arg = i;
+        if (arg < 0) break;
+        double m = a[arg], Z = 0.0;
+        for (int64_t i = 0; i < E; ++i)
+          if (!sel[i]) Z += exp((a[i] - m) / t);
+        double gq = 0.0;
+        for (int64_t i = 0; i < E; ++i)
+          if (!sel[i]) { q[i] = exp((a[i] - m) / t) / Z; gq += g[i] * q[i]; }
+        for (int64_t i = 0; i < E; ++i)
+          if (!sel[i]) da[i] += q[i] * (g[i] - gq) / t;
+        sel[arg] = 1;
+      }
+    }
+    free(sel); free(q);
+  }
+  return MSO_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* Keys for the assignment problem.                                     */
+
+/* Float mode: fixed-point image of the affinities, w = rne(A * 2^40).  */
+void mso_keys_from_scores(int64_t n, const double *A, int64_t *w) {
+  for (int64_t i = 0; i < n; ++i) w[i] = llrint(ldexp(A[i], 40));
+}
+
+/* 32-bit finaliser of MurmurHash3 (Appleby, public domain). */
+static uint32_t fmix32(uint32_t h) {
+  h ^= h >> 16; h *= 0x85ebca6bu; h ^= h >> 13; h *= 0xc2b2ae35u; h ^= h >> 16;
+  return h;
+}
+
+/* Integer mode: q = clamp(rne(L * 2^shift)) as int16; tie-break          */
+/* r = top 20 bits of fmix32(i*E + j + seed * 0x9E3779B9);                */
+/* w = q * 2^S + r with S = 20 + ceil(log2(T*k)), so that the summed      */
+/* perturbation of any assignment stays below one step of q.              */
+int mso_tiebreak_shift(int64_t T, int64_t k) {
+  int64_t n = T * k; int s = 0;
+  while (((int64_t)1 << s) < n) ++s;
+  return 20 + s;
+}
+
+void mso_keys_from_logits(int64_t T, int64_t E, int64_t k, const float *L, int shift,
+                          uint32_t seed, int64_t *w, int16_t *q_out) {
+  int S = mso_tiebreak_shift(T, k);
+  for (int64_t i = 0; i < T; ++i)
+    for (int64_t j = 0; j < E; ++j) {
+      /* the product by a power of two is exact in float; rintf is round-to-nearest-even */
+      float scaled = rintf(ldexpf(L[i * E + j], shift));
+      if (scaled > 32767.0f) scaled = 32767.0f;
+      if (scaled < -32768.0f) scaled = -32768.0f;
+      int64_t q = (int64_t)scaled;
+      uint32_t r = fmix32((uint32_t)(i * E + j) + seed * 0x9E3779B9u) >> 12;
+      w[i * E + j] = q * ((int64_t)1 << S) + (int64_t)r;
+      if (q_out) q_out[i * E + j] = (int16_t)q;
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* Textbook min-cost max-flow on the network of Table 1:                 */
+/*   source -> token_i   cap k  cost 0                                   */
+/*   token_i -> expert_j cap 1  cost -w_ij                               */
+/*   expert_j -> sink    cap C  cost 0                                   */
+/* Successive shortest augmenting paths, each found by SPFA (queue-based */
+/* Bellman-Ford), until the sink is unreachable.                         */
+typedef struct { int32_t to, cap; int64_t cost; } arc_t;
+
+int mso_flow_ssp(int64_t T, int64_t E, int64_t k, int64_t C, const int64_t *w,
+                 int32_t *expert_idx, int32_t *load, int64_t *flow_value) {
+  if (!mso_feasible(T, k, E, C)) return MSO_ERR_INFEASIBLE;
+  int64_t N = T + E + 2, S = 0, SINK = T + E + 1;
+  int64_t M = 2 * (T + T * E + E);
+  arc_t *arc = (arc_t *)malloc(sizeof(arc_t) * (size_t)M);
+  int64_t *first = (int64_t *)malloc(sizeof(int64_t) * (size_t)(N + 1));
+  i128 *dist = (i128 *)malloc(sizeof(i128) * (size_t)N);
+  int64_t *prev_arc = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
+  int64_t *queue = (int64_t *)malloc(sizeof(int64_t) * (size_t)(N + 1));
+  char *inq = (char *)malloc((size_t)N);
+  if (!arc || !first || !dist || !prev_arc || !queue || !inq) return MSO_ERR_ALLOC;
+  /* adjacency in CSR form; arc a and its reverse sit at a and rev(a) = partner[] */
+  int64_t *partner = (int64_t *)malloc(sizeof(int64_t) * (size_t)M);
+  int64_t *deg = (int64_t *)calloc((size_t)(N + 1), sizeof(int64_t));
+  /* degrees */
+  deg[S] = T;
+  for (int64_t i = 0; i < T; ++i) deg[1 + i] = 1 + E;
+  for (int64_t j = 0; j < E; ++j) deg[1 + T + j] = T + 1;
+  deg[SINK] = E;
+  first[0] = 0;
+  for (int64_t v = 0; v < N; ++v) first[v + 1] = first[v] + deg[v];
+  int64_t *fill = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
+  for (int64_t v = 0; v < N; ++v) fill[v] = first[v];
+#define ADD_ARC(u, v, c, cst)                                                   \
+  do {                                                                          \
+    int64_t a_ = fill[u]++, b_ = fill[v]++;                                     \
+    arc[a_].to = (int32_t)(v); arc[a_].cap = (int32_t)(c); arc[a_].cost = (cst); \
+    arc[b_].to = (int32_t)(u); arc[b_].cap = 0; arc[b_].cost = -(cst);          \
+    partner[a_] = b_; partner[b_] = a_;                                         \
+  } while (0)
+  for (int64_t i = 0; i < T; ++i) ADD_ARC(S, 1 + i, k, 0);
+  for (int64_t i = 0; i < T; ++i)
+    for (int64_t j = 0; j < E; ++j) ADD_ARC(1 + i, 1 + T + j, 1, -w[i * E + j]);
+  for (int64_t j = 0; j < E; ++j) ADD_ARC(1 + T + j, SINK, C, 0);
+#undef ADD_ARC
+  const i128 INF = ((i128)1) << 120;
+  int64_t flow = 0;
+  for (;;) {
+    for (int64_t v = 0; v < N; ++v) { dist[v] = INF; inq[v] = 0; prev_arc[v] = -1; }
+    int64_t qh = 0, qt = 0, qn = 0;
+    dist[S] = 0; queue[qt] = S; qt = (qt + 1) % (N + 1); qn = 1; inq[S] = 1;
+    while (qn > 0) {
+      int64_t u = queue[qh]; qh = (qh + 1) % (N + 1); --qn; inq[u] = 0;
+      for (int64_t a = first[u]; a < first[u + 1]; ++a) {
+        if (arc[a].cap <= 0) continue;
+        int64_t v = arc[a].to;
+        i128 nd = dist[u] + arc[a].cost;
+        if (nd < dist[v]) {
+          dist[v] = nd; prev_arc[v] = a;
+          if (!inq[v]) { queue[qt] = v; qt = (qt + 1) % (N + 1); ++qn; inq[v] = 1; }
+        }
+      }
+    }
+    if (prev_arc[SINK] < 0) break; /* no augmenting path remains */
+    /* bottleneck is 1 because every path crosses a unit token->expert arc */
+    for (int64_t v = SINK; v != S;) {
+      int64_t a = prev_arc[v];
+      arc[a].cap -= 1; arc[partner[a]].cap += 1;
+      v = arc[partner[a]].to;
+    }
+    ++flow;
+  }
+  /* read the assignment off the saturated token->expert arcs */
+  for (int64_t j = 0; j < E; ++j) load[j] = 0;
+  int rc = MSO_OK;
+  for (int64_t i = 0; i < T; ++i) {
+    int64_t c = 0;
+    for (int64_t a = first[1 + i]; a < first[2 + i]; ++a) {
+      int64_t v = arc[a].to;
+      if (v >= 1 + T && v < 1 + T + E && arc[a].cap == 0) {
+        if (c < k) expert_idx[i * k + c] = (int32_t)(v - 1 - T);
+        ++c; load[v - 1 - T] += 1;
+      }
+    }
+    if (c != k) rc = MSO_ERR_INFEASIBLE;
+    /* ascending expert index within the token */
+    for (int64_t x = 1; x < (c < k ? c : k); ++x)
+      for (int64_t y = x; y > 0 && expert_idx[i * k + y] < expert_idx[i * k + y - 1]; --y) {
+        int32_t tmp = expert_idx[i * k + y]; expert_idx[i * k + y] = expert_idx[i * k + y - 1];
+        expert_idx[i * k + y - 1] = tmp;
+      }
+  }
+  if (flow_value) *flow_value = flow;
+  free(arc); free(first); free(dist); free(prev_arc); free(queue); free(inq);
+  free(partner); free(deg); free(fill);
+  return rc;
+}
+
+/* ------------------------------------------------------------------ */
+/* Brute force for Eq. 7-8: enumerate every choice of k experts per     */
+/* token, keep those with all loads <= C, maximise sum of keys.         */
+/* Returns the optimum, how many assignments attain it, and the first   */
+/* optimal assignment in enumeration order.  For T <= 8, E <= 4 only.   */
+int mso_flow_bruteforce(int64_t T, int64_t E, int64_t k, int64_t C, const int64_t *w,
+                        int64_t *best_total, int64_t *n_optimal, int32_t *expert_idx) {
+  if (T > 10 || E > 6 || k > E) return MSO_ERR_ARG;
+  int masks[64]; int nm = 0;
+  for (int m = 0; m < (1 << E); ++m) if (__builtin_popcount(m) == k) masks[nm++] = m;
+  int choice[16]; int best_choice[16];
+  for (int i = 0; i < T; ++i) choice[i] = 0;
+  int found = 0; i128 best = 0; int64_t count = 0;
+  for (;;) {
+    int ld[8] = {0}; i128 tot = 0; int ok = 1;
+    for (int i = 0; i < T && ok; ++i)
+      for (int j = 0; j < E; ++j)
+        if (masks[choice[i]] >> j & 1) {
+          tot += w[i * E + j];
+          if (++ld[j] > C) { ok = 0; break; }
+        }
+    if (ok) {
+      if (!found || tot > best) { best = tot; count = 1; found = 1; memcpy(best_choice, choice, sizeof(choice)); }
+      else if (tot == best) ++count;
+    }
+    int p = (int)T - 1;
+    while (p >= 0 && ++choice[p] == nm) { choice[p] = 0; --p; }
+    if (p < 0) break;
+  }
+  if (!found) return MSO_ERR_INFEASIBLE;
+  *best_total = (int64_t)best; *n_optimal = count;
+  for (int i = 0; i < T; ++i) {
+    int c = 0;
+    for (int j = 0; j < E; ++j) if (masks[best_choice[i]] >> j & 1) expert_idx[i * k + c++] = j;
+  }
+  return MSO_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* Expert-level residual graph of an assignment P (nodes 0..E-1 are the */
+/* experts, node E is the sink side "Z"):                               */
+/*   D[e][f] = min over tokens i with P_ie = 1, P_if = 0 of w_ie - w_if */
+/*             (the loss of moving one token from e to f)               */
+/*   D[f][Z] = 0 if load_f < C ;  D[Z][e] = 0 if load_e > 0.            */
+/* P is optimal iff this graph has no negative cycle; it is the only    */
+/* optimum iff every cycle is strictly positive.                        */
+#define BIG ((i128)1 << 100)
+
+static void build_D(int64_t T, int64_t E, int64_t k, int64_t C, const int64_t *w,
+                    const int32_t *expert_idx, const int32_t *load, i128 *D, int32_t *who) {
+  int64_t n = E + 1;
+  for (int64_t a = 0; a < n * n; ++a) { D[a] = BIG; if (who) who[a] = -1; }
+  char *in = (char *)malloc((size_t)E);
+  for (int64_t i = 0; i < T; ++i) {
+    memset(in, 0, (size_t)E);
+    for (int64_t c = 0; c < k; ++c) in[expert_idx[i * k + c]] = 1;
+    for (int64_t c = 0; c < k; ++c) {
+      int64_t e = expert_idx[i * k + c];
+      for (int64_t f = 0; f < E; ++f) {
+        if (in[f]) continue;
+        i128 loss = (i128)w[i * E + e] - (i128)w[i * E + f];
+        if (loss < D[e * n + f]) { D[e * n + f] = loss; if (who) who[e * n + f] = (int32_t)i; }
+      }
+    }
+  }
+  for (int64_t e = 0; e < E; ++e) {
+    if (load[e] < C) D[e * n + E] = 0;
+    if (load[e] > 0) D[E * n + e] = 0;
+  }
+  free(in);
+}
+
+/* result: 0 = not optimal (negative cycle), 1 = optimal but a zero     */
+/* cycle exists (other optima), 2 = uniquely optimal.                   */
+/* prices[E] receives dual prices p_e >= 0 when optimal.                */
+/* Also checks the invariants: k distinct experts per token, ascending, */
+/* loads match and stay <= C; returns -1 if any fails.                  */
+int mso_flow_certificate(int64_t T, int64_t E, int64_t k, int64_t C, const int64_t *w,
+                         const int32_t *expert_idx, int64_t *prices) {
+  int64_t n = E + 1;
+  int32_t *load = (int32_t *)calloc((size_t)E, sizeof(int32_t));
+  for (int64_t i = 0; i < T; ++i)
+    for (int64_t c = 0; c < k; ++c) {
+      int32_t e = expert_idx[i * k + c];
+      if (e < 0 || e >= E) { free(load); return -1; }
+      if (c > 0 && expert_idx[i * k + c - 1] >= e) { free(load); return -1; }
+      load[e] += 1;
+    }
+  for (int64_t e = 0; e < E; ++e) if (load[e] > C) { free(load); return -1; }
+  i128 *D = (i128 *)malloc(sizeof(i128) * (size_t)(n * n));
+  build_D(T, E, k, C, w, expert_idx, load, D, NULL);
+  /* G = the expert-only part of D, kept apart for the uniqueness test: in  */
+  /* the full graph Z -> e -> Z is always a zero cycle (take a unit off the  */
+  /* arc expert_e -> sink and put it back), which is no second optimum.      */
+  i128 *G = (i128 *)malloc(sizeof(i128) * (size_t)(E * E));
+  for (int64_t a = 0; a < E; ++a)
+    for (int64_t b = 0; b < E; ++b) G[a * E + b] = D[a * n + b];
+  /* all-pairs shortest walks (Floyd-Warshall); diagonals start at +inf so  */
+  /* that [v][v] ends as the cheapest cycle through v                       */
+  for (int64_t m = 0; m < n; ++m)
+    for (int64_t a = 0; a < n; ++a) {
+      if (D[a * n + m] >= BIG) continue;
+      for (int64_t b = 0; b < n; ++b) {
+        if (D[m * n + b] >= BIG) continue;
+        i128 via = D[a * n + m] + D[m * n + b];
+        if (via < D[a * n + b]) D[a * n + b] = via;
+      }
+    }
+  for (int64_t m = 0; m < E; ++m)
+    for (int64_t a = 0; a < E; ++a) {
+      if (G[a * E + m] >= BIG) continue;
+      for (int64_t b = 0; b < E; ++b) {
+        if (G[m * E + b] >= BIG) continue;
+        i128 via = G[a * E + m] + G[m * E + b];
+        if (via < G[a * E + b]) G[a * E + b] = via;
+      }
+    }
+  int result = 2;
+  for (int64_t v = 0; v < n; ++v)
+    if (D[v * n + v] < 0) { result = 0; break; }
+  if (result) {
+    /* a zero cycle among the experts, or a zero walk from an expert to a    */
+    /* different expert with room (a cycle through Z), is a second optimum   */
+    for (int64_t a = 0; a < E && result == 2; ++a)
+      for (int64_t b = 0; b < E; ++b) {
+        if (a == b) { if (G[a * E + a] == 0) { result = 1; break; } }
+        else if (load[b] < C && G[a * E + b] == 0) { result = 1; break; }
+      }
+  }
+  free(G);
+  if (result > 0 && prices) {
+    /* potentials: pi_v = min(0, cheapest walk into v from any node), so    */
+    /* pi_f <= pi_e + D[e][f] on every arc.  The price of expert e is        */
+    /* p_e = pi_Z - pi_e: the arcs e -> f then say w_ie - p_e >= w_if - p_f  */
+    /* for every token in e and not in f, the arcs Z -> e give p_e >= 0      */
+    /* where load_e > 0 and the arcs f -> Z give p_f <= 0 where load_f < C.  */
+    /* An empty expert may come out negative; raising it to 0 keeps every    */
+    /* token's preference and no token sits there.                           */
+    i128 piZ = 0;
+    for (int64_t a = 0; a < n; ++a) if (D[a * n + E] < piZ) piZ = D[a * n + E];
+    for (int64_t e = 0; e < E; ++e) {
+      i128 pie = 0;
+      for (int64_t a = 0; a < n; ++a) if (D[a * n + e] < pie) pie = D[a * n + e];
+      i128 p = piZ - pie;
+      prices[e] = (int64_t)(p < 0 ? 0 : p);
+    }
+  }
+  free(D); free(load);
+  return result;
+}
+
+/* Dual objective of Eq. 8 at prices p:                                 */
+/*   sum_i (sum of the k largest of w_ie - p_e) + C * sum_e p_e.        */
+/* Equals the primal optimum exactly when p is optimal (strong duality   */
+/* of the totally unimodular flow LP).  Written as two int64 halves.     */
+void mso_dual_value(int64_t T, int64_t E, int64_t k, int64_t C, const int64_t *w,
+                    const int64_t *p, int64_t *hi, uint64_t *lo) {
+  i128 tot = 0;
+  i128 *v = (i128 *)malloc(sizeof(i128) * (size_t)E);
+  for (int64_t i = 0; i < T; ++i) {
+    for (int64_t e = 0; e < E; ++e) v[e] = (i128)w[i * E + e] - (i128)p[e];
+    for (int64_t c = 0; c < k; ++c) { /* selection of the k largest */
+      int64_t arg = c;
+      for (int64_t e = c + 1; e < E; ++e) if (v[e] > v[arg]) arg = e;
+      i128 tmp = v[c]; v[c] = v[arg]; v[arg] = tmp;
+      tot += v[c];
+    }
+  }
+  for (int64_t e = 0; e < E; ++e) tot += (i128)C * p[e];
+  free(v);
+  *hi = (int64_t)(tot >> 64); *lo = (uint64_t)tot;
+}
+
+void mso_primal_value(int64_t T, int64_t E, int64_t k, const int64_t *w,
+                      const int32_t *expert_idx, int64_t *hi, uint64_t *lo) {
+  i128 tot = 0;
+  for (int64_t i = 0; i < T; ++i)
+    for (int64_t c = 0; c < k; ++c) tot += w[i * E + expert_idx[i * k + c]];
+  *hi = (int64_t)(tot >> 64); *lo = (uint64_t)tot;
+}
+
+/* ------------------------------------------------------------------ */
+/* Successive shortest paths with the path search on the expert-level   */
+/* graph.  Start: every token takes its k largest keys (the min-cost    */
+/* flow when the expert->sink capacities are ignored).  Then, while an  */
+/* expert holds more than C tokens, find the cheapest walk from the set  */
+/* of overloaded experts to an expert with room (Bellman-Ford on E+1     */
+/* nodes; all cycles are non-negative, so it terminates) and move one    */
+/* token along each of its arcs.  The rows of D touched by the walk are  */
+/* rebuilt from the token lists.  Same optimum as mso_flow_ssp; checked  */
+/* against it in the tests.                                              */
+int mso_flow_condensed(int64_t T, int64_t E, int64_t k, int64_t C, const int64_t *w,
+                       int32_t *expert_idx, int32_t *load, int64_t *n_augment) {
+  if (!mso_feasible(T, k, E, C)) return MSO_ERR_INFEASIBLE;
+  int64_t n = E; /* expert nodes only; room is a node property here */
+  /* member[i*E+e] = 1 iff P_ie = 1 */
+  char *member = (char *)calloc((size_t)(T * E), 1);
+  for (int64_t e = 0; e < E; ++e) load[e] = 0;
+  for (int64_t i = 0; i < T; ++i) {
+    for (int64_t c = 0; c < k; ++c) {
+      int64_t arg = -1;
+      for (int64_t e = 0; e < E; ++e)
+        if (!member[i * E + e] && (arg < 0 || w[i * E + e] > w[i * E + arg])) arg = e;
+      member[i * E + arg] = 1; load[arg] += 1;
+    }
+  }
+  i128 *D = (i128 *)malloc(sizeof(i128) * (size_t)(n * n));
+  int32_t *who = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n * n));
+  i128 *dist = (i128 *)malloc(sizeof(i128) * (size_t)n);
+  int64_t *pred = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);
+  char *dirty = (char *)malloc((size_t)n);
+  for (int64_t e = 0; e < n; ++e) dirty[e] = 1;
+  int64_t aug = 0;
+  for (;;) {
+    /* rebuild the rows marked dirty: D[e][f] over tokens in e and not in f */
+    for (int64_t e = 0; e < n; ++e) {
+      if (!dirty[e]) continue;
+      for (int64_t f = 0; f < n; ++f) { D[e * n + f] = BIG; who[e * n + f] = -1; }
+    }
+    for (int64_t i = 0; i < T; ++i)
+      for (int64_t e = 0; e < n; ++e) {
+        if (!dirty[e] || !member[i * E + e]) continue;
+        for (int64_t f = 0; f < n; ++f) {
+          if (member[i * E + f]) continue;
+          i128 loss = (i128)w[i * E + e] - (i128)w[i * E + f];
+          if (loss < D[e * n + f]) { D[e * n + f] = loss; who[e * n + f] = (int32_t)i; }
+        }
+      }
+    /* a token that joined expert f may have been the cheapest mover of some
+       arc into f from another of its experts; those arcs' rows were marked too */
+    for (int64_t e = 0; e < n; ++e) dirty[e] = 0;
+    int any_over = 0;
+    for (int64_t e = 0; e < n; ++e) {
+      if (load[e] > C) { dist[e] = 0; any_over = 1; } else dist[e] = BIG;
+      pred[e] = -1;
+    }
+    if (!any_over) break;
+    for (int64_t round = 0; round < n; ++round) {
+      int changed = 0;
+      for (int64_t e = 0; e < n; ++e) {
+        if (dist[e] >= BIG) continue;
+        for (int64_t f = 0; f < n; ++f) {
+          if (D[e * n + f] >= BIG) continue;
+          i128 nd = dist[e] + D[e * n + f];
+          if (nd < dist[f]) { dist[f] = nd; pred[f] = e; changed = 1; }
+        }
+      }
+      if (!changed) break;
+    }
+    int64_t target = -1;
+    for (int64_t f = 0; f < n; ++f)
+      if (load[f] < C && dist[f] < BIG && (target < 0 || dist[f] < dist[target])) target = f;
+    if (target < 0) { free(member); free(D); free(who); free(dist); free(pred); free(dirty); return MSO_ERR_INFEASIBLE; }
+    /* move one token along each arc of the walk, from the far end back */
+    int64_t f = target;
+    load[target] += 1;
+    while (pred[f] >= 0) {
+      int64_t e = pred[f];
+      int64_t i = who[e * n + f];
+      member[i * E + e] = 0; member[i * E + f] = 1;
+      /* rows to rebuild: e (lost i), f (gained i), and every other expert of i
+         (its arc into f may have been using i, and its arc into e may now use i) */
+      for (int64_t g = 0; g < n; ++g) if (member[i * E + g]) dirty[g] = 1;
+      dirty[e] = 1;
+      f = e;
+    }
+    load[f] -= 1; /* f is now the overloaded start of the walk */
+    ++aug;
+  }
+  for (int64_t i = 0; i < T; ++i) {
+    int64_t c = 0;
+    for (int64_t e = 0; e < E; ++e) if (member[i * E + e]) expert_idx[i * k + c++] = (int32_t)e;
+  }
+  if (n_augment) *n_augment = aug;
+  free(member); free(D); free(who); free(dist); free(pred); free(dirty);
+  return MSO_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* Index build: the slot of token i in expert e is the rank of i among  */
+/* the tokens assigned to e, in ascending token index.  Unused slots of */
+/* slot_token hold -1 (padding of the capacity-shaped buffers, Sec. 2.3).*/
+int mso_index_build(int64_t T, int64_t E, int64_t k, int64_t C, const int32_t *expert_idx,
+                    int32_t *slot_idx, int32_t *slot_token, int32_t *load) {
+  for (int64_t e = 0; e < E; ++e) load[e] = 0;
+  for (int64_t a = 0; a < E * C; ++a) slot_token[a] = -1;
+  for (int64_t i = 0; i < T; ++i)
+    for (int64_t c = 0; c < k; ++c) {
+      int32_t e = expert_idx[i * k + c];
+      if (e < 0 || e >= E || load[e] >= C) return MSO_ERR_ARG;
+      slot_idx[i * k + c] = load[e];
+      slot_token[(int64_t)e * C + load[e]] = (int32_t)i;
+      load[e] += 1;
+    }
+  return MSO_OK;
+}
+
+/* Dispatch: xdisp[e][s][:] = src[slot_token[e][s]][:], zero rows for   */
+/* padding.  Pure data movement on rows of row_bytes bytes.             */
+void mso_dispatch(int64_t E, int64_t C, int64_t row_bytes, const void *src,
+                  const int32_t *slot_token, void *dst) {
+  for (int64_t a = 0; a < E * C; ++a) {
+    char *out = (char *)dst + a * row_bytes;
+    if (slot_token[a] < 0) memset(out, 0, (size_t)row_bytes);
+    else memcpy(out, (const char *)src + (int64_t)slot_token[a] * row_bytes, (size_t)row_bytes);
+  }
+}
+
+/* Combine, Eq. 1: Y[i][:] = sum over the token's experts, in ascending  */
+/* expert index, of gate_w[i][c] * yexp[e][slot][:].  gate_w NULL means  */
+/* unit weights (the adjoint of dispatch).                               */
+void mso_combine(int64_t T, int64_t d, int64_t k, int64_t C, const double *yexp,
+                 const int32_t *expert_idx, const int32_t *slot_idx, const double *gate_w,
+                 double *Y) {
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < T; ++i) {
+    for (int64_t m = 0; m < d; ++m) Y[i * d + m] = 0.0;
+    for (int64_t c = 0; c < k; ++c) {
+      int64_t row = (int64_t)expert_idx[i * k + c] * C + slot_idx[i * k + c];
+      double g = gate_w ? gate_w[i * k + c] : 1.0;
+      for (int64_t m = 0; m < d; ++m) Y[i * d + m] += g * yexp[row * d + m];
+    }
+  }
+}
+
+/* Derivative of Eq. 1 with P held fixed:                               */
+/*   dyexp[e][s][:] = gate_w[i][c] * dY[i][:]   (zero rows for padding)  */
+/*   dgate_w[i][c]  = <dY[i][:], yexp[e][s][:]>                          */
+void mso_combine_bwd(int64_t T, int64_t d, int64_t E, int64_t k, int64_t C, const double *dY,
+                     const double *yexp, const int32_t *expert_idx, const int32_t *slot_idx,
+                     const double *gate_w, double *dyexp, double *dgate_w) {
+  for (int64_t a = 0; a < E * C * d; ++a) dyexp[a] = 0.0;
+  for (int64_t i = 0; i < T; ++i)
+    for (int64_t c = 0; c < k; ++c) {
+      int64_t row = (int64_t)expert_idx[i * k + c] * C + slot_idx[i * k + c];
+      double dot = 0.0;
+      for (int64_t m = 0; m < d; ++m) {
+        dyexp[row * d + m] = gate_w[i * k + c] * dY[i * d + m];
+        dot += dY[i * d + m] * yexp[row * d + m];
+      }
+      dgate_w[i * k + c] = dot;
+    }
+}
+
+/* Derivative of Eq. 2:  dW = H^T dL  ([d,E]),  dH = dL W^T  ([T,d]).    */
+void mso_gate_bwd(int64_t T, int64_t d, int64_t E, const double *H, const double *W,
+                  const double *dL, double *dW, double *dH) {
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < d; ++m)
+    for (int64_t j = 0; j < E; ++j) {
+      double acc = 0.0;
+      for (int64_t i = 0; i < T; ++i) acc += H[i * d + m] * dL[i * E + j];
+      dW[m * E + j] = acc;
+    }
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < T; ++i)
+    for (int64_t m = 0; m < d; ++m) {
+      double acc = 0.0;
+      for (int64_t j = 0; j < E; ++j) acc += dL[i * E + j] * W[m * E + j];
+      dH[i * d + m] = acc;
+    }
+}
+
+/* Auxiliary load-balance loss, Eq. 9:                                  */
+/*   L_aux = lambda / e * sum_j mean_i(A_ij) * mean_i(P_ij).            */
+double mso_aux_loss(int64_t T, int64_t E, int64_t k, double lambda, const double *A,
+                    const int32_t *expert_idx) {
+  double tot = 0.0;
+  for (int64_t j = 0; j < E; ++j) {
+    double sa = 0.0, sp = 0.0;
+    for (int64_t i = 0; i < T; ++i) {
+      sa += A[i * E + j];
+      for (int64_t c = 0; c < k; ++c) if (expert_idx[i * k + c] == j) sp += 1.0;
+    }
+    tot += (sa / (double)T) * (sp / (double)T);
+  }
+  return lambda * tot / (double)E;
+}
