@@ -1,0 +1,677 @@
+// Token -> expert assignment: the min-cost max-flow of Eq. 7-8 on the network of Table 1, solved
+// exactly on the GPU.
+//
+// Structure used.  The dual of the flow problem has one price p_e >= 0 per expert; given prices every
+// token independently holds its k largest values of key(i, e) - p_e.  The solver therefore works on
+// the E prices, never on the T x E arcs:
+//
+//   sweeps    (data parallel, one thread per token)  every token re-picks its top-k under the
+//             current prices; per expert a load count and two small histograms of margins (how much
+//             a price rise makes a holder leave / how much a price cut makes an outsider join) are
+//             collected; the last CTA to finish moves each over- or under-loaded expert's price to
+//             the histogram quantile that balances it, plus a step eps that is halved as the sweeps
+//             go on.  This is an epsilon-scaled simultaneous price adjustment (auction-style); it
+//             ends a few dozen token moves away from the optimum.
+//   collect   every token's top-k under the final prices is written out; tokens whose k-th and
+//             (k+1)-th values differ by at most theta are listed as candidates.
+//   exact     one CTA runs successive shortest augmenting paths on the expert-level residual graph
+//             (E experts + one node Z for the sink side), arcs e->f costing the cheapest candidate
+//             token move; node potentials keep reduced costs non-negative, so each search is a
+//             Bellman-Ford over E+1 nodes held in shared memory.  It ends with every expert within
+//             capacity and complementary slackness satisfied for the candidates.
+//   verify    a last data-parallel pass checks complementary slackness for EVERY token under the
+//             final prices.  If a non-candidate token is violated, theta grows and collect/exact run
+//             again.  Passing this check is a proof of optimality (LP duality of Eq. 7-8).
+//
+// All arithmetic is on int64 keys: key = rne(A * 2^40) (+ a 12-bit position hash) for float
+// affinities, or the quantised logit with a hashed tie-break.
+#pragma once
+#include "common.cuh"
+
+namespace msr {
+
+constexpr int kNBLog = 6;
+constexpr int kNB = 1 << kNBLog;          // histogram bins per expert
+constexpr int kTopN = kMaxK + 2;          // sorted values kept per token in a sweep
+constexpr long long kInf = 1LL << 62;
+constexpr long long kArcLimit = 1LL << 55; // arcs with a larger reduced cost are ignored by the exact phase
+constexpr int kMaxCand = 4096;            // candidate tokens one exact-phase round can hold
+constexpr int kCapLogMax = 60;
+constexpr int kCapLogMin = kNBLog + 1;
+constexpr int kEPLf = kMaxE / 32;          // experts per lane when a warp spans one token row
+
+struct KeyGen {
+  int mode;            // 0: float affinities, 1: quantised logits
+  int quant_shift;
+  uint32_t seed_mul;   // tiebreak_seed * 0x9E3779B9
+  int S;               // shift of the quantised part
+};
+
+__device__ __forceinline__ uint32_t fmix32(uint32_t h) {   // 32-bit finaliser of MurmurHash3
+  h ^= h >> 16; h *= 0x85ebca6bu; h ^= h >> 13; h *= 0xc2b2ae35u; h ^= h >> 16;
+  return h;
+}
+
+__device__ __forceinline__ long long make_key(const KeyGen& g, float x, uint32_t flat_idx) {
+  if (!isfinite(x)) x = 0.f;   // reported separately by the collect pass
+  // x * 2^40 is exact in fp32; the low 12 bits carry a multiplicative hash of the entry's position so
+  // that identical rows do not tie exactly (it moves the optimum by less than 4e-9 per chosen pair)
+  if (g.mode == 0) return __float2ll_rn(x * 1099511627776.0f) + (long long)((flat_idx * 2654435761u) >> 20);
+  float sc = rintf(ldexpf(x, g.quant_shift));
+  sc = fminf(fmaxf(sc, -32768.f), 32767.f);
+  long long q = (long long)sc;
+  uint32_t r = fmix32(flat_idx + g.seed_mul) >> 12;
+  return q * (1LL << g.S) + (long long)r;
+}
+
+struct FlowState {
+  long long p[kMaxE];        // expert prices
+  long long eps, eps_min;
+  long long theta;           // candidate threshold of the current round
+  double total_score;
+  int load[kMaxE];           // accumulated by the running pass, consumed by its last CTA
+  int load_cur[kMaxE];       // loads of the assignment currently written in expert_idx
+  unsigned hist_up[kMaxE * kNB];
+  unsigned hist_dn[kMaxE * kNB];
+  int cap_up[kMaxE], cap_dn[kMaxE];   // log2 of the histogram ranges
+  int flag_dn[kMaxE];                 // expert whose join-histogram came out short: scan it in full next sweep
+  unsigned ticket;
+  int sweep, p1_done, balanced;
+  int round, converged, ncand, violations, naug, rerouted;
+  unsigned status;
+  int ncand_last;
+};
+
+// ---------------------------------------------------------------------------------------------
+__global__ void flow_init_kernel(FlowState* st, long long eps0, long long eps_min, int cap0,
+                                 long long theta0, int balanced, int E) {
+  for (int i = threadIdx.x; i < kMaxE * kNB; i += blockDim.x) { st->hist_up[i] = 0; st->hist_dn[i] = 0; }
+  for (int e = threadIdx.x; e < kMaxE; e += blockDim.x) {
+    st->p[e] = 0; st->load[e] = 0; st->load_cur[e] = 0; st->cap_up[e] = cap0; st->cap_dn[e] = cap0; st->flag_dn[e] = 0;
+  }
+  if (threadIdx.x == 0) {
+    st->eps = eps0; st->eps_min = eps_min; st->theta = theta0; st->total_score = 0.0;
+    st->ticket = 0; st->sweep = 0; st->p1_done = 0; st->balanced = balanced;
+    st->round = 0; st->converged = 0; st->ncand = 0; st->violations = 0; st->naug = 0;
+    st->rerouted = 0; st->status = 0; st->ncand_last = 0;
+  }
+}
+
+// Insert (val, id) into a list sorted by descending value; on equal values the earlier (lower id,
+// because ids arrive ascending) entry stays in front.
+template <int N>
+__device__ __forceinline__ void top_insert(long long (&v)[N], int (&id)[N], long long val, int e) {
+  if (val > v[N - 1]) {
+    v[N - 1] = val; id[N - 1] = e;
+#pragma unroll
+    for (int j = N - 1; j > 0; --j) {
+      if (v[j] > v[j - 1]) {
+        long long tv = v[j]; v[j] = v[j - 1]; v[j - 1] = tv;
+        int ti = id[j]; id[j] = id[j - 1]; id[j - 1] = ti;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ bool last_block_arrives(unsigned* ticket) {
+  __shared__ bool is_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned t = atomicAdd(ticket, 1u);
+    is_last = (t == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (is_last) __threadfence();
+  return is_last;
+}
+
+// Price step that moves `need` tokens across the threshold of one expert, from its margin histogram
+// (bins of width 2^(cl - kNBLog) over [0, 2^cl)).  If the bin that holds the need-th smallest margin
+// also holds many more tokens (a group of near-ties), the step stops at the bin's lower edge and the
+// window is narrowed to that bin, so that the next sweep resolves the group; otherwise the step goes
+// to the bin's upper edge plus eps.
+__device__ __forceinline__ long long price_step(const unsigned* hist, int need, long long eps, int& cl,
+                                                bool& window_short, int grow) {
+  window_short = false;
+  unsigned cum = 0, before = 0; int pos = kNB;
+  for (int b = 0; b < kNB; ++b) {
+    const unsigned h = __ldcg(hist + b);
+    if (cum + h >= (unsigned)need) { pos = b; before = cum; cum += h; break; }
+    cum += h;
+  }
+  const int wl = cl - kNBLog;                         // log2 of the bin width
+  if (pos >= kNB) {                                   // the window is too narrow
+    const long long step = (1LL << cl);
+    cl = min(cl + grow, kCapLogMax);
+    window_short = true;
+    return step;
+  }
+  const long long e_eff = eps < (8LL << wl) ? eps : (8LL << wl);
+  if (cum <= 2u * (unsigned)need || cl <= kCapLogMin) {
+    const long long step = ((long long)(pos + 1) << wl) + e_eff;
+    if (pos < 4 && cl > kCapLogMin + 1) cl -= 2;
+    return step;
+  }
+  (void)before;
+  const long long step = (long long)pos << wl;        // conservative: moves fewer than `need`
+  cl = max(wl + 1, kCapLogMin);
+  return step;
+}
+
+// ---------------------------------------------------------------------------------------------
+// One price sweep.
+constexpr int kSweepThreads = 128;
+
+__global__ void __launch_bounds__(kSweepThreads)
+flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int k, int C, KeyGen g,
+                  int n_sweeps, int decay_every) {
+  if (*(volatile int*)&st->p1_done) return;
+  __shared__ long long sp[kMaxE];
+  __shared__ int sload[kMaxE];
+  __shared__ int scu[kMaxE], scd[kMaxE];
+  __shared__ int sflag[kMaxE];
+  __shared__ int nflag;
+  if (threadIdx.x == 0) nflag = 0;
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    sp[e] = st->p[e]; sload[e] = 0; scu[e] = st->cap_up[e]; scd[e] = st->cap_dn[e];
+    if (st->flag_dn[e]) sflag[atomicAdd(&nflag, 1)] = e;
+  }
+  __syncthreads();
+  const int tok = blockIdx.x * blockDim.x + threadIdx.x;
+  if (tok < T) {
+    long long v[kTopN]; int id[kTopN];
+#pragma unroll
+    for (int j = 0; j < kTopN; ++j) { v[j] = -kInf; id[j] = -1; }
+    const float* row = M + (size_t)tok * E;
+    const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+    if ((E & 3) == 0) {
+      for (int e = 0; e < E; e += 4) {
+        float4 x = __ldg(reinterpret_cast<const float4*>(row + e));
+        top_insert(v, id, make_key(g, x.x, flat + e) - sp[e], e);
+        top_insert(v, id, make_key(g, x.y, flat + e + 1) - sp[e + 1], e + 1);
+        top_insert(v, id, make_key(g, x.z, flat + e + 2) - sp[e + 2], e + 2);
+        top_insert(v, id, make_key(g, x.w, flat + e + 3) - sp[e + 3], e + 3);
+      }
+    } else {
+      for (int e = 0; e < E; ++e) top_insert(v, id, make_key(g, __ldg(row + e), flat + e) - sp[e], e);
+    }
+    const bool has_alt = E > k;
+    long long vk = -kInf, vk1 = -kInf;                // k-th value and best alternative
+#pragma unroll
+    for (int j = 0; j < kTopN; ++j) { if (j == k - 1) vk = v[j]; if (j == k) vk1 = v[j]; }
+#pragma unroll
+    for (int j = 0; j < kMaxK; ++j) {
+      if (j < k) {
+        const int e = id[j];
+        atomicAdd(&sload[e], 1);
+        if (has_alt) {
+          const long long m = v[j] - vk1;             // price rise at which this token leaves e
+          const int cl = scu[e];
+          if (m < (1LL << cl)) atomicAdd(&st->hist_up[e * kNB + (int)(m >> (cl - kNBLog))], 1u);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 1; j < kTopN; ++j) {
+      if ((j == k || j == k + 1) && j < E) {
+        const int e = id[j];
+        if (e >= 0) {
+          const long long m = vk - v[j];              // price cut at which this token joins e
+          const int cl = scd[e];
+          if (m < (1LL << cl)) atomicAdd(&st->hist_dn[e * kNB + (int)(m >> (cl - kNBLog))], 1u);
+        }
+      }
+    }
+    // experts whose join-histogram was short last time: count this token even if the expert is not
+    // among its best alternatives
+    for (int q = 0; q < nflag; ++q) {
+      const int e = sflag[q];
+      bool seen = false;
+#pragma unroll
+      for (int j = 0; j < kTopN; ++j) seen |= (j <= k + 1 && id[j] == e);
+      if (seen) continue;
+      const long long m = vk - (make_key(g, __ldg(row + e), flat + e) - sp[e]);
+      const int cl = scd[e];
+      if (m >= 0 && m < (1LL << cl)) atomicAdd(&st->hist_dn[e * kNB + (int)(m >> (cl - kNBLog))], 1u);
+    }
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x)
+    if (sload[e]) atomicAdd(&st->load[e], sload[e]);
+
+  if (!last_block_arrives(&st->ticket)) return;
+  // ---- last CTA: move the prices -------------------------------------------------------------
+  __shared__ int s_imb;
+  __shared__ long long pmin;
+  if (threadIdx.x == 0) s_imb = 0;
+  __syncthreads();
+  const long long eps = st->eps;
+  const bool balanced = st->balanced != 0;
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    const int load = __ldcg(&st->load[e]);
+    long long p = sp[e];
+    const int x = load - C;
+    if (x > 0) {
+      int cl = scu[e]; bool shortw;
+      p += price_step(st->hist_up + e * kNB, x, eps, cl, shortw, 3);
+      st->cap_up[e] = cl;
+      st->flag_dn[e] = 0;
+      atomicAdd(&s_imb, x);
+    } else if (x < 0 && (balanced || p > 0)) {
+      int cl = scd[e]; bool shortw;
+      p -= price_step(st->hist_dn + e * kNB, -x, eps, cl, shortw, 2);
+      if (!balanced && p < 0) p = 0;
+      st->cap_dn[e] = cl;
+      st->flag_dn[e] = shortw ? 1 : 0;
+      atomicAdd(&s_imb, -x);
+    } else {
+      st->flag_dn[e] = 0;
+    }
+    st->load[e] = 0;
+    // when nothing was out of balance the prices stay put and the collect pass reproduces this state
+    if (x != 0) sp[e] = p;
+  }
+  __syncthreads();   // every expert's histogram has been read before any is cleared
+  for (int i = threadIdx.x; i < E * kNB; i += blockDim.x) { st->hist_up[i] = 0; st->hist_dn[i] = 0; }
+  const int sweep = st->sweep + 1;
+  const bool done = (s_imb == 0) || sweep >= n_sweeps;
+  if (threadIdx.x == 0) {
+    // prices are only defined up to a shift when every expert must be full; anchor the minimum at 0
+    long long m = 0;
+    if (done && balanced) { m = sp[0]; for (int e = 1; e < E; ++e) m = sp[e] < m ? sp[e] : m; }
+    pmin = m;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x) st->p[e] = sp[e] - pmin;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    st->sweep = sweep;
+    if (sweep % decay_every == 0) { long long ne = eps >> 1; st->eps = ne < st->eps_min ? st->eps_min : ne; }
+    st->ticket = 0;
+    __threadfence();
+    if (done) st->p1_done = 1;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Collect / verify pass.  round 0 picks every token's top-k under the sweep prices.  Later rounds
+// keep a token's experts when they still are a top-k under the current prices (ties included) and
+// re-pick otherwise.  verify_only never re-picks: it only counts violations and gathers statistics.
+__global__ void __launch_bounds__(kSweepThreads)
+flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restrict__ expert_idx,
+                    int32_t* __restrict__ cand, int T, int E, int k, int C, KeyGen g, int first,
+                    int verify_only, long long theta_scale, int32_t* __restrict__ expert_load_out,
+                    void* stats_out, const unsigned* __restrict__ error_flag) {
+  if (!verify_only && *(volatile int*)&st->converged) return;
+  __shared__ long long sp[kMaxE];
+  __shared__ int sload[kMaxE];
+  __shared__ int s_viol, s_rer;
+  __shared__ double s_score;
+  __shared__ unsigned s_flags;
+  for (int e = threadIdx.x; e < E; e += blockDim.x) { sp[e] = st->p[e]; sload[e] = 0; }
+  if (threadIdx.x == 0) { s_viol = 0; s_rer = 0; s_score = 0.0; s_flags = 0; }
+  __syncthreads();
+  const long long theta = st->theta;
+  const int tok = blockIdx.x * blockDim.x + threadIdx.x;
+  if (tok < T) {
+    unsigned held[4] = {0, 0, 0, 0};
+    if (!first)
+      for (int c = 0; c < k; ++c) {
+        int e = expert_idx[(size_t)tok * k + c];
+        if (e >= 0 && e < E) held[e >> 5] |= 1u << (e & 31);
+      }
+    long long v[kMaxK + 1]; int id[kMaxK + 1];
+    long long raw[kMaxK];                       // k largest raw keys (unconstrained top-k), verify only
+#pragma unroll
+    for (int j = 0; j <= kMaxK; ++j) { v[j] = -kInf; id[j] = -1; }
+#pragma unroll
+    for (int j = 0; j < kMaxK; ++j) raw[j] = -kInf;
+    long long min_held = kInf, max_non = -kInf;
+    const float* row = M + (size_t)tok * E;
+    const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+    bool bad = false;
+    for (int e = 0; e < E; ++e) {
+      const float x = __ldg(row + e);
+      bad |= !isfinite(x);
+      const long long key = make_key(g, x, flat + e);
+      const long long val = key - sp[e];
+      top_insert(v, id, val, e);
+      if (held[e >> 5] >> (e & 31) & 1u) min_held = val < min_held ? val : min_held;
+      else max_non = val > max_non ? val : max_non;
+      if (verify_only && key > raw[kMaxK - 1]) {
+        raw[kMaxK - 1] = key;
+#pragma unroll
+        for (int j = kMaxK - 1; j > 0; --j)
+          if (raw[j] > raw[j - 1]) { long long t = raw[j]; raw[j] = raw[j - 1]; raw[j - 1] = t; }
+      }
+    }
+    if (bad) atomicOr(&s_flags, 2u);
+    const bool keep = !first && (min_held >= max_non);
+    long long gap;
+    if (!keep) {
+      if (!first) atomicAdd(&s_viol, 1);
+      if (!verify_only) {
+        held[0] = held[1] = held[2] = held[3] = 0;
+#pragma unroll
+        for (int j = 0; j < kMaxK; ++j)
+          if (j < k) held[id[j] >> 5] |= 1u << (id[j] & 31);
+        // the k-th value sits at v[k-1], the best alternative at v[k]
+        long long vk = -kInf, vk1 = -kInf;
+#pragma unroll
+        for (int j = 0; j <= kMaxK; ++j) { if (j == k - 1) vk = v[j]; if (j == k) vk1 = v[j]; }
+        gap = (E > k) ? vk - vk1 : kInf;
+      } else gap = kInf;
+    } else gap = (E > k) ? min_held - max_non : kInf;
+    // write the experts in ascending order (bit order of the mask)
+    int c = 0;
+    double sc = 0.0; int rer = 0;
+    long long kth_raw = -kInf;
+    if (verify_only) {
+#pragma unroll
+      for (int j = 0; j < kMaxK; ++j) if (j == k - 1) kth_raw = raw[j];
+    }
+    for (int wd = 0; wd < 4; ++wd) {
+      unsigned m = held[wd];
+      while (m) {
+        int e = (wd << 5) + __ffs(m) - 1; m &= m - 1;
+        if (c < k) expert_idx[(size_t)tok * k + c] = e;
+        ++c;
+        atomicAdd(&sload[e], 1);
+        if (verify_only) {
+          const float x = __ldg(row + e);
+          const long long key = make_key(g, x, flat + e);
+          sc += (g.mode == 0) ? (double)x : (double)key;
+          if (key < kth_raw) ++rer;
+        }
+      }
+    }
+    if (verify_only) { atomicAdd(&s_score, sc); if (rer) atomicAdd(&s_rer, rer); }
+    if (!verify_only && gap < kInf && gap <= theta) {
+      int pos = atomicAdd(&st->ncand, 1);
+      if (pos < kMaxCand) cand[pos] = tok;
+    }
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x)
+    if (sload[e]) atomicAdd(&st->load[e], sload[e]);
+  if (threadIdx.x == 0) {
+    if (s_viol) atomicAdd(&st->violations, s_viol);
+    if (s_flags) atomicOr(&st->status, s_flags);
+    if (verify_only) { atomicAdd(&st->total_score, s_score); if (s_rer) atomicAdd(&st->rerouted, s_rer); }
+  }
+  if (!last_block_arrives(&st->ticket)) return;
+  // ---- last CTA: is the state a certificate? ---------------------------------------------------
+  __shared__ int s_badload;
+  if (threadIdx.x == 0) s_badload = 0;
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    const int load = __ldcg(&st->load[e]);
+    st->load_cur[e] = load;
+    st->load[e] = 0;
+    if (verify_only && expert_load_out) expert_load_out[e] = load;
+    // primal feasibility and complementary slackness on the expert -> sink arcs
+    if (load > C || (sp[e] > 0 && load < C)) atomicAdd(&s_badload, 1);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int viol = *(volatile int*)&st->violations;
+    const bool ok = (first || viol == 0) && s_badload == 0;
+    st->violations = 0;
+    st->ticket = 0;
+    if (!verify_only) {
+      st->round = st->round + 1;
+      if (st->ncand > kMaxCand) st->ncand = kMaxCand;
+      st->theta = (theta > (kInf >> 8)) ? kInf : theta * theta_scale;   // next round looks further
+    }
+    if (verify_only && !ok) atomicOr(&st->status, 1u);
+    if (verify_only && error_flag && *error_flag) atomicOr(&st->status, 4u);
+    __threadfence();
+    if (ok) st->converged = 1;
+    if (verify_only && stats_out) {
+      // layout of maxscore_stats: status, capacity, sweeps, augmentations, rounds, candidates,
+      // rerouted, reserved, total_score
+      int* so = reinterpret_cast<int*>(stats_out);
+      so[0] = (int)(*(volatile unsigned*)&st->status & 7u);
+      so[1] = C; so[2] = st->sweep; so[3] = st->naug; so[4] = st->round;
+      so[5] = st->ncand_last; so[6] = *(volatile int*)&st->rerouted; so[7] = 0;
+      *reinterpret_cast<double*>(so + 8) = *(volatile double*)&st->total_score;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Exact phase: successive shortest augmenting paths on the expert-level residual graph, one CTA.
+constexpr int kP2Threads = 1024;
+
+struct P2Shared {
+  long long p[kMaxE + 1];        // potentials: prices of the experts, then Z
+  long long dist[2][kMaxE + 1];
+  int pred[kMaxE + 1];
+  int imb[kMaxE + 1];            // + excess, - deficit
+  int flow[kMaxE];               // units on expert -> sink
+  int dirty[kMaxE];
+  int path[kMaxE + 2];
+  int npath, changed, who, target, stop, any_pos;
+  long long dt;
+};
+
+__device__ __forceinline__ bool holds(const unsigned char* h, int k, int e) {
+  bool r = false;
+  for (int c = 0; c < k; ++c) r |= (h[c] == e);
+  return r;
+}
+
+__global__ void __launch_bounds__(kP2Threads)
+flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restrict__ expert_idx,
+                  const int32_t* __restrict__ cand_g, int T, int E, int k, int C, KeyGen g, int max_aug) {
+  if (*(volatile int*)&st->converged) return;
+  extern __shared__ __align__(16) unsigned char p2smem[];
+  long long* D = reinterpret_cast<long long*>(p2smem);                       // [E][E] raw arc costs
+  int* cand = reinterpret_cast<int*>(D + (size_t)E * E);                       // [kMaxCand]
+  unsigned char* held = reinterpret_cast<unsigned char*>(cand + kMaxCand);     // [kMaxCand][kMaxK]
+  __shared__ P2Shared s;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n = min(st->ncand, kMaxCand);
+  const int nZ = E;   // index of Z
+
+  // ---- candidates, sorted so that every tie below is broken the same way on every run -------------
+  int npow = 1; while (npow < n) npow <<= 1;
+  for (int i = tid; i < npow; i += blockDim.x) cand[i] = i < n ? cand_g[i] : 0x7fffffff;
+  __syncthreads();
+  for (int size = 2; size <= npow; size <<= 1)
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int i = tid; i < npow; i += blockDim.x) {
+        int j = i ^ stride;
+        if (j > i) {
+          bool up = (i & size) == 0;
+          int a = cand[i], b = cand[j];
+          if ((a > b) == up) { cand[i] = b; cand[j] = a; }
+        }
+      }
+      __syncthreads();
+    }
+  for (int i = tid; i < n * k; i += blockDim.x) {
+    int c = i / k, j = i - c * k;
+    held[c * kMaxK + j] = (unsigned char)expert_idx[(size_t)cand[c] * k + j];
+  }
+  for (int e = tid; e < E; e += blockDim.x) {
+    s.p[e] = st->p[e];
+    const int load = st->load_cur[e];
+    const int fl = s.p[e] > 0 ? C : min(load, C);
+    s.flow[e] = fl; s.imb[e] = load - fl; s.dirty[e] = 1;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int tot = 0;
+    for (int e = 0; e < E; ++e) tot += s.imb[e];
+    s.imb[nZ] = -tot; s.p[nZ] = 0; s.stop = 0;
+  }
+  __syncthreads();
+
+  int naug = 0;
+  for (;;) {
+    // ---- rebuild the rows of D marked dirty: D[e][f] = min over candidates in e, not in f ----------
+    for (int i = tid; i < E * E; i += blockDim.x)
+      if (s.dirty[i / E]) D[i] = kInf;
+    __syncthreads();
+    for (int c = warp; c < n; c += kP2Threads / 32) {
+      const unsigned char* h = held + c * kMaxK;
+      bool any = false;
+      for (int j = 0; j < k; ++j) any |= (s.dirty[h[j]] != 0);
+      if (!any) continue;
+      const int tok = cand[c];
+      const float* row = M + (size_t)tok * E;
+      const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+      long long key[kEPLf];
+      bool in[kEPLf];
+#pragma unroll
+      for (int q = 0; q < kEPLf; ++q) {
+        const int f = lane + 32 * q;
+        key[q] = f < E ? make_key(g, __ldg(row + f), flat + f) : 0;
+        in[q] = f < E ? holds(h, k, f) : true;
+      }
+      for (int j = 0; j < k; ++j) {
+        const int e = h[j];
+        if (!s.dirty[e]) continue;
+        long long mine = 0;
+#pragma unroll
+        for (int q = 0; q < kEPLf; ++q) if ((e >> 5) == q) mine = key[q];
+        const long long we = __shfl_sync(0xffffffffu, mine, e & 31);
+#pragma unroll
+        for (int q = 0; q < kEPLf; ++q) {
+          const int f = lane + 32 * q;
+          if (!in[q]) atomicMin(&D[e * E + f], we - key[q]);
+        }
+      }
+    }
+    __syncthreads();
+    for (int e = tid; e < E; e += blockDim.x) s.dirty[e] = 0;
+    if (tid == 0) {
+      int any = 0;
+      for (int v = 0; v <= E; ++v) any |= (s.imb[v] > 0);
+      s.any_pos = any;
+    }
+    __syncthreads();
+    if (!s.any_pos || naug >= max_aug) break;
+
+    // ---- Bellman-Ford from every node with excess, reduced costs rc = cost - p[u] + p[v] >= 0 --------
+    for (int v = tid; v <= E; v += blockDim.x) {
+      s.dist[0][v] = s.imb[v] > 0 ? 0 : kInf;
+      s.pred[v] = -1;
+    }
+    __syncthreads();
+    int cur = 0;
+    for (int round = 0; round <= E + 1; ++round) {
+      if (tid == 0) s.changed = 0;
+      __syncthreads();
+      for (int v = warp; v <= E; v += kP2Threads / 32) {
+        long long best = s.dist[cur][v]; int bu = -1;
+        for (int u = lane; u <= E; u += 32) {
+          const long long du = s.dist[cur][u];
+          if (du >= kInf || u == v) continue;
+          long long rc;
+          if (u < E && v < E) {
+            const long long c = D[u * E + v];
+            if (c >= kInf) continue;
+            rc = c - s.p[u] + s.p[v];
+          } else if (v == nZ) {          // expert u -> Z: one more unit on u -> sink
+            if (s.flow[u] >= C) continue;
+            rc = -s.p[u] + s.p[nZ];
+          } else {                       // Z -> expert v: one unit less on v -> sink
+            if (s.flow[v] <= 0) continue;
+            rc = -s.p[nZ] + s.p[v];
+          }
+          if (rc < 0) rc = 0;            // cannot happen while the potentials are valid
+          if (rc >= kArcLimit) continue;
+          const long long nd = du + rc;
+          if (nd < best || (nd == best && bu >= 0 && u < bu)) { best = nd; bu = u; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+          const int ou = __shfl_xor_sync(0xffffffffu, bu, o);
+          if (ob < best || (ob == best && ou >= 0 && (bu < 0 || ou < bu))) { best = ob; bu = ou; }
+        }
+        if (lane == 0) {
+          s.dist[cur ^ 1][v] = best;
+          if (bu >= 0 && best < s.dist[cur][v]) { s.pred[v] = bu; s.changed = 1; }
+        }
+      }
+      __syncthreads();
+      cur ^= 1;
+      if (!s.changed) break;
+      __syncthreads();
+    }
+    // ---- nearest node with a deficit --------------------------------------------------------------
+    if (tid == 0) {
+      int t = -1; long long dt = kInf;
+      for (int v = 0; v <= E; ++v)
+        if (s.imb[v] < 0 && s.dist[cur][v] < dt) { dt = s.dist[cur][v]; t = v; }
+      s.target = t; s.dt = dt; s.npath = 0;
+      if (t >= 0) {
+        int len = 0, v = t;
+        while (v >= 0 && len <= E + 1) { s.path[len++] = v; v = s.pred[v]; }
+        s.npath = len;
+      }
+    }
+    __syncthreads();
+    if (s.target < 0) break;        // no augmenting path inside the candidate graph: a wider theta is needed
+    for (int v = tid; v <= E; v += blockDim.x) {
+      const long long d = s.dist[cur][v];
+      s.p[v] -= (d < s.dt ? d : s.dt);
+    }
+    __syncthreads();
+    // ---- push one unit along the path (stored target first) ------------------------------------------
+    for (int a = s.npath - 1; a >= 1; --a) {
+      const int u = s.path[a], v = s.path[a - 1];
+      if (u < E && v < E) {
+        if (tid == 0) s.who = 0x7fffffff;
+        __syncthreads();
+        const long long want = D[u * E + v];
+        for (int c = tid; c < n; c += blockDim.x) {
+          const unsigned char* h = held + c * kMaxK;
+          if (!holds(h, k, u) || holds(h, k, v)) continue;
+          const int tok = cand[c];
+          const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+          const long long cost = make_key(g, __ldg(M + (size_t)tok * E + u), flat + u) -
+                                 make_key(g, __ldg(M + (size_t)tok * E + v), flat + v);
+          if (cost == want) atomicMin(&s.who, c);
+        }
+        __syncthreads();
+        if (s.who == 0x7fffffff) {   // internal inconsistency: stop, the verify pass will report it
+          if (tid == 0) { atomicOr(&st->status, 4u); s.stop = 1; }
+        } else if (tid == 0) {
+          unsigned char* h = held + s.who * kMaxK;
+          for (int j = 0; j < k; ++j) {
+            s.dirty[h[j]] = 1;
+            if (h[j] == u) h[j] = (unsigned char)v;
+          }
+          s.dirty[v] = 1;
+        }
+        __syncthreads();
+        if (s.stop) break;
+      } else if (tid == 0) {
+        if (v == nZ) s.flow[u] += 1; else s.flow[v] -= 1;
+      }
+    }
+    if (s.stop) break;
+    if (tid == 0) { s.imb[s.path[s.npath - 1]] -= 1; s.imb[s.target] += 1; }
+    ++naug;
+    __syncthreads();
+  }
+  // ---- write back ---------------------------------------------------------------------------------
+  __syncthreads();
+  for (int i = tid; i < n * k; i += blockDim.x) {
+    int c = i / k, j = i - c * k;
+    expert_idx[(size_t)cand[c] * k + j] = held[c * kMaxK + j];
+  }
+  for (int e = tid; e < E; e += blockDim.x) {
+    long long pe = s.p[e] - s.p[nZ];
+    st->p[e] = pe < 0 ? 0 : pe;     // only an expert that holds nothing can come out negative
+  }
+  if (tid == 0) { st->naug += naug; st->ncand_last = n; st->ncand = 0; }
+}
+
+}  // namespace msr

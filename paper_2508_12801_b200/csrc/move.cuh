@@ -1,0 +1,262 @@
+// Index build, dispatch, combine and combine-backward: the data movement of Eq. 1 through the
+// capacity-shaped [E, C, d_model] expert buffers of Sec. 2.3.
+#pragma once
+#include "common.cuh"
+
+namespace msr {
+
+// ---------------------------------------------------------------------------------------------
+// Index build.  slot_idx[i, c] = rank of token i among the tokens of expert expert_idx[i, c], in
+// ascending token order; slot_token is the inverse map.  Deterministic: no atomic decides an order.
+//   pass 1: per block of kIdxTok tokens, count tokens per expert
+//   pass 2: a block's base offset per expert = sum of the counts of the blocks before it; inside the
+//           block, warps are ordered by a scan of per-warp counts and lanes by a ballot mask.
+constexpr int kIdxTok = 1024;   // tokens per block, one per thread
+
+__global__ void __launch_bounds__(kIdxTok)
+index_count_kernel(const int32_t* __restrict__ expert_idx, int32_t* __restrict__ block_counts, int T,
+                   int E, int k) {
+  __shared__ int cnt[kMaxE];
+  for (int e = threadIdx.x; e < E; e += blockDim.x) cnt[e] = 0;
+  __syncthreads();
+  int tok = blockIdx.x * kIdxTok + threadIdx.x;
+  if (tok < T)
+    for (int c = 0; c < k; ++c) {
+      int e = __ldg(expert_idx + (size_t)tok * k + c);
+      if (e >= 0 && e < E) atomicAdd(&cnt[e], 1);
+    }
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x) block_counts[(size_t)blockIdx.x * E + e] = cnt[e];
+}
+
+__global__ void __launch_bounds__(kIdxTok)
+index_fill_kernel(const int32_t* __restrict__ expert_idx, const int32_t* __restrict__ block_counts,
+                  int32_t* __restrict__ slot_idx, int32_t* __restrict__ slot_token,
+                  int32_t* __restrict__ expert_load, int T, int E, int k, int C) {
+  __shared__ int base[kMaxE];                       // first slot of this block per expert
+  __shared__ int wcnt[kIdxTok / 32][kMaxE + 1];     // per-warp counts, then exclusive offsets
+  __shared__ unsigned bits[kIdxTok / 32][kMaxE];    // lanes of the warp that hold the expert
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    int b = 0, total = 0;
+    for (int blk = 0; blk < (int)gridDim.x; ++blk) {
+      int v = __ldg(block_counts + (size_t)blk * E + e);
+      if (blk < (int)blockIdx.x) b += v;
+      total += v;
+    }
+    base[e] = b;
+    if (blockIdx.x == 0) expert_load[e] = total;
+  }
+  for (int e = lane; e < E; e += 32) bits[warp][e] = 0u;
+  __syncthreads();
+  const int tok = blockIdx.x * kIdxTok + threadIdx.x;
+  int mine[kMaxK];
+#pragma unroll
+  for (int c = 0; c < kMaxK; ++c) {
+    mine[c] = -1;
+    if (c < k && tok < T) {
+      int e = __ldg(expert_idx + (size_t)tok * k + c);
+      if (e >= 0 && e < E) { mine[c] = e; atomicOr(&bits[warp][e], 1u << lane); }
+    }
+  }
+  __syncthreads();
+  for (int e = lane; e < E; e += 32) wcnt[warp][e] = __popc(bits[warp][e]);
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {   // exclusive scan over the warps of the block
+    int run = 0;
+    for (int w = 0; w < kIdxTok / 32; ++w) { int v = wcnt[w][e]; wcnt[w][e] = run; run += v; }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int c = 0; c < kMaxK; ++c) {
+    if (mine[c] >= 0) {
+      int e = mine[c];
+      int slot = base[e] + wcnt[warp][e] + __popc(bits[warp][e] & ((1u << lane) - 1u));
+      slot_idx[(size_t)tok * k + c] = slot;
+      if (slot < C) slot_token[(size_t)e * C + slot] = tok;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Dispatch: each token row is staged once in shared memory by a 1-D bulk (TMA) copy and written
+// from there to its k slots by k bulk stores.  One elected thread per CTA drives a ring of stages;
+// the copy engines do all the data movement, so a CTA needs no more threads than that.
+// A "unit" is one chunk of one token row (rows wider than the stage are split in chunks).
+struct DispatchArgs {
+  const char* src; char* dst;
+  const int32_t* expert_idx; const int32_t* slot_idx;
+  int T, k, C;
+  uint32_t row_bytes, chunk_bytes, chunks_per_row;
+  int stages;
+  unsigned* error_flag;
+};
+
+__global__ void __launch_bounds__(32) dispatch_kernel(const DispatchArgs a) {
+  extern __shared__ __align__(128) unsigned char dsm[];
+  __shared__ __align__(8) uint64_t full[16];
+  if (threadIdx.x != 0) return;
+  const int S = a.stages;
+  for (int s = 0; s < S; ++s) mbar_init(&full[s], 1);
+  fence_barrier_init();
+  fence_proxy_async();
+  const long long units = (long long)a.T * a.chunks_per_row;
+  const long long per = (units + gridDim.x - 1) / gridDim.x;       // contiguous range per CTA
+  const long long u0 = per * blockIdx.x;
+  const long long u1 = u0 + per < units ? u0 + per : units;
+  if (u0 >= u1) return;
+  auto issue_load = [&](long long u, int s) {
+    long long tok = u / a.chunks_per_row;
+    uint32_t ch = (uint32_t)(u % a.chunks_per_row);
+    uint32_t off = ch * a.chunk_bytes;
+    uint32_t bytes = a.row_bytes - off < a.chunk_bytes ? a.row_bytes - off : a.chunk_bytes;
+    mbar_expect_tx(&full[s], bytes);
+    bulk_g2s(dsm + (size_t)s * a.chunk_bytes, a.src + tok * (long long)a.row_bytes + off, bytes, &full[s]);
+  };
+  // prologue: fill the ring
+  for (int s = 0; s < S && u0 + s < u1; ++s) issue_load(u0 + s, s);
+  bool ok = true;
+  for (long long u = u0; u < u1 && ok; ++u) {
+    const long long n = u - u0;
+    const int s = (int)(n % S);
+    const uint32_t phase = (uint32_t)((n / S) & 1);
+    ok = mbar_wait_bounded(&full[s], phase);
+    if (!ok) break;
+    long long tok = u / a.chunks_per_row;
+    uint32_t ch = (uint32_t)(u % a.chunks_per_row);
+    uint32_t off = ch * a.chunk_bytes;
+    uint32_t bytes = a.row_bytes - off < a.chunk_bytes ? a.row_bytes - off : a.chunk_bytes;
+    for (int c = 0; c < a.k; ++c) {
+      int e = __ldg(a.expert_idx + tok * a.k + c);
+      int sl = __ldg(a.slot_idx + tok * a.k + c);
+      if (e < 0 || sl < 0 || sl >= a.C) continue;
+      bulk_s2g(a.dst + ((long long)e * a.C + sl) * (long long)a.row_bytes + off,
+               dsm + (size_t)s * a.chunk_bytes, bytes);
+    }
+    bulk_commit();
+    // The stage used one iteration ago may be refilled once its stores have read shared memory.
+    if (n >= 1 && u - 1 + S < u1) {
+      bulk_wait_read<1>();
+      issue_load(u - 1 + S, (int)((n - 1) % S));
+    }
+  }
+  bulk_wait_all<0>();
+  if (!ok) atomicOr(a.error_flag, 4u);
+}
+
+// Zero the rows of padding slots (slot_token < 0) of an [E*C, row] buffer.
+__global__ void __launch_bounds__(256)
+zero_padding_kernel(const int32_t* __restrict__ slot_token, char* __restrict__ dst, long long n_slots,
+                    uint32_t row_bytes) {
+  const int warps = blockDim.x >> 5, lane = threadIdx.x & 31;
+  for (long long s = (long long)blockIdx.x * warps + (threadIdx.x >> 5); s < n_slots;
+       s += (long long)gridDim.x * warps) {
+    if (__ldg(slot_token + s) >= 0) continue;
+    uint4* row = reinterpret_cast<uint4*>(dst + s * (long long)row_bytes);
+    for (uint32_t v = lane; v < row_bytes / 16; v += 32) row[v] = make_uint4(0, 0, 0, 0);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Combine: dst[i, :] = sum_c w[i, c] * src[e_c, slot_c, :] in fp32, ascending c, rounded once.
+// One CTA per token at a time; a thread owns 16-byte column groups and keeps the k row loads of a
+// group in flight together.
+template <typename T>
+__global__ void __launch_bounds__(256)
+combine_kernel(const T* __restrict__ src, const int32_t* __restrict__ expert_idx,
+               const int32_t* __restrict__ slot_idx, const float* __restrict__ gate_w,
+               T* __restrict__ dst, int Tn, int d, int k, int C, int accumulate) {
+  constexpr int N = Vec16<T>::N;
+  __shared__ long long rowoff[kMaxK];
+  __shared__ float wgt[kMaxK];
+  const int nvec = d / N;
+  for (int tok = blockIdx.x; tok < Tn; tok += gridDim.x) {
+    __syncthreads();
+    if (threadIdx.x < k) {
+      int e = __ldg(expert_idx + (size_t)tok * k + threadIdx.x);
+      int sl = __ldg(slot_idx + (size_t)tok * k + threadIdx.x);
+      const bool valid = e >= 0 && sl >= 0 && sl < C;   // a malformed entry contributes nothing
+      rowoff[threadIdx.x] = valid ? ((long long)e * C + sl) * (long long)d : 0;
+      wgt[threadIdx.x] = !valid ? 0.f : gate_w ? __ldg(gate_w + (size_t)tok * k + threadIdx.x) : 1.f;
+    }
+    __syncthreads();
+    for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
+      float x[kMaxK][N];
+#pragma unroll
+      for (int c = 0; c < kMaxK; ++c)
+        if (c < k) Vec16<T>::load(src + rowoff[c] + (size_t)v * N, x[c]);
+      float acc[N];
+#pragma unroll
+      for (int j = 0; j < N; ++j) acc[j] = 0.f;
+      if (accumulate) Vec16<T>::load(dst + (size_t)tok * d + (size_t)v * N, acc);
+#pragma unroll
+      for (int c = 0; c < kMaxK; ++c)
+        if (c < k) {
+          const float w = wgt[c];
+#pragma unroll
+          for (int j = 0; j < N; ++j) acc[j] = fmaf(w, x[c][j], acc[j]);
+        }
+      Vec16<T>::store(dst + (size_t)tok * d + (size_t)v * N, acc);
+    }
+  }
+}
+
+// Combine backward: dyexp[e_c, slot_c, :] = w[i, c] * dY[i, :],  dgate_w[i, c] = <dY[i, :], yexp[e_c, slot_c, :]>.
+// One CTA per token; the dY chunk of a thread is read once and reused for the k experts.
+template <typename T>
+__global__ void __launch_bounds__(256)
+combine_bwd_kernel(const T* __restrict__ dY, const T* __restrict__ yexp,
+                   const int32_t* __restrict__ expert_idx, const int32_t* __restrict__ slot_idx,
+                   const float* __restrict__ gate_w, T* __restrict__ dyexp, float* __restrict__ dgate_w,
+                   int Tn, int d, int k, int C) {
+  constexpr int N = Vec16<T>::N;
+  __shared__ long long rowoff[kMaxK];
+  __shared__ float wgt[kMaxK];
+  __shared__ float red[8][kMaxK];
+  const int nvec = d / N;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int tok = blockIdx.x; tok < Tn; tok += gridDim.x) {
+    __syncthreads();
+    if (threadIdx.x < k) {
+      int e = __ldg(expert_idx + (size_t)tok * k + threadIdx.x);
+      int sl = __ldg(slot_idx + (size_t)tok * k + threadIdx.x);
+      const bool valid = e >= 0 && sl >= 0 && sl < C;   // a malformed entry is skipped
+      rowoff[threadIdx.x] = valid ? ((long long)e * C + sl) * (long long)d : -1;
+      wgt[threadIdx.x] = __ldg(gate_w + (size_t)tok * k + threadIdx.x);
+    }
+    __syncthreads();
+    float dot[kMaxK];
+#pragma unroll
+    for (int c = 0; c < kMaxK; ++c) dot[c] = 0.f;
+    for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
+      float g[N];
+      Vec16<T>::load(dY + (size_t)tok * d + (size_t)v * N, g);
+      float y[kMaxK][N];
+#pragma unroll
+      for (int c = 0; c < kMaxK; ++c)
+        if (c < k && rowoff[c] >= 0) Vec16<T>::load(yexp + rowoff[c] + (size_t)v * N, y[c]);
+#pragma unroll
+      for (int c = 0; c < kMaxK; ++c)
+        if (c < k && rowoff[c] >= 0) {
+          float o[N];
+          const float w = wgt[c];
+#pragma unroll
+          for (int j = 0; j < N; ++j) { dot[c] = fmaf(g[j], y[c][j], dot[c]); o[j] = w * g[j]; }
+          Vec16<T>::store(dyexp + rowoff[c] + (size_t)v * N, o);
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < kMaxK; ++c) {
+      float s = warp_sum(dot[c]);
+      if (lane == 0) red[warp][c] = s;
+    }
+    __syncthreads();
+    if (threadIdx.x < k) {
+      float s = 0.f;
+      for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w][threadIdx.x];
+      dgate_w[(size_t)tok * k + threadIdx.x] = s;
+    }
+  }
+}
+
+}  // namespace msr

@@ -1,0 +1,127 @@
+// SoftTopk forward and backward (Eq. 6 and its derivative), one warp per token.
+//
+// Level j (1-based) of Eq. 6 adds a softmax with temperature t over the entries that are not among
+// the j-1 largest (ties: lowest expert index).  A lane holds experts lane, lane+32, ... so every
+// global access of a warp is one contiguous row segment, and each level costs two shuffle
+// reductions (arg-max, sum).
+#pragma once
+#include "common.cuh"
+
+namespace msr {
+
+constexpr int kEPL = kMaxE / 32;  // experts per lane
+
+// arg-max over the warp of (value, index) pairs, lowest index on equal values
+__device__ __forceinline__ void warp_argmax(float& v, int& idx) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    float ov = __shfl_xor_sync(0xffffffffu, v, o);
+    int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+    if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+  }
+}
+
+__global__ void __launch_bounds__(256)
+softtopk_fwd_kernel(const float* __restrict__ logits, float* __restrict__ scores, int T, int E, int k,
+                    float t) {
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  for (int tok = blockIdx.x * warps_per_block + (threadIdx.x >> 5); tok < T;
+       tok += gridDim.x * warps_per_block) {
+    const float* row = logits + (size_t)tok * E;
+    float a[kEPL], y[kEPL];
+    bool live[kEPL];
+#pragma unroll
+    for (int j = 0; j < kEPL; ++j) {
+      int e = lane + 32 * j;
+      live[j] = e < E;
+      a[j] = live[j] ? __ldg(row + e) : 0.f;
+      y[j] = 0.f;
+    }
+    for (int level = 0; level < k; ++level) {
+      float best = -INFINITY; int bidx = 0x7fffffff;
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j)
+        if (live[j] && (a[j] > best || bidx == 0x7fffffff)) { best = a[j]; bidx = lane + 32 * j; }
+      warp_argmax(best, bidx);
+      float z[kEPL], zs = 0.f;
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j) {
+        z[j] = live[j] ? expf((a[j] - best) / t) : 0.f;
+        zs += z[j];
+      }
+      zs = warp_sum(zs);
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j) {
+        y[j] += z[j] / zs;
+        if (lane + 32 * j == bidx) live[j] = false;   // masked from the next level on
+      }
+    }
+    float* out = scores + (size_t)tok * E;
+#pragma unroll
+    for (int j = 0; j < kEPL; ++j) {
+      int e = lane + 32 * j;
+      if (e < E) out[e] = y[j];
+    }
+  }
+}
+
+// dlogits = J^T g with g non-zero only at the token's k assigned experts.  The masks are constants.
+//   da_l = (1/t) * sum_{levels j with l unmasked} q_l * (g_l - sum_i g_i q_i),  q = level-j softmax
+__global__ void __launch_bounds__(256)
+softtopk_bwd_kernel(const float* __restrict__ logits, const int32_t* __restrict__ expert_idx,
+                    const float* __restrict__ dgate_w, float* __restrict__ dlogits, int T, int E, int k,
+                    float t) {
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  for (int tok = blockIdx.x * warps_per_block + (threadIdx.x >> 5); tok < T;
+       tok += gridDim.x * warps_per_block) {
+    const float* row = logits + (size_t)tok * E;
+    float a[kEPL], g[kEPL], da[kEPL];
+    bool live[kEPL];
+#pragma unroll
+    for (int j = 0; j < kEPL; ++j) {
+      int e = lane + 32 * j;
+      live[j] = e < E;
+      a[j] = live[j] ? __ldg(row + e) : 0.f;
+      g[j] = 0.f; da[j] = 0.f;
+    }
+    for (int c = 0; c < k; ++c) {
+      int e = __ldg(expert_idx + (size_t)tok * k + c);
+      float gv = __ldg(dgate_w + (size_t)tok * k + c);
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j)
+        if (lane + 32 * j == e) g[j] = gv;
+    }
+    for (int level = 0; level < k; ++level) {
+      float best = -INFINITY; int bidx = 0x7fffffff;
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j)
+        if (live[j] && (a[j] > best || bidx == 0x7fffffff)) { best = a[j]; bidx = lane + 32 * j; }
+      warp_argmax(best, bidx);
+      float z[kEPL], zs = 0.f, gz = 0.f;
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j) {
+        z[j] = live[j] ? expf((a[j] - best) / t) : 0.f;
+        zs += z[j];
+        gz += g[j] * z[j];
+      }
+      zs = warp_sum(zs);
+      gz = warp_sum(gz);
+      const float gq = gz / zs;
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j) {
+        da[j] += (z[j] / zs) * (g[j] - gq) / t;
+        if (lane + 32 * j == bidx) live[j] = false;
+      }
+    }
+    float* out = dlogits + (size_t)tok * E;
+#pragma unroll
+    for (int j = 0; j < kEPL; ++j) {
+      int e = lane + 32 * j;
+      if (e < E) out[e] = da[j];
+    }
+  }
+}
+
+}  // namespace msr
