@@ -1,0 +1,215 @@
+/*
+ * maxscore.h -- C ABI of the MaxScore router for NVIDIA B200 (sm_100a).
+ *
+ * Maximum Score Routing (arXiv 2508.12801) for one MoE layer and one batch of T tokens:
+ *
+ *   gate logits      L = H . W_g                                   (Eq. 2)
+ *   affinities       A = SoftTopk(L; k, t)                         (Eq. 6)
+ *   assignment       P = argmax { sum_ij P_ij A_ij : P binary, every token has exactly k experts,
+ *                                 every expert at most C tokens }  (Eq. 7-8, network of Table 1)
+ *   capacity         C = ceil(cf * T * k / E)                      (Sec. 2.3; Algorithm 1, step 1)
+ *   dispatch/combine tokens into and out of dense [E, C, d_model] expert buffers   (Eq. 1)
+ *
+ * Conventions that hold for every entry point
+ *   - All tensor arguments are DEVICE pointers unless the name ends in _host.  Row-major, contiguous,
+ *     16-byte aligned.  The caller owns every buffer; the library allocates no device memory and
+ *     keeps no pointer after a call returns other than the workspace handed to maxscore_create.
+ *   - cuda_stream is a cudaStream_t passed as void*.  Calls enqueue work and return without
+ *     synchronising.  Calls on one context must not overlap on the GPU (they share the workspace).
+ *   - Host-detectable errors (NULL pointers, bad sizes, k > E, infeasible capacity, misalignment,
+ *     short workspace) return a status before anything is launched.  Conditions only the device sees
+ *     (solver gave up, non-finite input) set bits in maxscore_stats.status, which the caller reads
+ *     after synchronising.  Nothing aborts, throws or traps.
+ *   - expert_idx[i, :] is ascending.  slot_idx[i, c] is the rank of token i among the tokens of expert
+ *     expert_idx[i, c], in ascending token order.  Unused slots of slot_token hold -1.
+ *   - Limits of this build: 1 <= k <= 8, k <= E <= 128, bf16 I/O needs d_model % 8 == 0, fp32 I/O
+ *     needs d_model % 4 == 0, T * k < 2^31.
+ */
+#ifndef MAXSCORE_H_
+#define MAXSCORE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct maxscore_ctx maxscore_ctx; /* opaque; owns nothing but host bookkeeping */
+
+typedef enum {
+  MAXSCORE_OK = 0,
+  MAXSCORE_ERR_INVALID_ARG = 1,   /* NULL pointer, non-positive size, misaligned pointer        */
+  MAXSCORE_ERR_INFEASIBLE = 2,    /* k > E, or E * min(C, T) < T * k: no assignment exists       */
+  MAXSCORE_ERR_WORKSPACE = 3,     /* workspace smaller than maxscore_workspace_bytes()           */
+  MAXSCORE_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed (see maxscore_last_cuda_error) */
+  MAXSCORE_ERR_NOT_CONVERGED = 5, /* never returned by a call; mirrors the stats bit for readers */
+  MAXSCORE_ERR_UNSUPPORTED = 6    /* outside the limits listed above                             */
+} maxscore_status;
+
+typedef enum { MAXSCORE_F32 = 0, MAXSCORE_BF16 = 1 } maxscore_dtype;
+
+/* bits of maxscore_stats.status */
+#define MAXSCORE_STAT_NOT_CONVERGED 1u /* solver hit max_sweeps; the assignment returned is not certified optimal */
+#define MAXSCORE_STAT_NON_FINITE 2u    /* a NaN or Inf was seen in the score matrix                               */
+#define MAXSCORE_STAT_INTERNAL 4u      /* an internal bound (a bounded wait, a path search) was hit               */
+
+typedef struct {
+  int32_t T;               /* tokens in the batch (the paper's n)                                  */
+  int32_t d_model;         /* width of a token row                                                 */
+  int32_t E;               /* experts (the paper's e)                                              */
+  int32_t k;               /* experts per token                                                    */
+  float capacity_factor;   /* c_f of Sec. 2.3; C = ceil(c_f * T * k / E)                           */
+  int32_t capacity;        /* > 0 overrides the formula                                            */
+  float t;                 /* SoftTopk temperature, > 0                                            */
+  int32_t score_mode;      /* 0: maximise the float affinities A, as fixed-point keys              */
+                           /*    rne(A * 2^40) + (((i*E + j) * 2654435761 mod 2^32) >> 20): the    */
+                           /*    12-bit position hash only separates exact ties (< 4e-9 per pair); */
+                           /* 1: maximise integer keys from the logits: q * 2^S + r with           */
+                           /*    q = clamp_int16(rne(L * 2^quant_shift)),                          */
+                           /*    r = fmix32(i*E + j + tiebreak_seed * 0x9E3779B9) >> 12            */
+                           /*        (fmix32 = 32-bit finaliser of MurmurHash3),                   */
+                           /*    S = 20 + ceil(log2(T*k))                                          */
+  int32_t quant_shift;     /* score_mode 1 only                                                    */
+  uint32_t tiebreak_seed;  /* score_mode 1 only                                                    */
+  int32_t max_sweeps;      /* bound on price sweeps + augmentations of the solver; 0 = default     */
+  int32_t io_dtype;        /* maxscore_dtype of hidden, w_gate, xdisp, yexp, y, dY, dH             */
+  int32_t w_gate_layout;   /* 0: w_gate is [d_model, E] as in Eq. 2; 1: [E, d_model]               */
+} maxscore_params;
+
+typedef struct {           /* lives in DEVICE memory; written by route_fwd / assign                */
+  uint32_t status;         /* MAXSCORE_STAT_* bits                                                 */
+  int32_t capacity;        /* C used                                                               */
+  int32_t sweeps;          /* price sweeps run                                                     */
+  int32_t augmentations;   /* exact augmenting paths applied after the sweeps                      */
+  int32_t rounds;          /* candidate-collection rounds used by the exact phase                  */
+  int32_t candidates;      /* tokens in the last candidate list                                    */
+  int32_t rerouted;        /* token-slots assigned outside the token's own unconstrained top-k     */
+  int32_t reserved;
+  double total_score;      /* score_mode 0: sum of A over the chosen pairs; mode 1: sum of keys    */
+} maxscore_stats;
+
+/* C = ceil(c_f * T * k / E), or params->capacity when that is > 0 (Sec. 2.3).  Returns -1 on NULL. */
+int32_t maxscore_capacity(const maxscore_params* params);
+
+/* Bytes of device workspace a context for `params` needs.  Host only. */
+maxscore_status maxscore_workspace_bytes(const maxscore_params* params, size_t* bytes);
+
+/* Validate params, record the workspace (device memory, 256-byte aligned, at least the size above,
+ * owned by the caller and left untouched by other work while the context lives) and build a context.
+ * Performs no device work except one cudaMemsetAsync of the workspace head on the default stream,
+ * followed by a synchronise. */
+maxscore_status maxscore_create(maxscore_ctx** ctx, const maxscore_params* params, void* workspace,
+                                size_t workspace_bytes);
+void maxscore_destroy(maxscore_ctx* ctx);
+
+/* Text of the last CUDA error seen by this thread's calls ("" if none). Host only. */
+const char* maxscore_last_cuda_error(void);
+
+/* ---- the four calls of the hot path ------------------------------------------------------------ */
+
+/* Forward routing of one batch: Eq. 2, Eq. 6, Eq. 7-8, then the slot indices of the E x C buffers.
+ *   hidden      [T, d_model]  io_dtype          in
+ *   w_gate      per w_gate_layout, io_dtype     in
+ *   expert_bias [E] fp32 or NULL                in   added to the logits (not in the paper; used to
+ *                                                    skew the load in tests)
+ *   logits      [T, E] fp32                     out  L
+ *   scores      [T, E] fp32                     out  A
+ *   expert_idx  [T, k] int32                    out  the experts of each token, ascending
+ *   slot_idx    [T, k] int32                    out
+ *   gate_w      [T, k] fp32                     out  A at the chosen pairs (R(x) of Eq. 1-2, not renormalised)
+ *   slot_token  [E, C] int32                    out  token held by each slot, -1 = padding
+ *   expert_load [E] int32                       out
+ *   stats       device maxscore_stats           out */
+maxscore_status maxscore_route_fwd(maxscore_ctx* ctx, const void* hidden, const void* w_gate,
+                                   const float* expert_bias, float* logits, float* scores,
+                                   int32_t* expert_idx, int32_t* slot_idx, float* gate_w,
+                                   int32_t* slot_token, int32_t* expert_load, maxscore_stats* stats,
+                                   void* cuda_stream);
+
+/* Dispatch (Eq. 1, input side): dst[e, s, :] = src[slot_token[e, s], :], zero rows where the slot is
+ * padding.  src [T, d_model], dst [E, C, d_model], both io_dtype.  Needs slot_idx and expert_idx too:
+ * rows are read once per token and written to each of its k slots. */
+maxscore_status maxscore_dispatch(maxscore_ctx* ctx, const void* src, const int32_t* expert_idx,
+                                  const int32_t* slot_idx, const int32_t* slot_token, void* dst,
+                                  void* cuda_stream);
+
+/* Combine (Eq. 1, output side): dst[i, :] = sum_c gate_w[i, c] * src[expert_idx[i, c], slot_idx[i, c], :],
+ * summed in ascending expert index in fp32 and rounded once.  gate_w NULL = unit weights (this is the
+ * backward of dispatch).  accumulate != 0 adds to dst instead of overwriting it. */
+maxscore_status maxscore_combine(maxscore_ctx* ctx, const void* src, const int32_t* expert_idx,
+                                 const int32_t* slot_idx, const float* gate_w, void* dst,
+                                 int accumulate, void* cuda_stream);
+
+/* Backward of combine, SoftTopk and the gate with the assignment P held constant:
+ *   dyexp[e, s, :]   = gate_w * dY[i, :]        (zero rows at padding slots)     [E, C, d_model] io_dtype
+ *   dgate_w[i, c]    = <dY[i, :], yexp[e, s, :]>                                 [T, k] fp32
+ *   dlogits          = J_SoftTopk^T . scatter(dgate_w)                           [T, E] fp32
+ *   dw_gate          = H^T . dlogits            always [d_model, E] fp32
+ *   dH               = dlogits . W_g^T          [T, d_model] io_dtype
+ * slot_token is needed to zero the padding rows of dyexp. */
+maxscore_status maxscore_route_bwd(maxscore_ctx* ctx, const void* dY, const void* yexp,
+                                   const void* hidden, const void* w_gate, const float* logits,
+                                   const int32_t* expert_idx, const int32_t* slot_idx,
+                                   const float* gate_w, const int32_t* slot_token, void* dyexp,
+                                   float* dgate_w, float* dlogits, float* dw_gate, void* dH,
+                                   void* cuda_stream);
+
+/* ---- single stages (the same kernels route_fwd / route_bwd run), for stage-by-stage checks ------ */
+
+/* Eq. 2 only: logits = hidden . w_gate (+ expert_bias). */
+maxscore_status maxscore_gate(maxscore_ctx* ctx, const void* hidden, const void* w_gate,
+                              const float* expert_bias, float* logits, void* cuda_stream);
+
+/* Eq. 6 only: scores = SoftTopk(logits; k, t). */
+maxscore_status maxscore_softtopk_fwd(maxscore_ctx* ctx, const float* logits, float* scores,
+                                      void* cuda_stream);
+
+/* Derivative of Eq. 6: dlogits = J^T g where g is zero except g[i, expert_idx[i, c]] = dgate_w[i, c]. */
+maxscore_status maxscore_softtopk_bwd(maxscore_ctx* ctx, const float* logits,
+                                      const int32_t* expert_idx, const float* dgate_w,
+                                      float* dlogits, void* cuda_stream);
+
+/* Eq. 7-8 only: the solver on a caller-supplied [T, E] fp32 matrix (affinities in score_mode 0,
+ * logits in score_mode 1).  Writes expert_idx [T, k], expert_load [E] and stats. */
+maxscore_status maxscore_assign(maxscore_ctx* ctx, const float* matrix, int32_t* expert_idx,
+                                int32_t* expert_load, maxscore_stats* stats, void* cuda_stream);
+
+/* Slot indices of an assignment: slot_idx [T, k], slot_token [E, C], expert_load [E]. */
+maxscore_status maxscore_index_build(maxscore_ctx* ctx, const int32_t* expert_idx, int32_t* slot_idx,
+                                     int32_t* slot_token, int32_t* expert_load, void* cuda_stream);
+
+/* Derivative of Eq. 1 alone (first two outputs of route_bwd). */
+maxscore_status maxscore_combine_bwd(maxscore_ctx* ctx, const void* dY, const void* yexp,
+                                     const int32_t* expert_idx, const int32_t* slot_idx,
+                                     const float* gate_w, const int32_t* slot_token, void* dyexp,
+                                     float* dgate_w, void* cuda_stream);
+
+/* Derivative of Eq. 2 alone (last two outputs of route_bwd). */
+maxscore_status maxscore_gate_bwd(maxscore_ctx* ctx, const void* hidden, const void* w_gate,
+                                  const float* dlogits, float* dw_gate, void* dH, void* cuda_stream);
+
+/* ---- end-to-end from host memory ---------------------------------------------------------------- */
+
+/* route_fwd + dispatch for callers whose batch lives in HOST memory (pinned for full speed).
+ * Copies hidden_host (and w_gate_host, expert_bias_host) to the device buffers given in `dev`,
+ * runs maxscore_route_fwd and maxscore_dispatch, copies expert_idx, slot_idx, gate_w and stats back
+ * to the *_host outputs and synchronises the stream before returning.  xdisp stays on the device
+ * (dev->xdisp) for the experts to consume. */
+typedef struct {
+  void* hidden; void* w_gate; float* expert_bias; float* logits; float* scores; int32_t* expert_idx;
+  int32_t* slot_idx; float* gate_w; int32_t* slot_token; int32_t* expert_load; maxscore_stats* stats;
+  void* xdisp;
+} maxscore_device_buffers;
+
+maxscore_status maxscore_route_dispatch_host(maxscore_ctx* ctx, const void* hidden_host,
+                                             const void* w_gate_host, const float* expert_bias_host,
+                                             const maxscore_device_buffers* dev,
+                                             int32_t* expert_idx_host, int32_t* slot_idx_host,
+                                             float* gate_w_host, maxscore_stats* stats_host,
+                                             void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MAXSCORE_H_ */

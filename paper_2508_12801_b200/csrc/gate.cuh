@@ -1,0 +1,282 @@
+// Gate logits L = H . W_g (+ bias), Eq. 2, and the derivative GEMMs.
+//
+// bf16 path: tcgen05 tensor cores.  One CTA owns a 128-token tile; H streams through a ring of
+// 128x64 bf16 tiles loaded by TMA (128-byte swizzle), W_g (transposed and padded to [Npad, d] once
+// per call) rides along, the fp32 accumulator [128 x Npad] lives in tensor memory and is read back
+// by the four warps of the CTA, one TMEM lane quarter each, so that every thread ends up with one
+// token's full row of logits.  The contraction is HBM-bound (intensity ~ E flop per byte of H), so
+// the design goal is to keep as many H tiles in flight as shared memory allows: two CTAs per SM.
+//
+// fp32 path: plain FMA tiles (tensor cores would round the inputs to tf32).
+#pragma once
+#include <cuda.h>
+#include "common.cuh"
+
+namespace msr {
+
+// ---- tcgen05 / TMA wrappers ------------------------------------------------------------------
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* tmap, int x, int y,
+                                            uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_slot, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_slot)),
+               "r"(ncols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&r)[16]) {
+  uint32_t u[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+        "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) r[i] = __uint_as_float(u[i]);
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64 elements) and
+// were written by TMA with the 128-byte swizzle: groups of 8 rows are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_k128(uint32_t saddr) {
+  return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+         (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t idesc_bf16_m128(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+constexpr int kGateBM = 128, kGateBK = 64, kGateStages = 3;
+constexpr int kGateATile = kGateBM * kGateBK * 2;   // 16 KiB
+constexpr int kGateStageBytes = kGateATile + 16384; // the W_g tile is padded to 16 KiB to stay 1024-aligned
+constexpr int kGateSmemBytes = kGateStages * kGateStageBytes + 1024;
+
+struct GateSmem {
+  uint64_t full[kGateStages], empty[kGateStages], accum;
+  uint32_t tmem_base;
+  int failed;
+};
+
+__global__ void __launch_bounds__(128)
+gate_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW,
+                    const float* __restrict__ bias, float* __restrict__ logits, int T, int E, int Npad,
+                    int num_kb, unsigned* error_flag) {
+  extern __shared__ unsigned char gsm_raw[];
+  unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(gsm_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ GateSmem sm;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * kGateBM;
+  const uint32_t b_bytes = (uint32_t)Npad * kGateBK * 2;
+  uint32_t tmem_cols = 32; while ((int)tmem_cols < Npad) tmem_cols <<= 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kGateStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
+    mbar_init(&sm.accum, 1);
+    sm.failed = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) tmem_alloc(&sm.tmem_base, tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_acc = sm.tmem_base;
+
+  if (warp == 0 && lane == 0) {
+    // ---- producer: TMA loads of the H tile and the matching W_g columns ---------------------------
+    for (int kb = 0; kb < num_kb; ++kb) {
+      const int s = kb % kGateStages;
+      const uint32_t ph = (uint32_t)((kb / kGateStages) & 1);
+      if (kb >= kGateStages && !mbar_wait_bounded(&sm.empty[s], ph ^ 1)) { sm.failed = 1; break; }
+      unsigned char* a = tiles + (size_t)s * kGateStageBytes;
+      mbar_expect_tx(&sm.full[s], kGateATile + b_bytes);
+      tma_load_2d(a, &tmH, kb * kGateBK, m0, &sm.full[s]);
+      tma_load_2d(a + kGateATile, &tmW, kb * kGateBK, 0, &sm.full[s]);
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---- MMA issuer: four K=16 instructions per 64-wide stage ------------------------------------
+    const uint32_t idesc = idesc_bf16_m128(Npad);
+    bool ok = true;
+    for (int kb = 0; kb < num_kb && ok; ++kb) {
+      const int s = kb % kGateStages;
+      const uint32_t ph = (uint32_t)((kb / kGateStages) & 1);
+      ok = mbar_wait_bounded(&sm.full[s], ph);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t a_addr = smem_u32(tiles + (size_t)s * kGateStageBytes);
+      const uint64_t adesc = smem_desc_k128(a_addr), bdesc = smem_desc_k128(a_addr + kGateATile);
+#pragma unroll
+      for (int kk = 0; kk < kGateBK / 16; ++kk)      // +32 bytes along K inside the swizzle atom
+        umma_bf16(tmem_acc, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+      umma_commit(&sm.empty[s]);                      // frees the stage when these MMAs retire
+    }
+    if (!ok) sm.failed = 1;
+    umma_commit(&sm.accum);                           // accumulator complete
+  }
+  __syncwarp();
+  // ---- epilogue: warp w reads TMEM lanes [32w, 32w+32), i.e. tokens m0 + 32w + lane ------------------
+  const bool got = mbar_wait_bounded(&sm.accum, 0);
+  tc_fence_after();
+  if (got && !sm.failed) {
+    const int row = m0 + warp * 32 + lane;
+    for (int c0 = 0; c0 < Npad; c0 += 16) {
+      float r[16];
+      tmem_ld16(tmem_acc + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, r);
+      if (row < T) {
+#pragma unroll
+        for (int j = 0; j < 16; j += 4) {
+          const int c = c0 + j;
+          if (c + 3 < E && (E & 3) == 0) {
+            float4 o = make_float4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+            if (bias) { o.x += __ldg(bias + c); o.y += __ldg(bias + c + 1); o.z += __ldg(bias + c + 2); o.w += __ldg(bias + c + 3); }
+            *reinterpret_cast<float4*>(logits + (size_t)row * E + c) = o;
+          } else {
+            for (int jj = 0; jj < 4; ++jj)
+              if (c + jj < E) logits[(size_t)row * E + c + jj] = r[j + jj] + (bias ? __ldg(bias + c + jj) : 0.f);
+          }
+        }
+      }
+    }
+  } else if (threadIdx.x == 0) {
+    atomicOr(error_flag, 4u);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_acc, tmem_cols);
+}
+
+// W_g -> bf16 [Npad, d] with the contraction index contiguous; rows >= E are zero.
+__global__ void wgate_prepare_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wt, int d,
+                                     int E, int Npad, int layout) {
+  const long long n = (long long)Npad * d;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const int row = (int)(i / d), col = (int)(i % d);
+    __nv_bfloat16 v = __float2bfloat16(0.f);
+    if (row < E) v = layout == 0 ? w[(size_t)col * E + row] : w[(size_t)row * d + col];
+    wt[i] = v;
+  }
+}
+
+// ---- fp32 path and the derivative GEMMs: plain FMA tiles ------------------------------------------
+template <typename T>
+__device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// logits[i][j] = sum_m H[i][m] * W(m, j) + bias[j]; one thread per output, 16 x 16 thread tiles.
+template <typename T>
+__global__ void __launch_bounds__(256)
+gate_gemm_simt_kernel(const T* __restrict__ H, const T* __restrict__ W, const float* __restrict__ bias,
+                      float* __restrict__ logits, int Tn, int d, int E, int layout) {
+  __shared__ float sh[16][17], sw[16][17];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int row = blockIdx.x * 16 + ty, col = blockIdx.y * 16 + tx;
+  float acc = 0.f;
+  for (int m0 = 0; m0 < d; m0 += 16) {
+    const int hr = blockIdx.x * 16 + ty, hm = m0 + tx;
+    sh[ty][tx] = (hr < Tn && hm < d) ? to_f(H[(size_t)hr * d + hm]) : 0.f;
+    const int wm = m0 + ty, wc = blockIdx.y * 16 + tx;
+    sw[ty][tx] = (wm < d && wc < E) ? to_f(layout == 0 ? W[(size_t)wm * E + wc] : W[(size_t)wc * d + wm]) : 0.f;
+    __syncthreads();
+#pragma unroll
+    for (int m = 0; m < 16; ++m) acc = fmaf(sh[ty][m], sw[m][tx], acc);
+    __syncthreads();
+  }
+  if (row < Tn && col < E) logits[(size_t)row * E + col] = acc + (bias ? bias[col] : 0.f);
+}
+
+// dH[i][m] = sum_j dL[i][j] * W(m, j); a CTA caches its 16 rows of dL in shared memory.
+template <typename T>
+__global__ void __launch_bounds__(256)
+gate_bwd_dh_kernel(const float* __restrict__ dL, const T* __restrict__ W, T* __restrict__ dH, int Tn, int d,
+                   int E, int layout) {
+  __shared__ float sdl[16][kMaxE];
+  const int r0 = blockIdx.x * 16;
+  for (int i = threadIdx.x; i < 16 * E; i += blockDim.x) {
+    const int r = i / E, j = i - r * E;
+    sdl[r][j] = (r0 + r < Tn) ? dL[(size_t)(r0 + r) * E + j] : 0.f;
+  }
+  __syncthreads();
+  for (int m = threadIdx.x; m < d; m += blockDim.x) {
+    float acc[16];
+#pragma unroll
+    for (int r = 0; r < 16; ++r) acc[r] = 0.f;
+    for (int j = 0; j < E; ++j) {
+      const float w = to_f(layout == 0 ? W[(size_t)m * E + j] : W[(size_t)j * d + m]);
+#pragma unroll
+      for (int r = 0; r < 16; ++r) acc[r] = fmaf(sdl[r][j], w, acc[r]);
+    }
+#pragma unroll
+    for (int r = 0; r < 16; ++r)
+      if (r0 + r < Tn) {
+        if constexpr (sizeof(T) == 4) dH[(size_t)(r0 + r) * d + m] = acc[r];
+        else dH[(size_t)(r0 + r) * d + m] = __float2bfloat16(acc[r]);
+      }
+  }
+}
+
+// dW[m][j] = sum_i H[i][m] * dL[i][j].  A CTA owns a 64-wide slice of m and a chunk of tokens and adds
+// its partial sums to dW (fp32 atomics; dW is zeroed first).
+constexpr int kDwTok = 256;
+template <typename T>
+__global__ void __launch_bounds__(256)
+gate_bwd_dw_kernel(const T* __restrict__ H, const float* __restrict__ dL, float* __restrict__ dW, int Tn, int d,
+                   int E) {
+  __shared__ float sh[32][65];
+  __shared__ float sdl[32][kMaxE];
+  const int m0 = blockIdx.x * 64, i0 = blockIdx.y * kDwTok;
+  const int tm = threadIdx.x & 63, tj = threadIdx.x >> 6;    // thread: column m0+tm, experts tj, tj+4, ...
+  float acc[kMaxE / 4];
+#pragma unroll
+  for (int q = 0; q < kMaxE / 4; ++q) acc[q] = 0.f;
+  for (int ib = 0; ib < kDwTok; ib += 32) {
+    for (int x = threadIdx.x; x < 32 * 64; x += blockDim.x) {
+      const int r = x >> 6, c = x & 63, i = i0 + ib + r;
+      sh[r][c] = (i < Tn && m0 + c < d) ? to_f(H[(size_t)i * d + m0 + c]) : 0.f;
+    }
+    for (int x = threadIdx.x; x < 32 * E; x += blockDim.x) {
+      const int r = x / E, j = x - r * E, i = i0 + ib + r;
+      sdl[r][j] = (i < Tn) ? dL[(size_t)i * E + j] : 0.f;
+    }
+    __syncthreads();
+    for (int r = 0; r < 32; ++r) {
+      const float h = sh[r][tm];
+#pragma unroll
+      for (int q = 0; q < kMaxE / 4; ++q) {
+        const int j = tj + 4 * q;
+        if (j < E) acc[q] = fmaf(h, sdl[r][j], acc[q]);
+      }
+    }
+    __syncthreads();
+  }
+  if (m0 + tm < d) {
+#pragma unroll
+    for (int q = 0; q < kMaxE / 4; ++q) {
+      const int j = tj + 4 * q;
+      if (j < E) atomicAdd(dW + (size_t)(m0 + tm) * E + j, acc[q]);
+    }
+  }
+}
+
+}  // namespace msr

@@ -1,0 +1,488 @@
+// C ABI of the MaxScore router (see include/maxscore.h): argument checks, workspace carving and
+// kernel launches on the caller's stream.  No device memory is allocated here.
+#include "../../include/maxscore.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "common.cuh"
+#include "flow.cuh"
+#include "gate.cuh"
+#include "move.cuh"
+#include "softtopk.cuh"
+
+using namespace msr;
+
+namespace {
+
+thread_local char g_last_error[256] = "";
+
+maxscore_status cuda_fail(cudaError_t e, const char* where) {
+  snprintf(g_last_error, sizeof(g_last_error), "%s: %s", where, cudaGetErrorString(e));
+  return MAXSCORE_ERR_CUDA;
+}
+#define MS_CUDA(call)                                              \
+  do {                                                             \
+    cudaError_t e_ = (call);                                       \
+    if (e_ != cudaSuccess) return cuda_fail(e_, #call);            \
+  } while (0)
+#define MS_LAUNCH_CHECK(name)                                      \
+  do {                                                             \
+    cudaError_t e_ = cudaGetLastError();                           \
+    if (e_ != cudaSuccess) return cuda_fail(e_, name);             \
+  } while (0)
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int32_t capacity_of(const maxscore_params& p) {
+  if (p.capacity > 0) return p.capacity;
+  // ceil(cf * T * k / E) with cf read as a multiple of 2^-20 (exact for 1.0, 1.25, 1.5, ...)
+  const long long cfq = llround((double)p.capacity_factor * 1048576.0);
+  const __int128 num = (__int128)cfq * p.T * p.k;
+  const __int128 den = (__int128)1048576 * p.E;
+  return (int32_t)((num + den - 1) / den);
+}
+
+struct Layout {          // byte offsets inside the workspace
+  size_t state, cand, block_counts, wt, error_flag, total;
+  int Npad, n_idx_blocks;
+};
+
+Layout layout_of(const maxscore_params& p) {
+  Layout l{};
+  l.Npad = (int)align_up((size_t)p.E, 16);
+  l.n_idx_blocks = (p.T + kIdxTok - 1) / kIdxTok;
+  size_t off = 0;
+  l.state = off; off = align_up(off + sizeof(FlowState), 256);
+  l.error_flag = off; off = align_up(off + 16, 256);
+  l.cand = off; off = align_up(off + sizeof(int32_t) * kMaxCand, 256);
+  l.block_counts = off; off = align_up(off + sizeof(int32_t) * (size_t)l.n_idx_blocks * p.E, 1024);
+  l.wt = off;
+  off = align_up(off + (p.io_dtype == MAXSCORE_BF16 ? sizeof(__nv_bfloat16) * (size_t)l.Npad * p.d_model : 0), 1024);
+  l.total = off;
+  return l;
+}
+
+maxscore_status check_params(const maxscore_params* p) {
+  if (!p) return MAXSCORE_ERR_INVALID_ARG;
+  if (p->T <= 0 || p->d_model <= 0 || p->E <= 0 || p->k <= 0) return MAXSCORE_ERR_INVALID_ARG;
+  if (!(p->t > 0.f) || !isfinite(p->t)) return MAXSCORE_ERR_INVALID_ARG;
+  if (p->io_dtype != MAXSCORE_F32 && p->io_dtype != MAXSCORE_BF16) return MAXSCORE_ERR_INVALID_ARG;
+  if (p->score_mode != 0 && p->score_mode != 1) return MAXSCORE_ERR_INVALID_ARG;
+  if (p->w_gate_layout != 0 && p->w_gate_layout != 1) return MAXSCORE_ERR_INVALID_ARG;
+  if (p->capacity <= 0 && !(p->capacity_factor > 0.f)) return MAXSCORE_ERR_INVALID_ARG;
+  if (p->score_mode == 1 && (p->quant_shift < 0 || p->quant_shift > 14)) return MAXSCORE_ERR_INVALID_ARG;
+  if (p->max_sweeps < 0) return MAXSCORE_ERR_INVALID_ARG;
+  if (p->k > p->E) return MAXSCORE_ERR_INFEASIBLE;
+  if (p->E > kMaxE || p->k > kMaxK) return MAXSCORE_ERR_UNSUPPORTED;
+  if ((long long)p->T * p->k >= (1LL << 31)) return MAXSCORE_ERR_UNSUPPORTED;
+  if (p->io_dtype == MAXSCORE_BF16 && p->d_model % 8) return MAXSCORE_ERR_UNSUPPORTED;
+  if (p->io_dtype == MAXSCORE_F32 && p->d_model % 4) return MAXSCORE_ERR_UNSUPPORTED;
+  const long long C = capacity_of(*p);
+  if (C <= 0 || C > (1LL << 30)) return MAXSCORE_ERR_INVALID_ARG;
+  const long long cap = C < p->T ? C : p->T;
+  if ((long long)p->E * cap < (long long)p->T * p->k) return MAXSCORE_ERR_INFEASIBLE;
+  return MAXSCORE_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr int kP2SmemMax = (int)(sizeof(long long) * kMaxE * kMaxE + sizeof(int) * kMaxCand + kMaxCand * kMaxK);
+constexpr int kDispatchSmem = 64 * 1024;
+
+}  // namespace
+
+struct maxscore_ctx {
+  maxscore_params p;
+  int32_t C;
+  Layout lay;
+  char* ws;
+  EncodeTiledFn encode;
+  int sm_count;
+};
+
+namespace {
+
+KeyGen keygen_of(const maxscore_ctx* c) {
+  KeyGen g{};
+  g.mode = c->p.score_mode;
+  g.quant_shift = c->p.quant_shift;
+  g.seed_mul = c->p.tiebreak_seed * 0x9E3779B9u;
+  int s = 0;
+  const long long n = (long long)c->p.T * c->p.k;
+  while ((1LL << s) < n) ++s;
+  g.S = 20 + s;
+  return g;
+}
+
+maxscore_status make_tmap_bf16(const maxscore_ctx* c, CUtensorMap* tm, const void* base, uint64_t inner,
+                               uint64_t outer, uint32_t box_inner, uint32_t box_outer) {
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {inner * 2};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = c->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(g_last_error, sizeof(g_last_error), "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+    return MAXSCORE_ERR_CUDA;
+  }
+  return MAXSCORE_OK;
+}
+
+unsigned* error_flag_of(const maxscore_ctx* c) { return reinterpret_cast<unsigned*>(c->ws + c->lay.error_flag); }
+size_t elem_bytes(const maxscore_ctx* c) { return c->p.io_dtype == MAXSCORE_BF16 ? 2 : 4; }
+
+maxscore_status launch_gate(maxscore_ctx* c, const void* hidden, const void* w_gate, const float* bias,
+                            float* logits, cudaStream_t st) {
+  const maxscore_params& p = c->p;
+  if (p.io_dtype == MAXSCORE_F32) {
+    dim3 grid((p.T + 15) / 16, (p.E + 15) / 16);
+    gate_gemm_simt_kernel<float><<<grid, 256, 0, st>>>((const float*)hidden, (const float*)w_gate, bias, logits,
+                                                        p.T, p.d_model, p.E, p.w_gate_layout);
+    MS_LAUNCH_CHECK("gate_gemm_simt_kernel");
+    return MAXSCORE_OK;
+  }
+  __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(c->ws + c->lay.wt);
+  const int Npad = c->lay.Npad;
+  {
+    const long long n = (long long)Npad * p.d_model;
+    int blocks = (int)((n + 255) / 256); if (blocks > 1184) blocks = 1184;
+    wgate_prepare_kernel<<<blocks, 256, 0, st>>>((const __nv_bfloat16*)w_gate, wt, p.d_model, p.E, Npad, p.w_gate_layout);
+    MS_LAUNCH_CHECK("wgate_prepare_kernel");
+  }
+  CUtensorMap tmH, tmW;
+  maxscore_status s = make_tmap_bf16(c, &tmH, hidden, (uint64_t)p.d_model, (uint64_t)p.T, kGateBK, kGateBM);
+  if (s) return s;
+  s = make_tmap_bf16(c, &tmW, wt, (uint64_t)p.d_model, (uint64_t)Npad, kGateBK, (uint32_t)Npad);
+  if (s) return s;
+  const int num_kb = (p.d_model + kGateBK - 1) / kGateBK;
+  gate_gemm_tc_kernel<<<(p.T + kGateBM - 1) / kGateBM, 128, kGateSmemBytes, st>>>(tmH, tmW, bias, logits, p.T, p.E,
+                                                                                   Npad, num_kb, error_flag_of(c));
+  MS_LAUNCH_CHECK("gate_gemm_tc_kernel");
+  return MAXSCORE_OK;
+}
+
+maxscore_status launch_softtopk_fwd(maxscore_ctx* c, const float* logits, float* scores, cudaStream_t st) {
+  const maxscore_params& p = c->p;
+  int blocks = (p.T + 7) / 8; if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
+  softtopk_fwd_kernel<<<blocks, 256, 0, st>>>(logits, scores, p.T, p.E, p.k, p.t);
+  MS_LAUNCH_CHECK("softtopk_fwd_kernel");
+  return MAXSCORE_OK;
+}
+
+constexpr int kSweeps = 40, kRounds = 4, kDefaultAug = 4096;
+
+maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_idx, int32_t* expert_load,
+                              maxscore_stats* stats, cudaStream_t st) {
+  const maxscore_params& p = c->p;
+  FlowState* fs = reinterpret_cast<FlowState*>(c->ws + c->lay.state);
+  int32_t* cand = reinterpret_cast<int32_t*>(c->ws + c->lay.cand);
+  const KeyGen g = keygen_of(c);
+  const int scale_bits = p.score_mode == 0 ? 40 : g.S + p.quant_shift;   // log2 of one unit of score
+  const long long eps0 = 1LL << (scale_bits - 10);
+  const long long eps_min = p.score_mode == 0 ? (1LL << 20) : (1LL << 12);
+  const int cap0 = scale_bits - 8;
+  const long long theta0 = 1LL << (scale_bits - 13);
+  const int balanced = ((long long)p.E * c->C == (long long)p.T * p.k) ? 1 : 0;
+  const int budget = p.max_sweeps > 0 ? p.max_sweeps : kSweeps + kDefaultAug;
+  const int n_sweeps = budget < kSweeps ? budget : kSweeps;
+  const int max_aug = budget - n_sweeps;
+
+  flow_init_kernel<<<1, 256, 0, st>>>(fs, eps0, eps_min, cap0, theta0, balanced, p.E);
+  MS_LAUNCH_CHECK("flow_init_kernel");
+  const int blocks = (p.T + kSweepThreads - 1) / kSweepThreads;
+  for (int s = 0; s < n_sweeps; ++s) {
+    flow_sweep_kernel<<<blocks, kSweepThreads, 0, st>>>(M, fs, p.T, p.E, p.k, c->C, g, n_sweeps, 2);
+    MS_LAUNCH_CHECK("flow_sweep_kernel");
+  }
+  const size_t p2smem = sizeof(long long) * (size_t)p.E * p.E + sizeof(int) * kMaxCand + (size_t)kMaxCand * kMaxK;
+  for (int r = 0; r < kRounds; ++r) {
+    flow_collect_kernel<<<blocks, kSweepThreads, 0, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, r == 0, 0,
+                                                         32LL, nullptr, nullptr, nullptr);
+    MS_LAUNCH_CHECK("flow_collect_kernel");
+    flow_exact_kernel<<<1, kP2Threads, p2smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, max_aug);
+    MS_LAUNCH_CHECK("flow_exact_kernel");
+  }
+  flow_collect_kernel<<<blocks, kSweepThreads, 0, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, 0, 1, 32LL,
+                                                       expert_load, stats, error_flag_of(c));
+  MS_LAUNCH_CHECK("flow_collect_kernel(verify)");
+  return MAXSCORE_OK;
+}
+
+maxscore_status launch_index_build(maxscore_ctx* c, const int32_t* expert_idx, int32_t* slot_idx, int32_t* slot_token,
+                                   int32_t* expert_load, cudaStream_t st) {
+  const maxscore_params& p = c->p;
+  int32_t* bc = reinterpret_cast<int32_t*>(c->ws + c->lay.block_counts);
+  MS_CUDA(cudaMemsetAsync(slot_token, 0xFF, sizeof(int32_t) * (size_t)p.E * c->C, st));
+  index_count_kernel<<<c->lay.n_idx_blocks, kIdxTok, 0, st>>>(expert_idx, bc, p.T, p.E, p.k);
+  MS_LAUNCH_CHECK("index_count_kernel");
+  index_fill_kernel<<<c->lay.n_idx_blocks, kIdxTok, 0, st>>>(expert_idx, bc, slot_idx, slot_token, expert_load, p.T,
+                                                            p.E, p.k, c->C);
+  MS_LAUNCH_CHECK("index_fill_kernel");
+  return MAXSCORE_OK;
+}
+
+__global__ void gather_gate_w_kernel(const float* __restrict__ scores, const int32_t* __restrict__ expert_idx,
+                                     float* __restrict__ gate_w, long long n, int E, int k) {
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const long long tok = i / k;
+    const int e = expert_idx[i];
+    gate_w[i] = (e >= 0 && e < E) ? scores[tok * E + e] : 0.f;
+  }
+}
+
+maxscore_status launch_zero_padding(maxscore_ctx* c, const int32_t* slot_token, void* dst, cudaStream_t st) {
+  const long long n_slots = (long long)c->p.E * c->C;
+  int blocks = (int)((n_slots + 7) / 8); if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
+  zero_padding_kernel<<<blocks, 256, 0, st>>>(slot_token, (char*)dst, n_slots, (uint32_t)(c->p.d_model * elem_bytes(c)));
+  MS_LAUNCH_CHECK("zero_padding_kernel");
+  return MAXSCORE_OK;
+}
+
+}  // namespace
+
+// ==================================================================================================
+extern "C" {
+
+int32_t maxscore_capacity(const maxscore_params* params) {
+  if (!params || params->E <= 0) return -1;
+  return capacity_of(*params);
+}
+
+const char* maxscore_last_cuda_error(void) { return g_last_error; }
+
+maxscore_status maxscore_workspace_bytes(const maxscore_params* params, size_t* bytes) {
+  if (!bytes) return MAXSCORE_ERR_INVALID_ARG;
+  maxscore_status s = check_params(params);
+  if (s) return s;
+  *bytes = layout_of(*params).total;
+  return MAXSCORE_OK;
+}
+
+maxscore_status maxscore_create(maxscore_ctx** out, const maxscore_params* params, void* workspace,
+                                size_t workspace_bytes) {
+  if (!out) return MAXSCORE_ERR_INVALID_ARG;
+  *out = nullptr;
+  maxscore_status s = check_params(params);
+  if (s) return s;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MAXSCORE_ERR_INVALID_ARG;
+  const Layout lay = layout_of(*params);
+  if (workspace_bytes < lay.total) return MAXSCORE_ERR_WORKSPACE;
+  int dev = 0, sms = 0;
+  MS_CUDA(cudaGetDevice(&dev));
+  MS_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  MS_CUDA(cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres));
+  if (!fn || qres != cudaDriverEntryPointSuccess) {
+    snprintf(g_last_error, sizeof(g_last_error), "cuTensorMapEncodeTiled not available from the driver");
+    return MAXSCORE_ERR_CUDA;
+  }
+  MS_CUDA(cudaFuncSetAttribute(gate_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGateSmemBytes));
+  MS_CUDA(cudaFuncSetAttribute(flow_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kP2SmemMax));
+  MS_CUDA(cudaFuncSetAttribute(dispatch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDispatchSmem));
+  MS_CUDA(cudaMemsetAsync(workspace, 0, lay.wt, 0));
+  MS_CUDA(cudaStreamSynchronize(0));
+  maxscore_ctx* c = new (std::nothrow) maxscore_ctx();
+  if (!c) return MAXSCORE_ERR_INVALID_ARG;
+  c->p = *params; c->C = capacity_of(*params); c->lay = lay; c->ws = static_cast<char*>(workspace);
+  c->encode = reinterpret_cast<EncodeTiledFn>(fn); c->sm_count = sms;
+  *out = c;
+  return MAXSCORE_OK;
+}
+
+void maxscore_destroy(maxscore_ctx* ctx) { delete ctx; }
+
+maxscore_status maxscore_gate(maxscore_ctx* c, const void* hidden, const void* w_gate, const float* bias,
+                              float* logits, void* stream) {
+  if (!c || !hidden || !w_gate || !logits) return MAXSCORE_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(w_gate) || !aligned16(logits)) return MAXSCORE_ERR_INVALID_ARG;
+  return launch_gate(c, hidden, w_gate, bias, logits, (cudaStream_t)stream);
+}
+
+maxscore_status maxscore_softtopk_fwd(maxscore_ctx* c, const float* logits, float* scores, void* stream) {
+  if (!c || !logits || !scores) return MAXSCORE_ERR_INVALID_ARG;
+  return launch_softtopk_fwd(c, logits, scores, (cudaStream_t)stream);
+}
+
+maxscore_status maxscore_softtopk_bwd(maxscore_ctx* c, const float* logits, const int32_t* expert_idx,
+                                      const float* dgate_w, float* dlogits, void* stream) {
+  if (!c || !logits || !expert_idx || !dgate_w || !dlogits) return MAXSCORE_ERR_INVALID_ARG;
+  const maxscore_params& p = c->p;
+  int blocks = (p.T + 7) / 8; if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
+  softtopk_bwd_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, dlogits, p.T, p.E, p.k, p.t);
+  MS_LAUNCH_CHECK("softtopk_bwd_kernel");
+  return MAXSCORE_OK;
+}
+
+maxscore_status maxscore_assign(maxscore_ctx* c, const float* matrix, int32_t* expert_idx, int32_t* expert_load,
+                                maxscore_stats* stats, void* stream) {
+  if (!c || !matrix || !expert_idx || !expert_load || !stats) return MAXSCORE_ERR_INVALID_ARG;
+  if (!aligned16(matrix)) return MAXSCORE_ERR_INVALID_ARG;
+  return launch_assign(c, matrix, expert_idx, expert_load, stats, (cudaStream_t)stream);
+}
+
+maxscore_status maxscore_index_build(maxscore_ctx* c, const int32_t* expert_idx, int32_t* slot_idx,
+                                     int32_t* slot_token, int32_t* expert_load, void* stream) {
+  if (!c || !expert_idx || !slot_idx || !slot_token || !expert_load) return MAXSCORE_ERR_INVALID_ARG;
+  return launch_index_build(c, expert_idx, slot_idx, slot_token, expert_load, (cudaStream_t)stream);
+}
+
+maxscore_status maxscore_route_fwd(maxscore_ctx* c, const void* hidden, const void* w_gate, const float* bias,
+                                   float* logits, float* scores, int32_t* expert_idx, int32_t* slot_idx,
+                                   float* gate_w, int32_t* slot_token, int32_t* expert_load, maxscore_stats* stats,
+                                   void* stream) {
+  if (!c || !hidden || !w_gate || !logits || !scores || !expert_idx || !slot_idx || !gate_w || !slot_token ||
+      !expert_load || !stats)
+    return MAXSCORE_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(w_gate) || !aligned16(logits) || !aligned16(scores))
+    return MAXSCORE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  maxscore_status s = launch_gate(c, hidden, w_gate, bias, logits, st);
+  if (s) return s;
+  s = launch_softtopk_fwd(c, logits, scores, st);
+  if (s) return s;
+  s = launch_assign(c, c->p.score_mode == 0 ? scores : logits, expert_idx, expert_load, stats, st);
+  if (s) return s;
+  s = launch_index_build(c, expert_idx, slot_idx, slot_token, expert_load, st);
+  if (s) return s;
+  const long long n = (long long)c->p.T * c->p.k;
+  int blocks = (int)((n + 255) / 256); if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
+  gather_gate_w_kernel<<<blocks, 256, 0, st>>>(scores, expert_idx, gate_w, n, c->p.E, c->p.k);
+  MS_LAUNCH_CHECK("gather_gate_w_kernel");
+  return MAXSCORE_OK;
+}
+
+maxscore_status maxscore_dispatch(maxscore_ctx* c, const void* src, const int32_t* expert_idx,
+                                  const int32_t* slot_idx, const int32_t* slot_token, void* dst, void* stream) {
+  if (!c || !src || !expert_idx || !slot_idx || !slot_token || !dst) return MAXSCORE_ERR_INVALID_ARG;
+  if (!aligned16(src) || !aligned16(dst)) return MAXSCORE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const maxscore_params& p = c->p;
+  DispatchArgs a{};
+  a.src = (const char*)src; a.dst = (char*)dst; a.expert_idx = expert_idx; a.slot_idx = slot_idx;
+  a.T = p.T; a.k = p.k; a.C = c->C;
+  a.row_bytes = (uint32_t)(p.d_model * elem_bytes(c));
+  a.chunk_bytes = a.row_bytes < 8192 ? (uint32_t)align_up(a.row_bytes, 128) : 8192;
+  a.chunks_per_row = (a.row_bytes + a.chunk_bytes - 1) / a.chunk_bytes;
+  a.stages = (int)(kDispatchSmem / a.chunk_bytes); if (a.stages > 16) a.stages = 16;
+  a.error_flag = error_flag_of(c);
+  const long long units = (long long)p.T * a.chunks_per_row;
+  long long grid = c->sm_count * 3; if (grid > units) grid = units;
+  dispatch_kernel<<<(int)grid, 32, (size_t)a.stages * a.chunk_bytes, st>>>(a);
+  MS_LAUNCH_CHECK("dispatch_kernel");
+  return launch_zero_padding(c, slot_token, dst, st);
+}
+
+maxscore_status maxscore_combine(maxscore_ctx* c, const void* src, const int32_t* expert_idx,
+                                 const int32_t* slot_idx, const float* gate_w, void* dst, int accumulate,
+                                 void* stream) {
+  if (!c || !src || !expert_idx || !slot_idx || !dst) return MAXSCORE_ERR_INVALID_ARG;
+  if (!aligned16(src) || !aligned16(dst)) return MAXSCORE_ERR_INVALID_ARG;
+  const maxscore_params& p = c->p;
+  int blocks = p.T < c->sm_count * 8 ? p.T : c->sm_count * 8;
+  if (p.io_dtype == MAXSCORE_BF16)
+    combine_kernel<__nv_bfloat16><<<blocks, 256, 0, (cudaStream_t)stream>>>(
+        (const __nv_bfloat16*)src, expert_idx, slot_idx, gate_w, (__nv_bfloat16*)dst, p.T, p.d_model, p.k, c->C, accumulate);
+  else
+    combine_kernel<float><<<blocks, 256, 0, (cudaStream_t)stream>>>((const float*)src, expert_idx, slot_idx, gate_w,
+                                                                     (float*)dst, p.T, p.d_model, p.k, c->C, accumulate);
+  MS_LAUNCH_CHECK("combine_kernel");
+  return MAXSCORE_OK;
+}
+
+maxscore_status maxscore_combine_bwd(maxscore_ctx* c, const void* dY, const void* yexp, const int32_t* expert_idx,
+                                     const int32_t* slot_idx, const float* gate_w, const int32_t* slot_token,
+                                     void* dyexp, float* dgate_w, void* stream) {
+  if (!c || !dY || !yexp || !expert_idx || !slot_idx || !gate_w || !slot_token || !dyexp || !dgate_w)
+    return MAXSCORE_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(yexp) || !aligned16(dyexp)) return MAXSCORE_ERR_INVALID_ARG;
+  const maxscore_params& p = c->p;
+  cudaStream_t st = (cudaStream_t)stream;
+  int blocks = p.T < c->sm_count * 8 ? p.T : c->sm_count * 8;
+  if (p.io_dtype == MAXSCORE_BF16)
+    combine_bwd_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dY, (const __nv_bfloat16*)yexp,
+                                                              expert_idx, slot_idx, gate_w, (__nv_bfloat16*)dyexp,
+                                                              dgate_w, p.T, p.d_model, p.k, c->C);
+  else
+    combine_bwd_kernel<float><<<blocks, 256, 0, st>>>((const float*)dY, (const float*)yexp, expert_idx, slot_idx, gate_w,
+                                                      (float*)dyexp, dgate_w, p.T, p.d_model, p.k, c->C);
+  MS_LAUNCH_CHECK("combine_bwd_kernel");
+  return launch_zero_padding(c, slot_token, dyexp, st);
+}
+
+maxscore_status maxscore_gate_bwd(maxscore_ctx* c, const void* hidden, const void* w_gate, const float* dlogits,
+                                  float* dw_gate, void* dH, void* stream) {
+  if (!c || !hidden || !w_gate || !dlogits || !dw_gate || !dH) return MAXSCORE_ERR_INVALID_ARG;
+  const maxscore_params& p = c->p;
+  cudaStream_t st = (cudaStream_t)stream;
+  MS_CUDA(cudaMemsetAsync(dw_gate, 0, sizeof(float) * (size_t)p.d_model * p.E, st));
+  dim3 gw((p.d_model + 63) / 64, (p.T + kDwTok - 1) / kDwTok);
+  const int gh = (p.T + 15) / 16;
+  if (p.io_dtype == MAXSCORE_BF16) {
+    gate_bwd_dw_kernel<__nv_bfloat16><<<gw, 256, 0, st>>>((const __nv_bfloat16*)hidden, dlogits, dw_gate, p.T, p.d_model, p.E);
+    MS_LAUNCH_CHECK("gate_bwd_dw_kernel");
+    gate_bwd_dh_kernel<__nv_bfloat16><<<gh, 256, 0, st>>>(dlogits, (const __nv_bfloat16*)w_gate, (__nv_bfloat16*)dH, p.T,
+                                                          p.d_model, p.E, p.w_gate_layout);
+  } else {
+    gate_bwd_dw_kernel<float><<<gw, 256, 0, st>>>((const float*)hidden, dlogits, dw_gate, p.T, p.d_model, p.E);
+    MS_LAUNCH_CHECK("gate_bwd_dw_kernel");
+    gate_bwd_dh_kernel<float><<<gh, 256, 0, st>>>(dlogits, (const float*)w_gate, (float*)dH, p.T, p.d_model, p.E,
+                                                  p.w_gate_layout);
+  }
+  MS_LAUNCH_CHECK("gate_bwd_dh_kernel");
+  return MAXSCORE_OK;
+}
+
+maxscore_status maxscore_route_bwd(maxscore_ctx* c, const void* dY, const void* yexp, const void* hidden,
+                                   const void* w_gate, const float* logits, const int32_t* expert_idx,
+                                   const int32_t* slot_idx, const float* gate_w, const int32_t* slot_token,
+                                   void* dyexp, float* dgate_w, float* dlogits, float* dw_gate, void* dH,
+                                   void* stream) {
+  if (!logits || !dlogits) return MAXSCORE_ERR_INVALID_ARG;
+  maxscore_status s = maxscore_combine_bwd(c, dY, yexp, expert_idx, slot_idx, gate_w, slot_token, dyexp, dgate_w, stream);
+  if (s) return s;
+  s = maxscore_softtopk_bwd(c, logits, expert_idx, dgate_w, dlogits, stream);
+  if (s) return s;
+  return maxscore_gate_bwd(c, hidden, w_gate, dlogits, dw_gate, dH, stream);
+}
+
+maxscore_status maxscore_route_dispatch_host(maxscore_ctx* c, const void* hidden_host, const void* w_gate_host,
+                                             const float* bias_host, const maxscore_device_buffers* dev,
+                                             int32_t* expert_idx_host, int32_t* slot_idx_host, float* gate_w_host,
+                                             maxscore_stats* stats_host, void* stream) {
+  if (!c || !hidden_host || !w_gate_host || !dev || !expert_idx_host || !slot_idx_host || !gate_w_host || !stats_host)
+    return MAXSCORE_ERR_INVALID_ARG;
+  if (!dev->hidden || !dev->w_gate || !dev->xdisp || (bias_host && !dev->expert_bias)) return MAXSCORE_ERR_INVALID_ARG;
+  const maxscore_params& p = c->p;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t eb = elem_bytes(c);
+  MS_CUDA(cudaMemcpyAsync(dev->hidden, hidden_host, eb * (size_t)p.T * p.d_model, cudaMemcpyHostToDevice, st));
+  MS_CUDA(cudaMemcpyAsync(dev->w_gate, w_gate_host, eb * (size_t)p.d_model * p.E, cudaMemcpyHostToDevice, st));
+  if (bias_host) MS_CUDA(cudaMemcpyAsync(dev->expert_bias, bias_host, sizeof(float) * p.E, cudaMemcpyHostToDevice, st));
+  maxscore_status s = maxscore_route_fwd(c, dev->hidden, dev->w_gate, bias_host ? dev->expert_bias : nullptr, dev->logits,
+                                         dev->scores, dev->expert_idx, dev->slot_idx, dev->gate_w, dev->slot_token,
+                                         dev->expert_load, dev->stats, stream);
+  if (s) return s;
+  s = maxscore_dispatch(c, dev->hidden, dev->expert_idx, dev->slot_idx, dev->slot_token, dev->xdisp, stream);
+  if (s) return s;
+  const size_t nk = (size_t)p.T * p.k;
+  MS_CUDA(cudaMemcpyAsync(expert_idx_host, dev->expert_idx, sizeof(int32_t) * nk, cudaMemcpyDeviceToHost, st));
+  MS_CUDA(cudaMemcpyAsync(slot_idx_host, dev->slot_idx, sizeof(int32_t) * nk, cudaMemcpyDeviceToHost, st));
+  MS_CUDA(cudaMemcpyAsync(gate_w_host, dev->gate_w, sizeof(float) * nk, cudaMemcpyDeviceToHost, st));
+  MS_CUDA(cudaMemcpyAsync(stats_host, dev->stats, sizeof(maxscore_stats), cudaMemcpyDeviceToHost, st));
+  MS_CUDA(cudaStreamSynchronize(st));
+  return MAXSCORE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,51 @@
+"""Helpers shared by the GPU parity tests (no routing arithmetic here)."""
+import numpy as np
+import torch
+
+
+def f64(t: torch.Tensor) -> np.ndarray:
+    """Exact float64 image of an fp32 / bf16 tensor."""
+    return t.detach().to("cpu").to(torch.float64).numpy()
+
+
+def np32(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to("cpu").to(torch.float32).numpy()
+
+
+def raw16(t: torch.Tensor) -> np.ndarray:
+    """Bit pattern of a bf16 tensor as uint16 (for bit-exact row comparisons)."""
+    return t.detach().to("cpu").view(torch.int16).numpy().view(np.uint16)
+
+
+def assert_rel(got, ref, tol, what=""):
+    """For outputs whose terms all have one sign (no cancellation): per row
+    max_i |d_i| <= tol * max_i |ref_i|, and elementwise |d| <= tol*|ref| wherever
+    |ref| >= 1e-4 * rowmax."""
+    got = np.asarray(got, dtype=np.float64).reshape(-1, got.shape[-1])
+    ref = np.asarray(ref, dtype=np.float64).reshape(-1, ref.shape[-1])
+    rowmax = np.abs(ref).max(axis=1, keepdims=True)
+    d = np.abs(got - ref)
+    assert (d <= tol * rowmax + 1e-300).all(), f"{what}: row-relative error {np.max(d / (rowmax + 1e-300)):.3e} > {tol}"
+    big = (np.abs(ref) >= 1e-4 * rowmax) & (rowmax > 0)
+    rel = d[big] / np.abs(ref[big])
+    assert rel.size == 0 or rel.max() <= tol, f"{what}: elementwise relative error {rel.max():.3e} > {tol}"
+
+
+def assert_sum_close(got, ref, mag, tol, what=""):
+    """For outputs that are sums of signed products: |got - ref| <= tol * mag elementwise, where mag is
+    the same sum taken over absolute values (the magnitude the rounding errors scale with).  Entries
+    whose magnitude is zero must be exactly zero."""
+    got = np.asarray(got, dtype=np.float64); ref = np.asarray(ref, dtype=np.float64)
+    mag = np.asarray(mag, dtype=np.float64)
+    d = np.abs(got - ref)
+    bad = d > tol * mag
+    assert not bad.any(), f"{what}: {bad.sum()} entries off, worst {np.max(d / (mag + 1e-300)):.3e} > {tol}"
+
+
+def float_keys(scores32: np.ndarray) -> np.ndarray:
+    """The keys the library documents for score_mode 0: rne(A * 2^40) plus the 12-bit position hash
+    ((i*E + j) * 2654435761 mod 2^32) >> 20, restated here from include/maxscore.h's description."""
+    T, E = scores32.shape
+    base = np.rint(scores32.astype(np.float64) * float(1 << 40)).astype(np.int64)
+    flat = (np.arange(T * E, dtype=np.uint64).reshape(T, E) * np.uint64(2654435761)) & np.uint64(0xFFFFFFFF)
+    return base + (flat >> np.uint64(20)).astype(np.int64)
