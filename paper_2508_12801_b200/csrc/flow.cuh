@@ -30,14 +30,12 @@
 
 namespace msr {
 
-constexpr int kNBLog = 6;
-constexpr int kNB = 1 << kNBLog;          // histogram bins per expert
+constexpr int kNB = 256;                  // histogram bins per expert: 4 per octave of the margin
 constexpr int kTopN = kMaxK + 2;          // sorted values kept per token in a sweep
 constexpr long long kInf = 1LL << 62;
 constexpr long long kArcLimit = 1LL << 55; // arcs with a larger reduced cost are ignored by the exact phase
 constexpr int kMaxCand = 4096;            // candidate tokens one exact-phase round can hold
 constexpr int kCapLogMax = 60;
-constexpr int kCapLogMin = kNBLog + 1;
 constexpr int kEPLf = kMaxE / 32;          // experts per lane when a warp spans one token row
 
 struct KeyGen {
@@ -65,6 +63,7 @@ __device__ __forceinline__ long long make_key(const KeyGen& g, float x, uint32_t
 }
 
 struct FlowState {
+  int trace[64];             // total imbalance seen by each sweep (diagnostics)
   long long p[kMaxE];        // expert prices
   long long eps, eps_min;
   long long theta;           // candidate threshold of the current round
@@ -73,7 +72,7 @@ struct FlowState {
   int load_cur[kMaxE];       // loads of the assignment currently written in expert_idx
   unsigned hist_up[kMaxE * kNB];
   unsigned hist_dn[kMaxE * kNB];
-  int cap_up[kMaxE], cap_dn[kMaxE];   // log2 of the histogram ranges
+  int cap_up[kMaxE], cap_dn[kMaxE];   // log2 of the largest margin worth recording
   int flag_dn[kMaxE];                 // expert whose join-histogram came out short: scan it in full next sweep
   unsigned ticket;
   int sweep, p1_done, balanced;
@@ -126,37 +125,62 @@ __device__ __forceinline__ bool last_block_arrives(unsigned* ticket) {
   return is_last;
 }
 
-// Price step that moves `need` tokens across the threshold of one expert, from its margin histogram
-// (bins of width 2^(cl - kNBLog) over [0, 2^cl)).  If the bin that holds the need-th smallest margin
-// also holds many more tokens (a group of near-ties), the step stops at the bin's lower edge and the
-// window is narrowed to that bin, so that the next sweep resolves the group; otherwise the step goes
-// to the bin's upper edge plus eps.
-__device__ __forceinline__ long long price_step(const unsigned* hist, int need, long long eps, int& cl,
-                                                bool& window_short, int grow) {
+// Margin histograms are logarithmic with four bins per octave (a 2-bit mantissa): margins 0..3 have
+// their own bins, a margin m >= 4 with top bit o falls in bin 4*(o-1) + (next two bits).  Every scale
+// is resolved to 25 % at once, which matters when the scores are quantised (margins then cluster at
+// multiples of the quantum, separated by gaps that a linear window would have to zoom across).
+__device__ __forceinline__ int log_bin(long long m) {
+  if (m < 4) return (int)m;
+  const int o = 63 - __clzll(m);
+  return 4 * (o - 1) + (int)((m >> (o - 2)) & 3);
+}
+__device__ __forceinline__ long long bin_lower_edge(int b) {
+  if (b < 4) return b;
+  const int o = b / 4 + 1, sub = b & 3;
+  return (long long)(4 + sub) << (o - 2);
+}
+
+// Price step that moves `need` tokens across the threshold of one expert.  If the bin holding the
+// need-th smallest margin also holds many more tokens, the step stops at that bin's lower edge:
+// fewer tokens move, and the rest of the group then sits near zero margin, where the bins are fine.
+// Otherwise the step goes to the bin's upper edge plus eps (capped by the bin width).  `cut` is the
+// log2 of the largest margin the tokens were asked to record; if fewer than `need` lie below it the
+// step goes to 2^cut and the cut-off is lifted for the next sweep.
+__device__ __forceinline__ long long price_step(const unsigned* hist, int need, long long eps, int& cut,
+                                                bool& window_short) {
   window_short = false;
-  unsigned cum = 0, before = 0; int pos = kNB;
-  for (int b = 0; b < kNB; ++b) {
-    const unsigned h = __ldcg(hist + b);
-    if (cum + h >= (unsigned)need) { pos = b; before = cum; cum += h; break; }
-    cum += h;
+  const int nb = min(kNB, 4 * cut);                   // bins at or above 2^cut are empty
+  unsigned cum = 0, before = 0; int pos = -1, last = -1;
+  for (int b0 = 0; b0 < nb && pos < 0; b0 += 16) {
+    uint4 h[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) h[q] = __ldcg(reinterpret_cast<const uint4*>(hist + b0) + q);
+    const unsigned* hv = reinterpret_cast<const unsigned*>(h);
+#pragma unroll
+    for (int q = 0; q < 16; ++q) {
+      if (pos < 0) {
+        if (cum + hv[q] >= (unsigned)need) { pos = b0 + q; before = cum; }
+        if (hv[q]) last = b0 + q;
+        cum += hv[q];
+      }
+    }
   }
-  const int wl = cl - kNBLog;                         // log2 of the bin width
-  if (pos >= kNB) {                                   // the window is too narrow
-    const long long step = (1LL << cl);
-    cl = min(cl + grow, kCapLogMax);
+  if (pos < 0) {
+    // fewer than `need` margins were recorded.  Under a cut-off, everything below it may move; with
+    // no cut-off, move what was recorded (an outsider list can be incomplete) and ask for a full scan.
+    const long long step = cut < kCapLogMax ? (1LL << cut) : (last >= 0 ? bin_lower_edge(last + 1) : 0);
+    cut = kCapLogMax;
     window_short = true;
     return step;
   }
-  const long long e_eff = eps < (8LL << wl) ? eps : (8LL << wl);
-  if (cum <= 2u * (unsigned)need || cl <= kCapLogMin) {
-    const long long step = ((long long)(pos + 1) << wl) + e_eff;
-    if (pos < 4 && cl > kCapLogMin + 1) cl -= 2;
-    return step;
-  }
+  const long long lo = bin_lower_edge(pos), hi = bin_lower_edge(pos + 1);
+  cut = min(kCapLogMax, max(12, (pos >> 2) + 8));      // next sweep: record up to ~64x this margin
   (void)before;
-  const long long step = (long long)pos << wl;        // conservative: moves fewer than `need`
-  cl = max(wl + 1, kCapLogMin);
-  return step;
+  if (cum <= 2u * (unsigned)need || lo == 0) {
+    const long long w = hi - lo;
+    return hi + (eps < w ? eps : w);
+  }
+  return lo;                                          // conservative: moves `before` < need tokens
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -209,7 +233,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
         if (has_alt) {
           const long long m = v[j] - vk1;             // price rise at which this token leaves e
           const int cl = scu[e];
-          if (m < (1LL << cl)) atomicAdd(&st->hist_up[e * kNB + (int)(m >> (cl - kNBLog))], 1u);
+          if (m < (1LL << cl)) atomicAdd(&st->hist_up[e * kNB + log_bin(m)], 1u);
         }
       }
     }
@@ -220,7 +244,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
         if (e >= 0) {
           const long long m = vk - v[j];              // price cut at which this token joins e
           const int cl = scd[e];
-          if (m < (1LL << cl)) atomicAdd(&st->hist_dn[e * kNB + (int)(m >> (cl - kNBLog))], 1u);
+          if (m < (1LL << cl)) atomicAdd(&st->hist_dn[e * kNB + log_bin(m)], 1u);
         }
       }
     }
@@ -234,7 +258,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
       if (seen) continue;
       const long long m = vk - (make_key(g, __ldg(row + e), flat + e) - sp[e]);
       const int cl = scd[e];
-      if (m >= 0 && m < (1LL << cl)) atomicAdd(&st->hist_dn[e * kNB + (int)(m >> (cl - kNBLog))], 1u);
+      if (m >= 0 && m < (1LL << cl)) atomicAdd(&st->hist_dn[e * kNB + log_bin(m)], 1u);
     }
   }
   __syncthreads();
@@ -255,13 +279,13 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
     const int x = load - C;
     if (x > 0) {
       int cl = scu[e]; bool shortw;
-      p += price_step(st->hist_up + e * kNB, x, eps, cl, shortw, 3);
+      p += price_step(st->hist_up + e * kNB, x, eps, cl, shortw);
       st->cap_up[e] = cl;
       st->flag_dn[e] = 0;
       atomicAdd(&s_imb, x);
     } else if (x < 0 && (balanced || p > 0)) {
       int cl = scd[e]; bool shortw;
-      p -= price_step(st->hist_dn + e * kNB, -x, eps, cl, shortw, 2);
+      p -= price_step(st->hist_dn + e * kNB, -x, eps, cl, shortw);
       if (!balanced && p < 0) p = 0;
       st->cap_dn[e] = cl;
       st->flag_dn[e] = shortw ? 1 : 0;
@@ -274,7 +298,10 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
     if (x != 0) sp[e] = p;
   }
   __syncthreads();   // every expert's histogram has been read before any is cleared
-  for (int i = threadIdx.x; i < E * kNB; i += blockDim.x) { st->hist_up[i] = 0; st->hist_dn[i] = 0; }
+  {
+    uint4* hu = reinterpret_cast<uint4*>(st->hist_up); uint4* hd = reinterpret_cast<uint4*>(st->hist_dn);
+    for (int i = threadIdx.x; i < E * kNB / 4; i += blockDim.x) { hu[i] = make_uint4(0, 0, 0, 0); hd[i] = make_uint4(0, 0, 0, 0); }
+  }
   const int sweep = st->sweep + 1;
   const bool done = (s_imb == 0) || sweep >= n_sweeps;
   if (threadIdx.x == 0) {
@@ -287,6 +314,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
   for (int e = threadIdx.x; e < E; e += blockDim.x) st->p[e] = sp[e] - pmin;
   __syncthreads();
   if (threadIdx.x == 0) {
+    if (sweep <= 64) st->trace[sweep - 1] = s_imb;
     st->sweep = sweep;
     if (sweep % decay_every == 0) { long long ne = eps >> 1; st->eps = ne < st->eps_min ? st->eps_min : ne; }
     st->ticket = 0;

@@ -191,7 +191,7 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   const int scale_bits = p.score_mode == 0 ? 40 : g.S + p.quant_shift;   // log2 of one unit of score
   const long long eps0 = 1LL << (scale_bits - 10);
   const long long eps_min = p.score_mode == 0 ? (1LL << 20) : (1LL << 12);
-  const int cap0 = scale_bits - 8;
+  const int cap0 = kCapLogMax;   // the first sweep records every margin
   const long long theta0 = 1LL << (scale_bits - 13);
   const int balanced = ((long long)p.E * c->C == (long long)p.T * p.k) ? 1 : 0;
   const int budget = p.max_sweeps > 0 ? p.max_sweeps : kSweeps + kDefaultAug;

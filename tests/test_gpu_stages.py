@@ -1,0 +1,292 @@
+"""GPU parity, stage by stage: every CUDA stage is called through the C ABI and compared with the
+CPU oracle on the same seeded inputs.  Downstream stages are fed the GPU's own upstream output, so
+that a flipped near-tie upstream cannot pass for a downstream bug.
+
+Tolerances.  SoftTopk sums positive terms, so it is held to 1e-5 relative elementwise.  Outputs that
+are sums of signed products (gate, combine, the backward GEMMs) are held to tol * (the same sum over
+absolute values): 1e-5 for fp32 I/O, 2e-2 for bf16 I/O (one rounding to bf16 is 2^-9)."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import assert_rel, assert_sum_close, f64, float_keys, np32, raw16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ms():
+    from paper_2508_12801_b200 import binding
+    assert torch.cuda.is_available()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def synth():
+    from paper_2508_12801_b200 import synth
+    return synth
+
+
+DEV = "cuda:0"
+
+
+def _ctx(ms, T, d, E, k, cf=1.0, dtype="bf16", **kw):
+    p = ms.make_params(T, d, E, k, cf, io_dtype=ms.BF16 if dtype == "bf16" else ms.F32, **kw)
+    return ms.create(p, DEV)
+
+
+def _tol(dtype):
+    return 2e-2 if dtype == "bf16" else 1e-5
+
+
+# ------------------------------------------------------------------------------------------- gate
+@pytest.mark.parametrize("T,d,E,dtype,layout,bias", [
+    (512, 256, 8, "f32", 0, False), (300, 100, 12, "f32", 1, True),
+    (512, 256, 8, "bf16", 0, False), (4096, 1024, 16, "bf16", 0, True),
+    (1000, 2048, 64, "bf16", 1, False), (257, 4096, 128, "bf16", 0, True),
+    (129, 72, 20, "bf16", 0, False),
+])
+def test_gate(ms, orc, synth, T, d, E, dtype, layout, bias):
+    w = synth.Workload("g", T, d, E, 2, 1.0, dtype)
+    H, W = synth.hidden(w, 1), synth.w_gate(w, 1)
+    b = torch.linspace(-1, 1, E) if bias else None
+    ctx = _ctx(ms, T, d, E, min(2, E), dtype=dtype, w_gate_layout=layout)
+    Wd = (W if layout == 0 else W.t().contiguous()).to(DEV)
+    L = torch.empty(T, E, dtype=torch.float32, device=DEV)
+    ms.gate(ctx, H.to(DEV), Wd, b.to(DEV) if bias else None, L)
+    torch.cuda.synchronize()
+    ref = orc.gate(f64(H), f64(W), f64(b) if bias else None)
+    mag = orc.gate(np.abs(f64(H)), np.abs(f64(W)), np.abs(f64(b)) if bias else None)
+    assert_sum_close(np32(L), ref, mag, 1e-5, "gate")      # logits are fp32 in both I/O modes
+
+
+# ------------------------------------------------------------------------------------------- SoftTopk
+@pytest.mark.parametrize("T,E,k,t", [(512, 8, 2, 1.0), (512, 8, 2, 4.0), (1000, 16, 2, 1.0), (777, 64, 8, 1.0),
+                                      (515, 128, 8, 0.25), (64, 20, 3, 2.0), (33, 5, 5, 1.0), (40, 128, 1, 1.0)])
+def test_softtopk_fwd_bwd(ms, orc, synth, T, E, k, t):
+    L = synth.logits_like(T, E, seed=3)
+    ctx = _ctx(ms, T, 64, E, k, cf=float(E), t=t)       # capacity irrelevant here
+    Ld = L.to(DEV)
+    A = torch.empty_like(Ld)
+    ms.softtopk_fwd(ctx, Ld, A)
+    ref = orc.softtopk_fwd(f64(L), k, t)
+    assert_rel(np32(A), ref, 1e-5, "SoftTopk fwd")
+    # backward with a sparse upstream gradient at k "assigned" experts per token
+    g = torch.Generator().manual_seed(5)
+    idx = torch.stack([torch.randperm(E, generator=g)[:k].sort().values for _ in range(T)]).to(torch.int32)
+    dg = torch.randn(T, k, generator=g)
+    dL = torch.empty_like(Ld)
+    ms.softtopk_bwd(ctx, Ld, idx.to(DEV), dg.to(DEV), dL)
+    G = np.zeros((T, E)); np.put_along_axis(G, idx.numpy().astype(np.int64), f64(dg), axis=1)
+    refb = orc.softtopk_bwd(f64(L), G, k, t)
+    got = np32(dL)
+    rowmax = np.abs(refb).max(axis=1, keepdims=True)
+    assert (np.abs(got - refb) <= 1e-5 * rowmax + 1e-9).all()
+
+
+# ------------------------------------------------------------------------------------------- assignment
+def _run_assign(ms, M, T, E, k, cf, **kw):
+    ctx = _ctx(ms, T, 64, E, k, cf=cf, **kw)
+    idx = torch.empty(T, k, dtype=torch.int32, device=DEV)
+    load = torch.empty(E, dtype=torch.int32, device=DEV)
+    stats = ms.new_stats(DEV)
+    Md = M.to(DEV)
+    ms.assign(ctx, Md, idx, load, stats)
+    torch.cuda.synchronize()
+    return ctx, idx.cpu().numpy(), load.cpu().numpy(), ms.read_stats(stats)
+
+
+def _describe(st):
+    return (f"status={st.status} sweeps={st.sweeps} aug={st.augmentations} rounds={st.rounds} "
+            f"cand={st.candidates} rerouted={st.rerouted}")
+
+
+def _check_feasible(idx, load, T, E, k, C, st=None):
+    msg = _describe(st) if st is not None else ""
+    assert (idx >= 0).all() and (idx < E).all(), msg
+    assert k == 1 or (np.diff(idx, axis=1) > 0).all(), msg
+    np.testing.assert_array_equal(np.bincount(idx.ravel(), minlength=E), load, err_msg=msg)
+    assert (load <= C).all() and load.sum() == T * k, f"{msg} load max {load.max()} C {C}"
+
+
+@pytest.mark.parametrize("T,E,k,cf,skew", [(512, 8, 2, 1.0, False), (4096, 16, 2, 1.0, False),
+                                            (1000, 16, 4, 1.0, False), (2048, 64, 8, 1.0, False),
+                                            (2048, 64, 8, 1.25, True), (300, 8, 2, 1.5, True),
+                                            (8192, 64, 8, 1.0, False), (129, 5, 5, 1.0, False),
+                                            (257, 12, 1, 1.0, True)])
+def test_assign_float_scores(ms, orc, synth, T, E, k, cf, skew):
+    wl = synth.Workload("a", T, 64, E, k, cf, "bf16", skew=skew)
+    L = synth.logits_like(T, E, seed=7, bias=synth.expert_bias(wl, 7))
+    A = torch.from_numpy(orc.softtopk_fwd(f64(L), k, 1.0).astype(np.float32))
+    ctx, idx, load, st = _run_assign(ms, A, T, E, k, cf)
+    C = ctx.capacity
+    assert C == orc.capacity(T, k, E, cf)
+    _check_feasible(idx, load, T, E, k, C, st)
+    assert st.status == 0, _describe(st)
+    # optimal for the keys the library documents ...
+    keys = float_keys(A.numpy())
+    res, prices = orc.flow_certificate(keys, idx, C)
+    assert res >= 1, _describe(st)
+    assert orc.dual_value(keys, prices, k, C) == orc.primal_value(keys, idx)
+    # ... and within 1e-5 relative of the oracle's optimum of the float problem
+    oidx, oload, _ = orc.flow_condensed(orc.keys_from_scores(f64(A)), k, C)
+    best = orc.total_score(f64(A), oidx)
+    got = orc.total_score(f64(A), idx)
+    assert abs(got - best) <= 1e-5 * abs(best)
+    assert abs(st.total_score - got) <= 1e-6 * abs(got)
+    if cf == 1.0 and (T * k) % E == 0:
+        assert (load == C).all()
+    # rerouted = token-slots outside the token's own top-k
+    topk = np.argsort(-keys, axis=1, kind="stable")[:, :k]
+    inside = (idx[:, :, None] == topk[:, None, :]).any(2)
+    assert st.rerouted == int((~inside).sum())
+
+
+@pytest.mark.parametrize("T,E,k,cf,skew,seed", [(512, 8, 2, 1.0, False, 0), (2048, 64, 8, 1.0, False, 0),
+                                                 (2048, 64, 8, 1.25, True, 1), (8192, 64, 8, 1.0, False, 0),
+                                                 (1000, 16, 3, 1.0, False, 2)])
+def test_assign_integer_keys_bit_exact(ms, orc, synth, T, E, k, cf, skew, seed):
+    wl = synth.Workload("a", T, 64, E, k, cf, "bf16", skew=skew)
+    L = synth.logits_like(T, E, seed=11, bias=synth.expert_bias(wl, 11))
+    ctx, idx, load, st = _run_assign(ms, L, T, E, k, cf, score_mode=1, quant_shift=11, tiebreak_seed=seed)
+    C = ctx.capacity
+    _check_feasible(idx, load, T, E, k, C, st)
+    keys, _ = orc.keys_from_logits(np32(L), k, 11, seed)
+    oidx, oload, _ = orc.flow_condensed(keys, k, C)
+    res, _ = orc.flow_certificate(keys, oidx, C)
+    assert res == 2, "oracle optimum not unique for this seed"
+    np.testing.assert_array_equal(idx, oidx, err_msg=_describe(st))
+    np.testing.assert_array_equal(load, oload)
+    assert st.status == 0
+
+
+def test_assign_degenerate_inputs(ms, orc):
+    # all scores equal: every assignment within capacity is optimal; must stay feasible and certified
+    T, E, k = 256, 8, 2
+    A = torch.full((T, E), 0.25)
+    ctx, idx, load, st = _run_assign(ms, A, T, E, k, 1.0)
+    _check_feasible(idx, load, T, E, k, ctx.capacity, st)
+    assert orc.flow_certificate(float_keys(A.numpy()), idx, ctx.capacity)[0] >= 1
+    # one hot expert for everybody
+    A = torch.zeros(T, E); A[:, 3] = 1.0; A += torch.arange(E) * 1e-3
+    ctx, idx, load, st = _run_assign(ms, A, T, E, k, 1.0)
+    _check_feasible(idx, load, T, E, k, ctx.capacity, st)
+    assert orc.flow_certificate(float_keys(A.numpy()), idx, ctx.capacity)[0] >= 1
+    # loose capacity: plain per-token top-k
+    g = torch.Generator().manual_seed(1)
+    A = torch.rand(T, E, generator=g)
+    ctx, idx, load, st = _run_assign(ms, A, T, E, k, float(E))
+    want = np.sort(np.argsort(-float_keys(A.numpy()), axis=1, kind="stable")[:, :k], axis=1)
+    np.testing.assert_array_equal(idx, want)
+    assert st.augmentations == 0 and st.rerouted == 0
+
+
+# ------------------------------------------------------------------------------------------- index / dispatch / combine
+@pytest.mark.parametrize("T,d,E,k,cf,dtype", [(512, 256, 8, 2, 1.0, "f32"), (1000, 512, 16, 2, 1.25, "bf16"),
+                                               (2048, 2048, 64, 8, 1.0, "bf16"), (333, 4096, 128, 8, 1.5, "bf16"),
+                                               (100, 8200, 8, 2, 1.0, "bf16"), (65, 40, 4, 1, 2.0, "f32")])
+def test_index_dispatch_combine_and_backward(ms, orc, synth, T, d, E, k, cf, dtype):
+    wl = synth.Workload("m", T, d, E, k, cf, dtype)
+    H = synth.hidden(wl, 2)
+    L = synth.logits_like(T, E, seed=2)
+    A = orc.softtopk_fwd(f64(L), k, 1.0)
+    C = orc.capacity(T, k, E, cf)
+    oidx, _, _ = orc.flow_condensed(orc.keys_from_scores(A), k, C)
+    ctx = _ctx(ms, T, d, E, k, cf=cf, dtype=dtype)
+    assert ctx.capacity == C
+    idx = torch.from_numpy(oidx).to(DEV)
+    slot_idx = torch.empty(T, k, dtype=torch.int32, device=DEV)
+    slot_token = torch.empty(E, C, dtype=torch.int32, device=DEV)
+    load = torch.empty(E, dtype=torch.int32, device=DEV)
+    ms.index_build(ctx, idx, slot_idx, slot_token, load)
+    o_slot, o_tok, o_load = orc.index_build(oidx, E, C)
+    np.testing.assert_array_equal(slot_idx.cpu().numpy(), o_slot)
+    np.testing.assert_array_equal(slot_token.cpu().numpy(), o_tok)
+    np.testing.assert_array_equal(load.cpu().numpy(), o_load)
+    # dispatch: bit-exact rows, zero padding
+    Hd = H.to(DEV)
+    xd = torch.full((E, C, d), 7.0, dtype=H.dtype, device=DEV)      # poison: padding must be overwritten
+    ms.dispatch(ctx, Hd, idx, slot_idx, slot_token, xd)
+    torch.cuda.synchronize()
+    if dtype == "bf16":
+        np.testing.assert_array_equal(raw16(xd), orc.dispatch(raw16(H), o_tok))
+    else:
+        np.testing.assert_array_equal(xd.cpu().numpy(), orc.dispatch(H.numpy(), o_tok))
+    # combine on independent expert outputs
+    g = torch.Generator().manual_seed(9)
+    yexp = torch.randn(E, C, d, generator=g).to(H.dtype)
+    gw = torch.from_numpy(orc.gate_weights(A, oidx).astype(np.float32))
+    Y = torch.empty(T, d, dtype=H.dtype, device=DEV)
+    yd, gwd = yexp.to(DEV), gw.to(DEV)
+    ms.combine(ctx, yd, idx, slot_idx, gwd, Y)
+    refY = orc.combine(f64(yexp), oidx, o_slot, f64(gw))
+    magY = orc.combine(np.abs(f64(yexp)), oidx, o_slot, np.abs(f64(gw)))
+    assert_sum_close(f64(Y), refY, magY, _tol(dtype), "combine")
+    # unit weights + accumulate (dispatch backward into an existing gradient)
+    base = torch.randn(T, d, generator=g).to(H.dtype)
+    Y2 = base.clone().to(DEV)
+    ms.combine(ctx, yd, idx, slot_idx, None, Y2, accumulate=1)
+    ref2 = f64(base) + orc.combine(f64(yexp), oidx, o_slot, None)
+    mag2 = np.abs(f64(base)) + orc.combine(np.abs(f64(yexp)), oidx, o_slot, None)
+    assert_sum_close(f64(Y2), ref2, mag2, _tol(dtype), "combine accumulate")
+    # combine backward
+    dY = synth.upstream_grad(wl, 2)
+    dyexp = torch.full((E, C, d), 3.0, dtype=H.dtype, device=DEV)
+    dgw = torch.empty(T, k, dtype=torch.float32, device=DEV)
+    ms.combine_bwd(ctx, dY.to(DEV), yd, idx, slot_idx, gwd, slot_token, dyexp, dgw)
+    r_dyexp, r_dgw = orc.combine_bwd(f64(dY), f64(yexp), oidx, o_slot, f64(gw))
+    assert_sum_close(f64(dyexp), r_dyexp, np.abs(r_dyexp), _tol(dtype), "dyexp")      # padding rows exactly zero
+    _, m_dgw = orc.combine_bwd(np.abs(f64(dY)), np.abs(f64(yexp)), oidx, o_slot, np.abs(f64(gw)))
+    assert_sum_close(np32(dgw), r_dgw, m_dgw, 1e-5, "dgate_w")                         # fp32 dot of exact products
+
+
+@pytest.mark.parametrize("T,d,E,dtype,layout", [(512, 256, 8, "f32", 0), (1000, 1024, 16, "bf16", 0),
+                                                 (700, 2048, 64, "bf16", 1), (130, 72, 20, "f32", 1)])
+def test_gate_bwd(ms, orc, synth, T, d, E, dtype, layout):
+    wl = synth.Workload("b", T, d, E, 2, 1.0, dtype)
+    H, W = synth.hidden(wl, 4), synth.w_gate(wl, 4)
+    dL = synth.logits_like(T, E, seed=4) * 0.1
+    ctx = _ctx(ms, T, d, E, 2, dtype=dtype, w_gate_layout=layout)
+    Wd = (W if layout == 0 else W.t().contiguous()).to(DEV)
+    dW = torch.empty(d, E, dtype=torch.float32, device=DEV)
+    dH = torch.empty(T, d, dtype=H.dtype, device=DEV)
+    ms.gate_bwd(ctx, H.to(DEV), Wd, dL.to(DEV), dW, dH)
+    r_dW, r_dH = orc.gate_bwd(f64(H), f64(W), f64(dL))
+    m_dW, m_dH = orc.gate_bwd(np.abs(f64(H)), np.abs(f64(W)), np.abs(f64(dL)))
+    assert_sum_close(np32(dW), r_dW, m_dW, 1e-5, "dW")
+    assert_sum_close(f64(dH), r_dH, m_dH, _tol(dtype), "dH")
+
+
+# ------------------------------------------------------------------------------------------- whole path
+@pytest.mark.parametrize("name,T", [("tiny", None), ("k2e16", None), ("k8e64", 2048), ("skew", 2048)])
+def test_route_fwd_end_to_end(ms, orc, synth, name, T):
+    wl = synth.WORKLOADS[name]
+    if T:
+        wl = synth.scaled(wl, T=T)
+    T, d, E, k = wl.T, wl.d_model, wl.E, wl.k
+    H, W, b = synth.hidden(wl), synth.w_gate(wl), synth.expert_bias(wl)
+    ctx = _ctx(ms, T, d, E, k, cf=wl.capacity_factor, dtype=wl.dtype)
+    C = ctx.capacity
+    buf = ms.RouterBuffers(ctx)
+    Hd, Wd, bd = H.to(DEV), W.to(DEV), (b.to(DEV) if b is not None else None)
+    ms.route_fwd(ctx, Hd, Wd, bd, *buf.args())
+    torch.cuda.synchronize()
+    st = ms.read_stats(buf.stats)
+    assert st.status == 0 and st.capacity == C, _describe(st)
+    L = np32(buf.logits); A = np32(buf.scores)
+    refL = orc.gate(f64(H), f64(W), f64(b) if b is not None else None)
+    magL = orc.gate(np.abs(f64(H)), np.abs(f64(W)), np.abs(f64(b)) if b is not None else None)
+    assert_sum_close(L, refL, magL, 1e-5, "logits")
+    assert_rel(A, orc.softtopk_fwd(L.astype(np.float64), k, 1.0), 1e-5, "scores from GPU logits")
+    idx = buf.expert_idx.cpu().numpy(); load = buf.expert_load.cpu().numpy()
+    _check_feasible(idx, load, T, E, k, C, st)
+    keys = float_keys(A)
+    assert orc.flow_certificate(keys, idx, C)[0] >= 1
+    oidx, _, _ = orc.flow_condensed(orc.keys_from_scores(A.astype(np.float64)), k, C)
+    best = orc.total_score(A.astype(np.float64), oidx)
+    assert abs(orc.total_score(A.astype(np.float64), idx) - best) <= 1e-5 * abs(best)
+    o_slot, o_tok, o_load = orc.index_build(idx, E, C)
+    np.testing.assert_array_equal(buf.slot_idx.cpu().numpy(), o_slot)
+    np.testing.assert_array_equal(buf.slot_token.cpu().numpy(), o_tok)
+    np.testing.assert_array_equal(load, o_load)
+    np.testing.assert_array_equal(np32(buf.gate_w), np.take_along_axis(A, idx.astype(np.int64), axis=1))
