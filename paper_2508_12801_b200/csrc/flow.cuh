@@ -26,6 +26,7 @@
 // All arithmetic is on int64 keys: key = rne(A * 2^40) (+ a 12-bit position hash) for float
 // affinities, or the quantised logit with a hashed tie-break.
 #pragma once
+#include <cstddef>
 #include "common.cuh"
 
 namespace msr {
@@ -34,7 +35,6 @@ constexpr int kNB = 256;                  // histogram bins per expert: 4 per oc
 constexpr int kTopN = kMaxK + 2;          // sorted values kept per token in a sweep
 constexpr long long kInf = 1LL << 62;
 constexpr long long kArcLimit = 1LL << 55; // arcs with a larger reduced cost are ignored by the exact phase
-constexpr int kMaxCand = 4096;            // candidate tokens one exact-phase round can hold
 constexpr int kCapLogMax = 60;
 constexpr int kEPLf = kMaxE / 32;          // experts per lane when a warp spans one token row
 
@@ -66,12 +66,13 @@ struct FlowState {
   int trace[64];             // total imbalance seen by each sweep (diagnostics)
   long long p[kMaxE];        // expert prices
   long long eps, eps_min;
-  long long theta;           // candidate threshold of the current round
+  long long theta;           // candidate threshold of the next collect pass
+  long long theta_used;      // threshold the current candidate list was collected with
   double total_score;
   int load[kMaxE];           // accumulated by the running pass, consumed by its last CTA
   int load_cur[kMaxE];       // loads of the assignment currently written in expert_idx
-  unsigned hist_up[kMaxE * kNB];
-  unsigned hist_dn[kMaxE * kNB];
+  alignas(16) unsigned hist_up[kMaxE * kNB];   // read and cleared with 16-byte accesses
+  alignas(16) unsigned hist_dn[kMaxE * kNB];
   int cap_up[kMaxE], cap_dn[kMaxE];   // log2 of the largest margin worth recording
   int flag_dn[kMaxE];                 // expert whose join-histogram came out short: scan it in full next sweep
   unsigned ticket;
@@ -80,6 +81,9 @@ struct FlowState {
   unsigned status;
   int ncand_last;
 };
+
+static_assert(offsetof(FlowState, hist_up) % 16 == 0 && offsetof(FlowState, hist_dn) % 16 == 0,
+              "histograms are accessed as uint4");
 
 // ---------------------------------------------------------------------------------------------
 __global__ void flow_init_kernel(FlowState* st, long long eps0, long long eps_min, int cap0,
@@ -314,7 +318,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
   for (int e = threadIdx.x; e < E; e += blockDim.x) st->p[e] = sp[e] - pmin;
   __syncthreads();
   if (threadIdx.x == 0) {
-    if (sweep <= 64) st->trace[sweep - 1] = s_imb;
+    if (sweep <= 48) st->trace[sweep - 1] = s_imb;
     st->sweep = sweep;
     if (sweep % decay_every == 0) { long long ne = eps >> 1; st->eps = ne < st->eps_min ? st->eps_min : ne; }
     st->ticket = 0;
@@ -331,7 +335,7 @@ __global__ void __launch_bounds__(kSweepThreads)
 flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restrict__ expert_idx,
                     int32_t* __restrict__ cand, int T, int E, int k, int C, KeyGen g, int first,
                     int verify_only, long long theta_scale, int32_t* __restrict__ expert_load_out,
-                    void* stats_out, const unsigned* __restrict__ error_flag) {
+                    void* stats_out, const unsigned* __restrict__ error_flag, int unbounded) {
   if (!verify_only && *(volatile int*)&st->converged) return;
   __shared__ long long sp[kMaxE];
   __shared__ int sload[kMaxE];
@@ -341,7 +345,7 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
   for (int e = threadIdx.x; e < E; e += blockDim.x) { sp[e] = st->p[e]; sload[e] = 0; }
   if (threadIdx.x == 0) { s_viol = 0; s_rer = 0; s_score = 0.0; s_flags = 0; }
   __syncthreads();
-  const long long theta = st->theta;
+  const long long theta = unbounded ? kInf : st->theta;   // the last round lists every token
   const int tok = blockIdx.x * blockDim.x + threadIdx.x;
   if (tok < T) {
     unsigned held[4] = {0, 0, 0, 0};
@@ -417,8 +421,7 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
     }
     if (verify_only) { atomicAdd(&s_score, sc); if (rer) atomicAdd(&s_rer, rer); }
     if (!verify_only && gap < kInf && gap <= theta) {
-      int pos = atomicAdd(&st->ncand, 1);
-      if (pos < kMaxCand) cand[pos] = tok;
+      cand[atomicAdd(&st->ncand, 1)] = tok;   // the list has room for every token
     }
   }
   __syncthreads();
@@ -446,11 +449,16 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
   if (threadIdx.x == 0) {
     const int viol = *(volatile int*)&st->violations;
     const bool ok = (first || viol == 0) && s_badload == 0;
+    {   // diagnostics: per round, violations / experts out of balance / augmentations so far / candidates
+      const int r = st->round < 4 ? st->round : 3;
+      st->trace[48 + 4 * r] = viol; st->trace[49 + 4 * r] = s_badload; st->trace[50 + 4 * r] = st->naug;
+      st->trace[51 + 4 * r] = st->ncand;
+    }
     st->violations = 0;
     st->ticket = 0;
     if (!verify_only) {
       st->round = st->round + 1;
-      if (st->ncand > kMaxCand) st->ncand = kMaxCand;
+      st->theta_used = theta;
       st->theta = (theta > (kInf >> 8)) ? kInf : theta * theta_scale;   // next round looks further
     }
     if (verify_only && !ok) atomicOr(&st->status, 1u);
@@ -471,10 +479,18 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
 
 // ---------------------------------------------------------------------------------------------
 // Exact phase: successive shortest augmenting paths on the expert-level residual graph, one CTA.
+//
+// Only candidate tokens (gap <= theta) are in the graph.  A round stops BEFORE an augmentation whose
+// price update would spread the experts' price changes of this round by more than theta: up to that
+// point no token outside the list can have lost its top-k, so the state handed to the next collect
+// pass is consistent, and that pass only has to list more tokens.  The experts held by a candidate
+// live in expert_idx itself and are edited in place; ties are broken by the smallest token index, so
+// the result does not depend on the order of the candidate list.
 constexpr int kP2Threads = 1024;
 
 struct P2Shared {
   long long p[kMaxE + 1];        // potentials: prices of the experts, then Z
+  long long p0[kMaxE + 1];       // potentials at the start of the round
   long long dist[2][kMaxE + 1];
   int pred[kMaxE + 1];
   int imb[kMaxE + 1];            // + excess, - deficit
@@ -482,50 +498,23 @@ struct P2Shared {
   int dirty[kMaxE];
   int path[kMaxE + 2];
   int npath, changed, who, target, stop, any_pos;
-  long long dt;
+  long long dt, spread_lo, spread_hi;
 };
 
-__device__ __forceinline__ bool holds(const unsigned char* h, int k, int e) {
-  bool r = false;
-  for (int c = 0; c < k; ++c) r |= (h[c] == e);
-  return r;
-}
-
 __global__ void __launch_bounds__(kP2Threads)
-flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restrict__ expert_idx,
-                  const int32_t* __restrict__ cand_g, int T, int E, int k, int C, KeyGen g, int max_aug) {
+flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_idx,
+                  const int32_t* __restrict__ cand, int T, int E, int k, int C, KeyGen g, int max_aug) {
   if (*(volatile int*)&st->converged) return;
   extern __shared__ __align__(16) unsigned char p2smem[];
   long long* D = reinterpret_cast<long long*>(p2smem);                       // [E][E] raw arc costs
-  int* cand = reinterpret_cast<int*>(D + (size_t)E * E);                       // [kMaxCand]
-  unsigned char* held = reinterpret_cast<unsigned char*>(cand + kMaxCand);     // [kMaxCand][kMaxK]
   __shared__ P2Shared s;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int n = min(st->ncand, kMaxCand);
+  const int n = min(st->ncand, T);
   const int nZ = E;   // index of Z
+  const long long theta = st->theta_used;
 
-  // ---- candidates, sorted so that every tie below is broken the same way on every run -------------
-  int npow = 1; while (npow < n) npow <<= 1;
-  for (int i = tid; i < npow; i += blockDim.x) cand[i] = i < n ? cand_g[i] : 0x7fffffff;
-  __syncthreads();
-  for (int size = 2; size <= npow; size <<= 1)
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      for (int i = tid; i < npow; i += blockDim.x) {
-        int j = i ^ stride;
-        if (j > i) {
-          bool up = (i & size) == 0;
-          int a = cand[i], b = cand[j];
-          if ((a > b) == up) { cand[i] = b; cand[j] = a; }
-        }
-      }
-      __syncthreads();
-    }
-  for (int i = tid; i < n * k; i += blockDim.x) {
-    int c = i / k, j = i - c * k;
-    held[c * kMaxK + j] = (unsigned char)expert_idx[(size_t)cand[c] * k + j];
-  }
   for (int e = tid; e < E; e += blockDim.x) {
-    s.p[e] = st->p[e];
+    s.p[e] = st->p[e]; s.p0[e] = s.p[e];
     const int load = st->load_cur[e];
     const int fl = s.p[e] > 0 ? C : min(load, C);
     s.flow[e] = fl; s.imb[e] = load - fl; s.dirty[e] = 1;
@@ -534,7 +523,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restric
   if (tid == 0) {
     int tot = 0;
     for (int e = 0; e < E; ++e) tot += s.imb[e];
-    s.imb[nZ] = -tot; s.p[nZ] = 0; s.stop = 0;
+    s.imb[nZ] = -tot; s.p[nZ] = 0; s.p0[nZ] = 0; s.stop = 0;
   }
   __syncthreads();
 
@@ -545,11 +534,15 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restric
       if (s.dirty[i / E]) D[i] = kInf;
     __syncthreads();
     for (int c = warp; c < n; c += kP2Threads / 32) {
-      const unsigned char* h = held + c * kMaxK;
-      bool any = false;
-      for (int j = 0; j < k; ++j) any |= (s.dirty[h[j]] != 0);
-      if (!any) continue;
       const int tok = cand[c];
+      int h[kMaxK];
+      bool any = false;
+#pragma unroll
+      for (int j = 0; j < kMaxK; ++j) {
+        h[j] = j < k ? expert_idx[(size_t)tok * k + j] : -1;
+        if (j < k) any |= (s.dirty[h[j]] != 0);
+      }
+      if (!any) continue;
       const float* row = M + (size_t)tok * E;
       const uint32_t flat = (uint32_t)tok * (uint32_t)E;
       long long key[kEPLf];
@@ -558,9 +551,14 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restric
       for (int q = 0; q < kEPLf; ++q) {
         const int f = lane + 32 * q;
         key[q] = f < E ? make_key(g, __ldg(row + f), flat + f) : 0;
-        in[q] = f < E ? holds(h, k, f) : true;
+        bool held = f >= E;
+#pragma unroll
+        for (int j = 0; j < kMaxK; ++j) held |= (h[j] == f);
+        in[q] = held;
       }
-      for (int j = 0; j < k; ++j) {
+#pragma unroll
+      for (int j = 0; j < kMaxK; ++j) {
+        if (j >= k) continue;
         const int e = h[j];
         if (!s.dirty[e]) continue;
         long long mine = 0;
@@ -632,7 +630,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restric
       if (!s.changed) break;
       __syncthreads();
     }
-    // ---- nearest node with a deficit --------------------------------------------------------------
+    // ---- nearest node with a deficit; would the price update stay within theta? -----------------------
     if (tid == 0) {
       int t = -1; long long dt = kInf;
       for (int v = 0; v <= E; ++v)
@@ -642,10 +640,17 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restric
         int len = 0, v = t;
         while (v >= 0 && len <= E + 1) { s.path[len++] = v; v = s.pred[v]; }
         s.npath = len;
+        long long lo = kInf, hi = -kInf;
+        for (int e = 0; e < E; ++e) {
+          const long long d = s.dist[cur][e];
+          const long long chg = s.p[e] - (d < dt ? d : dt) - s.p0[e];
+          lo = chg < lo ? chg : lo; hi = chg > hi ? chg : hi;
+        }
+        if (theta < kInf && hi - lo > theta) s.target = -2;   // stop here; the next round lists more tokens
       }
     }
     __syncthreads();
-    if (s.target < 0) break;        // no augmenting path inside the candidate graph: a wider theta is needed
+    if (s.target < 0) break;        // -1: no augmenting path inside the candidate graph
     for (int v = tid; v <= E; v += blockDim.x) {
       const long long d = s.dist[cur][v];
       s.p[v] -= (d < s.dt ? d : s.dt);
@@ -659,22 +664,26 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restric
         __syncthreads();
         const long long want = D[u * E + v];
         for (int c = tid; c < n; c += blockDim.x) {
-          const unsigned char* h = held + c * kMaxK;
-          if (!holds(h, k, u) || holds(h, k, v)) continue;
           const int tok = cand[c];
+          bool hu = false, hv = false;
+          for (int j = 0; j < k; ++j) {
+            const int e = expert_idx[(size_t)tok * k + j];
+            hu |= (e == u); hv |= (e == v);
+          }
+          if (!hu || hv) continue;
           const uint32_t flat = (uint32_t)tok * (uint32_t)E;
           const long long cost = make_key(g, __ldg(M + (size_t)tok * E + u), flat + u) -
                                  make_key(g, __ldg(M + (size_t)tok * E + v), flat + v);
-          if (cost == want) atomicMin(&s.who, c);
+          if (cost == want) atomicMin(&s.who, tok);
         }
         __syncthreads();
         if (s.who == 0x7fffffff) {   // internal inconsistency: stop, the verify pass will report it
           if (tid == 0) { atomicOr(&st->status, 4u); s.stop = 1; }
         } else if (tid == 0) {
-          unsigned char* h = held + s.who * kMaxK;
+          int32_t* h = expert_idx + (size_t)s.who * k;
           for (int j = 0; j < k; ++j) {
             s.dirty[h[j]] = 1;
-            if (h[j] == u) h[j] = (unsigned char)v;
+            if (h[j] == u) h[j] = v;
           }
           s.dirty[v] = 1;
         }
@@ -691,10 +700,6 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restric
   }
   // ---- write back ---------------------------------------------------------------------------------
   __syncthreads();
-  for (int i = tid; i < n * k; i += blockDim.x) {
-    int c = i / k, j = i - c * k;
-    expert_idx[(size_t)cand[c] * k + j] = held[c * kMaxK + j];
-  }
   for (int e = tid; e < E; e += blockDim.x) {
     long long pe = s.p[e] - s.p[nZ];
     st->p[e] = pe < 0 ? 0 : pe;     // only an expert that holds nothing can come out negative

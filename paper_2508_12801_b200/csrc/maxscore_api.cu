@@ -61,7 +61,7 @@ Layout layout_of(const maxscore_params& p) {
   size_t off = 0;
   l.state = off; off = align_up(off + sizeof(FlowState), 256);
   l.error_flag = off; off = align_up(off + 16, 256);
-  l.cand = off; off = align_up(off + sizeof(int32_t) * kMaxCand, 256);
+  l.cand = off; off = align_up(off + sizeof(int32_t) * (size_t)p.T, 256);
   l.block_counts = off; off = align_up(off + sizeof(int32_t) * (size_t)l.n_idx_blocks * p.E, 1024);
   l.wt = off;
   off = align_up(off + (p.io_dtype == MAXSCORE_BF16 ? sizeof(__nv_bfloat16) * (size_t)l.Npad * p.d_model : 0), 1024);
@@ -95,7 +95,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-constexpr int kP2SmemMax = (int)(sizeof(long long) * kMaxE * kMaxE + sizeof(int) * kMaxCand + kMaxCand * kMaxK);
+constexpr int kP2SmemMax = (int)(sizeof(long long) * kMaxE * kMaxE);
 constexpr int kDispatchSmem = 64 * 1024;
 
 }  // namespace
@@ -205,16 +205,16 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
     flow_sweep_kernel<<<blocks, kSweepThreads, 0, st>>>(M, fs, p.T, p.E, p.k, c->C, g, n_sweeps, 2);
     MS_LAUNCH_CHECK("flow_sweep_kernel");
   }
-  const size_t p2smem = sizeof(long long) * (size_t)p.E * p.E + sizeof(int) * kMaxCand + (size_t)kMaxCand * kMaxK;
+  const size_t p2smem = sizeof(long long) * (size_t)p.E * p.E;
   for (int r = 0; r < kRounds; ++r) {
     flow_collect_kernel<<<blocks, kSweepThreads, 0, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, r == 0, 0,
-                                                         32LL, nullptr, nullptr, nullptr);
+                                                         32LL, nullptr, nullptr, nullptr, r == kRounds - 1);
     MS_LAUNCH_CHECK("flow_collect_kernel");
     flow_exact_kernel<<<1, kP2Threads, p2smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, max_aug);
     MS_LAUNCH_CHECK("flow_exact_kernel");
   }
   flow_collect_kernel<<<blocks, kSweepThreads, 0, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, 0, 1, 32LL,
-                                                       expert_load, stats, error_flag_of(c));
+                                                       expert_load, stats, error_flag_of(c), 0);
   MS_LAUNCH_CHECK("flow_collect_kernel(verify)");
   return MAXSCORE_OK;
 }
@@ -291,7 +291,7 @@ maxscore_status maxscore_create(maxscore_ctx** out, const maxscore_params* param
   MS_CUDA(cudaFuncSetAttribute(gate_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGateSmemBytes));
   MS_CUDA(cudaFuncSetAttribute(flow_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kP2SmemMax));
   MS_CUDA(cudaFuncSetAttribute(dispatch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDispatchSmem));
-  MS_CUDA(cudaMemsetAsync(workspace, 0, lay.wt, 0));
+  MS_CUDA(cudaMemsetAsync(workspace, 0, lay.cand, 0));
   MS_CUDA(cudaStreamSynchronize(0));
   maxscore_ctx* c = new (std::nothrow) maxscore_ctx();
   if (!c) return MAXSCORE_ERR_INVALID_ARG;
