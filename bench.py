@@ -1,0 +1,355 @@
+#!/usr/bin/env python
+"""Benchmark of the MaxScore router hot path on B200.
+
+A step is one pass of the whole path over one synthetic batch: gate -> SoftTopk -> flow assignment ->
+index build -> dispatch -> combine, then the backward (combine-bwd, SoftTopk-bwd, gate-bwd, dispatch-bwd).
+Workload "stress": T=65536 tokens, d_model=4096, E=128, k=8, capacity factor 1.0 (C=4096), bf16 rows.
+Inputs (0.5 GiB of tokens, 4 GiB expert buffers) exceed the 126 MB L2, so no flush is needed between steps.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload stress] [--impl ours|reference]
+
+N > 1 (under torchrun): independent replicas, one per GPU, no collective on the data path.
+--impl reference times the CPU checker (oracle/) on the host cores on a bounded sample of the workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "routed tokens/s per MoE layer (gate->flow->dispatch) on 1 B200; % of roofline"
+UNIT = "tokens/s"
+SWEEPS, ROUNDS = 40, 4
+
+
+def launches_per_step():
+    """Kernels of this library launched by one step (memsets not counted)."""
+    gate = 2                       # W_g transpose/pad + tcgen05 GEMM
+    assign = 1 + SWEEPS + 2 * ROUNDS + 1
+    route_fwd = gate + 1 + assign + 2 + 1          # + SoftTopk + index (count, fill) + gate_w gather
+    dispatch, combine = 2, 1
+    route_bwd = 2 + 1 + 2                          # combine-bwd (+padding), SoftTopk-bwd, gate-bwd (dW, dH)
+    return route_fwd + dispatch + combine + route_bwd + combine   # last combine = dispatch backward
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append(parts)
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm = sorted(int(r[0]) for r in self.rows if r[0].isdigit())
+        mx = [int(r[1]) for r in self.rows if r[1].isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i].lower().startswith("active") for r in self.rows)]
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(self.rows)}
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return 6650.0, "fallback (6.65 TB/s)"
+
+
+# ------------------------------------------------------------------------------------------------ reference arm
+def oracle_step(wl, Ts, seed=0):
+    """One pass of the whole path by the CPU checker on the first Ts tokens of the workload."""
+    import numpy as np
+    import torch
+
+    import oracle
+    from paper_2508_12801_b200 import synth
+
+    sub = synth.scaled(wl, T=Ts)
+    f64 = lambda t: t.to(torch.float64).numpy()
+    H, W, b, dY = synth.hidden(sub, seed), synth.w_gate(sub, seed), synth.expert_bias(sub, seed), synth.upstream_grad(sub, seed)
+    H64, W64, dY64 = f64(H), f64(W), f64(dY)
+    t0 = time.perf_counter()
+    k, E = sub.k, sub.E
+    C = oracle.capacity(Ts, k, E, sub.capacity_factor)
+    L = oracle.gate(H64, W64, f64(b) if b is not None else None).astype(np.float32)
+    A = oracle.softtopk_fwd(L, k, sub.temperature).astype(np.float32)
+    idx, load, _ = oracle.flow_condensed(oracle.keys_from_scores(A), k, C)
+    slot_idx, slot_token, _ = oracle.index_build(idx, E, C)
+    xd = oracle.dispatch(H64, slot_token)
+    gw = oracle.gate_weights(A, idx)
+    Y = oracle.combine(xd, idx, slot_idx, gw)
+    dyexp, dgw = oracle.combine_bwd(dY64, xd, idx, slot_idx, gw)
+    G = np.zeros((Ts, E)); np.put_along_axis(G, idx.astype(np.int64), dgw, axis=1)
+    dL = oracle.softtopk_bwd(L, G, k, sub.temperature)
+    dW, dH = oracle.gate_bwd(H64, W64, dL)
+    dH += oracle.combine(dyexp, idx, slot_idx, None)
+    return time.perf_counter() - t0, float(Y[0, 0] + dH[0, 0] + dW[0, 0])
+
+
+def run_reference(args, wl):
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    oracle.build()
+    Ts = args.ref_tokens
+    for _ in range(args.warmup):
+        oracle_step(wl, min(Ts, 256))
+    times = [oracle_step(wl, Ts)[0] for _ in range(args.steps)]
+    dt = sum(times) / len(times)
+    val = Ts / dt
+    sample = f"first {Ts} tokens of the workload per step (same d_model, E, k, capacity factor), whole path fwd+bwd"
+    out = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": wl.name, "T": wl.T, "d_model": wl.d_model, "E": wl.E, "k": wl.k,
+                      "capacity_factor": wl.capacity_factor, "sample_tokens": Ts},
+           "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+           "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+# ------------------------------------------------------------------------------------------------ our arm
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2508_12801_b200 import binding as ms
+    from paper_2508_12801_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the router has no CPU path")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    T, d, E, k = wl.T, wl.d_model, wl.E, wl.k
+    seed = rank                                           # replicas route different batches
+    H_host = synth.hidden(wl, seed).pin_memory()
+    W_host = synth.w_gate(wl, seed).pin_memory()
+    b = synth.expert_bias(wl, seed)
+    dY = synth.upstream_grad(wl, seed).to(dev)
+    ctx = ms.create(ms.make_params(T, d, E, k, wl.capacity_factor, t=wl.temperature,
+                                   io_dtype=ms.BF16 if wl.dtype == "bf16" else ms.F32), dev)
+    C = ctx.capacity
+    buf = ms.RouterBuffers(ctx)
+    Hd, Wd = H_host.to(dev), W_host.to(dev)
+    bd = b.to(dev) if b is not None else None
+    dt_t = H_host.dtype
+    xd = torch.empty(E, C, d, dtype=dt_t, device=dev)       # dispatch output; identity experts: yexp = xdisp
+    Y = torch.empty(T, d, dtype=dt_t, device=dev)
+    dyexp = torch.empty(E, C, d, dtype=dt_t, device=dev)
+    dgw = torch.empty(T, k, dtype=torch.float32, device=dev)
+    dL = torch.empty(T, E, dtype=torch.float32, device=dev)
+    dW = torch.empty(d, E, dtype=torch.float32, device=dev)
+    dH = torch.empty(T, d, dtype=dt_t, device=dev)
+    idx_host = torch.empty(T, k, dtype=torch.int32).pin_memory()
+    slot_host = torch.empty(T, k, dtype=torch.int32).pin_memory()
+    gw_host = torch.empty(T, k, dtype=torch.float32).pin_memory()
+    stats_host = torch.zeros(40, dtype=torch.uint8).pin_memory()
+    devbuf = buf.device_buffers(Hd, Wd, bd, xd)
+    stage_names = ["route_fwd", "dispatch", "combine", "combine_bwd", "softtopk_bwd", "gate_bwd", "dispatch_bwd"]
+
+    def rest_of_step(ev=None):
+        mark = (lambda i: ev[i].record()) if ev else (lambda i: None)
+        ms.combine(ctx, xd, buf.expert_idx, buf.slot_idx, buf.gate_w, Y); mark(3)
+        ms.combine_bwd(ctx, dY, xd, buf.expert_idx, buf.slot_idx, buf.gate_w, buf.slot_token, dyexp, dgw); mark(4)
+        ms.softtopk_bwd(ctx, buf.logits, buf.expert_idx, dgw, dL); mark(5)
+        ms.gate_bwd(ctx, Hd, Wd, dL, dW, dH); mark(6)
+        ms.combine(ctx, dyexp, buf.expert_idx, buf.slot_idx, None, dH, accumulate=1); mark(7)
+
+    def step(ev=None):
+        if ev:
+            ev[0].record()
+        ms.route_fwd(ctx, Hd, Wd, bd, *buf.args())
+        if ev:
+            ev[1].record()
+        ms.dispatch(ctx, Hd, buf.expert_idx, buf.slot_idx, buf.slot_token, xd)
+        if ev:
+            ev[2].record()
+        rest_of_step(ev)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sync_all()
+    st = ms.read_stats(buf.stats)
+
+    # ---- timed region: K steps, device-timed, per-stage events inside --------------------------------
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.2)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(8)] for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    e0.record()
+    for i in range(args.steps):
+        step(evs[i])
+    e1.record()
+    sync_all()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = e0.elapsed_time(e1)
+    stage_ms = [sum(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(args.steps)) / args.steps for j in range(7)]
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    st2 = ms.read_stats(buf.stats)
+
+    # ---- end to end: the same step, batch coming from pinned host memory through the C ABI ---------------
+    for _ in range(2):
+        ms.route_dispatch_host(ctx, H_host, W_host, None, devbuf, idx_host, slot_host, gw_host, stats_host)
+        rest_of_step()
+    sync_all()
+    t0 = time.perf_counter()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record()
+    for _ in range(args.steps):
+        ms.route_dispatch_host(ctx, H_host, W_host, None, devbuf, idx_host, slot_host, gw_host, stats_host)
+        rest_of_step()
+    g1.record()
+    sync_all()
+    e2e_ms = g0.elapsed_time(g1) / args.steps
+    wall_ms = (time.perf_counter() - t0) * 1e3 / args.steps
+    te = torch.tensor([max(e2e_ms, wall_ms)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_ms = float(te.item())
+    eb = H_host.element_size()
+    h2d = eb * (T * d + d * E)
+    d2h = 3 * 4 * T * k + 40
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel -------------------------------------------------------------
+    peak, peak_src = measured_peak_gbs()
+    row = d * eb
+    alg_bytes = {   # algorithmic bytes per launch
+        "route_fwd": T * row + T * E * 4 * 4,                      # read H once; logits and scores written and read
+        "dispatch": T * row + T * k * row,                         # read each row once, write it k times
+        "combine": T * k * row + T * row,
+        "combine_bwd": T * row + 2 * T * k * row,                  # read dY and k yexp rows, write k dyexp rows
+        "softtopk_bwd": 2 * T * E * 4,
+        "gate_bwd": 2 * T * row + T * E * 4,                       # read H (dW) and dL, write dH
+        "dispatch_bwd": T * k * row + 2 * T * row,                 # read k rows, read-modify-write dH
+    }
+    dom = max(range(7), key=lambda j: stage_ms[j])
+    dom_name = stage_names[dom]
+    achieved = alg_bytes[dom_name] / (stage_ms[dom] * 1e-3) / 1e9
+    stages = {n: {"ms": round(stage_ms[j], 4), "alg_GB": round(alg_bytes[n] / 1e9, 4),
+                  "GBps": round(alg_bytes[n] / (stage_ms[j] * 1e-3) / 1e9, 1),
+                  "frac_of_hbm_peak": round(alg_bytes[n] / (stage_ms[j] * 1e-3) / 1e9 / peak, 4)}
+              for j, n in enumerate(stage_names)}
+    fwd_ms = stage_ms[0] + stage_ms[1]
+
+    # ---- the CPU checker on the host cores, bounded sample ------------------------------------------------
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        Ts = args.ref_tokens
+        oracle_step(wl, 128)
+        dt_cpu, _ = oracle_step(wl, Ts)
+        cpu = {"value": Ts / dt_cpu, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+               "sample": f"first {Ts} tokens of the workload, whole path fwd+bwd, {dt_cpu:.1f} s"}
+
+    out = {
+        "metric": METRIC, "value": world * T / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+        "config": {"workload": wl.name, "T": T, "d_model": d, "E": E, "k": k, "capacity_factor": wl.capacity_factor,
+                   "C": C, "step": "route_fwd+dispatch+combine+route_bwd+dispatch_bwd",
+                   "l2": "inputs exceed L2 (0.5 GiB tokens, 4 GiB expert buffers); no flush",
+                   "replicas": world},
+        "route_dispatch_tokens_per_s": world * T / (fwd_ms * 1e-3),
+        "stages": stages,
+        "solver": {"status": st2.status, "sweeps": st2.sweeps, "augmentations": st2.augmentations,
+                   "rounds": st2.rounds, "candidates": st2.candidates, "rerouted": st2.rerouted,
+                   "total_score": st2.total_score},
+        "roofline": {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None, "peak_source": peak_src},
+        "cpu_baseline": cpu,
+        "e2e": {"value": world * T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
+                "covers": "maxscore_route_dispatch_host (pinned host batch in, indices out) + rest of the step on device"},
+        "gpu_launches": launches_per_step() * args.steps,
+        "clocks": clocks,
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="stress")
+    ap.add_argument("--tokens", type=int, default=0, help="override T (profiling on a smaller case)")
+    ap.add_argument("--ref-tokens", type=int, default=2048, help="tokens per step of the CPU checker's sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from paper_2508_12801_b200 import synth
+    wl = synth.WORKLOADS[args.workload]
+    if args.tokens:
+        wl = synth.scaled(wl, T=args.tokens)
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()
