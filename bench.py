@@ -338,7 +338,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="stress")
     ap.add_argument("--tokens", type=int, default=0, help="override T (profiling on a smaller case)")
-    ap.add_argument("--ref-tokens", type=int, default=2048, help="tokens per step of the CPU checker's sample")
+    ap.add_argument("--ref-tokens", type=int, default=4096, help="tokens per step of the CPU checker's sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     from paper_2508_12801_b200 import synth
