@@ -209,6 +209,33 @@ maxscore_status maxscore_route_dispatch_host(maxscore_ctx* ctx, const void* hidd
                                              float* gate_w_host, maxscore_stats* stats_host,
                                              void* cuda_stream);
 
+/* ---- index build for callers that cannot allocate device memory ---------------------------------- */
+
+/* The paper has no counterpart to this call; it exists for integration reasons only.
+ *
+ * Same result as maxscore_index_build (slot_idx [T, k], slot_token [E, C] with -1 padding,
+ * expert_load [E]), but it needs neither a context nor a workspace: its scratch (per-block expert
+ * counts) lives in a fixed array inside the library's device image.  It is meant for callers that must
+ * not allocate while they run: code inside a region where cudaMalloc is forbidden or would
+ * synchronise the device (a latency-critical serving loop, a plugin that only receives tensors its
+ * host framework owns, a memory pool that is already fully handed out).  It calls no cudaMalloc,
+ * cudaFree or any other allocating routine; the caller passes inputs and outputs only.
+ *
+ *   Limits: T <= MAXSCORE_NOALLOC_MAX_T (1,048,576 tokens), E <= 128, k <= 8, C >= 1.  Larger sizes
+ *   return MAXSCORE_ERR_UNSUPPORTED before anything is launched.  The scratch array is 512 KiB and is
+ *   held by every GPU that loads the library until the process exits.
+ *   First call on a device: looks up the device address of the scratch array (cudaGetSymbolAddress,
+ *   with that device current) and caches it for that device; make this first call outside any stream
+ *   capture.  The call uses whichever device is current.
+ *   Sharing: all calls on a device use the same scratch array.  Nothing in it has to start at zero
+ *   (every entry read by a call is first written by that call), but two calls that overlap on the GPU
+ *   (different streams, no ordering between them) race on it; order them on one stream or with events. */
+#define MAXSCORE_NOALLOC_MAX_T 1048576
+maxscore_status maxscore_index_build_noalloc(int32_t T, int32_t E, int32_t k, int32_t C,
+                                             const int32_t* expert_idx, int32_t* slot_idx,
+                                             int32_t* slot_token, int32_t* expert_load,
+                                             void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -14,6 +14,8 @@ import torch
 
 from . import build as _build
 
+C_int32 = C.c_int32
+
 F32, BF16 = 0, 1
 STAT_NOT_CONVERGED, STAT_NON_FINITE, STAT_INTERNAL = 1, 2, 4
 STATUS_NAMES = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_INFEASIBLE", 3: "ERR_WORKSPACE", 4: "ERR_CUDA",
@@ -43,7 +45,7 @@ EXPORTS = ["maxscore_capacity", "maxscore_workspace_bytes", "maxscore_create", "
            "maxscore_last_cuda_error", "maxscore_route_fwd", "maxscore_dispatch", "maxscore_combine",
            "maxscore_route_bwd", "maxscore_gate", "maxscore_softtopk_fwd", "maxscore_softtopk_bwd",
            "maxscore_assign", "maxscore_index_build", "maxscore_combine_bwd", "maxscore_gate_bwd",
-           "maxscore_route_dispatch_host"]
+           "maxscore_route_dispatch_host", "maxscore_index_build_noalloc"]
 
 
 def _load():
@@ -209,6 +211,13 @@ def route_dispatch_host(ctx, hidden_host, w_gate_host, expert_bias_host, dev: De
                                              _ptr(expert_bias_host), C.byref(dev), _ptr(expert_idx_host),
                                              _ptr(slot_idx_host), _ptr(gate_w_host), _ptr(stats_host),
                                              _stream(stream)), "maxscore_route_dispatch_host")
+
+
+def index_build_noalloc(T, E, k, C, expert_idx, slot_idx, slot_token, expert_load, stream=None):
+    """Index build with no context and no workspace (scratch inside the library); see the header."""
+    _check(_lib.maxscore_index_build_noalloc(C_int32(T), C_int32(E), C_int32(k), C_int32(C), _ptr(expert_idx),
+                                             _ptr(slot_idx), _ptr(slot_token), _ptr(expert_load), _stream(stream)),
+           "maxscore_index_build_noalloc")
 
 
 # ---- conveniences for callers that keep everything in torch tensors -----------------------------------

@@ -486,3 +486,61 @@ maxscore_status maxscore_route_dispatch_host(maxscore_ctx* c, const void* hidden
 }
 
 }  // extern "C"
+
+// ==================================================================================================
+// Index build without a context or a workspace, for callers that cannot allocate device memory.
+// The scratch of the two-pass index build (expert counts per block of kIdxTok tokens) is a fixed array
+// in the device image.  In host code the array's name is only a handle: the device address each GPU
+// gave it is fetched once per device with cudaGetSymbolAddress and handed to the kernels.
+namespace {
+
+constexpr int kNoAllocMaxBlocks = MAXSCORE_NOALLOC_MAX_T / kIdxTok;          // 1024 blocks
+static __device__ __align__(256) int32_t g_noalloc_block_counts[kNoAllocMaxBlocks * kMaxE];   // 512 KiB
+
+constexpr int kMaxDevices = 64;
+int32_t* g_noalloc_scratch_ptr[kMaxDevices] = {};      // per device, filled on the first call there
+
+maxscore_status noalloc_scratch(int32_t** out) {
+  int dev = 0;
+  MS_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return MAXSCORE_ERR_UNSUPPORTED;
+  int32_t* p = __atomic_load_n(&g_noalloc_scratch_ptr[dev], __ATOMIC_ACQUIRE);
+  if (!p) {
+    void* addr = nullptr;
+    MS_CUDA(cudaGetSymbolAddress(&addr, g_noalloc_block_counts));   // address on the current device
+    p = static_cast<int32_t*>(addr);
+    __atomic_store_n(&g_noalloc_scratch_ptr[dev], p, __ATOMIC_RELEASE);   // racing first calls store the same value
+  }
+  *out = p;
+  return MAXSCORE_OK;
+}
+
+}  // namespace
+
+extern "C" maxscore_status maxscore_index_build_noalloc(int32_t T, int32_t E, int32_t k, int32_t C,
+                                                        const int32_t* expert_idx, int32_t* slot_idx,
+                                                        int32_t* slot_token, int32_t* expert_load,
+                                                        void* cuda_stream) {
+  if (!expert_idx || !slot_idx || !slot_token || !expert_load) return MAXSCORE_ERR_INVALID_ARG;
+  if (T <= 0 || E <= 0 || k <= 0 || C <= 0) return MAXSCORE_ERR_INVALID_ARG;
+  if (k > E) return MAXSCORE_ERR_INFEASIBLE;
+  if (T > MAXSCORE_NOALLOC_MAX_T || E > kMaxE || k > kMaxK) {
+    snprintf(g_last_error, sizeof(g_last_error),
+             "maxscore_index_build_noalloc: T=%d E=%d k=%d exceeds the fixed scratch (T <= %d, E <= %d, k <= %d)",
+             T, E, k, MAXSCORE_NOALLOC_MAX_T, kMaxE, kMaxK);
+    return MAXSCORE_ERR_UNSUPPORTED;
+  }
+  int32_t* scratch = nullptr;
+  maxscore_status s = noalloc_scratch(&scratch);
+  if (s) return s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const int blocks = (T + kIdxTok - 1) / kIdxTok;
+  // every scratch entry the fill pass reads (blocks x E counts) is written by the count pass first,
+  // so what an earlier call left in the array does not matter
+  MS_CUDA(cudaMemsetAsync(slot_token, 0xFF, sizeof(int32_t) * (size_t)E * C, st));
+  index_count_kernel<<<blocks, kIdxTok, 0, st>>>(expert_idx, scratch, T, E, k);
+  MS_LAUNCH_CHECK("index_count_kernel");
+  index_fill_kernel<<<blocks, kIdxTok, 0, st>>>(expert_idx, scratch, slot_idx, slot_token, expert_load, T, E, k, C);
+  MS_LAUNCH_CHECK("index_fill_kernel");
+  return MAXSCORE_OK;
+}
