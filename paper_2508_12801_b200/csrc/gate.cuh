@@ -280,3 +280,277 @@ gate_bwd_dw_kernel(const T* __restrict__ H, const float* __restrict__ dL, float*
 }
 
 }  // namespace msr
+
+// =================================================================================================
+// Tensor-core derivative GEMMs (bf16 I/O).
+//
+// dlogits is fp32.  It is split into bf16 hi + lo parts (dL = hi + lo up to 2^-17 relative), laid
+// out as dLs[T][2*Kpad] = [hi | lo] with Kpad = E rounded up to 64, so that the products against the
+// exact bf16 H and W_g keep close to fp32 accuracy while running on the bf16 tensor pipe.
+namespace msr {
+
+__global__ void split_dlogits_kernel(const float* __restrict__ dL, __nv_bfloat16* __restrict__ dLs, int T, int E,
+                                     int Kpad) {
+  const long long n = (long long)T * Kpad;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const long long t = i / Kpad; const int j = (int)(i - t * Kpad);
+    float x = j < E ? dL[t * E + j] : 0.f;
+    const __nv_bfloat16 hi = __float2bfloat16(x);
+    const __nv_bfloat16 lo = __float2bfloat16(x - __bfloat162float(hi));
+    dLs[t * 2 * Kpad + j] = hi;
+    dLs[t * 2 * Kpad + Kpad + j] = lo;
+  }
+}
+
+// W_g as bf16 [d][Kpad] (expert index contiguous, zero padded): the K-major B operand of dH = dL . W_g^T
+__global__ void wgate_kmajor_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wk, int d, int E,
+                                    int Kpad, int layout) {
+  const long long n = (long long)d * Kpad;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const int m = (int)(i / Kpad), j = (int)(i % Kpad);
+    __nv_bfloat16 v = __float2bfloat16(0.f);
+    if (j < E) v = layout == 0 ? w[(size_t)m * E + j] : w[(size_t)j * d + m];
+    wk[i] = v;
+  }
+}
+
+// Descriptor of an MN-major bf16 operand tile written by TMA boxes of 64 (M or N) x rows (K) with the
+// 128-byte swizzle: a K row is 128 bytes, groups of 8 K rows are 1024 bytes apart, and the next
+// 64-wide chunk along M/N starts `chunk_bytes` further.
+__device__ __forceinline__ uint64_t smem_desc_mn128(uint32_t saddr, uint32_t chunk_bytes) {
+  return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)((chunk_bytes >> 4) & 0x3FFF) << 16) |
+         ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+__host__ __device__ constexpr uint32_t idesc_bf16_m128_mn(int n) {   // both operands MN-major
+  return idesc_bf16_m128(n) | (1u << 15) | (1u << 16);
+}
+
+// ---- dH[T, d] = dL[T, E] . W_g^T -------------------------------------------------------------------
+// One CTA per 128-token tile.  The dL tile (hi and lo) is loaded once; 128-column tiles of W_g stream
+// through a 3-stage ring; two TMEM accumulators alternate so that the four epilogue warps convert and
+// store tile n while the MMA warp works on tile n+1.
+constexpr int kDhBN = 128, kDhStages = 3;
+struct DhSmem {
+  uint64_t a_full, b_full[kDhStages], b_empty[kDhStages], acc_full[2], acc_empty[2];
+  uint32_t tmem_base;
+  int failed;
+};
+
+__global__ void __launch_bounds__(192)
+gate_bwd_dh_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                      __nv_bfloat16* __restrict__ dH, int T, int d, int Kpad, unsigned* error_flag) {
+  extern __shared__ unsigned char dsm_raw[];
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(dsm_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ DhSmem sm;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * 128;
+  const int kboxes = Kpad / 64;                       // 64-wide K boxes per part
+  const uint32_t a_bytes = 2u * kboxes * 16384u;      // hi and lo
+  const uint32_t b_bytes = kboxes * 16384u;
+  unsigned char* a_tile = base;                       // [2*kboxes][128 rows][128 B]
+  unsigned char* b_ring = base + a_bytes;             // [stage][kboxes][128 rows][128 B]
+  const int n_tiles = (d + kDhBN - 1) / kDhBN;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&sm.a_full, 1);
+    for (int s = 0; s < kDhStages; ++s) { mbar_init(&sm.b_full[s], 1); mbar_init(&sm.b_empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&sm.acc_full[b], 1); mbar_init(&sm.acc_empty[b], 4); }
+    sm.failed = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) tmem_alloc(&sm.tmem_base, 256);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sm.tmem_base;
+
+  if (warp == 0 && lane == 0) {
+    mbar_expect_tx(&sm.a_full, a_bytes);
+    for (int kb = 0; kb < kboxes; ++kb) {
+      tma_load_2d(a_tile + (size_t)kb * 16384, &tmA, kb * 64, m0, &sm.a_full);                      // hi
+      tma_load_2d(a_tile + (size_t)(kboxes + kb) * 16384, &tmA, Kpad + kb * 64, m0, &sm.a_full);    // lo
+    }
+    for (int nt = 0; nt < n_tiles; ++nt) {
+      const int s = nt % kDhStages;
+      const uint32_t ph = (uint32_t)((nt / kDhStages) & 1);
+      if (nt >= kDhStages && !mbar_wait_bounded(&sm.b_empty[s], ph ^ 1)) { sm.failed = 1; break; }
+      mbar_expect_tx(&sm.b_full[s], b_bytes);
+      for (int kb = 0; kb < kboxes; ++kb)
+        tma_load_2d(b_ring + (size_t)s * b_bytes + (size_t)kb * 16384, &tmB, kb * 64, nt * kDhBN, &sm.b_full[s]);
+    }
+  } else if (warp == 1 && lane == 0) {
+    const uint32_t idesc = idesc_bf16_m128(kDhBN);
+    bool ok = mbar_wait_bounded(&sm.a_full, 0);
+    for (int nt = 0; nt < n_tiles && ok; ++nt) {
+      const int s = nt % kDhStages, buf = nt & 1;
+      if (nt >= 2) ok = mbar_wait_bounded(&sm.acc_empty[buf], (uint32_t)(((nt >> 1) & 1) ^ 1));
+      if (ok) ok = mbar_wait_bounded(&sm.b_full[s], (uint32_t)((nt / kDhStages) & 1));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t acc = tmem + (uint32_t)(buf * kDhBN);
+      uint32_t first = 0;
+      for (int kb = 0; kb < kboxes; ++kb) {
+        const uint64_t bd = smem_desc_k128(smem_u32(b_ring + (size_t)s * b_bytes + (size_t)kb * 16384));
+        const uint64_t ah = smem_desc_k128(smem_u32(a_tile + (size_t)kb * 16384));
+        const uint64_t al = smem_desc_k128(smem_u32(a_tile + (size_t)(kboxes + kb) * 16384));
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          umma_bf16(acc, ah + 2 * kk, bd + 2 * kk, idesc, first); first = 1;
+          umma_bf16(acc, al + 2 * kk, bd + 2 * kk, idesc, 1u);
+        }
+      }
+      umma_commit(&sm.b_empty[s]);
+      umma_commit(&sm.acc_full[buf]);
+    }
+    if (!ok) sm.failed = 1;
+  } else if (warp >= 2) {
+    const int quarter = warp & 3;                      // TMEM lanes this warp may read
+    const int row = m0 + quarter * 32 + lane;
+    bool ok = true;
+    for (int nt = 0; nt < n_tiles && ok; ++nt) {
+      const int buf = nt & 1;
+      ok = mbar_wait_bounded(&sm.acc_full[buf], (uint32_t)((nt >> 1) & 1));
+      if (!ok) break;
+      tc_fence_after();
+      for (int c0 = 0; c0 < kDhBN; c0 += 16) {
+        float r[16];
+        tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kDhBN + c0), r);
+        const int col = nt * kDhBN + c0;
+        if (row < T && col < d) {
+          __nv_bfloat16* out = dH + (size_t)row * d + col;
+          if (col + 16 <= d) {
+            uint32_t w[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              __nv_bfloat162 h = __floats2bfloat162_rn(r[2 * j], r[2 * j + 1]);
+              w[j] = *reinterpret_cast<uint32_t*>(&h);
+            }
+            reinterpret_cast<uint4*>(out)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            reinterpret_cast<uint4*>(out)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+          } else {
+            for (int j = 0; j < 16 && col + j < d; ++j) out[j] = __float2bfloat16(r[j]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);
+    }
+    if (!ok && lane == 0) sm.failed = 1;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && sm.failed) atomicOr(error_flag, 4u);
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem, 256);
+}
+
+// ---- dW[d, E] = H^T . dL ---------------------------------------------------------------------------
+// The contraction runs over tokens while both operands are stored with tokens as rows, so both are
+// MN-major for the tensor core: a TMA box of 64 columns x 64 tokens lands in exactly the layout the
+// MN-major descriptor names.  A CTA owns 128 columns of H (rows of dW) and one chunk of tokens
+// (split-K); partial results go to a workspace and are summed in a fixed order by a second kernel.
+constexpr int kDwStages = 4, kDwBK = 64;
+struct DwSmem {
+  uint64_t full[kDwStages], empty[kDwStages], accum;
+  uint32_t tmem_base;
+  int failed;
+};
+
+__global__ void __launch_bounds__(128)
+gate_bwd_dw_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmL,
+                      float* __restrict__ partial, int T, int d, int E, int Kpad, int tokens_per_split,
+                      unsigned* error_flag) {
+  extern __shared__ unsigned char wsm_raw[];
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(wsm_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ DwSmem sm;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * 128;
+  const int t_begin = blockIdx.y * tokens_per_split;
+  const int t_end = min(T, t_begin + tokens_per_split);
+  const int num_kb = (t_end - t_begin + kDwBK - 1) / kDwBK;
+  const int nboxes = Kpad / 64;                                   // 64-wide N chunks
+  const uint32_t a_bytes = 2u * 8192u, b_bytes = 2u * nboxes * 8192u;   // B: hi and lo
+  const uint32_t stage_bytes = a_bytes + b_bytes;
+  uint32_t tmem_cols = 32; while ((int)tmem_cols < Kpad) tmem_cols <<= 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kDwStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
+    mbar_init(&sm.accum, 1);
+    sm.failed = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) tmem_alloc(&sm.tmem_base, tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sm.tmem_base;
+
+  if (warp == 0 && lane == 0) {
+    for (int kb = 0; kb < num_kb; ++kb) {
+      const int s = kb % kDwStages;
+      const uint32_t ph = (uint32_t)((kb / kDwStages) & 1);
+      if (kb >= kDwStages && !mbar_wait_bounded(&sm.empty[s], ph ^ 1)) { sm.failed = 1; break; }
+      unsigned char* st = base + (size_t)s * stage_bytes;
+      const int t0 = t_begin + kb * kDwBK;
+      mbar_expect_tx(&sm.full[s], stage_bytes);
+      tma_load_2d(st, &tmH, m0, t0, &sm.full[s]);
+      tma_load_2d(st + 8192, &tmH, m0 + 64, t0, &sm.full[s]);
+      for (int nb = 0; nb < nboxes; ++nb) {
+        tma_load_2d(st + a_bytes + (size_t)nb * 8192, &tmL, nb * 64, t0, &sm.full[s]);                          // hi
+        tma_load_2d(st + a_bytes + (size_t)(nboxes + nb) * 8192, &tmL, Kpad + nb * 64, t0, &sm.full[s]);        // lo
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    const uint32_t idesc = idesc_bf16_m128_mn(Kpad);
+    bool ok = true;
+    for (int kb = 0; kb < num_kb && ok; ++kb) {
+      const int s = kb % kDwStages;
+      ok = mbar_wait_bounded(&sm.full[s], (uint32_t)((kb / kDwStages) & 1));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t sa = smem_u32(base + (size_t)s * stage_bytes);
+      const uint32_t sbh = sa + a_bytes, sbl = sbh + nboxes * 8192u;
+#pragma unroll
+      for (int kk = 0; kk < kDwBK / 16; ++kk) {           // 16 tokens = 2048 bytes further down each box
+        const uint64_t ad = smem_desc_mn128(sa + kk * 2048u, 8192u);
+        umma_bf16(tmem, ad, smem_desc_mn128(sbh + kk * 2048u, 8192u), idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+        umma_bf16(tmem, ad, smem_desc_mn128(sbl + kk * 2048u, 8192u), idesc, 1u);
+      }
+      umma_commit(&sm.empty[s]);
+    }
+    if (!ok) sm.failed = 1;
+    umma_commit(&sm.accum);
+  }
+  __syncwarp();
+  const bool got = mbar_wait_bounded(&sm.accum, 0);
+  tc_fence_after();
+  if (got && !sm.failed && num_kb > 0) {
+    const int row = m0 + warp * 32 + lane;              // row of dW = column of H
+    float* out = partial + ((size_t)blockIdx.y * d + row) * E;
+    for (int c0 = 0; c0 < Kpad; c0 += 16) {
+      float r[16];
+      tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, r);
+      if (row < d)
+        for (int j = 0; j < 16; ++j)
+          if (c0 + j < E) out[c0 + j] = r[j];
+    }
+  } else if (num_kb <= 0) {
+    const int row = m0 + warp * 32 + lane;
+    if (row < d) for (int j = 0; j < E; ++j) partial[((size_t)blockIdx.y * d + row) * E + j] = 0.f;
+  } else if (threadIdx.x == 0) {
+    atomicOr(error_flag, 4u);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, tmem_cols);
+}
+
+__global__ void reduce_dw_kernel(const float* __restrict__ partial, float* __restrict__ dW, long long n, int nsplit) {
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    float acc = 0.f;
+    for (int s = 0; s < nsplit; ++s) acc += partial[(size_t)s * n + i];   // fixed order: reproducible
+    dW[i] = acc;
+  }
+}
+
+}  // namespace msr

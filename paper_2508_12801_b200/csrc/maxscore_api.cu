@@ -50,8 +50,9 @@ int32_t capacity_of(const maxscore_params& p) {
 }
 
 struct Layout {          // byte offsets inside the workspace
-  size_t state, cand, block_counts, wt, error_flag, total;
+  size_t state, cand, block_counts, wt, error_flag, dls, wk, dwpart, total;
   int Npad, n_idx_blocks;
+  int Kpad, dw_splits, dw_tokens_per_split;   // tensor-core backward GEMMs (bf16 I/O)
 };
 
 Layout layout_of(const maxscore_params& p) {
@@ -65,6 +66,21 @@ Layout layout_of(const maxscore_params& p) {
   l.block_counts = off; off = align_up(off + sizeof(int32_t) * (size_t)l.n_idx_blocks * p.E, 1024);
   l.wt = off;
   off = align_up(off + (p.io_dtype == MAXSCORE_BF16 ? sizeof(__nv_bfloat16) * (size_t)l.Npad * p.d_model : 0), 1024);
+  l.Kpad = (int)align_up((size_t)p.E, 64);
+  {   // split the token dimension of dW so that about two CTAs per SM are busy
+    const int mtiles = (p.d_model + 127) / 128;
+    int splits = (296 + mtiles - 1) / mtiles;
+    const int max_splits = (p.T + 255) / 256;
+    if (splits > max_splits) splits = max_splits;
+    if (splits > 64) splits = 64;
+    if (splits < 1) splits = 1;
+    l.dw_tokens_per_split = (int)align_up((size_t)((p.T + splits - 1) / splits), 64);
+    l.dw_splits = (p.T + l.dw_tokens_per_split - 1) / l.dw_tokens_per_split;
+  }
+  const bool bf = p.io_dtype == MAXSCORE_BF16;
+  l.dls = off; off = align_up(off + (bf ? sizeof(__nv_bfloat16) * (size_t)p.T * 2 * l.Kpad : 0), 1024);
+  l.wk = off; off = align_up(off + (bf ? sizeof(__nv_bfloat16) * (size_t)p.d_model * l.Kpad : 0), 1024);
+  l.dwpart = off; off = align_up(off + (bf ? sizeof(float) * (size_t)l.dw_splits * p.d_model * p.E : 0), 1024);
   l.total = off;
   return l;
 }
@@ -97,6 +113,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 constexpr int kP2SmemMax = (int)(sizeof(long long) * kMaxE * kMaxE);
 constexpr int kDispatchSmem = 64 * 1024;
+constexpr int kDhSmemMax = 2 * 2 * 16384 + kDhStages * 2 * 16384 + 1024;     // Kpad = 128
+constexpr int kDwSmemMax = kDwStages * (16384 + 2 * 2 * 8192) + 1024;
 
 }  // namespace
 
@@ -291,6 +309,8 @@ maxscore_status maxscore_create(maxscore_ctx** out, const maxscore_params* param
   MS_CUDA(cudaFuncSetAttribute(gate_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGateSmemBytes));
   MS_CUDA(cudaFuncSetAttribute(flow_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kP2SmemMax));
   MS_CUDA(cudaFuncSetAttribute(dispatch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDispatchSmem));
+  MS_CUDA(cudaFuncSetAttribute(gate_bwd_dh_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDhSmemMax));
+  MS_CUDA(cudaFuncSetAttribute(gate_bwd_dw_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDwSmemMax));
   MS_CUDA(cudaMemsetAsync(workspace, 0, lay.cand, 0));
   MS_CUDA(cudaStreamSynchronize(0));
   maxscore_ctx* c = new (std::nothrow) maxscore_ctx();
@@ -426,14 +446,44 @@ maxscore_status maxscore_gate_bwd(maxscore_ctx* c, const void* hidden, const voi
   if (!c || !hidden || !w_gate || !dlogits || !dw_gate || !dH) return MAXSCORE_ERR_INVALID_ARG;
   const maxscore_params& p = c->p;
   cudaStream_t st = (cudaStream_t)stream;
-  MS_CUDA(cudaMemsetAsync(dw_gate, 0, sizeof(float) * (size_t)p.d_model * p.E, st));
+  if (p.io_dtype != MAXSCORE_BF16) MS_CUDA(cudaMemsetAsync(dw_gate, 0, sizeof(float) * (size_t)p.d_model * p.E, st));
   dim3 gw((p.d_model + 63) / 64, (p.T + kDwTok - 1) / kDwTok);
   const int gh = (p.T + 15) / 16;
   if (p.io_dtype == MAXSCORE_BF16) {
-    gate_bwd_dw_kernel<__nv_bfloat16><<<gw, 256, 0, st>>>((const __nv_bfloat16*)hidden, dlogits, dw_gate, p.T, p.d_model, p.E);
-    MS_LAUNCH_CHECK("gate_bwd_dw_kernel");
-    gate_bwd_dh_kernel<__nv_bfloat16><<<gh, 256, 0, st>>>(dlogits, (const __nv_bfloat16*)w_gate, (__nv_bfloat16*)dH, p.T,
-                                                          p.d_model, p.E, p.w_gate_layout);
+    const Layout& l = c->lay;
+    __nv_bfloat16* dls = reinterpret_cast<__nv_bfloat16*>(c->ws + l.dls);
+    __nv_bfloat16* wk = reinterpret_cast<__nv_bfloat16*>(c->ws + l.wk);
+    float* part = reinterpret_cast<float*>(c->ws + l.dwpart);
+    const int Kpad = l.Kpad;
+    {
+      long long n = (long long)p.T * Kpad;
+      int blocks = (int)((n + 255) / 256); if (blocks > c->sm_count * 16) blocks = c->sm_count * 16;
+      split_dlogits_kernel<<<blocks, 256, 0, st>>>(dlogits, dls, p.T, p.E, Kpad);
+      MS_LAUNCH_CHECK("split_dlogits_kernel");
+      n = (long long)p.d_model * Kpad;
+      blocks = (int)((n + 255) / 256); if (blocks > c->sm_count * 16) blocks = c->sm_count * 16;
+      wgate_kmajor_kernel<<<blocks, 256, 0, st>>>((const __nv_bfloat16*)w_gate, wk, p.d_model, p.E, Kpad, p.w_gate_layout);
+      MS_LAUNCH_CHECK("wgate_kmajor_kernel");
+    }
+    CUtensorMap tmA, tmB, tmH2, tmL2;
+    maxscore_status s2 = make_tmap_bf16(c, &tmA, dls, (uint64_t)2 * Kpad, (uint64_t)p.T, 64, 128);
+    if (!s2) s2 = make_tmap_bf16(c, &tmB, wk, (uint64_t)Kpad, (uint64_t)p.d_model, 64, 128);
+    if (!s2) s2 = make_tmap_bf16(c, &tmH2, hidden, (uint64_t)p.d_model, (uint64_t)p.T, 64, 64);
+    if (!s2) s2 = make_tmap_bf16(c, &tmL2, dls, (uint64_t)2 * Kpad, (uint64_t)p.T, 64, 64);
+    if (s2) return s2;
+    const int kboxes = Kpad / 64;
+    const size_t dh_smem = (size_t)2 * kboxes * 16384 + (size_t)kDhStages * kboxes * 16384 + 1024;
+    gate_bwd_dh_tc_kernel<<<(p.T + 127) / 128, 192, dh_smem, st>>>(tmA, tmB, (__nv_bfloat16*)dH, p.T, p.d_model, Kpad,
+                                                                  error_flag_of(c));
+    MS_LAUNCH_CHECK("gate_bwd_dh_tc_kernel");
+    const size_t dw_smem = (size_t)kDwStages * (16384 + (size_t)2 * kboxes * 8192) + 1024;
+    dim3 gdw((p.d_model + 127) / 128, l.dw_splits);
+    gate_bwd_dw_tc_kernel<<<gdw, 128, dw_smem, st>>>(tmH2, tmL2, part, p.T, p.d_model, p.E, Kpad, l.dw_tokens_per_split,
+                                                    error_flag_of(c));
+    MS_LAUNCH_CHECK("gate_bwd_dw_tc_kernel");
+    const long long nw = (long long)p.d_model * p.E;
+    int rblocks = (int)((nw + 255) / 256); if (rblocks > c->sm_count * 8) rblocks = c->sm_count * 8;
+    reduce_dw_kernel<<<rblocks, 256, 0, st>>>(part, dw_gate, nw, l.dw_splits);
   } else {
     gate_bwd_dw_kernel<float><<<gw, 256, 0, st>>>((const float*)hidden, dlogits, dw_gate, p.T, p.d_model, p.E);
     MS_LAUNCH_CHECK("gate_bwd_dw_kernel");
