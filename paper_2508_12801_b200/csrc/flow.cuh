@@ -34,7 +34,8 @@ namespace msr {
 constexpr int kNB = 256;                  // histogram bins per expert: 4 per octave of the margin
 constexpr int kTopN = kMaxK + 2;          // sorted values kept per token in a sweep
 constexpr long long kInf = 1LL << 62;
-constexpr long long kArcLimit = 1LL << 55; // arcs with a larger reduced cost are ignored by the exact phase
+constexpr long long kArcLimit = 1LL << 58; // arcs with a larger reduced cost are ignored by the exact phase
+constexpr long long kPriceLimit = 1LL << 56; // sweeps keep |price| below this
 constexpr int kCapLogMax = 60;
 constexpr int kEPLf = kMaxE / 32;          // experts per lane when a warp spans one token row
 
@@ -43,6 +44,7 @@ struct KeyGen {
   int quant_shift;
   uint32_t seed_mul;   // tiebreak_seed * 0x9E3779B9
   int S;               // shift of the quantised part
+  float fshift, fS;    // 2^quant_shift and 2^S as floats (approximate keys)
 };
 
 __device__ __forceinline__ uint32_t fmix32(uint32_t h) {   // 32-bit finaliser of MurmurHash3
@@ -116,6 +118,104 @@ __device__ __forceinline__ void top_insert(long long (&v)[N], int (&id)[N], long
   }
 }
 
+// Same, but with the order made explicit: larger value first, lower expert index first on equal values.
+// Needed where entries do not arrive in ascending index order.
+template <int N>
+__device__ __forceinline__ void top_insert_tb(long long (&v)[N], int (&id)[N], long long val, int e) {
+  if (val > v[N - 1] || (val == v[N - 1] && e < id[N - 1])) {
+    v[N - 1] = val; id[N - 1] = e;
+#pragma unroll
+    for (int j = N - 1; j > 0; --j) {
+      if (v[j] > v[j - 1] || (v[j] == v[j - 1] && id[j] < id[j - 1])) {
+        long long tv = v[j]; v[j] = v[j - 1]; v[j - 1] = tv;
+        int ti = id[j]; id[j] = id[j - 1]; id[j - 1] = ti;
+      }
+    }
+  }
+}
+
+// Key in fp32 (24 significant bits): good enough to FIND the largest few entries of a row cheaply.
+__device__ __forceinline__ float approx_key(const KeyGen& g, float x) {
+  if (!isfinite(x)) x = 0.f;
+  if (g.mode == 0) return x * 1099511627776.0f;
+  return fminf(fmaxf(rintf(x * g.fshift), -32768.f), 32767.f) * g.fS;
+}
+
+// The N largest entries of key(e) - price(e) over one row, exact and sorted (value descending, lower
+// expert index first on equal values).
+//   1. a branch-free pass keeps the N largest fp32 approximations; the expert index rides in the low
+//      7 mantissa bits, so each slot costs one max and one min;
+//   2. the exact int64 values of those N experts are computed and sorted;
+//   3. if `exact`, a second pass checks that no other expert beats the N-th one exactly; in the rare
+//      case one does (values closer than fp32 resolves), the row is redone by exact insertion.
+// Without `exact` the result may miss an entry that differs from the N-th by less than ~2^-17 relative.
+template <int N>
+__device__ __forceinline__ void select_top(const float* row, const long long* sp, const float* spf, const KeyGen& g,
+                                           uint32_t flat, int E, int start, bool exact, long long (&v)[N],
+                                           int (&id)[N]) {
+  float pk[N];
+#pragma unroll
+  for (int j = 0; j < N; ++j) pk[j] = -INFINITY;
+  int e = start;
+  for (int jj = 0; jj < E; ++jj) {
+    const float vf = approx_key(g, row[e]) - (spf ? spf[e] : 0.f);
+    float x = __uint_as_float((__float_as_uint(vf) & ~127u) | (unsigned)e);
+#pragma unroll
+    for (int j = 0; j < N; ++j) { const float hi = fmaxf(pk[j], x); x = fminf(pk[j], x); pk[j] = hi; }
+    if (++e == E) e = 0;
+  }
+#pragma unroll
+  for (int j = 0; j < N; ++j) {
+    const bool ok = pk[j] != -INFINITY;
+    const int ee = (int)(__float_as_uint(pk[j]) & 127u);
+    id[j] = ok ? ee : -1;
+    v[j] = ok ? make_key(g, row[ee], flat + ee) - (sp ? sp[ee] : 0) : -kInf;
+  }
+#pragma unroll
+  for (int pass = 0; pass < N; ++pass) {
+#pragma unroll
+    for (int j = (pass & 1); j + 1 < N; j += 2) {
+      if (v[j + 1] > v[j] || (v[j + 1] == v[j] && id[j + 1] >= 0 && id[j + 1] < id[j])) {
+        const long long tv = v[j]; v[j] = v[j + 1]; v[j + 1] = tv;
+        const int ti = id[j]; id[j] = id[j + 1]; id[j + 1] = ti;
+      }
+    }
+  }
+  if (!exact || id[N - 1] < 0) return;                 // E <= N: every expert is in the list
+  const long long tv = v[N - 1]; const int ti = id[N - 1];
+  bool missed = false;
+  e = start;
+  for (int jj = 0; jj < E; ++jj) {
+    const long long val = make_key(g, row[e], flat + e) - (sp ? sp[e] : 0);
+    if (val > tv || (val == tv && e < ti)) {
+      bool in = false;
+#pragma unroll
+      for (int j = 0; j < N; ++j) in |= (id[j] == e);
+      missed |= !in;
+    }
+    if (++e == E) e = 0;
+  }
+  if (!missed) return;
+#pragma unroll
+  for (int j = 0; j < N; ++j) { v[j] = -kInf; id[j] = -1; }
+  for (e = 0; e < E; ++e) top_insert_tb(v, id, make_key(g, row[e], flat + e) - (sp ? sp[e] : 0), e);
+}
+
+// Copy the score rows of this CTA's tokens (contiguous in memory) into shared memory with coalesced
+// loads.  A thread then walks its own row starting at a column rotated by its index, so that the lanes
+// of a warp hit different banks although the rows are E floats apart.
+__device__ __forceinline__ void stage_rows(const float* __restrict__ M, float* tile, int tok0, int ntok, int E) {
+  const long long n = (long long)ntok * E;
+  const float* src = M + (size_t)tok0 * E;
+  if ((E & 3) == 0) {
+    const float4* s4 = reinterpret_cast<const float4*>(src);
+    float4* d4 = reinterpret_cast<float4*>(tile);
+    for (int i = threadIdx.x; i < n / 4; i += blockDim.x) d4[i] = __ldg(s4 + i);
+  } else {
+    for (int i = threadIdx.x; i < n; i += blockDim.x) tile[i] = __ldg(src + i);
+  }
+}
+
 __device__ __forceinline__ bool last_block_arrives(unsigned* ticket) {
   __shared__ bool is_last;
   __threadfence();
@@ -178,7 +278,7 @@ __device__ __forceinline__ long long price_step(const unsigned* hist, int need, 
     return step;
   }
   const long long lo = bin_lower_edge(pos), hi = bin_lower_edge(pos + 1);
-  cut = min(kCapLogMax, max(12, (pos >> 2) + 8));      // next sweep: record up to ~64x this margin
+  cut = min(kCapLogMax, max(12, (pos >> 2) + 5));      // next sweep: record up to ~16x this margin
   (void)before;
   if (cum <= 2u * (unsigned)need || lo == 0) {
     const long long w = hi - lo;
@@ -198,33 +298,27 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
   __shared__ long long sp[kMaxE];
   __shared__ int sload[kMaxE];
   __shared__ int scu[kMaxE], scd[kMaxE];
+  __shared__ float spf[kMaxE];
   __shared__ int sflag[kMaxE];
   __shared__ int nflag;
   if (threadIdx.x == 0) nflag = 0;
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += blockDim.x) {
-    sp[e] = st->p[e]; sload[e] = 0; scu[e] = st->cap_up[e]; scd[e] = st->cap_dn[e];
+    sp[e] = st->p[e]; spf[e] = (float)sp[e]; sload[e] = 0; scu[e] = st->cap_up[e]; scd[e] = st->cap_dn[e];
     if (st->flag_dn[e]) sflag[atomicAdd(&nflag, 1)] = e;
   }
+  extern __shared__ __align__(16) float sweep_tile[];
+  const int tok0 = blockIdx.x * blockDim.x;
+  stage_rows(M, sweep_tile, tok0, min((int)blockDim.x, T - tok0), E);
   __syncthreads();
-  const int tok = blockIdx.x * blockDim.x + threadIdx.x;
+  const int tok = tok0 + threadIdx.x;
   if (tok < T) {
     long long v[kTopN]; int id[kTopN];
-#pragma unroll
-    for (int j = 0; j < kTopN; ++j) { v[j] = -kInf; id[j] = -1; }
-    const float* row = M + (size_t)tok * E;
+    const float* row = sweep_tile + (size_t)threadIdx.x * E;
     const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-    if ((E & 3) == 0) {
-      for (int e = 0; e < E; e += 4) {
-        float4 x = __ldg(reinterpret_cast<const float4*>(row + e));
-        top_insert(v, id, make_key(g, x.x, flat + e) - sp[e], e);
-        top_insert(v, id, make_key(g, x.y, flat + e + 1) - sp[e + 1], e + 1);
-        top_insert(v, id, make_key(g, x.z, flat + e + 2) - sp[e + 2], e + 2);
-        top_insert(v, id, make_key(g, x.w, flat + e + 3) - sp[e + 3], e + 3);
-      }
-    } else {
-      for (int e = 0; e < E; ++e) top_insert(v, id, make_key(g, __ldg(row + e), flat + e) - sp[e], e);
-    }
+    // rotated start: conflict-free shared-memory reads.  The sweeps are a heuristic, so the cheap
+    // (fp32-filtered) selection is enough here.
+    select_top(row, sp, spf, g, flat, E, threadIdx.x % E, false, v, id);
     const bool has_alt = E > k;
     long long vk = -kInf, vk1 = -kInf;                // k-th value and best alternative
 #pragma unroll
@@ -260,7 +354,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
 #pragma unroll
       for (int j = 0; j < kTopN; ++j) seen |= (j <= k + 1 && id[j] == e);
       if (seen) continue;
-      const long long m = vk - (make_key(g, __ldg(row + e), flat + e) - sp[e]);
+      const long long m = vk - (make_key(g, row[e], flat + e) - sp[e]);
       const int cl = scd[e];
       if (m >= 0 && m < (1LL << cl)) atomicAdd(&st->hist_dn[e * kNB + log_bin(m)], 1u);
     }
@@ -298,6 +392,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
       st->flag_dn[e] = 0;
     }
     st->load[e] = 0;
+    p = p > kPriceLimit ? kPriceLimit : (p < -kPriceLimit ? -kPriceLimit : p);
     // when nothing was out of balance the prices stay put and the collect pass reproduces this state
     if (x != 0) sp[e] = p;
   }
@@ -338,15 +433,20 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
                     void* stats_out, const unsigned* __restrict__ error_flag, int unbounded) {
   if (!verify_only && *(volatile int*)&st->converged) return;
   __shared__ long long sp[kMaxE];
+  __shared__ float spf[kMaxE];
   __shared__ int sload[kMaxE];
   __shared__ int s_viol, s_rer;
   __shared__ double s_score;
   __shared__ unsigned s_flags;
-  for (int e = threadIdx.x; e < E; e += blockDim.x) { sp[e] = st->p[e]; sload[e] = 0; }
+  for (int e = threadIdx.x; e < E; e += blockDim.x) { sp[e] = st->p[e]; spf[e] = (float)sp[e]; sload[e] = 0; }
   if (threadIdx.x == 0) { s_viol = 0; s_rer = 0; s_score = 0.0; s_flags = 0; }
   __syncthreads();
   const long long theta = unbounded ? kInf : st->theta;   // the last round lists every token
-  const int tok = blockIdx.x * blockDim.x + threadIdx.x;
+  extern __shared__ __align__(16) float collect_tile[];
+  const int tok0 = blockIdx.x * blockDim.x;
+  stage_rows(M, collect_tile, tok0, min((int)blockDim.x, T - tok0), E);
+  __syncthreads();
+  const int tok = tok0 + threadIdx.x;
   if (tok < T) {
     unsigned held[4] = {0, 0, 0, 0};
     if (!first)
@@ -354,30 +454,31 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
         int e = expert_idx[(size_t)tok * k + c];
         if (e >= 0 && e < E) held[e >> 5] |= 1u << (e & 31);
       }
-    long long v[kMaxK + 1]; int id[kMaxK + 1];
-    long long raw[kMaxK];                       // k largest raw keys (unconstrained top-k), verify only
-#pragma unroll
-    for (int j = 0; j <= kMaxK; ++j) { v[j] = -kInf; id[j] = -1; }
-#pragma unroll
-    for (int j = 0; j < kMaxK; ++j) raw[j] = -kInf;
+    long long v[kTopN]; int id[kTopN];
     long long min_held = kInf, max_non = -kInf;
-    const float* row = M + (size_t)tok * E;
+    const float* row = collect_tile + (size_t)threadIdx.x * E;
     const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+    const int start = threadIdx.x % E;
     bool bad = false;
-    for (int e = 0; e < E; ++e) {
-      const float x = __ldg(row + e);
-      bad |= !isfinite(x);
-      const long long key = make_key(g, x, flat + e);
-      const long long val = key - sp[e];
-      top_insert(v, id, val, e);
-      if (held[e >> 5] >> (e & 31) & 1u) min_held = val < min_held ? val : min_held;
-      else max_non = val > max_non ? val : max_non;
-      if (verify_only && key > raw[kMaxK - 1]) {
-        raw[kMaxK - 1] = key;
-#pragma unroll
-        for (int j = kMaxK - 1; j > 0; --j)
-          if (raw[j] > raw[j - 1]) { long long t = raw[j]; raw[j] = raw[j - 1]; raw[j - 1] = t; }
+    if (!first) {                                     // exact check of the experts the token holds now
+      int e = start;
+      for (int jj = 0; jj < E; ++jj) {
+        const float x = row[e];
+        bad |= !isfinite(x);
+        const long long val = make_key(g, x, flat + e) - sp[e];
+        if (held[e >> 5] >> (e & 31) & 1u) min_held = val < min_held ? val : min_held;
+        else max_non = val > max_non ? val : max_non;
+        if (++e == E) e = 0;
       }
+    }
+    const bool repick = !verify_only && (first || min_held < max_non);
+    if (repick) select_top(row, sp, spf, g, flat, E, start, true, v, id);
+    long long kth_raw = -kInf;                        // k-th largest raw key: the token's own top-k boundary
+    if (verify_only) {
+      long long rv[kTopN]; int rid[kTopN];
+      select_top(row, (const long long*)nullptr, (const float*)nullptr, g, flat, E, start, true, rv, rid);
+#pragma unroll
+      for (int j = 0; j < kTopN; ++j) if (j == k - 1) kth_raw = rv[j];
     }
     if (bad) atomicOr(&s_flags, 2u);
     const bool keep = !first && (min_held >= max_non);
@@ -392,18 +493,13 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
         // the k-th value sits at v[k-1], the best alternative at v[k]
         long long vk = -kInf, vk1 = -kInf;
 #pragma unroll
-        for (int j = 0; j <= kMaxK; ++j) { if (j == k - 1) vk = v[j]; if (j == k) vk1 = v[j]; }
+        for (int j = 0; j < kTopN; ++j) { if (j == k - 1) vk = v[j]; if (j == k) vk1 = v[j]; }
         gap = (E > k) ? vk - vk1 : kInf;
       } else gap = kInf;
     } else gap = (E > k) ? min_held - max_non : kInf;
     // write the experts in ascending order (bit order of the mask)
     int c = 0;
     double sc = 0.0; int rer = 0;
-    long long kth_raw = -kInf;
-    if (verify_only) {
-#pragma unroll
-      for (int j = 0; j < kMaxK; ++j) if (j == k - 1) kth_raw = raw[j];
-    }
     for (int wd = 0; wd < 4; ++wd) {
       unsigned m = held[wd];
       while (m) {
@@ -412,7 +508,7 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
         ++c;
         atomicAdd(&sload[e], 1);
         if (verify_only) {
-          const float x = __ldg(row + e);
+          const float x = row[e];
           const long long key = make_key(g, x, flat + e);
           sc += (g.mode == 0) ? (double)x : (double)key;
           if (key < kth_raw) ++rer;

@@ -138,6 +138,8 @@ KeyGen keygen_of(const maxscore_ctx* c) {
   const long long n = (long long)c->p.T * c->p.k;
   while ((1LL << s) < n) ++s;
   g.S = 20 + s;
+  g.fshift = ldexpf(1.f, g.quant_shift);
+  g.fS = ldexpf(1.f, g.S);
   return g;
 }
 
@@ -219,19 +221,20 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   flow_init_kernel<<<1, 256, 0, st>>>(fs, eps0, eps_min, cap0, theta0, balanced, p.E);
   MS_LAUNCH_CHECK("flow_init_kernel");
   const int blocks = (p.T + kSweepThreads - 1) / kSweepThreads;
+  const size_t tile_smem = sizeof(float) * (size_t)kSweepThreads * p.E;
   for (int s = 0; s < n_sweeps; ++s) {
-    flow_sweep_kernel<<<blocks, kSweepThreads, 0, st>>>(M, fs, p.T, p.E, p.k, c->C, g, n_sweeps, 2);
+    flow_sweep_kernel<<<blocks, kSweepThreads, tile_smem, st>>>(M, fs, p.T, p.E, p.k, c->C, g, n_sweeps, 2);
     MS_LAUNCH_CHECK("flow_sweep_kernel");
   }
   const size_t p2smem = sizeof(long long) * (size_t)p.E * p.E;
   for (int r = 0; r < kRounds; ++r) {
-    flow_collect_kernel<<<blocks, kSweepThreads, 0, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, r == 0, 0,
+    flow_collect_kernel<<<blocks, kSweepThreads, tile_smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, r == 0, 0,
                                                          32LL, nullptr, nullptr, nullptr, r == kRounds - 1);
     MS_LAUNCH_CHECK("flow_collect_kernel");
     flow_exact_kernel<<<1, kP2Threads, p2smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, max_aug);
     MS_LAUNCH_CHECK("flow_exact_kernel");
   }
-  flow_collect_kernel<<<blocks, kSweepThreads, 0, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, 0, 1, 32LL,
+  flow_collect_kernel<<<blocks, kSweepThreads, tile_smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, 0, 1, 32LL,
                                                        expert_load, stats, error_flag_of(c), 0);
   MS_LAUNCH_CHECK("flow_collect_kernel(verify)");
   return MAXSCORE_OK;
@@ -307,6 +310,8 @@ maxscore_status maxscore_create(maxscore_ctx** out, const maxscore_params* param
     return MAXSCORE_ERR_CUDA;
   }
   MS_CUDA(cudaFuncSetAttribute(gate_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGateSmemBytes));
+  MS_CUDA(cudaFuncSetAttribute(flow_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * kSweepThreads * kMaxE)));
+  MS_CUDA(cudaFuncSetAttribute(flow_collect_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * kSweepThreads * kMaxE)));
   MS_CUDA(cudaFuncSetAttribute(flow_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kP2SmemMax));
   MS_CUDA(cudaFuncSetAttribute(dispatch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDispatchSmem));
   MS_CUDA(cudaFuncSetAttribute(gate_bwd_dh_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDhSmemMax));

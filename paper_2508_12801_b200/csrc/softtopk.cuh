@@ -3,7 +3,10 @@
 // Level j (1-based) of Eq. 6 adds a softmax with temperature t over the entries that are not among
 // the j-1 largest (ties: lowest expert index).  A lane holds experts lane, lane+32, ... so every
 // global access of a warp is one contiguous row segment, and each level costs two shuffle
-// reductions (arg-max, sum).
+// reductions (arg-max, sum).  The exponentials are taken once, relative to the row maximum: a level's
+// softmax is z_i / (sum of z over its unmasked entries) whatever the reference point.  Only when a
+// level's own maximum lies so far below the row maximum that z would leave the normal fp32 range are
+// they recomputed relative to that level's maximum.
 #pragma once
 #include "common.cuh"
 
@@ -38,23 +41,28 @@ softtopk_fwd_kernel(const float* __restrict__ logits, float* __restrict__ scores
       a[j] = live[j] ? __ldg(row + e) : 0.f;
       y[j] = 0.f;
     }
+    float z[kEPL];
+    float ref = 0.f;                                  // reference point of the current z
     for (int level = 0; level < k; ++level) {
       float best = -INFINITY; int bidx = 0x7fffffff;
 #pragma unroll
       for (int j = 0; j < kEPL; ++j)
         if (live[j] && (a[j] > best || bidx == 0x7fffffff)) { best = a[j]; bidx = lane + 32 * j; }
       warp_argmax(best, bidx);
-      float z[kEPL], zs = 0.f;
+      if (level == 0 || (ref - best) > 60.f * t) {    // (re)base the exponentials on this level's maximum
+        ref = best;
 #pragma unroll
-      for (int j = 0; j < kEPL; ++j) {
-        z[j] = live[j] ? expf((a[j] - best) / t) : 0.f;
-        zs += z[j];
+        for (int j = 0; j < kEPL; ++j) z[j] = live[j] ? expf((a[j] - ref) / t) : 0.f;
       }
+      float zs = 0.f;
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j) zs += z[j];
       zs = warp_sum(zs);
+      const float inv = 1.f / zs;
 #pragma unroll
       for (int j = 0; j < kEPL; ++j) {
-        y[j] += z[j] / zs;
-        if (lane + 32 * j == bidx) live[j] = false;   // masked from the next level on
+        y[j] = fmaf(z[j], inv, y[j]);
+        if (lane + 32 * j == bidx) { live[j] = false; z[j] = 0.f; }   // masked from the next level on
       }
     }
     float* out = scores + (size_t)tok * E;
@@ -93,26 +101,31 @@ softtopk_bwd_kernel(const float* __restrict__ logits, const int32_t* __restrict_
       for (int j = 0; j < kEPL; ++j)
         if (lane + 32 * j == e) g[j] = gv;
     }
+    float z[kEPL];
+    float ref = 0.f;
+    const float inv_t = 1.f / t;
     for (int level = 0; level < k; ++level) {
       float best = -INFINITY; int bidx = 0x7fffffff;
 #pragma unroll
       for (int j = 0; j < kEPL; ++j)
         if (live[j] && (a[j] > best || bidx == 0x7fffffff)) { best = a[j]; bidx = lane + 32 * j; }
       warp_argmax(best, bidx);
-      float z[kEPL], zs = 0.f, gz = 0.f;
+      if (level == 0 || (ref - best) > 60.f * t) {
+        ref = best;
 #pragma unroll
-      for (int j = 0; j < kEPL; ++j) {
-        z[j] = live[j] ? expf((a[j] - best) / t) : 0.f;
-        zs += z[j];
-        gz += g[j] * z[j];
+        for (int j = 0; j < kEPL; ++j) z[j] = live[j] ? expf((a[j] - ref) / t) : 0.f;
       }
+      float zs = 0.f, gz = 0.f;
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j) { zs += z[j]; gz += g[j] * z[j]; }
       zs = warp_sum(zs);
       gz = warp_sum(gz);
-      const float gq = gz / zs;
+      const float inv = 1.f / zs;
+      const float gq = gz * inv;
 #pragma unroll
       for (int j = 0; j < kEPL; ++j) {
-        da[j] += (z[j] / zs) * (g[j] - gq) / t;
-        if (lane + 32 * j == bidx) live[j] = false;
+        da[j] = fmaf(z[j] * inv, (g[j] - gq) * inv_t, da[j]);
+        if (lane + 32 * j == bidx) { live[j] = false; z[j] = 0.f; }
       }
     }
     float* out = dlogits + (size_t)tok * E;
