@@ -579,35 +579,81 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
 // Only candidate tokens (gap <= theta) are in the graph.  A round stops BEFORE an augmentation whose
 // price update would spread the experts' price changes of this round by more than theta: up to that
 // point no token outside the list can have lost its top-k, so the state handed to the next collect
-// pass is consistent, and that pass only has to list more tokens.  The experts held by a candidate
-// live in expert_idx itself and are edited in place; ties are broken by the smallest token index, so
-// the result does not depend on the order of the candidate list.
+// pass is consistent, and that pass only has to list more tokens.
+//
+// D[e][f] (shared memory) is the cheapest move of one candidate token from e to f.  After a token
+// moves u -> v only row u is rebuilt; the rows of its other experts and of v are patched from the
+// token's own keys.  The experts of the first kHeldCache candidates are mirrored in shared memory
+// (expert_idx itself is edited in place as well); the list is sorted first, so ties are broken by
+// the smallest token index whatever order the collect pass appended the tokens in.
 constexpr int kP2Threads = 1024;
+constexpr int kHeldCache = 2048;
+constexpr int kSortMax = 16384;     // candidate lists up to this length are sorted (they fit in D's space)
 
 struct P2Shared {
   long long p[kMaxE + 1];        // potentials: prices of the experts, then Z
   long long p0[kMaxE + 1];       // potentials at the start of the round
-  long long dist[2][kMaxE + 1];
+  long long dist[2][kMaxE + 1];  // [0] current, [1] snapshot of the previous round
   int pred[kMaxE + 1];
+  unsigned char act[2][kMaxE + 4];   // nodes whose distance changed in the last round
   int imb[kMaxE + 1];            // + excess, - deficit
   int flow[kMaxE];               // units on expert -> sink
   int dirty[kMaxE];
   int path[kMaxE + 2];
   int npath, changed, who, target, stop, any_pos;
-  long long dt, spread_lo, spread_hi;
+  long long dt;
 };
 
 __global__ void __launch_bounds__(kP2Threads)
-flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_idx,
-                  const int32_t* __restrict__ cand, int T, int E, int k, int C, KeyGen g, int max_aug) {
+flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_idx, int32_t* cand, int T, int E,
+                  int k, int C, KeyGen g, int max_aug) {
   if (*(volatile int*)&st->converged) return;
   extern __shared__ __align__(16) unsigned char p2smem[];
-  long long* D = reinterpret_cast<long long*>(p2smem);                       // [E][E] raw arc costs
+  long long* D = reinterpret_cast<long long*>(p2smem);                              // [E][E] raw arc costs
+  unsigned char* held_s = reinterpret_cast<unsigned char*>(D + (size_t)E * (E | 1));       // [kHeldCache][kMaxK]
+  int* cand_s = reinterpret_cast<int*>(held_s + (size_t)kHeldCache * kMaxK);          // [kHeldCache]
   __shared__ P2Shared s;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = min(st->ncand, T);
   const int nZ = E;   // index of Z
+  const int ES = E | 1;   // odd row stride of D: a warp walking down a column hits different banks
   const long long theta = st->theta_used;
+  const long long arc_window = theta >= (kInf >> 2) ? kInf : 2 * theta;
+
+  // ---- sort the candidate list (in D's space, not yet in use) ----------------------------------------
+  if (n > 1 && n <= kSortMax && (size_t)n * 4 <= (size_t)E * (E | 1) * 8) {
+    int* buf = reinterpret_cast<int*>(D);
+    int npow = 1; while (npow < n) npow <<= 1;
+    if ((size_t)npow * 4 <= (size_t)E * (E | 1) * 8) {
+      for (int i = tid; i < npow; i += blockDim.x) buf[i] = i < n ? cand[i] : 0x7fffffff;
+      __syncthreads();
+      for (int size = 2; size <= npow; size <<= 1)
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+          for (int i = tid; i < npow; i += blockDim.x) {
+            const int j = i ^ stride;
+            if (j > i) {
+              const bool up = (i & size) == 0;
+              const int a = buf[i], b = buf[j];
+              if ((a > b) == up) { buf[i] = b; buf[j] = a; }
+            }
+          }
+          __syncthreads();
+        }
+      for (int i = tid; i < n; i += blockDim.x) cand[i] = buf[i];
+      __syncthreads();
+    }
+  }
+  const int nc = min(n, kHeldCache);
+  for (int i = tid; i < nc; i += blockDim.x) cand_s[i] = cand[i];
+  __syncthreads();
+  for (int i = tid; i < nc * k; i += blockDim.x) {
+    const int c = i / k, j = i - c * k;
+    held_s[c * kMaxK + j] = (unsigned char)expert_idx[(size_t)cand_s[c] * k + j];
+  }
+  auto tok_of = [&](int c) -> int { return c < nc ? cand_s[c] : cand[c]; };
+  auto held_of = [&](int c, int tok, int j) -> int {
+    return c < nc ? (int)held_s[c * kMaxK + j] : expert_idx[(size_t)tok * k + j];
+  };
 
   for (int e = tid; e < E; e += blockDim.x) {
     s.p[e] = st->p[e]; s.p0[e] = s.p[e];
@@ -624,18 +670,20 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
   __syncthreads();
 
   int naug = 0;
+  int bf_rounds = 0;
+  long long t_rebuild = 0, t_bf = 0, t_move = 0, t0 = clock64();   // phase timers (thread 0), diagnostics
   for (;;) {
     // ---- rebuild the rows of D marked dirty: D[e][f] = min over candidates in e, not in f ----------
-    for (int i = tid; i < E * E; i += blockDim.x)
-      if (s.dirty[i / E]) D[i] = kInf;
+    for (int i = tid; i < E * ES; i += blockDim.x)
+      if (s.dirty[i / ES]) D[i] = kInf;
     __syncthreads();
     for (int c = warp; c < n; c += kP2Threads / 32) {
-      const int tok = cand[c];
+      const int tok = tok_of(c);
       int h[kMaxK];
       bool any = false;
 #pragma unroll
       for (int j = 0; j < kMaxK; ++j) {
-        h[j] = j < k ? expert_idx[(size_t)tok * k + j] : -1;
+        h[j] = j < k ? held_of(c, tok, j) : -1;
         if (j < k) any |= (s.dirty[h[j]] != 0);
       }
       if (!any) continue;
@@ -647,10 +695,10 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
       for (int q = 0; q < kEPLf; ++q) {
         const int f = lane + 32 * q;
         key[q] = f < E ? make_key(g, __ldg(row + f), flat + f) : 0;
-        bool held = f >= E;
+        bool hd = f >= E;
 #pragma unroll
-        for (int j = 0; j < kMaxK; ++j) held |= (h[j] == f);
-        in[q] = held;
+        for (int j = 0; j < kMaxK; ++j) hd |= (h[j] == f);
+        in[q] = hd;
       }
 #pragma unroll
       for (int j = 0; j < kMaxK; ++j) {
@@ -661,10 +709,15 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
 #pragma unroll
         for (int q = 0; q < kEPLf; ++q) if ((e >> 5) == q) mine = key[q];
         const long long we = __shfl_sync(0xffffffffu, mine, e & 31);
+        // only moves whose reduced cost is within 2*theta can be used before this round ends
+        const long long pe = s.p[e];
 #pragma unroll
         for (int q = 0; q < kEPLf; ++q) {
           const int f = lane + 32 * q;
-          if (!in[q]) atomicMin(&D[e * E + f], we - key[q]);
+          if (!in[q]) {
+            const long long cst = we - key[q];
+            if (cst - pe + s.p[f] <= arc_window) atomicMin(&D[e * ES + f], cst);
+          }
         }
       }
     }
@@ -676,62 +729,79 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
       s.any_pos = any;
     }
     __syncthreads();
+    { const long long t1 = clock64(); t_rebuild += t1 - t0; t0 = t1; }
     if (!s.any_pos || naug >= max_aug) break;
 
-    // ---- Bellman-Ford from every node with excess, reduced costs rc = cost - p[u] + p[v] >= 0 --------
-    for (int v = tid; v <= E; v += blockDim.x) {
-      s.dist[0][v] = s.imb[v] > 0 ? 0 : kInf;
-      s.pred[v] = -1;
-    }
-    __syncthreads();
-    int cur = 0;
-    for (int round = 0; round <= E + 1; ++round) {
-      if (tid == 0) s.changed = 0;
-      __syncthreads();
-      for (int v = warp; v <= E; v += kP2Threads / 32) {
-        long long best = s.dist[cur][v]; int bu = -1;
-        for (int u = lane; u <= E; u += 32) {
-          const long long du = s.dist[cur][u];
-          if (du >= kInf || u == v) continue;
-          long long rc;
-          if (u < E && v < E) {
-            const long long c = D[u * E + v];
-            if (c >= kInf) continue;
-            rc = c - s.p[u] + s.p[v];
-          } else if (v == nZ) {          // expert u -> Z: one more unit on u -> sink
-            if (s.flow[u] >= C) continue;
-            rc = -s.p[u] + s.p[nZ];
-          } else {                       // Z -> expert v: one unit less on v -> sink
-            if (s.flow[v] <= 0) continue;
-            rc = -s.p[nZ] + s.p[v];
-          }
-          if (rc < 0) rc = 0;            // cannot happen while the potentials are valid
-          if (rc >= kArcLimit) continue;
-          const long long nd = du + rc;
-          if (nd < best || (nd == best && bu >= 0 && u < bu)) { best = nd; bu = u; }
-        }
+    // ---- Dijkstra from every node with excess (reduced costs rc = cost - p[u] + p[v] are >= 0) ---------
+    // One warp, nodes spread over its lanes; it stops when the first node with a deficit is settled:
+    // every node still open is at least that far away, which is all the price update needs to know.
+    if (warp == 0) {
+      constexpr int NQ = (kMaxE + 1 + 31) / 32;
+      long long d[NQ]; int pr[NQ]; bool open[NQ];
+#pragma unroll
+      for (int q = 0; q < NQ; ++q) {
+        const int v = lane + 32 * q;
+        open[q] = v <= E;
+        d[q] = (v <= E && s.imb[v] > 0) ? 0 : kInf;
+        pr[q] = -1;
+      }
+      int target = -1; long long dt = kInf;
+      for (int it = 0; it <= E; ++it) {
+        long long best = kInf; int bv = 0x7fffffff;
+#pragma unroll
+        for (int q = 0; q < NQ; ++q)
+          if (open[q] && d[q] < best) { best = d[q]; bv = lane + 32 * q; }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
           const long long ob = __shfl_xor_sync(0xffffffffu, best, o);
-          const int ou = __shfl_xor_sync(0xffffffffu, bu, o);
-          if (ob < best || (ob == best && ou >= 0 && (bu < 0 || ou < bu))) { best = ob; bu = ou; }
+          const int ov = __shfl_xor_sync(0xffffffffu, bv, o);
+          if (ob < best || (ob == best && ov < bv)) { best = ob; bv = ov; }
         }
-        if (lane == 0) {
-          s.dist[cur ^ 1][v] = best;
-          if (bu >= 0 && best < s.dist[cur][v]) { s.pred[v] = bu; s.changed = 1; }
+        if (best >= kInf) break;                       // nothing reachable is left
+        const int u = bv; const long long du = best;
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) if (lane + 32 * q == u) open[q] = false;
+        ++bf_rounds;
+        if (s.imb[u] < 0) { target = u; dt = du; break; }
+        const long long pu = s.p[u];
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+          const int v = lane + 32 * q;
+          if (!open[q]) continue;
+          long long rc;
+          if (u < E && v < E) {
+            const long long c = D[u * ES + v];
+            if (c >= kInf) continue;
+            rc = c - pu + s.p[v];
+          } else if (v == nZ) {          // expert u -> Z: one more unit on u -> sink
+            if (s.flow[u] >= C) continue;
+            rc = -pu + s.p[nZ];
+          } else {                       // Z -> expert v: one unit less on v -> sink
+            if (s.flow[v] <= 0) continue;
+            rc = -pu + s.p[v];
+          }
+          if (rc < 0) rc = 0;            // cannot happen while the potentials are valid
+          if (rc >= kArcLimit) continue;
+          if (du + rc < d[q]) { d[q] = du + rc; pr[q] = u; }
         }
       }
-      __syncthreads();
-      cur ^= 1;
-      if (!s.changed) break;
-      __syncthreads();
+#pragma unroll
+      for (int q = 0; q < NQ; ++q) {
+        const int v = lane + 32 * q;
+        if (v <= E) {
+          // settled nodes keep their distance; open ones are at least dt away
+          s.dist[0][v] = open[q] ? kInf : d[q];
+          s.pred[v] = pr[q];
+        }
+      }
+      if (lane == 0) { s.target = target; s.dt = dt; }
     }
+    __syncthreads();
+    const int cur = 0;
     // ---- nearest node with a deficit; would the price update stay within theta? -----------------------
     if (tid == 0) {
-      int t = -1; long long dt = kInf;
-      for (int v = 0; v <= E; ++v)
-        if (s.imb[v] < 0 && s.dist[cur][v] < dt) { dt = s.dist[cur][v]; t = v; }
-      s.target = t; s.dt = dt; s.npath = 0;
+      const int t = s.target; const long long dt = s.dt;
+      s.npath = 0;
       if (t >= 0) {
         int len = 0, v = t;
         while (v >= 0 && len <= E + 1) { s.path[len++] = v; v = s.pred[v]; }
@@ -746,6 +816,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
       }
     }
     __syncthreads();
+    { const long long t1 = clock64(); t_bf += t1 - t0; t0 = t1; }
     if (s.target < 0) break;        // -1: no augmenting path inside the candidate graph
     for (int v = tid; v <= E; v += blockDim.x) {
       const long long d = s.dist[cur][v];
@@ -758,33 +829,83 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
       if (u < E && v < E) {
         if (tid == 0) s.who = 0x7fffffff;
         __syncthreads();
-        const long long want = D[u * E + v];
+        const long long want = D[u * ES + v];
         for (int c = tid; c < n; c += blockDim.x) {
-          const int tok = cand[c];
+          const int tok = tok_of(c);
           bool hu = false, hv = false;
           for (int j = 0; j < k; ++j) {
-            const int e = expert_idx[(size_t)tok * k + j];
+            const int e = held_of(c, tok, j);
             hu |= (e == u); hv |= (e == v);
           }
           if (!hu || hv) continue;
           const uint32_t flat = (uint32_t)tok * (uint32_t)E;
           const long long cost = make_key(g, __ldg(M + (size_t)tok * E + u), flat + u) -
                                  make_key(g, __ldg(M + (size_t)tok * E + v), flat + v);
-          if (cost == want) atomicMin(&s.who, tok);
+          if (cost == want) atomicMin(&s.who, c);      // the list is sorted: smallest c = smallest token
         }
         __syncthreads();
         if (s.who == 0x7fffffff) {   // internal inconsistency: stop, the verify pass will report it
           if (tid == 0) { atomicOr(&st->status, 4u); s.stop = 1; }
-        } else if (tid == 0) {
-          int32_t* h = expert_idx + (size_t)s.who * k;
-          for (int j = 0; j < k; ++j) {
-            s.dirty[h[j]] = 1;
-            if (h[j] == u) h[j] = v;
+          __syncthreads();
+          break;
+        }
+        if (warp == 0) {
+          // the token leaves u for v: patch D from its own keys instead of rebuilding every row it touches
+          const int c = s.who, tok = tok_of(c);
+          int h[kMaxK];
+#pragma unroll
+          for (int j = 0; j < kMaxK; ++j) {
+            h[j] = j < k ? held_of(c, tok, j) : -1;
+            if (h[j] == u) h[j] = v;                   // experts after the move
           }
-          s.dirty[v] = 1;
+          const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+          long long key[kEPLf]; bool in[kEPLf];
+#pragma unroll
+          for (int q = 0; q < kEPLf; ++q) {
+            const int f = lane + 32 * q;
+            key[q] = f < E ? make_key(g, __ldg(M + (size_t)tok * E + f), flat + f) : 0;
+            bool hd = f >= E;
+#pragma unroll
+            for (int j = 0; j < kMaxK; ++j) hd |= (h[j] == f);
+            in[q] = hd;
+          }
+          auto key_of = [&](int e) -> long long {
+            long long mine = 0;
+#pragma unroll
+            for (int q = 0; q < kEPLf; ++q) if ((e >> 5) == q) mine = key[q];
+            return __shfl_sync(0xffffffffu, mine, e & 31);
+          };
+          const long long ku = key_of(u), kv = key_of(v);
+          // row v gains the token: new moves v -> f for every expert f it does not hold
+#pragma unroll
+          for (int q = 0; q < kEPLf; ++q) {
+            const int f = lane + 32 * q;
+            if (!in[q]) { const long long cst = kv - key[q]; if (cst < D[v * ES + f]) D[v * ES + f] = cst; }
+          }
+          // its other experts g: g -> u is a new move; g -> v is gone, and if it was the cheapest one
+          // row g has to be rebuilt
+#pragma unroll
+          for (int j = 0; j < kMaxK; ++j) {
+            if (j >= k || h[j] == v) continue;
+            const int gg = h[j];
+            const long long kg = key_of(gg);
+            if (lane == 0) {
+              if (kg - ku < D[gg * ES + u]) D[gg * ES + u] = kg - ku;
+              if (D[gg * ES + v] == kg - kv) s.dirty[gg] = 1;
+            }
+          }
+          if (lane == 0) {
+            s.dirty[u] = 1;                            // row u lost the token
+            for (int j = 0; j < k; ++j) {
+              const int e = held_of(c, tok, j);
+              if (e == u) {
+                if (c < nc) held_s[c * kMaxK + j] = (unsigned char)v;
+                expert_idx[(size_t)tok * k + j] = v;
+              }
+            }
+          }
         }
         __syncthreads();
-        if (s.stop) break;
       } else if (tid == 0) {
         if (v == nZ) s.flow[u] += 1; else s.flow[v] -= 1;
       }
@@ -793,6 +914,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
     if (tid == 0) { s.imb[s.path[s.npath - 1]] -= 1; s.imb[s.target] += 1; }
     ++naug;
     __syncthreads();
+    { const long long t1 = clock64(); t_move += t1 - t0; t0 = t1; }
   }
   // ---- write back ---------------------------------------------------------------------------------
   __syncthreads();
@@ -800,7 +922,10 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
     long long pe = s.p[e] - s.p[nZ];
     st->p[e] = pe < 0 ? 0 : pe;     // only an expert that holds nothing can come out negative
   }
-  if (tid == 0) { st->naug += naug; st->ncand_last = n; st->ncand = 0; }
+  if (tid == 0) {
+    st->naug += naug; st->ncand_last = n; st->ncand = 0;
+    st->trace[44] = (int)(t_rebuild >> 10); st->trace[45] = (int)(t_bf >> 10); st->trace[46] = (int)(t_move >> 10); st->trace[47] = bf_rounds;   // kilo-cycles
+  }
 }
 
 }  // namespace msr

@@ -32,6 +32,9 @@ def main():
         st = ms.read_stats(stats)
         print(f"assign T={T} E={E} k={k}: {e0.elapsed_time(e1):.3f} ms status={st.status} sweeps={st.sweeps} "
               f"aug={st.augmentations} rounds={st.rounds} cand={st.candidates}")
+        base = (ctx.workspace.data_ptr() + 255) // 256 * 256 - ctx.workspace.data_ptr()
+        tr = ctx.workspace[base:base + 256].cpu().numpy().view("int32")
+        print("  exact-phase kilo-cycles (rebuild, path search, moves), path-search rounds, of the last round run:", tr[44:48].tolist())
 
 
 if __name__ == "__main__":
