@@ -600,7 +600,7 @@ struct P2Shared {
   int flow[kMaxE];               // units on expert -> sink
   int dirty[kMaxE];
   int path[kMaxE + 2];
-  int npath, changed, who, target, stop, any_pos;
+  int npath, changed, who, target, stop, any_pos, qn;
   long long dt;
 };
 
@@ -612,6 +612,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
   long long* D = reinterpret_cast<long long*>(p2smem);                              // [E][E] raw arc costs
   unsigned char* held_s = reinterpret_cast<unsigned char*>(D + (size_t)E * (E | 1));       // [kHeldCache][kMaxK]
   int* cand_s = reinterpret_cast<int*>(held_s + (size_t)kHeldCache * kMaxK);          // [kHeldCache]
+  int* queue_s = cand_s + kHeldCache;                                                // [kHeldCache]
   __shared__ P2Shared s;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = min(st->ncand, T);
@@ -677,7 +678,19 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
     for (int i = tid; i < E * ES; i += blockDim.x)
       if (s.dirty[i / ES]) D[i] = kInf;
     __syncthreads();
-    for (int c = warp; c < n; c += kP2Threads / 32) {
+    // cached candidates that hold a dirty row are queued first (one thread each, shared memory only);
+    // the warps then work through the queue and through the uncached tail of the list
+    if (tid == 0) s.qn = 0;
+    __syncthreads();
+    for (int c = tid; c < nc; c += blockDim.x) {
+      bool any = false;
+      for (int j = 0; j < k; ++j) any |= (s.dirty[held_s[c * kMaxK + j]] != 0);
+      if (any) queue_s[atomicAdd(&s.qn, 1)] = c;
+    }
+    __syncthreads();
+    const int work = s.qn + (n - nc);
+    for (int i = warp; i < work; i += kP2Threads / 32) {
+      const int c = i < s.qn ? queue_s[i] : nc + (i - s.qn);
       const int tok = tok_of(c);
       int h[kMaxK];
       bool any = false;
