@@ -713,6 +713,19 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
         for (int j = 0; j < kMaxK; ++j) hd |= (h[j] == f);
         in[q] = hd;
       }
+      // best value among the experts the token does not hold: a held expert further than the arc
+      // window above it has no usable move at all
+      long long vmax = -kInf;
+#pragma unroll
+      for (int q = 0; q < kEPLf; ++q) {
+        const int f = lane + 32 * q;
+        if (!in[q]) { const long long val = key[q] - s.p[f]; vmax = val > vmax ? val : vmax; }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const long long ov = __shfl_xor_sync(0xffffffffu, vmax, o);
+        vmax = ov > vmax ? ov : vmax;
+      }
 #pragma unroll
       for (int j = 0; j < kMaxK; ++j) {
         if (j >= k) continue;
@@ -724,6 +737,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
         const long long we = __shfl_sync(0xffffffffu, mine, e & 31);
         // only moves whose reduced cost is within 2*theta can be used before this round ends
         const long long pe = s.p[e];
+        if (arc_window < kInf && (we - pe) - vmax > arc_window) continue;
 #pragma unroll
         for (int q = 0; q < kEPLf; ++q) {
           const int f = lane + 32 * q;
@@ -759,6 +773,33 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
         pr[q] = -1;
       }
       int target = -1; long long dt = kInf;
+      // all nodes with excess start at distance 0: settle them together and relax their arcs in one go
+#pragma unroll
+      for (int q = 0; q < NQ; ++q) if (open[q] && d[q] == 0) open[q] = false;
+      for (int u = 0; u <= E; ++u) {
+        if (s.imb[u] <= 0) continue;
+        const long long pu = s.p[u];
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+          const int v = lane + 32 * q;
+          if (!open[q]) continue;
+          long long rc;
+          if (u < E && v < E) {
+            const long long c = D[u * ES + v];
+            if (c >= kInf) continue;
+            rc = c - pu + s.p[v];
+          } else if (v == nZ) {
+            if (s.flow[u] >= C) continue;
+            rc = -pu + s.p[nZ];
+          } else {
+            if (s.flow[v] <= 0) continue;
+            rc = -pu + s.p[v];
+          }
+          if (rc < 0) rc = 0;
+          if (rc >= kArcLimit) continue;
+          if (rc < d[q]) { d[q] = rc; pr[q] = u; }
+        }
+      }
       for (int it = 0; it <= E; ++it) {
         long long best = kInf; int bv = 0x7fffffff;
 #pragma unroll

@@ -200,7 +200,7 @@ maxscore_status launch_softtopk_fwd(maxscore_ctx* c, const float* logits, float*
   return MAXSCORE_OK;
 }
 
-constexpr int kSweeps = 40, kRounds = 4, kDefaultAug = 4096;
+constexpr int kSweeps = 24, kRounds = 4, kDefaultAug = 4096;
 
 maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_idx, int32_t* expert_load,
                               maxscore_stats* stats, cudaStream_t st) {
@@ -223,7 +223,7 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   const int blocks = (p.T + kSweepThreads - 1) / kSweepThreads;
   const size_t tile_smem = sizeof(float) * (size_t)kSweepThreads * p.E;
   for (int s = 0; s < n_sweeps; ++s) {
-    flow_sweep_kernel<<<blocks, kSweepThreads, tile_smem, st>>>(M, fs, p.T, p.E, p.k, c->C, g, n_sweeps, 2);
+    flow_sweep_kernel<<<blocks, kSweepThreads, tile_smem, st>>>(M, fs, p.T, p.E, p.k, c->C, g, n_sweeps, 1);
     MS_LAUNCH_CHECK("flow_sweep_kernel");
   }
   const size_t p2smem = sizeof(long long) * (size_t)p.E * (p.E | 1) + (size_t)kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache;
