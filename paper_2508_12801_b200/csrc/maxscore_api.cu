@@ -415,7 +415,7 @@ maxscore_status maxscore_combine(maxscore_ctx* c, const void* src, const int32_t
   if (!c || !src || !expert_idx || !slot_idx || !dst) return MAXSCORE_ERR_INVALID_ARG;
   if (!aligned16(src) || !aligned16(dst)) return MAXSCORE_ERR_INVALID_ARG;
   const maxscore_params& p = c->p;
-  int blocks = p.T < c->sm_count * 8 ? p.T : c->sm_count * 8;
+  int blocks = (p.T + 7) / 8 < c->sm_count * 8 ? (p.T + 7) / 8 : c->sm_count * 8;   // a warp per token
   if (p.io_dtype == MAXSCORE_BF16)
     combine_kernel<__nv_bfloat16><<<blocks, 256, 0, (cudaStream_t)stream>>>(
         (const __nv_bfloat16*)src, expert_idx, slot_idx, gate_w, (__nv_bfloat16*)dst, p.T, p.d_model, p.k, c->C, accumulate);

@@ -159,43 +159,53 @@ zero_padding_kernel(const int32_t* __restrict__ slot_token, char* __restrict__ d
 
 // ---------------------------------------------------------------------------------------------
 // Combine: dst[i, :] = sum_c w[i, c] * src[e_c, slot_c, :] in fp32, ascending c, rounded once.
-// One CTA per token at a time; a thread owns 16-byte column groups and keeps the k row loads of a
-// group in flight together.
+// One warp per token: lanes < k fetch the token's slots and weights and share them by shuffle, so no
+// block barrier sits between a token's index loads and its row loads; a lane owns 16-byte column
+// groups and keeps the k row loads of a group in flight together.
 template <typename T>
 __global__ void __launch_bounds__(256)
 combine_kernel(const T* __restrict__ src, const int32_t* __restrict__ expert_idx,
                const int32_t* __restrict__ slot_idx, const float* __restrict__ gate_w,
                T* __restrict__ dst, int Tn, int d, int k, int C, int accumulate) {
   constexpr int N = Vec16<T>::N;
-  __shared__ long long rowoff[kMaxK];
-  __shared__ float wgt[kMaxK];
   const int nvec = d / N;
-  for (int tok = blockIdx.x; tok < Tn; tok += gridDim.x) {
-    __syncthreads();
-    if (threadIdx.x < k) {
-      int e = __ldg(expert_idx + (size_t)tok * k + threadIdx.x);
-      int sl = __ldg(slot_idx + (size_t)tok * k + threadIdx.x);
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  for (int tok = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; tok < Tn; tok += warps) {
+    long long my_off = 0; float my_w = 0.f;
+    if (lane < k) {
+      const int e = __ldg(expert_idx + (size_t)tok * k + lane);
+      const int sl = __ldg(slot_idx + (size_t)tok * k + lane);
       const bool valid = e >= 0 && sl >= 0 && sl < C;   // a malformed entry contributes nothing
-      rowoff[threadIdx.x] = valid ? ((long long)e * C + sl) * (long long)d : 0;
-      wgt[threadIdx.x] = !valid ? 0.f : gate_w ? __ldg(gate_w + (size_t)tok * k + threadIdx.x) : 1.f;
+      my_off = valid ? ((long long)e * C + sl) * (long long)d : 0;
+      my_w = !valid ? 0.f : gate_w ? __ldg(gate_w + (size_t)tok * k + lane) : 1.f;
     }
-    __syncthreads();
-    for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
-      float x[kMaxK][N];
+    long long rowoff[kMaxK]; float wgt[kMaxK];
 #pragma unroll
-      for (int c = 0; c < kMaxK; ++c)
-        if (c < k) Vec16<T>::load(src + rowoff[c] + (size_t)v * N, x[c]);
+    for (int c = 0; c < kMaxK; ++c) {
+      rowoff[c] = __shfl_sync(0xffffffffu, my_off, c);
+      wgt[c] = __shfl_sync(0xffffffffu, my_w, c);
+    }
+    for (int v = lane; v < nvec; v += 32) {
       float acc[N];
 #pragma unroll
       for (int j = 0; j < N; ++j) acc[j] = 0.f;
       if (accumulate) Vec16<T>::load(dst + (size_t)tok * d + (size_t)v * N, acc);
 #pragma unroll
-      for (int c = 0; c < kMaxK; ++c)
-        if (c < k) {
-          const float w = wgt[c];
+      for (int c0 = 0; c0 < kMaxK; c0 += 4) {           // four rows in flight at a time keeps registers low
+        if (c0 >= k) break;
+        float x[4][N];
 #pragma unroll
-          for (int j = 0; j < N; ++j) acc[j] = fmaf(w, x[c][j], acc[j]);
-        }
+        for (int c = 0; c < 4; ++c)
+          if (c0 + c < k) Vec16<T>::load(src + rowoff[c0 + c] + (size_t)v * N, x[c]);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (c0 + c < k) {
+            const float w = wgt[c0 + c];
+#pragma unroll
+            for (int j = 0; j < N; ++j) acc[j] = fmaf(w, x[c][j], acc[j]);
+          }
+      }
       Vec16<T>::store(dst + (size_t)tok * d + (size_t)v * N, acc);
     }
   }
