@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 
 METRIC = "routed tokens/s per MoE layer (gate->flow->dispatch) on 1 B200; % of roofline"
 UNIT = "tokens/s"
-SWEEPS, ROUNDS = 40, 4
+SWEEPS, ROUNDS = 24, 4
 
 
 def launches_per_step():
@@ -36,7 +36,7 @@ def launches_per_step():
     assign = 1 + SWEEPS + 2 * ROUNDS + 1
     route_fwd = gate + 1 + assign + 2 + 1          # + SoftTopk + index (count, fill) + gate_w gather
     dispatch, combine = 2, 1
-    route_bwd = 2 + 1 + 2                          # combine-bwd (+padding), SoftTopk-bwd, gate-bwd (dW, dH)
+    route_bwd = 2 + 1 + 5                          # combine-bwd (+padding), SoftTopk-bwd, gate-bwd (split, W_g, dH, dW, reduce)
     return route_fwd + dispatch + combine + route_bwd + combine   # last combine = dispatch backward
 
 

@@ -293,7 +293,7 @@ constexpr int kSweepThreads = 128;
 
 __global__ void __launch_bounds__(kSweepThreads)
 flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int k, int C, KeyGen g,
-                  int n_sweeps, int decay_every) {
+                  int n_sweeps, int decay_every, int staged) {
   if (*(volatile int*)&st->p1_done) return;
   __shared__ long long sp[kMaxE];
   __shared__ int sload[kMaxE];
@@ -309,12 +309,12 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
   }
   extern __shared__ __align__(16) float sweep_tile[];
   const int tok0 = blockIdx.x * blockDim.x;
-  stage_rows(M, sweep_tile, tok0, min((int)blockDim.x, T - tok0), E);
+  if (staged) stage_rows(M, sweep_tile, tok0, min((int)blockDim.x, T - tok0), E);
   __syncthreads();
   const int tok = tok0 + threadIdx.x;
   if (tok < T) {
     long long v[kTopN]; int id[kTopN];
-    const float* row = sweep_tile + (size_t)threadIdx.x * E;
+    const float* row = staged ? sweep_tile + (size_t)threadIdx.x * E : M + (size_t)tok * E;
     const uint32_t flat = (uint32_t)tok * (uint32_t)E;
     // rotated start: conflict-free shared-memory reads.  The sweeps are a heuristic, so the cheap
     // (fp32-filtered) selection is enough here.
@@ -363,6 +363,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
   for (int e = threadIdx.x; e < E; e += blockDim.x)
     if (sload[e]) atomicAdd(&st->load[e], sload[e]);
 
+  const long long tail_t0 = clock64();
   if (!last_block_arrives(&st->ticket)) return;
   // ---- last CTA: move the prices -------------------------------------------------------------
   __shared__ int s_imb;
@@ -413,7 +414,8 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
   for (int e = threadIdx.x; e < E; e += blockDim.x) st->p[e] = sp[e] - pmin;
   __syncthreads();
   if (threadIdx.x == 0) {
-    if (sweep <= 48) st->trace[sweep - 1] = s_imb;
+    if (sweep <= 40) st->trace[sweep - 1] = s_imb;
+    st->trace[40] = (int)((clock64() - tail_t0) >> 4);   // cycles/16 the last CTA spent on the price update
     st->sweep = sweep;
     if (sweep % decay_every == 0) { long long ne = eps >> 1; st->eps = ne < st->eps_min ? st->eps_min : ne; }
     st->ticket = 0;

@@ -222,8 +222,10 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   MS_LAUNCH_CHECK("flow_init_kernel");
   const int blocks = (p.T + kSweepThreads - 1) / kSweepThreads;
   const size_t tile_smem = sizeof(float) * (size_t)kSweepThreads * p.E;
+  // measured on B200: reading the rows straight from L2 beats staging them (more CTAs per SM)
+  const int sweep_staged = 0;
   for (int s = 0; s < n_sweeps; ++s) {
-    flow_sweep_kernel<<<blocks, kSweepThreads, tile_smem, st>>>(M, fs, p.T, p.E, p.k, c->C, g, n_sweeps, 1);
+    flow_sweep_kernel<<<blocks, kSweepThreads, sweep_staged ? tile_smem : 0, st>>>(M, fs, p.T, p.E, p.k, c->C, g, n_sweeps, 1, sweep_staged);
     MS_LAUNCH_CHECK("flow_sweep_kernel");
   }
   const size_t p2smem = sizeof(long long) * (size_t)p.E * (p.E | 1) + (size_t)kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache;
