@@ -191,21 +191,20 @@ combine_kernel(const T* __restrict__ src, const int32_t* __restrict__ expert_idx
 #pragma unroll
       for (int j = 0; j < N; ++j) acc[j] = 0.f;
       if (accumulate) Vec16<T>::load(dst + (size_t)tok * d + (size_t)v * N, acc);
+      // all k row loads are issued before any is used; they stay packed (4 registers each) until then
+      uint4 raw[kMaxK];
 #pragma unroll
-      for (int c0 = 0; c0 < kMaxK; c0 += 4) {           // four rows in flight at a time keeps registers low
-        if (c0 >= k) break;
-        float x[4][N];
+      for (int c = 0; c < kMaxK; ++c)
+        if (c < k) raw[c] = ldg16(src + rowoff[c] + (size_t)v * N);
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-          if (c0 + c < k) Vec16<T>::load(src + rowoff[c0 + c] + (size_t)v * N, x[c]);
+      for (int c = 0; c < kMaxK; ++c)
+        if (c < k) {
+          float x[N];
+          Vec16<T>::unpack(raw[c], x);
+          const float w = wgt[c];
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-          if (c0 + c < k) {
-            const float w = wgt[c0 + c];
-#pragma unroll
-            for (int j = 0; j < N; ++j) acc[j] = fmaf(w, x[c][j], acc[j]);
-          }
-      }
+          for (int j = 0; j < N; ++j) acc[j] = fmaf(w, x[j], acc[j]);
+        }
       Vec16<T>::store(dst + (size_t)tok * d + (size_t)v * N, acc);
     }
   }
@@ -241,17 +240,18 @@ combine_bwd_kernel(const T* __restrict__ dY, const T* __restrict__ yexp,
     for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
       float g[N];
       Vec16<T>::load(dY + (size_t)tok * d + (size_t)v * N, g);
-      float y[kMaxK][N];
+      uint4 raw[kMaxK];                                  // the k row loads stay packed until they are used
 #pragma unroll
       for (int c = 0; c < kMaxK; ++c)
-        if (c < k && rowoff[c] >= 0) Vec16<T>::load(yexp + rowoff[c] + (size_t)v * N, y[c]);
+        if (c < k && rowoff[c] >= 0) raw[c] = ldg16(yexp + rowoff[c] + (size_t)v * N);
 #pragma unroll
       for (int c = 0; c < kMaxK; ++c)
         if (c < k && rowoff[c] >= 0) {
-          float o[N];
+          float y[N], o[N];
+          Vec16<T>::unpack(raw[c], y);
           const float w = wgt[c];
 #pragma unroll
-          for (int j = 0; j < N; ++j) { dot[c] = fmaf(g[j], y[c][j], dot[c]); o[j] = w * g[j]; }
+          for (int j = 0; j < N; ++j) { dot[c] = fmaf(g[j], y[j], dot[c]); o[j] = w * g[j]; }
           Vec16<T>::store(dyexp + rowoff[c] + (size_t)v * N, o);
         }
     }
