@@ -157,12 +157,25 @@ __device__ __forceinline__ void select_top(const float* row, const long long* sp
 #pragma unroll
   for (int j = 0; j < N; ++j) pk[j] = -INFINITY;
   int e = start;
-  for (int jj = 0; jj < E; ++jj) {
-    const float vf = approx_key(g, row[e]) - (spf ? spf[e] : 0.f);
-    float x = __uint_as_float((__float_as_uint(vf) & ~127u) | (unsigned)e);
+  auto feed = [&](float val, int ee) {
+    const float vf = approx_key(g, val) - (spf ? spf[ee] : 0.f);
+    float x = __uint_as_float((__float_as_uint(vf) & ~127u) | (unsigned)ee);
 #pragma unroll
     for (int j = 0; j < N; ++j) { const float hi = fmaxf(pk[j], x); x = fminf(pk[j], x); pk[j] = hi; }
-    if (++e == E) e = 0;
+  };
+  if (start < 0) {
+    // row in global memory: 16-byte loads, so that each 32-byte sector is fetched by two adjacent
+    // instructions instead of eight that the L1 may not keep apart
+    for (int e4 = 0; e4 < E; e4 += 4) {
+      const float4 x4 = __ldg(reinterpret_cast<const float4*>(row + e4));
+      feed(x4.x, e4); feed(x4.y, e4 + 1); feed(x4.z, e4 + 2); feed(x4.w, e4 + 3);
+    }
+    start = 0;
+  } else {
+    for (int jj = 0; jj < E; ++jj) {
+      feed(row[e], e);
+      if (++e == E) e = 0;
+    }
   }
 #pragma unroll
   for (int j = 0; j < N; ++j) {
@@ -318,7 +331,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
     const uint32_t flat = (uint32_t)tok * (uint32_t)E;
     // rotated start: conflict-free shared-memory reads.  The sweeps are a heuristic, so the cheap
     // (fp32-filtered) selection is enough here.
-    select_top(row, sp, spf, g, flat, E, threadIdx.x % E, false, v, id);
+    select_top(row, sp, spf, g, flat, E, staged ? (int)(threadIdx.x % E) : ((E & 3) == 0 ? -1 : 0), false, v, id);
     const bool has_alt = E > k;
     long long vk = -kInf, vk1 = -kInf;                // k-th value and best alternative
 #pragma unroll
@@ -590,6 +603,7 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
 // the smallest token index whatever order the collect pass appended the tokens in.
 constexpr int kP2Threads = 1024;
 constexpr int kHeldCache = 2048;
+constexpr int kMaxFix = 48;
 constexpr int kSortMax = 16384;     // candidate lists up to this length are sorted (they fit in D's space)
 
 struct P2Shared {
@@ -602,7 +616,8 @@ struct P2Shared {
   int flow[kMaxE];               // units on expert -> sink
   int dirty[kMaxE];
   int path[kMaxE + 2];
-  int npath, changed, who, target, stop, any_pos, qn;
+  int npath, changed, who, target, stop, any_pos, qn, nfix;
+  int fix_e[kMaxFix], fix_f[kMaxFix];   // stale D entries to recompute after a move
   long long dt;
 };
 
@@ -673,7 +688,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
   __syncthreads();
 
   int naug = 0;
-  int bf_rounds = 0;
+  int bf_rounds = 0; long long q_total = 0, t_first = 0;
   long long t_rebuild = 0, t_bf = 0, t_move = 0, t0 = clock64();   // phase timers (thread 0), diagnostics
   for (;;) {
     // ---- rebuild the rows of D marked dirty: D[e][f] = min over candidates in e, not in f ----------
@@ -691,6 +706,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
     }
     __syncthreads();
     const int work = s.qn + (n - nc);
+    q_total += work; if (naug == 0 && t_first == 0) t_first = -1;
     for (int i = warp; i < work; i += kP2Threads / 32) {
       const int c = i < s.qn ? queue_s[i] : nc + (i - s.qn);
       const int tok = tok_of(c);
@@ -758,7 +774,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
       s.any_pos = any;
     }
     __syncthreads();
-    { const long long t1 = clock64(); t_rebuild += t1 - t0; t0 = t1; }
+    { const long long t1 = clock64(); t_rebuild += t1 - t0; if (t_first == -1) t_first = t1 - t0; t0 = t1; }
     if (!s.any_pos || naug >= max_aug) break;
 
     // ---- Dijkstra from every node with excess (reduced costs rc = cost - p[u] + p[v] are >= 0) ---------
@@ -936,22 +952,46 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
 #pragma unroll
           for (int q = 0; q < kEPLf; ++q) {
             const int f = lane + 32 * q;
-            if (!in[q]) { const long long cst = kv - key[q]; if (cst < D[v * ES + f]) D[v * ES + f] = cst; }
+            if (!in[q]) {
+              const long long cst = kv - key[q];
+              if (cst - s.p[v] + s.p[f] <= arc_window && cst < D[v * ES + f]) D[v * ES + f] = cst;
+            }
           }
-          // its other experts g: g -> u is a new move; g -> v is gone, and if it was the cheapest one
-          // row g has to be rebuilt
+          // D entries whose cheapest move was this token's become stale: (u, f) for the experts f it
+          // offered from u, and (g, v) for its other experts g.  They are listed and recomputed below
+          // from the candidates that hold the row's expert; a full row rebuild is the fallback.
+          if (lane == 0) s.nfix = 0;
+          __syncwarp();
+#pragma unroll
+          for (int q = 0; q < kEPLf; ++q) {
+            const int f = lane + 32 * q;
+            // before the move the token held u and not f (f != v is covered by in[], v itself is the used arc)
+            const bool was_out = f < E && f != u && (!in[q] || f == v);
+            if (was_out && D[u * ES + f] == ku - key[q]) {
+              const int slot = atomicAdd(&s.nfix, 1);
+              if (slot < kMaxFix) { s.fix_e[slot] = u; s.fix_f[slot] = f; }
+            }
+          }
 #pragma unroll
           for (int j = 0; j < kMaxK; ++j) {
             if (j >= k || h[j] == v) continue;
             const int gg = h[j];
             const long long kg = key_of(gg);
             if (lane == 0) {
-              if (kg - ku < D[gg * ES + u]) D[gg * ES + u] = kg - ku;
-              if (D[gg * ES + v] == kg - kv) s.dirty[gg] = 1;
+              if (kg - ku - s.p[gg] + s.p[u] <= arc_window && kg - ku < D[gg * ES + u]) D[gg * ES + u] = kg - ku;   // g -> u is a new move
+              if (D[gg * ES + v] == kg - kv) {                            // g -> v is gone
+                const int slot = atomicAdd(&s.nfix, 1);
+                if (slot < kMaxFix) { s.fix_e[slot] = gg; s.fix_f[slot] = v; }
+              }
             }
           }
+          __syncwarp();
           if (lane == 0) {
-            s.dirty[u] = 1;                            // row u lost the token
+            if (s.nfix > kMaxFix) {                    // too many: rebuild the rows instead
+              s.dirty[u] = 1;
+              for (int j = 0; j < k; ++j) if (h[j] != v) s.dirty[h[j]] = 1;
+              s.nfix = 0;
+            }
             for (int j = 0; j < k; ++j) {
               const int e = held_of(c, tok, j);
               if (e == u) {
@@ -960,8 +1000,31 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
               }
             }
           }
+          __syncwarp();
+          for (int i = lane; i < s.nfix; i += 32) D[s.fix_e[i] * ES + s.fix_f[i]] = kInf;
         }
         __syncthreads();
+        if (s.nfix > 0) {
+          // one thread per candidate: recompute the listed entries from the tokens that hold the row
+          for (int c = tid; c < n; c += blockDim.x) {
+            const int tok = tok_of(c);
+            int h[kMaxK];
+#pragma unroll
+            for (int j = 0; j < kMaxK; ++j) h[j] = j < k ? held_of(c, tok, j) : -1;
+            const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+            for (int i = 0; i < s.nfix; ++i) {
+              const int e = s.fix_e[i], f = s.fix_f[i];
+              bool he = false, hf = false;
+#pragma unroll
+              for (int j = 0; j < kMaxK; ++j) { he |= (h[j] == e); hf |= (h[j] == f); }
+              if (!he || hf) continue;
+              const long long cst = make_key(g, __ldg(M + (size_t)tok * E + e), flat + e) -
+                                    make_key(g, __ldg(M + (size_t)tok * E + f), flat + f);
+              if (cst - s.p[e] + s.p[f] <= arc_window) atomicMin(&D[e * ES + f], cst);
+            }
+          }
+          __syncthreads();
+        }
       } else if (tid == 0) {
         if (v == nZ) s.flow[u] += 1; else s.flow[v] -= 1;
       }
@@ -980,7 +1043,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
   }
   if (tid == 0) {
     st->naug += naug; st->ncand_last = n; st->ncand = 0;
-    st->trace[44] = (int)(t_rebuild >> 10); st->trace[45] = (int)(t_bf >> 10); st->trace[46] = (int)(t_move >> 10); st->trace[47] = bf_rounds;   // kilo-cycles
+    st->trace[44] = (int)(t_rebuild >> 10); st->trace[45] = (int)(t_bf >> 10); st->trace[46] = (int)(t_move >> 10); st->trace[47] = bf_rounds; st->trace[41] = (int)q_total; st->trace[42] = (int)(t_first >> 10);   // kilo-cycles
   }
 }
 
