@@ -604,6 +604,7 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
 constexpr int kP2Threads = 1024;
 constexpr int kHeldCache = 2048;
 constexpr int kMaxFix = 48;
+constexpr int kMaxArcs = 8192;      // finite arcs of D the Bellman-Ford search can list
 constexpr int kSortMax = 16384;     // candidate lists up to this length are sorted (they fit in D's space)
 
 struct P2Shared {
@@ -616,7 +617,7 @@ struct P2Shared {
   int flow[kMaxE];               // units on expert -> sink
   int dirty[kMaxE];
   int path[kMaxE + 2];
-  int npath, changed, who, target, stop, any_pos, qn, nfix;
+  int npath, changed, who, target, stop, any_pos, qn, nfix, narc, bf_bad;
   int fix_e[kMaxFix], fix_f[kMaxFix];   // stale D entries to recompute after a move
   long long dt;
 };
@@ -630,6 +631,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
   unsigned char* held_s = reinterpret_cast<unsigned char*>(D + (size_t)E * (E | 1));       // [kHeldCache][kMaxK]
   int* cand_s = reinterpret_cast<int*>(held_s + (size_t)kHeldCache * kMaxK);          // [kHeldCache]
   int* queue_s = cand_s + kHeldCache;                                                // [kHeldCache]
+  unsigned short* arcs_s = reinterpret_cast<unsigned short*>(queue_s + kHeldCache);  // [kMaxArcs] (u << 8 | v)
   __shared__ P2Shared s;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = min(st->ncand, T);
@@ -777,7 +779,94 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
     { const long long t1 = clock64(); t_rebuild += t1 - t0; if (t_first == -1) t_first = t1 - t0; t0 = t1; }
     if (!s.any_pos || naug >= max_aug) break;
 
+    // ---- shortest paths from every node with excess ---------------------------------------------------
+    // First choice: synchronous Bellman-Ford over the list of finite arcs of D (a few thousand after the
+    // window filter), all threads, distance and predecessor packed in one word (dist << 8 | pred) so
+    // that one atomicMin keeps them consistent.  A node is only updated when its distance strictly
+    // drops against the previous round, so the predecessor graph has no cycle.  If the arc list does
+    // not fit, or distances leave the packed range, the single-warp Dijkstra below takes over.
+    bool have_paths = false;
+    {
+      if (tid == 0) s.narc = 0;
+      __syncthreads();
+      for (int i = tid; i < E * ES; i += blockDim.x) {
+        const int u = i / ES, v = i - u * ES;
+        if (v < E && D[i] < kInf) {
+          const int slot = atomicAdd(&s.narc, 1);
+          if (slot < kMaxArcs) arcs_s[slot] = (unsigned short)((u << 8) | v);
+        }
+      }
+      __syncthreads();
+      if (s.narc <= kMaxArcs) {
+        const int narc = s.narc;
+        constexpr long long kPInf = 0x7fffffffffffffffLL;
+        constexpr long long kBfLimit = 1LL << 46;     // arcs and distances beyond this leave the packed range
+        long long* pd0 = s.dist[0]; long long* pd1 = s.dist[1];
+        for (int v = tid; v <= E; v += blockDim.x) pd0[v] = s.imb[v] > 0 ? 255LL : kPInf;   // dist 0, no pred
+        if (tid == 0) s.bf_bad = 0;
+        __syncthreads();
+        for (int round = 0; round <= E + 1; ++round) {
+          for (int v = tid; v <= E; v += blockDim.x) pd1[v] = pd0[v];
+          if (tid == 0) s.changed = 0;
+          __syncthreads();
+          for (int a = tid; a < narc; a += blockDim.x) {
+            const int u = arcs_s[a] >> 8, v = arcs_s[a] & 255;
+            const long long pu = pd0[u];
+            if (pu == kPInf) continue;
+            long long rc = D[u * ES + v] - s.p[u] + s.p[v];
+            if (rc < 0) rc = 0;
+            if (rc >= kBfLimit) { s.bf_bad = 1; continue; }
+            const long long nd = (pu >> 8) + rc;
+            if (nd >= kBfLimit) { s.bf_bad = 1; continue; }
+            const long long old = pd0[v];
+            if (old == kPInf || nd < (old >> 8)) { atomicMin(&pd1[v], (nd << 8) | u); s.changed = 1; }
+          }
+          for (int e = tid; e < E; e += blockDim.x) {      // the arcs through Z
+            const long long pe = pd0[e], pz = pd0[nZ];
+            if (pe != kPInf && s.flow[e] < C) {
+              long long rc = -s.p[e] + s.p[nZ]; if (rc < 0) rc = 0;
+              const long long nd = (pe >> 8) + rc;
+              if (rc >= kBfLimit || nd >= kBfLimit) s.bf_bad = 1;
+              else if (pz == kPInf || nd < (pz >> 8)) { atomicMin(&pd1[nZ], (nd << 8) | e); s.changed = 1; }
+            }
+            if (pz != kPInf && s.flow[e] > 0) {
+              long long rc = -s.p[nZ] + s.p[e]; if (rc < 0) rc = 0;
+              const long long nd = (pz >> 8) + rc;
+              if (rc >= kBfLimit || nd >= kBfLimit) s.bf_bad = 1;
+              else if (pe == kPInf || nd < (pe >> 8)) { atomicMin(&pd1[e], (nd << 8) | nZ); s.changed = 1; }
+            }
+          }
+          __syncthreads();
+          long long* t = pd0; pd0 = pd1; pd1 = t;
+          ++bf_rounds;
+          const bool more = s.changed != 0;
+          __syncthreads();
+          if (!more) break;
+        }
+        if (!s.bf_bad) {
+          // unpack; nearest node with a deficit (lowest index on ties)
+          long long dv = kInf; int pv = -1;
+          if (tid <= E) {
+            const long long w = pd0[tid];
+            if (w != kPInf) { dv = w >> 8; pv = (int)(w & 255); if (pv == 255) pv = -1; }
+          }
+          __syncthreads();
+          if (tid <= E) { s.dist[0][tid] = dv; s.pred[tid] = pv; }
+          __syncthreads();
+          if (tid == 0) {
+            int t = -1; long long dt = kInf;
+            for (int v = 0; v <= E; ++v)
+              if (s.imb[v] < 0 && s.dist[0][v] < dt) { dt = s.dist[0][v]; t = v; }
+            s.target = t; s.dt = dt;
+          }
+          __syncthreads();
+          have_paths = s.target >= 0;
+        }
+      }
+    }
     // ---- Dijkstra from every node with excess (reduced costs rc = cost - p[u] + p[v] are >= 0) ---------
+    if (!have_paths)
+
     // One warp, nodes spread over its lanes; it stops when the first node with a deficit is settled:
     // every node still open is at least that far away, which is all the price update needs to know.
     if (warp == 0) {

@@ -111,7 +111,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-constexpr int kP2SmemMax = (int)(sizeof(long long) * kMaxE * (kMaxE | 1) + kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache);
+constexpr int kP2SmemMax = (int)(sizeof(long long) * kMaxE * (kMaxE | 1) + kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache + 2 * kMaxArcs);
 constexpr int kDispatchSmem = 64 * 1024;
 constexpr int kDhSmemMax = 2 * 2 * 16384 + kDhStages * 2 * 16384 + 1024;     // Kpad = 128
 constexpr int kDwSmemMax = kDwStages * (16384 + 2 * 2 * 8192) + 1024;
@@ -228,7 +228,7 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
     flow_sweep_kernel<<<blocks, kSweepThreads, sweep_staged ? tile_smem : 0, st>>>(M, fs, p.T, p.E, p.k, c->C, g, n_sweeps, 1, sweep_staged);
     MS_LAUNCH_CHECK("flow_sweep_kernel");
   }
-  const size_t p2smem = sizeof(long long) * (size_t)p.E * (p.E | 1) + (size_t)kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache;
+  const size_t p2smem = sizeof(long long) * (size_t)p.E * (p.E | 1) + (size_t)kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache + 2 * kMaxArcs;
   for (int r = 0; r < kRounds; ++r) {
     flow_collect_kernel<<<blocks, kSweepThreads, tile_smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, r == 0, 0,
                                                          32LL, nullptr, nullptr, nullptr, r == kRounds - 1);
