@@ -73,8 +73,9 @@ struct FlowState {
   double total_score;
   int load[kMaxE];           // accumulated by the running pass, consumed by its last CTA
   int load_cur[kMaxE];       // loads of the assignment currently written in expert_idx
-  alignas(16) unsigned hist_up[kMaxE * kNB];   // read and cleared with 16-byte accesses
-  alignas(16) unsigned hist_dn[kMaxE * kNB];
+  alignas(16) unsigned hist_up[2][kMaxE * kNB];   // [sweep parity]; read and cleared with 16-byte accesses
+  alignas(16) unsigned hist_dn[2][kMaxE * kNB];
+  int cut_max;                                    // log2 of the largest margin worth recording at all
   int cap_up[kMaxE], cap_dn[kMaxE];   // log2 of the largest margin worth recording
   int flag_dn[kMaxE];                 // expert whose join-histogram came out short: scan it in full next sweep
   unsigned ticket;
@@ -84,13 +85,13 @@ struct FlowState {
   int ncand_last;
 };
 
-static_assert(offsetof(FlowState, hist_up) % 16 == 0 && offsetof(FlowState, hist_dn) % 16 == 0,
+static_assert(offsetof(FlowState, hist_up) % 16 == 0 && offsetof(FlowState, hist_dn) % 16 == 0 && (kMaxE * kNB * 4) % 16 == 0,
               "histograms are accessed as uint4");
 
 // ---------------------------------------------------------------------------------------------
 __global__ void flow_init_kernel(FlowState* st, long long eps0, long long eps_min, int cap0,
                                  long long theta0, int balanced, int E) {
-  for (int i = threadIdx.x; i < kMaxE * kNB; i += blockDim.x) { st->hist_up[i] = 0; st->hist_dn[i] = 0; }
+  for (int i = threadIdx.x; i < 2 * kMaxE * kNB; i += blockDim.x) { st->hist_up[0][i] = 0; st->hist_dn[0][i] = 0; }
   for (int e = threadIdx.x; e < kMaxE; e += blockDim.x) {
     st->p[e] = 0; st->load[e] = 0; st->load_cur[e] = 0; st->cap_up[e] = cap0; st->cap_dn[e] = cap0; st->flag_dn[e] = 0;
   }
@@ -98,7 +99,7 @@ __global__ void flow_init_kernel(FlowState* st, long long eps0, long long eps_mi
     st->eps = eps0; st->eps_min = eps_min; st->theta = theta0; st->total_score = 0.0;
     st->ticket = 0; st->sweep = 0; st->p1_done = 0; st->balanced = balanced;
     st->round = 0; st->converged = 0; st->ncand = 0; st->violations = 0; st->naug = 0;
-    st->rerouted = 0; st->status = 0; st->ncand_last = 0;
+    st->rerouted = 0; st->status = 0; st->ncand_last = 0; st->cut_max = cap0;
   }
 }
 
@@ -251,6 +252,7 @@ __device__ __forceinline__ int log_bin(long long m) {
   const int o = 63 - __clzll(m);
   return 4 * (o - 1) + (int)((m >> (o - 2)) & 3);
 }
+__device__ __forceinline__ int rel_bin(long long m, int) { return log_bin(m); }
 __device__ __forceinline__ long long bin_lower_edge(int b) {
   if (b < 4) return b;
   const int o = b / 4 + 1, sub = b & 3;
@@ -264,8 +266,9 @@ __device__ __forceinline__ long long bin_lower_edge(int b) {
 // log2 of the largest margin the tokens were asked to record; if fewer than `need` lie below it the
 // step goes to 2^cut and the cut-off is lifted for the next sweep.
 __device__ __forceinline__ long long price_step(const unsigned* hist, int need, long long eps, int& cut,
-                                                bool& window_short) {
+                                                bool& window_short, int cut_max) {
   window_short = false;
+  const int base = 0;
   const int nb = min(kNB, 4 * cut);                   // bins at or above 2^cut are empty
   unsigned cum = 0, before = 0; int pos = -1, last = -1;
   for (int b0 = 0; b0 < nb && pos < 0; b0 += 16) {
@@ -285,13 +288,13 @@ __device__ __forceinline__ long long price_step(const unsigned* hist, int need, 
   if (pos < 0) {
     // fewer than `need` margins were recorded.  Under a cut-off, everything below it may move; with
     // no cut-off, move what was recorded (an outsider list can be incomplete) and ask for a full scan.
-    const long long step = cut < kCapLogMax ? (1LL << cut) : (last >= 0 ? bin_lower_edge(last + 1) : 0);
-    cut = kCapLogMax;
+    const long long step = cut < cut_max ? (1LL << cut) : (last >= 0 ? bin_lower_edge(last + 1 + base) : 0);
+    cut = cut_max;
     window_short = true;
     return step;
   }
-  const long long lo = bin_lower_edge(pos), hi = bin_lower_edge(pos + 1);
-  cut = min(kCapLogMax, max(12, (pos >> 2) + 5));      // next sweep: record up to ~16x this margin
+  const long long lo = pos == 0 ? 0 : bin_lower_edge(pos + base), hi = bin_lower_edge(pos + 1 + base);
+  cut = min(cut_max, max(12, ((pos + base) >> 2) + 5));   // next sweep: record up to ~16x this margin
   (void)before;
   if (cum <= 2u * (unsigned)need || lo == 0) {
     const long long w = hi - lo;
@@ -308,6 +311,16 @@ __global__ void __launch_bounds__(kSweepThreads)
 flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int k, int C, KeyGen g,
                   int n_sweeps, int decay_every, int staged) {
   if (*(volatile int*)&st->p1_done) return;
+  // histograms alternate between two buffers: this sweep fills one while every CTA clears a slice of
+  // the other for the next sweep (its last reader, the previous sweep's last CTA, has finished)
+  const int par = st->sweep & 1;
+  unsigned* hup = st->hist_up[par]; unsigned* hdn = st->hist_dn[par];
+  {
+    uint4* zu = reinterpret_cast<uint4*>(st->hist_up[par ^ 1]); uint4* zd = reinterpret_cast<uint4*>(st->hist_dn[par ^ 1]);
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < kMaxE * kNB / 4; i += gridDim.x * blockDim.x) {
+      zu[i] = make_uint4(0, 0, 0, 0); zd[i] = make_uint4(0, 0, 0, 0);
+    }
+  }
   __shared__ long long sp[kMaxE];
   __shared__ int sload[kMaxE];
   __shared__ int scu[kMaxE], scd[kMaxE];
@@ -344,7 +357,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
         if (has_alt) {
           const long long m = v[j] - vk1;             // price rise at which this token leaves e
           const int cl = scu[e];
-          if (m < (1LL << cl)) atomicAdd(&st->hist_up[e * kNB + log_bin(m)], 1u);
+          if (m < (1LL << cl)) atomicAdd(&hup[e * kNB + rel_bin(m, cl)], 1u);
         }
       }
     }
@@ -355,7 +368,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
         if (e >= 0) {
           const long long m = vk - v[j];              // price cut at which this token joins e
           const int cl = scd[e];
-          if (m < (1LL << cl)) atomicAdd(&st->hist_dn[e * kNB + log_bin(m)], 1u);
+          if (m < (1LL << cl)) atomicAdd(&hdn[e * kNB + rel_bin(m, cl)], 1u);
         }
       }
     }
@@ -369,7 +382,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
       if (seen) continue;
       const long long m = vk - (make_key(g, row[e], flat + e) - sp[e]);
       const int cl = scd[e];
-      if (m >= 0 && m < (1LL << cl)) atomicAdd(&st->hist_dn[e * kNB + log_bin(m)], 1u);
+      if (m >= 0 && m < (1LL << cl)) atomicAdd(&hdn[e * kNB + rel_bin(m, cl)], 1u);
     }
   }
   __syncthreads();
@@ -379,6 +392,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
   const long long tail_t0 = clock64();
   if (!last_block_arrives(&st->ticket)) return;
   // ---- last CTA: move the prices -------------------------------------------------------------
+  const long long tA = clock64();
   __shared__ int s_imb;
   __shared__ long long pmin;
   if (threadIdx.x == 0) s_imb = 0;
@@ -391,13 +405,13 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
     const int x = load - C;
     if (x > 0) {
       int cl = scu[e]; bool shortw;
-      p += price_step(st->hist_up + e * kNB, x, eps, cl, shortw);
+      p += price_step(hup + e * kNB, x, eps, cl, shortw, st->cut_max);
       st->cap_up[e] = cl;
       st->flag_dn[e] = 0;
       atomicAdd(&s_imb, x);
     } else if (x < 0 && (balanced || p > 0)) {
       int cl = scd[e]; bool shortw;
-      p -= price_step(st->hist_dn + e * kNB, -x, eps, cl, shortw);
+      p -= price_step(hdn + e * kNB, -x, eps, cl, shortw, st->cut_max);
       if (!balanced && p < 0) p = 0;
       st->cap_dn[e] = cl;
       st->flag_dn[e] = shortw ? 1 : 0;
@@ -411,10 +425,8 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
     if (x != 0) sp[e] = p;
   }
   __syncthreads();   // every expert's histogram has been read before any is cleared
-  {
-    uint4* hu = reinterpret_cast<uint4*>(st->hist_up); uint4* hd = reinterpret_cast<uint4*>(st->hist_dn);
-    for (int i = threadIdx.x; i < E * kNB / 4; i += blockDim.x) { hu[i] = make_uint4(0, 0, 0, 0); hd[i] = make_uint4(0, 0, 0, 0); }
-  }
+  const long long tB = clock64();
+  const long long tC = clock64();
   const int sweep = st->sweep + 1;
   const bool done = (s_imb == 0) || sweep >= n_sweeps;
   if (threadIdx.x == 0) {
@@ -428,7 +440,8 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
   __syncthreads();
   if (threadIdx.x == 0) {
     if (sweep <= 40) st->trace[sweep - 1] = s_imb;
-    st->trace[40] = (int)((clock64() - tail_t0) >> 4);   // cycles/16 the last CTA spent on the price update
+    st->trace[40] = (int)((clock64() - tail_t0) >> 4);
+    st->trace[30] = (int)(tA - tail_t0); st->trace[31] = (int)(tB - tA); st->trace[32] = (int)(tC - tB); st->trace[33] = (int)(clock64() - tC);   // cycles/16 the last CTA spent on the price update
     st->sweep = sweep;
     if (sweep % decay_every == 0) { long long ne = eps >> 1; st->eps = ne < st->eps_min ? st->eps_min : ne; }
     st->ticket = 0;
