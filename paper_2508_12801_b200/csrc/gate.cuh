@@ -327,9 +327,10 @@ __host__ __device__ constexpr uint32_t idesc_bf16_m128_mn(int n) {   // both ope
 
 // ---- dH[T, d] = dL[T, E] . W_g^T -------------------------------------------------------------------
 // One CTA per 128-token tile.  The dL tile (hi and lo) is loaded once; 128-column tiles of W_g stream
-// through a 3-stage ring; two TMEM accumulators alternate so that the four epilogue warps convert and
-// store tile n while the MMA warp works on tile n+1.
-constexpr int kDhBN = 128, kDhStages = 3;
+// through a 2-stage ring; two TMEM accumulators alternate so that the four epilogue warps convert and
+// stage tile n in shared memory (one bulk store per row) while the MMA warp works on tile n+1.
+constexpr int kDhBN = 128, kDhStages = 2;
+constexpr int kDhOutStride = kDhBN * 2 + 16;     // bytes per staged output row (padded against bank conflicts)
 struct DhSmem {
   uint64_t a_full, b_full[kDhStages], b_empty[kDhStages], acc_full[2], acc_empty[2];
   uint32_t tmem_base;
@@ -349,6 +350,7 @@ gate_bwd_dh_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   const uint32_t b_bytes = kboxes * 16384u;
   unsigned char* a_tile = base;                       // [2*kboxes][128 rows][128 B]
   unsigned char* b_ring = base + a_bytes;             // [stage][kboxes][128 rows][128 B]
+  unsigned char* out_stage = b_ring + (size_t)kDhStages * b_bytes;   // [2][128 rows][kDhOutStride]
   const int n_tiles = (d + kDhBN - 1) / kDhBN;
 
   if (threadIdx.x == 0) {
@@ -412,30 +414,34 @@ gate_bwd_dh_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       ok = mbar_wait_bounded(&sm.acc_full[buf], (uint32_t)((nt >> 1) & 1));
       if (!ok) break;
       tc_fence_after();
+      // the staged copy of this buffer from two tiles ago must have been read by its bulk store
+      if (nt >= 2) bulk_wait_read<1>();
+      unsigned char* my_row = out_stage + ((size_t)buf * 128 + quarter * 32 + lane) * kDhOutStride;
       for (int c0 = 0; c0 < kDhBN; c0 += 16) {
         float r[16];
         tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kDhBN + c0), r);
-        const int col = nt * kDhBN + c0;
-        if (row < T && col < d) {
-          __nv_bfloat16* out = dH + (size_t)row * d + col;
-          if (col + 16 <= d) {
-            uint32_t w[8];
+        uint32_t w[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              __nv_bfloat162 h = __floats2bfloat162_rn(r[2 * j], r[2 * j + 1]);
-              w[j] = *reinterpret_cast<uint32_t*>(&h);
-            }
-            reinterpret_cast<uint4*>(out)[0] = make_uint4(w[0], w[1], w[2], w[3]);
-            reinterpret_cast<uint4*>(out)[1] = make_uint4(w[4], w[5], w[6], w[7]);
-          } else {
-            for (int j = 0; j < 16 && col + j < d; ++j) out[j] = __float2bfloat16(r[j]);
-          }
+        for (int j = 0; j < 8; ++j) {
+          __nv_bfloat162 h = __floats2bfloat162_rn(r[2 * j], r[2 * j + 1]);
+          w[j] = *reinterpret_cast<uint32_t*>(&h);
         }
+        reinterpret_cast<uint4*>(my_row + c0 * 2)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        reinterpret_cast<uint4*>(my_row + c0 * 2)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+      }
+      // each lane ships its own row: one 256-byte bulk store instead of sixteen scattered 16-byte ones
+      fence_proxy_async();
+      {
+        const int col0 = nt * kDhBN;
+        const int ncol = min(kDhBN, d - col0);
+        if (row < T && ncol > 0) bulk_s2g(dH + (size_t)row * d + col0, my_row, (uint32_t)ncol * 2);
+        bulk_commit();
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);
     }
+    bulk_wait_all<0>();
     if (!ok && lane == 0) sm.failed = 1;
   }
   __syncthreads();

@@ -113,7 +113,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 constexpr int kP2SmemMax = (int)(sizeof(long long) * kMaxE * (kMaxE | 1) + kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache + 2 * kMaxArcs);
 constexpr int kDispatchSmem = 64 * 1024;
-constexpr int kDhSmemMax = 2 * 2 * 16384 + kDhStages * 2 * 16384 + 1024;     // Kpad = 128
+constexpr int kDhSmemMax = 2 * 2 * 16384 + kDhStages * 2 * 16384 + 2 * 128 * kDhOutStride + 1024;     // Kpad = 128
 constexpr int kDwSmemMax = kDwStages * (16384 + 2 * 2 * 8192) + 1024;
 
 }  // namespace
@@ -479,7 +479,7 @@ maxscore_status maxscore_gate_bwd(maxscore_ctx* c, const void* hidden, const voi
     if (!s2) s2 = make_tmap_bf16(c, &tmL2, dls, (uint64_t)2 * Kpad, (uint64_t)p.T, 64, 64);
     if (s2) return s2;
     const int kboxes = Kpad / 64;
-    const size_t dh_smem = (size_t)2 * kboxes * 16384 + (size_t)kDhStages * kboxes * 16384 + 1024;
+    const size_t dh_smem = (size_t)2 * kboxes * 16384 + (size_t)kDhStages * kboxes * 16384 + (size_t)2 * 128 * kDhOutStride + 1024;
     gate_bwd_dh_tc_kernel<<<(p.T + 127) / 128, 192, dh_smem, st>>>(tmA, tmB, (__nv_bfloat16*)dH, p.T, p.d_model, Kpad,
                                                                   error_flag_of(c));
     MS_LAUNCH_CHECK("gate_bwd_dh_tc_kernel");
