@@ -65,7 +65,7 @@ __device__ __forceinline__ long long make_key(const KeyGen& g, float x, uint32_t
 }
 
 struct FlowState {
-  int trace[64];             // total imbalance seen by each sweep (diagnostics)
+  int trace[128];            // diagnostics: [0..23] imbalance per sweep, [64..] rows scanned in full per sweep
   long long p[kMaxE];        // expert prices
   long long eps, eps_min;
   long long theta;           // candidate threshold of the next collect pass
@@ -75,6 +75,7 @@ struct FlowState {
   int load_cur[kMaxE];       // loads of the assignment currently written in expert_idx
   alignas(16) unsigned hist_up[2][kMaxE * kNB];   // [sweep parity]; read and cleared with 16-byte accesses
   alignas(16) unsigned hist_dn[2][kMaxE * kNB];
+  long long cumdrop;                              // sum over sweeps of the largest price decrease of that sweep
   int cut_max;                                    // log2 of the largest margin worth recording at all
   int cap_up[kMaxE], cap_dn[kMaxE];   // log2 of the largest margin worth recording
   int flag_dn[kMaxE];                 // expert whose join-histogram came out short: scan it in full next sweep
@@ -98,8 +99,9 @@ __global__ void flow_init_kernel(FlowState* st, long long eps0, long long eps_mi
   if (threadIdx.x == 0) {
     st->eps = eps0; st->eps_min = eps_min; st->theta = theta0; st->total_score = 0.0;
     st->ticket = 0; st->sweep = 0; st->p1_done = 0; st->balanced = balanced;
+    for (int i = 64; i < 128; ++i) st->trace[i] = 0;
     st->round = 0; st->converged = 0; st->ncand = 0; st->violations = 0; st->naug = 0;
-    st->rerouted = 0; st->status = 0; st->ncand_last = 0; st->cut_max = cap0;
+    st->rerouted = 0; st->status = 0; st->ncand_last = 0; st->cut_max = cap0; st->cumdrop = 0;
   }
 }
 
@@ -303,17 +305,88 @@ __device__ __forceinline__ long long price_step(const unsigned* hist, int need, 
   return lo;                                          // conservative: moves `before` < need tokens
 }
 
+// The same step computed by a whole warp: lane l holds bins 8l .. 8l+7 of the expert's histogram.
+__device__ __forceinline__ long long price_step_warp(const uint4& ha, const uint4& hb, int need, long long eps, int& cut,
+                                                     bool& window_short, int cut_max) {
+  const int lane = threadIdx.x & 31;
+  const unsigned hv[8] = {ha.x, ha.y, ha.z, ha.w, hb.x, hb.y, hb.z, hb.w};
+  unsigned mine = 0; int top = -1;
+#pragma unroll
+  for (int q = 0; q < 8; ++q) { mine += hv[q]; if (hv[q]) top = 8 * lane + q; }
+  unsigned incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  const unsigned reach = __ballot_sync(0xffffffffu, incl >= (unsigned)need);
+  window_short = false;
+  if (!reach) {
+    const int last = __reduce_max_sync(0xffffffffu, top);
+    const long long step = cut < cut_max ? (1LL << cut) : (last >= 0 ? bin_lower_edge(last + 1) : 0);
+    cut = cut_max;
+    window_short = true;
+    return step;
+  }
+  const int src = __ffs(reach) - 1;
+  int pos = 0; unsigned cum = incl - mine;
+  if (lane == src) {
+    unsigned c = incl - mine; bool found = false;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {                        // first bin of this lane at which the count is reached
+      c += hv[q];
+      if (!found && c >= (unsigned)need) { pos = 8 * lane + q; cum = c; found = true; }
+    }
+  }
+  pos = __shfl_sync(0xffffffffu, pos, src);
+  cum = __shfl_sync(0xffffffffu, cum, src);
+  const long long lo = pos == 0 ? 0 : bin_lower_edge(pos), hi = bin_lower_edge(pos + 1);
+  cut = min(cut_max, max(12, (pos >> 2) + 5));
+  if (cum <= 2u * (unsigned)need || lo == 0) {
+    const long long w = hi - lo;
+    return hi + (eps < w ? eps : w);
+  }
+  return lo;
+}
+
 // ---------------------------------------------------------------------------------------------
 // One price sweep.
 constexpr int kSweepThreads = 128;
 
+// Per-token candidate cache of the sweeps.  A full scan of a token's row keeps its kCacheN best experts
+// (score and index) and `bound` = the smallest of their values minus the total price drop so far.  A
+// later sweep re-evaluates only those kCacheN entries; every other expert is worth at most
+// bound + (total price drop now), so while the (k+2)-th cached value stays at or above that, the cached
+// entries still contain the token's k+2 best experts and the row need not be read again.
+constexpr int kCacheN = 16;
+struct SweepCache {
+  float* x;              // [kCacheN][T] scores of the cached experts
+  unsigned char* id;     // [T][kCacheN] their indices (255 = none)
+  long long* bound;      // [T]
+};
+
+struct SweepShared {
+  long long sp[kMaxE];
+  float spf[kMaxE];
+  int sload[kMaxE], scu[kMaxE], scd[kMaxE], sflag[kMaxE];
+  int nflag, nslow;
+  unsigned short slow[kSweepThreads];
+};
+
+__device__ __forceinline__ void emit_margin(unsigned* hist, const int* caplog, int e, long long m) {
+  if (m >= 0 && m < (1LL << caplog[e])) atomicAdd(&hist[e * kNB + log_bin(m)], 1u);
+}
+
+template <bool kFirst>   // the first sweep scans every row (one thread per token) and fills the cache
 __global__ void __launch_bounds__(kSweepThreads)
-flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int k, int C, KeyGen g,
-                  int n_sweeps, int decay_every, int staged) {
+flow_sweep_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, int T, int E, int k, int C,
+                  KeyGen g) {
   if (*(volatile int*)&st->p1_done) return;
   // histograms alternate between two buffers: this sweep fills one while every CTA clears a slice of
-  // the other for the next sweep (its last reader, the previous sweep's last CTA, has finished)
-  const int par = st->sweep & 1;
+  // the other for the next sweep (its last reader, the previous price update, has finished)
+  const int sweep0 = st->sweep;
+  const long long cumdrop = st->cumdrop;
+  const int par = sweep0 & 1;
   unsigned* hup = st->hist_up[par]; unsigned* hdn = st->hist_dn[par];
   {
     uint4* zu = reinterpret_cast<uint4*>(st->hist_up[par ^ 1]); uint4* zd = reinterpret_cast<uint4*>(st->hist_dn[par ^ 1]);
@@ -321,112 +394,253 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
       zu[i] = make_uint4(0, 0, 0, 0); zd[i] = make_uint4(0, 0, 0, 0);
     }
   }
-  __shared__ long long sp[kMaxE];
-  __shared__ int sload[kMaxE];
-  __shared__ int scu[kMaxE], scd[kMaxE];
-  __shared__ float spf[kMaxE];
-  __shared__ int sflag[kMaxE];
-  __shared__ int nflag;
-  if (threadIdx.x == 0) nflag = 0;
+  __shared__ SweepShared sh;
+  long long (&sp)[kMaxE] = sh.sp;
+  int (&sload)[kMaxE] = sh.sload; int (&scu)[kMaxE] = sh.scu; int (&scd)[kMaxE] = sh.scd;
+  if (threadIdx.x == 0) { sh.nflag = 0; sh.nslow = 0; }
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += blockDim.x) {
-    sp[e] = st->p[e]; spf[e] = (float)sp[e]; sload[e] = 0; scu[e] = st->cap_up[e]; scd[e] = st->cap_dn[e];
-    if (st->flag_dn[e]) sflag[atomicAdd(&nflag, 1)] = e;
+    sp[e] = st->p[e]; sh.spf[e] = (float)sp[e]; sload[e] = 0; scu[e] = st->cap_up[e]; scd[e] = st->cap_dn[e];
+    if (st->flag_dn[e]) sh.sflag[atomicAdd(&sh.nflag, 1)] = e;
   }
-  extern __shared__ __align__(16) float sweep_tile[];
-  const int tok0 = blockIdx.x * blockDim.x;
-  if (staged) stage_rows(M, sweep_tile, tok0, min((int)blockDim.x, T - tok0), E);
   __syncthreads();
-  const int tok = tok0 + threadIdx.x;
-  if (tok < T) {
-    long long v[kTopN]; int id[kTopN];
-    const float* row = staged ? sweep_tile + (size_t)threadIdx.x * E : M + (size_t)tok * E;
-    const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-    // rotated start: conflict-free shared-memory reads.  The sweeps are a heuristic, so the cheap
-    // (fp32-filtered) selection is enough here.
-    select_top(row, sp, spf, g, flat, E, staged ? (int)(threadIdx.x % E) : ((E & 3) == 0 ? -1 : 0), false, v, id);
-    const bool has_alt = E > k;
-    long long vk = -kInf, vk1 = -kInf;                // k-th value and best alternative
+  const int tok0 = blockIdx.x * blockDim.x;
+  const int need = min(k + 2, E);                       // sorted values a token has to know
+  const int nflag = sh.nflag;
+  // ---- pass A, one thread per token: re-evaluate the cached experts -----------------------------
+  {
+    const int tok = tok0 + threadIdx.x;
+    if (tok < T) {
+      bool valid = false;
+      if (kFirst) {
+        const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+        const float* row = M + (size_t)tok * E;
+        long long v[kCacheN]; int id[kCacheN];
+        select_top(row, sp, sh.spf, g, flat, E, (E & 3) == 0 ? -1 : 0, false, v, id);
+        unsigned idws[4] = {0, 0, 0, 0};
 #pragma unroll
-    for (int j = 0; j < kTopN; ++j) { if (j == k - 1) vk = v[j]; if (j == k) vk1 = v[j]; }
+        for (int j = 0; j < kCacheN; ++j) {
+          cache.x[(size_t)j * T + tok] = id[j] >= 0 ? __ldg(row + id[j]) : 0.f;
+          idws[j >> 2] |= (unsigned)(id[j] >= 0 ? id[j] : 255) << (8 * (j & 3));
+        }
+        *reinterpret_cast<uint4*>(cache.id + (size_t)tok * kCacheN) = make_uint4(idws[0], idws[1], idws[2], idws[3]);
+        cache.bound[tok] = id[kCacheN - 1] >= 0 ? v[kCacheN - 1] - cumdrop : -kInf;
+        long long vk = -kInf, vk1 = -kInf;
 #pragma unroll
-    for (int j = 0; j < kMaxK; ++j) {
-      if (j < k) {
-        const int e = id[j];
-        atomicAdd(&sload[e], 1);
-        if (has_alt) {
-          const long long m = v[j] - vk1;             // price rise at which this token leaves e
-          const int cl = scu[e];
-          if (m < (1LL << cl)) atomicAdd(&hup[e * kNB + rel_bin(m, cl)], 1u);
+        for (int j = 0; j < kCacheN; ++j) { if (j == k - 1) vk = v[j]; if (j == k) vk1 = v[j]; }
+#pragma unroll
+        for (int j = 0; j < kMaxK + 2; ++j) {
+          const int e = id[j];
+          if (j < k) {
+            atomicAdd(&sload[e], 1);
+            if (E > k) emit_margin(hup, scu, e, v[j] - vk1);
+          } else if (j <= k + 1 && e >= 0) {
+            emit_margin(hdn, scd, e, vk - v[j]);
+          }
+        }
+        valid = true;                                   // no expert is flagged before the first sweep
+      } else if (sweep0 > 0) {
+        const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+        const uint4 idw = *reinterpret_cast<const uint4*>(cache.id + (size_t)tok * kCacheN);
+        const unsigned idws[4] = {idw.x, idw.y, idw.z, idw.w};
+        long long v[kCacheN]; int rank[kCacheN];
+#pragma unroll
+        for (int j = 0; j < kCacheN; ++j) {
+          const int e = (int)((idws[j >> 2] >> (8 * (j & 3))) & 255u);
+          const float x = cache.x[(size_t)j * T + tok];
+          v[j] = e < E ? make_key(g, x, flat + e) - sp[e] : -kInf;
+          rank[j] = 0;
+        }
+#pragma unroll
+        for (int j = 1; j < kCacheN; ++j)
+#pragma unroll
+          for (int i = 0; i < j; ++i) {
+            const bool first = v[i] >= v[j];            // the earlier entry wins a tie
+            rank[j] += first ? 1 : 0; rank[i] += first ? 0 : 1;
+          }
+        long long vk = -kInf, vk1 = -kInf, vneed = -kInf;
+#pragma unroll
+        for (int j = 0; j < kCacheN; ++j) {
+          if (rank[j] == k - 1) vk = v[j];
+          if (rank[j] == k) vk1 = v[j];
+          if (rank[j] == need - 1) vneed = v[j];
+        }
+        const long long bound = cache.bound[tok];
+        valid = bound <= -kInf || vneed >= bound + cumdrop;
+        if (valid) {
+          const bool has_alt = E > k;
+#pragma unroll
+          for (int j = 0; j < kCacheN; ++j) {
+            const int e = (int)((idws[j >> 2] >> (8 * (j & 3))) & 255u);
+            if (rank[j] < k) {
+              atomicAdd(&sload[e], 1);
+              if (has_alt) emit_margin(hup, scu, e, v[j] - vk1);        // price rise at which the token leaves e
+            } else if (rank[j] <= k + 1 && e < E) {
+              emit_margin(hdn, scd, e, vk - v[j]);                      // price cut at which the token joins e
+            }
+          }
+          // experts whose join-histogram was short last time: count this token even if the expert is
+          // not among its best alternatives
+          for (int q = 0; q < nflag; ++q) {
+            const int e = sh.sflag[q];
+            bool seen = false;
+#pragma unroll
+            for (int j = 0; j < kCacheN; ++j)
+              seen |= (rank[j] <= k + 1) && ((int)((idws[j >> 2] >> (8 * (j & 3))) & 255u) == e);
+            if (seen) continue;
+            emit_margin(hdn, scd, e, vk - (make_key(g, __ldg(M + (size_t)tok * E + e), flat + e) - sp[e]));
+          }
         }
       }
+      if (!valid) sh.slow[atomicAdd(&sh.nslow, 1)] = (unsigned short)threadIdx.x;
     }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && sweep0 < 64 && sh.nslow) atomicAdd(&st->trace[64 + sweep0], sh.nslow);
+  // ---- pass B, one warp per token whose cache no longer vouches for itself: scan the whole row ----
+  {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int nslow = sh.nslow;
+    for (int s = warp; s < nslow; s += kSweepThreads / 32) {
+      const int tok = tok0 + sh.slow[s];
+      const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+      const float* row = M + (size_t)tok * E;
+      // lane l looks at experts l, l+32, l+64, l+96.  fp32 approximations, the expert index in the low
+      // 7 mantissa bits, mapped to unsigned integers that order the same way; 0 = absent
+      unsigned u[kEPLf];
 #pragma unroll
-    for (int j = 1; j < kTopN; ++j) {
-      if ((j == k || j == k + 1) && j < E) {
-        const int e = id[j];
-        if (e >= 0) {
-          const long long m = vk - v[j];              // price cut at which this token joins e
-          const int cl = scd[e];
-          if (m < (1LL << cl)) atomicAdd(&hdn[e * kNB + rel_bin(m, cl)], 1u);
+      for (int q = 0; q < kEPLf; ++q) {
+        const int e = lane + 32 * q;
+        u[q] = 0;
+        if (e < E) {
+          const float vf = approx_key(g, __ldg(row + e)) - sh.spf[e];
+          const unsigned bits = (__float_as_uint(vf) & ~127u) | (unsigned)e;
+          u[q] = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
         }
       }
-    }
-    // experts whose join-histogram was short last time: count this token even if the expert is not
-    // among its best alternatives
-    for (int q = 0; q < nflag; ++q) {
-      const int e = sflag[q];
-      bool seen = false;
+      unsigned mine = 0;
+      for (int r = 0; r < kCacheN; ++r) {
+        unsigned m = u[0];
 #pragma unroll
-      for (int j = 0; j < kTopN; ++j) seen |= (j <= k + 1 && id[j] == e);
-      if (seen) continue;
-      const long long m = vk - (make_key(g, row[e], flat + e) - sp[e]);
-      const int cl = scd[e];
-      if (m >= 0 && m < (1LL << cl)) atomicAdd(&hdn[e * kNB + rel_bin(m, cl)], 1u);
+        for (int q = 1; q < kEPLf; ++q) m = max(m, u[q]);
+        const unsigned w = __reduce_max_sync(0xffffffffu, m);
+        if (lane == r) mine = w;
+#pragma unroll
+        for (int q = 0; q < kEPLf; ++q) u[q] = (u[q] == w) ? 0u : u[q];
+      }
+      // lanes 0..kCacheN-1 now hold the winners in descending approximate order; make them exact
+      int ee = 255; float xv = 0.f; long long val = -kInf;
+      if (lane < kCacheN && mine != 0) {
+        const unsigned bits = (mine & 0x80000000u) ? (mine & 0x7fffffffu) : ~mine;
+        ee = (int)(bits & 127u);
+        xv = __ldg(row + ee);
+        val = make_key(g, xv, flat + ee) - sp[ee];
+      }
+      if (lane < kCacheN) {
+        cache.x[(size_t)lane * T + tok] = xv;
+        cache.id[(size_t)tok * kCacheN + lane] = (unsigned char)ee;
+      }
+      // every expert outside the cache is worth no more than the last winner (none if E <= kCacheN)
+      const long long vlast = __shfl_sync(0xffffffffu, val, kCacheN - 1);
+      if (lane == 0) cache.bound[tok] = (vlast <= -kInf) ? -kInf : vlast - cumdrop;
+      int rank = 0;
+#pragma unroll
+      for (int i = 0; i < kCacheN; ++i) {
+        const long long vi = __shfl_sync(0xffffffffu, val, i);
+        rank += (vi > val || (vi == val && i < lane)) ? 1 : 0;
+      }
+      const bool listed = lane < kCacheN && ee < E;
+      const unsigned bk = __ballot_sync(0xffffffffu, listed && rank == k - 1);
+      const unsigned bk1 = __ballot_sync(0xffffffffu, listed && rank == k);
+      const long long vk = __shfl_sync(0xffffffffu, val, bk ? __ffs(bk) - 1 : 0);
+      const long long vk1 = bk1 ? __shfl_sync(0xffffffffu, val, __ffs(bk1) - 1) : -kInf;
+      if (listed) {
+        if (rank < k) {
+          atomicAdd(&sload[ee], 1);
+          if (E > k) emit_margin(hup, scu, ee, val - vk1);
+        } else if (rank <= k + 1) {
+          emit_margin(hdn, scd, ee, vk - val);
+        }
+      }
+      for (int q = 0; q < nflag; ++q) {
+        const int e = sh.sflag[q];
+        const unsigned seen = __ballot_sync(0xffffffffu, listed && rank <= k + 1 && ee == e);
+        if (!seen && lane == 0) emit_margin(hdn, scd, e, vk - (make_key(g, __ldg(row + e), flat + e) - sp[e]));
+      }
     }
   }
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += blockDim.x)
     if (sload[e]) atomicAdd(&st->load[e], sload[e]);
 
-  const long long tail_t0 = clock64();
-  if (!last_block_arrives(&st->ticket)) return;
-  // ---- last CTA: move the prices -------------------------------------------------------------
-  const long long tA = clock64();
+}
+
+// Price update that closes a sweep: one CTA, one warp per expert (four experts per warp, all their
+// histograms in flight at once).
+constexpr int kPriceThreads = 1024;
+__global__ void __launch_bounds__(kPriceThreads)
+flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every) {
+  if (*(volatile int*)&st->p1_done) return;
+  __shared__ long long sp[kMaxE];
   __shared__ int s_imb;
-  __shared__ long long pmin;
-  if (threadIdx.x == 0) s_imb = 0;
-  __syncthreads();
+  __shared__ long long pmin, s_drop;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  constexpr int kWarps = kPriceThreads / 32, kBatch = kMaxE / kWarps;
+  const int par = st->sweep & 1;
+  const unsigned* hup = st->hist_up[par]; const unsigned* hdn = st->hist_dn[par];
   const long long eps = st->eps;
   const bool balanced = st->balanced != 0;
-  for (int e = threadIdx.x; e < E; e += blockDim.x) {
-    const int load = __ldcg(&st->load[e]);
-    long long p = sp[e];
-    const int x = load - C;
-    if (x > 0) {
-      int cl = scu[e]; bool shortw;
-      p += price_step(hup + e * kNB, x, eps, cl, shortw, st->cut_max);
-      st->cap_up[e] = cl;
-      st->flag_dn[e] = 0;
-      atomicAdd(&s_imb, x);
-    } else if (x < 0 && (balanced || p > 0)) {
-      int cl = scd[e]; bool shortw;
-      p -= price_step(hdn + e * kNB, -x, eps, cl, shortw, st->cut_max);
-      if (!balanced && p < 0) p = 0;
-      st->cap_dn[e] = cl;
-      st->flag_dn[e] = shortw ? 1 : 0;
-      atomicAdd(&s_imb, -x);
-    } else {
-      st->flag_dn[e] = 0;
+  const int cut_max = st->cut_max;
+  if (threadIdx.x == 0) { s_imb = 0; s_drop = 0; }
+  uint4 ha[kBatch], hb[kBatch]; int xs[kBatch]; long long ps[kBatch];
+#pragma unroll
+  for (int b = 0; b < kBatch; ++b) {
+    const int e = warp + b * kWarps;
+    xs[b] = 0; ps[b] = 0; ha[b] = make_uint4(0, 0, 0, 0); hb[b] = ha[b];
+    if (e < E) {
+      const int x = st->load[e] - C;
+      xs[b] = x; ps[b] = st->p[e];
+      const bool up = x > 0, dn = x < 0 && (balanced || ps[b] > 0);
+      if (up || dn) {
+        const uint4* h = reinterpret_cast<const uint4*>((up ? hup : hdn) + e * kNB) + 2 * lane;
+        ha[b] = h[0]; hb[b] = h[1];
+      }
     }
-    st->load[e] = 0;
+  }
+  __syncthreads();
+  int imb = 0; long long drop = 0;
+#pragma unroll
+  for (int b = 0; b < kBatch; ++b) {
+    const int e = warp + b * kWarps;
+    if (e >= E) continue;
+    const int x = xs[b];
+    long long p = ps[b];
+    int flag = 0;
+    if (x > 0) {
+      int cl = st->cap_up[e]; bool shortw;
+      p += price_step_warp(ha[b], hb[b], x, eps, cl, shortw, cut_max);
+      if (lane == 0) st->cap_up[e] = cl;
+      imb += x;
+    } else if (x < 0 && (balanced || p > 0)) {
+      int cl = st->cap_dn[e]; bool shortw;
+      p -= price_step_warp(ha[b], hb[b], -x, eps, cl, shortw, cut_max);
+      if (!balanced && p < 0) p = 0;
+      if (lane == 0) st->cap_dn[e] = cl;
+      flag = shortw ? 1 : 0;
+      imb += -x;
+    }
     p = p > kPriceLimit ? kPriceLimit : (p < -kPriceLimit ? -kPriceLimit : p);
     // when nothing was out of balance the prices stay put and the collect pass reproduces this state
-    if (x != 0) sp[e] = p;
+    if (x == 0) p = ps[b];
+    if (lane == 0) {
+      st->flag_dn[e] = flag;
+      st->load[e] = 0;
+      if (ps[b] - p > drop) drop = ps[b] - p;
+      sp[e] = p;
+    }
   }
-  __syncthreads();   // every expert's histogram has been read before any is cleared
-  const long long tB = clock64();
-  const long long tC = clock64();
+  if (lane == 0) { if (imb) atomicAdd(&s_imb, imb); if (drop > 0) atomicMax(&s_drop, drop); }
+  __syncthreads();
   const int sweep = st->sweep + 1;
   const bool done = (s_imb == 0) || sweep >= n_sweeps;
   if (threadIdx.x == 0) {
@@ -437,15 +651,11 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, int T, int E, int 
   }
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += blockDim.x) st->p[e] = sp[e] - pmin;
-  __syncthreads();
   if (threadIdx.x == 0) {
     if (sweep <= 40) st->trace[sweep - 1] = s_imb;
-    st->trace[40] = (int)((clock64() - tail_t0) >> 4);
-    st->trace[30] = (int)(tA - tail_t0); st->trace[31] = (int)(tB - tA); st->trace[32] = (int)(tC - tB); st->trace[33] = (int)(clock64() - tC);   // cycles/16 the last CTA spent on the price update
     st->sweep = sweep;
+    st->cumdrop += s_drop;
     if (sweep % decay_every == 0) { long long ne = eps >> 1; st->eps = ne < st->eps_min ? st->eps_min : ne; }
-    st->ticket = 0;
-    __threadfence();
     if (done) st->p1_done = 1;
   }
 }
@@ -714,10 +924,16 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
     // the warps then work through the queue and through the uncached tail of the list
     if (tid == 0) s.qn = 0;
     __syncthreads();
-    for (int c = tid; c < nc; c += blockDim.x) {
+    for (int c0 = 0; c0 < nc; c0 += blockDim.x) {
+      const int c = c0 + tid;
       bool any = false;
-      for (int j = 0; j < k; ++j) any |= (s.dirty[held_s[c * kMaxK + j]] != 0);
-      if (any) queue_s[atomicAdd(&s.qn, 1)] = c;
+      if (c < nc)
+        for (int j = 0; j < k; ++j) any |= (s.dirty[held_s[c * kMaxK + j]] != 0);
+      const unsigned mask = __ballot_sync(0xffffffffu, any);
+      int base = 0;
+      if (lane == 0 && mask) base = atomicAdd(&s.qn, __popc(mask));
+      base = __shfl_sync(0xffffffffu, base, 0);
+      if (any) queue_s[base + __popc(mask & ((1u << lane) - 1u))] = c;
     }
     __syncthreads();
     const int work = s.qn + (n - nc);
@@ -802,12 +1018,16 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
     {
       if (tid == 0) s.narc = 0;
       __syncthreads();
-      for (int i = tid; i < E * ES; i += blockDim.x) {
+      for (int i0 = 0; i0 < E * ES; i0 += blockDim.x) {      // one counter update per warp, not per arc
+        const int i = i0 + tid;
         const int u = i / ES, v = i - u * ES;
-        if (v < E && D[i] < kInf) {
-          const int slot = atomicAdd(&s.narc, 1);
-          if (slot < kMaxArcs) arcs_s[slot] = (unsigned short)((u << 8) | v);
-        }
+        const bool finite = i < E * ES && v < E && D[i] < kInf;
+        const unsigned mask = __ballot_sync(0xffffffffu, finite);
+        int base = 0;
+        if (lane == 0 && mask) base = atomicAdd(&s.narc, __popc(mask));
+        base = __shfl_sync(0xffffffffu, base, 0);
+        const int slot = base + __popc(mask & ((1u << lane) - 1u));
+        if (finite && slot < kMaxArcs) arcs_s[slot] = (unsigned short)((u << 8) | v);
       }
       __syncthreads();
       if (s.narc <= kMaxArcs) {

@@ -50,7 +50,7 @@ int32_t capacity_of(const maxscore_params& p) {
 }
 
 struct Layout {          // byte offsets inside the workspace
-  size_t state, cand, block_counts, wt, error_flag, dls, wk, dwpart, total;
+  size_t state, cand, cache_x, cache_id, cache_bound, block_counts, wt, error_flag, dls, wk, dwpart, total;
   int Npad, n_idx_blocks;
   int Kpad, dw_splits, dw_tokens_per_split;   // tensor-core backward GEMMs (bf16 I/O)
 };
@@ -63,6 +63,9 @@ Layout layout_of(const maxscore_params& p) {
   l.state = off; off = align_up(off + sizeof(FlowState), 256);
   l.error_flag = off; off = align_up(off + 16, 256);
   l.cand = off; off = align_up(off + sizeof(int32_t) * (size_t)p.T, 256);
+  l.cache_x = off; off = align_up(off + sizeof(float) * (size_t)kCacheN * p.T, 256);
+  l.cache_id = off; off = align_up(off + (size_t)kCacheN * p.T, 256);
+  l.cache_bound = off; off = align_up(off + sizeof(long long) * (size_t)p.T, 256);
   l.block_counts = off; off = align_up(off + sizeof(int32_t) * (size_t)l.n_idx_blocks * p.E, 1024);
   l.wt = off;
   off = align_up(off + (p.io_dtype == MAXSCORE_BF16 ? sizeof(__nv_bfloat16) * (size_t)l.Npad * p.d_model : 0), 1024);
@@ -222,10 +225,12 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   MS_LAUNCH_CHECK("flow_init_kernel");
   const int blocks = (p.T + kSweepThreads - 1) / kSweepThreads;
   const size_t tile_smem = sizeof(float) * (size_t)kSweepThreads * p.E;
-  // measured on B200: reading the rows straight from L2 beats staging them (more CTAs per SM)
-  const int sweep_staged = 0;
+  SweepCache cache{reinterpret_cast<float*>(c->ws + c->lay.cache_x), reinterpret_cast<unsigned char*>(c->ws + c->lay.cache_id),
+                   reinterpret_cast<long long*>(c->ws + c->lay.cache_bound)};
   for (int s = 0; s < n_sweeps; ++s) {
-    flow_sweep_kernel<<<blocks, kSweepThreads, sweep_staged ? tile_smem : 0, st>>>(M, fs, p.T, p.E, p.k, c->C, g, n_sweeps, 1, sweep_staged);
+    if (s == 0) flow_sweep_kernel<true><<<blocks, kSweepThreads, 0, st>>>(M, fs, cache, p.T, p.E, p.k, c->C, g);
+    else flow_sweep_kernel<false><<<blocks, kSweepThreads, 0, st>>>(M, fs, cache, p.T, p.E, p.k, c->C, g);
+    flow_price_kernel<<<1, kPriceThreads, 0, st>>>(fs, p.E, c->C, n_sweeps, 1);
     MS_LAUNCH_CHECK("flow_sweep_kernel");
   }
   const size_t p2smem = sizeof(long long) * (size_t)p.E * (p.E | 1) + (size_t)kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache + 2 * kMaxArcs;
@@ -312,7 +317,6 @@ maxscore_status maxscore_create(maxscore_ctx** out, const maxscore_params* param
     return MAXSCORE_ERR_CUDA;
   }
   MS_CUDA(cudaFuncSetAttribute(gate_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGateSmemBytes));
-  MS_CUDA(cudaFuncSetAttribute(flow_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * kSweepThreads * kMaxE)));
   MS_CUDA(cudaFuncSetAttribute(flow_collect_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * kSweepThreads * kMaxE)));
   MS_CUDA(cudaFuncSetAttribute(flow_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kP2SmemMax));
   MS_CUDA(cudaFuncSetAttribute(dispatch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDispatchSmem));
