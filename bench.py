@@ -33,7 +33,7 @@ SWEEPS, ROUNDS = 24, 4
 def launches_per_step():
     """Kernels of this library launched by one step (memsets not counted)."""
     gate = 2                       # W_g transpose/pad + tcgen05 GEMM
-    assign = 1 + 2 * SWEEPS + 2 * ROUNDS + 1      # init, (sweep + price update) x SWEEPS, (collect + exact) x ROUNDS, verify
+    assign = 1 + 2 * SWEEPS + 3 * ROUNDS + 1      # init, (sweep + price update) x SWEEPS, (collect + build + exact) x ROUNDS, verify
     route_fwd = gate + 1 + assign + 2 + 1          # + SoftTopk + index (count, fill) + gate_w gather
     dispatch, combine = 2, 1
     route_bwd = 2 + 1 + 5                          # combine-bwd (+padding), SoftTopk-bwd, gate-bwd (split, W_g, dH, dW, reduce)

@@ -37,6 +37,8 @@ constexpr long long kInf = 1LL << 62;
 constexpr long long kArcLimit = 1LL << 58; // arcs with a larger reduced cost are ignored by the exact phase
 constexpr long long kPriceLimit = 1LL << 56; // sweeps keep |price| below this
 constexpr int kCapLogMax = 60;
+constexpr int kStallSweeps = 3, kStallImbalance = 256;
+constexpr int kExactNeed = 8;              // imbalances up to this are closed one exact margin at a time
 constexpr int kEPLf = kMaxE / 32;          // experts per lane when a warp spans one token row
 
 struct KeyGen {
@@ -77,10 +79,12 @@ struct FlowState {
   alignas(16) unsigned hist_dn[2][kMaxE * kNB];
   long long cumdrop;                              // sum over sweeps of the largest price decrease of that sweep
   int cut_max;                                    // log2 of the largest margin worth recording at all
+  long long min_up[kMaxE], min_dn[kMaxE];   // smallest margin recorded by the running sweep (reset by the price update)
   int cap_up[kMaxE], cap_dn[kMaxE];   // log2 of the largest margin worth recording
   int flag_dn[kMaxE];                 // expert whose join-histogram came out short: scan it in full next sweep
   unsigned ticket;
   int sweep, p1_done, balanced;
+  int best_imb, stall;                // smallest imbalance seen so far; sweeps since it last improved
   int round, converged, ncand, violations, naug, rerouted;
   unsigned status;
   int ncand_last;
@@ -94,11 +98,11 @@ __global__ void flow_init_kernel(FlowState* st, long long eps0, long long eps_mi
                                  long long theta0, int balanced, int E) {
   for (int i = threadIdx.x; i < 2 * kMaxE * kNB; i += blockDim.x) { st->hist_up[0][i] = 0; st->hist_dn[0][i] = 0; }
   for (int e = threadIdx.x; e < kMaxE; e += blockDim.x) {
-    st->p[e] = 0; st->load[e] = 0; st->load_cur[e] = 0; st->cap_up[e] = cap0; st->cap_dn[e] = cap0; st->flag_dn[e] = 0;
+    st->p[e] = 0; st->load[e] = 0; st->load_cur[e] = 0; st->min_up[e] = kInf; st->min_dn[e] = kInf; st->cap_up[e] = cap0; st->cap_dn[e] = cap0; st->flag_dn[e] = 0;
   }
   if (threadIdx.x == 0) {
     st->eps = eps0; st->eps_min = eps_min; st->theta = theta0; st->total_score = 0.0;
-    st->ticket = 0; st->sweep = 0; st->p1_done = 0; st->balanced = balanced;
+    st->ticket = 0; st->sweep = 0; st->p1_done = 0; st->balanced = balanced; st->best_imb = 0x7fffffff; st->stall = 0;
     for (int i = 64; i < 128; ++i) st->trace[i] = 0;
     st->round = 0; st->converged = 0; st->ncand = 0; st->violations = 0; st->naug = 0;
     st->rerouted = 0; st->status = 0; st->ncand_last = 0; st->cut_max = cap0; st->cumdrop = 0;
@@ -307,7 +311,7 @@ __device__ __forceinline__ long long price_step(const unsigned* hist, int need, 
 
 // The same step computed by a whole warp: lane l holds bins 8l .. 8l+7 of the expert's histogram.
 __device__ __forceinline__ long long price_step_warp(const uint4& ha, const uint4& hb, int need, long long eps, int& cut,
-                                                     bool& window_short, int cut_max) {
+                                                     bool& window_short, int cut_max, long long m1) {
   const int lane = threadIdx.x & 31;
   const unsigned hv[8] = {ha.x, ha.y, ha.z, ha.w, hb.x, hb.y, hb.z, hb.w};
   unsigned mine = 0; int top = -1;
@@ -329,19 +333,26 @@ __device__ __forceinline__ long long price_step_warp(const uint4& ha, const uint
     return step;
   }
   const int src = __ffs(reach) - 1;
-  int pos = 0; unsigned cum = incl - mine;
+  int pos = 0; unsigned cum = incl - mine, before = 0;
   if (lane == src) {
     unsigned c = incl - mine; bool found = false;
 #pragma unroll
     for (int q = 0; q < 8; ++q) {                        // first bin of this lane at which the count is reached
+      if (!found && c + hv[q] >= (unsigned)need) { pos = 8 * lane + q; before = c; cum = c + hv[q]; found = true; }
       c += hv[q];
-      if (!found && c >= (unsigned)need) { pos = 8 * lane + q; cum = c; found = true; }
     }
   }
   pos = __shfl_sync(0xffffffffu, pos, src);
   cum = __shfl_sync(0xffffffffu, cum, src);
+  before = __shfl_sync(0xffffffffu, before, src);
   const long long lo = pos == 0 ? 0 : bin_lower_edge(pos), hi = bin_lower_edge(pos + 1);
   cut = min(cut_max, max(12, (pos >> 2) + 5));
+  // end game: when a handful of tokens have to move and the bin would move more than that, move fewer
+  // but exactly: everything below the bin, or else the single token with the smallest margin
+  if (need <= kExactNeed && cum > (unsigned)need) {
+    if (before > 0 && lo > 0) return lo;
+    if (m1 < kInf) return m1 + 1;
+  }
   if (cum <= 2u * (unsigned)need || lo == 0) {
     const long long w = hi - lo;
     return hi + (eps < w ? eps : w);
@@ -373,8 +384,11 @@ struct SweepShared {
   unsigned short slow[kSweepThreads];
 };
 
-__device__ __forceinline__ void emit_margin(unsigned* hist, const int* caplog, int e, long long m) {
-  if (m >= 0 && m < (1LL << caplog[e])) atomicAdd(&hist[e * kNB + log_bin(m)], 1u);
+__device__ __forceinline__ void emit_margin(unsigned* hist, long long* mins, const int* caplog, int e, long long m) {
+  if (m >= 0 && m < (1LL << caplog[e])) {
+    atomicAdd(&hist[e * kNB + log_bin(m)], 1u);
+    atomicMin(&mins[e], m);                             // the exact smallest margin, for steps that move one token
+  }
 }
 
 template <bool kFirst>   // the first sweep scans every row (one thread per token) and fills the cache
@@ -388,6 +402,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, 
   const long long cumdrop = st->cumdrop;
   const int par = sweep0 & 1;
   unsigned* hup = st->hist_up[par]; unsigned* hdn = st->hist_dn[par];
+  long long* mup = st->min_up; long long* mdn = st->min_dn;
   {
     uint4* zu = reinterpret_cast<uint4*>(st->hist_up[par ^ 1]); uint4* zd = reinterpret_cast<uint4*>(st->hist_dn[par ^ 1]);
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < kMaxE * kNB / 4; i += gridDim.x * blockDim.x) {
@@ -433,9 +448,9 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, 
           const int e = id[j];
           if (j < k) {
             atomicAdd(&sload[e], 1);
-            if (E > k) emit_margin(hup, scu, e, v[j] - vk1);
+            if (E > k) emit_margin(hup, mup, scu, e, v[j] - vk1);
           } else if (j <= k + 1 && e >= 0) {
-            emit_margin(hdn, scd, e, vk - v[j]);
+            emit_margin(hdn, mdn, scd, e, vk - v[j]);
           }
         }
         valid = true;                                   // no expert is flagged before the first sweep
@@ -474,9 +489,9 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, 
             const int e = (int)((idws[j >> 2] >> (8 * (j & 3))) & 255u);
             if (rank[j] < k) {
               atomicAdd(&sload[e], 1);
-              if (has_alt) emit_margin(hup, scu, e, v[j] - vk1);        // price rise at which the token leaves e
+              if (has_alt) emit_margin(hup, mup, scu, e, v[j] - vk1);        // price rise at which the token leaves e
             } else if (rank[j] <= k + 1 && e < E) {
-              emit_margin(hdn, scd, e, vk - v[j]);                      // price cut at which the token joins e
+              emit_margin(hdn, mdn, scd, e, vk - v[j]);                      // price cut at which the token joins e
             }
           }
           // experts whose join-histogram was short last time: count this token even if the expert is
@@ -488,7 +503,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, 
             for (int j = 0; j < kCacheN; ++j)
               seen |= (rank[j] <= k + 1) && ((int)((idws[j >> 2] >> (8 * (j & 3))) & 255u) == e);
             if (seen) continue;
-            emit_margin(hdn, scd, e, vk - (make_key(g, __ldg(M + (size_t)tok * E + e), flat + e) - sp[e]));
+            emit_margin(hdn, mdn, scd, e, vk - (make_key(g, __ldg(M + (size_t)tok * E + e), flat + e) - sp[e]));
           }
         }
       }
@@ -557,15 +572,15 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, 
       if (listed) {
         if (rank < k) {
           atomicAdd(&sload[ee], 1);
-          if (E > k) emit_margin(hup, scu, ee, val - vk1);
+          if (E > k) emit_margin(hup, mup, scu, ee, val - vk1);
         } else if (rank <= k + 1) {
-          emit_margin(hdn, scd, ee, vk - val);
+          emit_margin(hdn, mdn, scd, ee, vk - val);
         }
       }
       for (int q = 0; q < nflag; ++q) {
         const int e = sh.sflag[q];
         const unsigned seen = __ballot_sync(0xffffffffu, listed && rank <= k + 1 && ee == e);
-        if (!seen && lane == 0) emit_margin(hdn, scd, e, vk - (make_key(g, __ldg(row + e), flat + e) - sp[e]));
+        if (!seen && lane == 0) emit_margin(hdn, mdn, scd, e, vk - (make_key(g, __ldg(row + e), flat + e) - sp[e]));
       }
     }
   }
@@ -592,11 +607,11 @@ flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every) {
   const bool balanced = st->balanced != 0;
   const int cut_max = st->cut_max;
   if (threadIdx.x == 0) { s_imb = 0; s_drop = 0; }
-  uint4 ha[kBatch], hb[kBatch]; int xs[kBatch]; long long ps[kBatch];
+  uint4 ha[kBatch], hb[kBatch]; int xs[kBatch]; long long ps[kBatch], m1[kBatch];
 #pragma unroll
   for (int b = 0; b < kBatch; ++b) {
     const int e = warp + b * kWarps;
-    xs[b] = 0; ps[b] = 0; ha[b] = make_uint4(0, 0, 0, 0); hb[b] = ha[b];
+    xs[b] = 0; ps[b] = 0; m1[b] = kInf; ha[b] = make_uint4(0, 0, 0, 0); hb[b] = ha[b];
     if (e < E) {
       const int x = st->load[e] - C;
       xs[b] = x; ps[b] = st->p[e];
@@ -604,6 +619,7 @@ flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every) {
       if (up || dn) {
         const uint4* h = reinterpret_cast<const uint4*>((up ? hup : hdn) + e * kNB) + 2 * lane;
         ha[b] = h[0]; hb[b] = h[1];
+        m1[b] = up ? st->min_up[e] : st->min_dn[e];
       }
     }
   }
@@ -618,12 +634,12 @@ flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every) {
     int flag = 0;
     if (x > 0) {
       int cl = st->cap_up[e]; bool shortw;
-      p += price_step_warp(ha[b], hb[b], x, eps, cl, shortw, cut_max);
+      p += price_step_warp(ha[b], hb[b], x, eps, cl, shortw, cut_max, m1[b]);
       if (lane == 0) st->cap_up[e] = cl;
       imb += x;
     } else if (x < 0 && (balanced || p > 0)) {
       int cl = st->cap_dn[e]; bool shortw;
-      p -= price_step_warp(ha[b], hb[b], -x, eps, cl, shortw, cut_max);
+      p -= price_step_warp(ha[b], hb[b], -x, eps, cl, shortw, cut_max, m1[b]);
       if (!balanced && p < 0) p = 0;
       if (lane == 0) st->cap_dn[e] = cl;
       flag = shortw ? 1 : 0;
@@ -635,6 +651,7 @@ flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every) {
     if (lane == 0) {
       st->flag_dn[e] = flag;
       st->load[e] = 0;
+      st->min_up[e] = kInf; st->min_dn[e] = kInf;
       if (ps[b] - p > drop) drop = ps[b] - p;
       sp[e] = p;
     }
@@ -642,7 +659,10 @@ flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every) {
   if (lane == 0) { if (imb) atomicAdd(&s_imb, imb); if (drop > 0) atomicMax(&s_drop, drop); }
   __syncthreads();
   const int sweep = st->sweep + 1;
-  const bool done = (s_imb == 0) || sweep >= n_sweeps;
+  // a small imbalance that has stopped shrinking is a price war between a few experts: the exact phase
+  // ends it faster than more sweeps would
+  const int stall = s_imb < st->best_imb ? 0 : st->stall + 1;
+  const bool done = (s_imb == 0) || sweep >= n_sweeps || (stall >= kStallSweeps && s_imb <= kStallImbalance);
   if (threadIdx.x == 0) {
     // prices are only defined up to a shift when every expert must be full; anchor the minimum at 0
     long long m = 0;
@@ -654,6 +674,7 @@ flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every) {
   if (threadIdx.x == 0) {
     if (sweep <= 40) st->trace[sweep - 1] = s_imb;
     st->sweep = sweep;
+    st->stall = stall; if (stall == 0) st->best_imb = s_imb;
     st->cumdrop += s_drop;
     if (sweep % decay_every == 0) { long long ne = eps >> 1; st->eps = ne < st->eps_min ? st->eps_min : ne; }
     if (done) st->p1_done = 1;
@@ -668,8 +689,10 @@ __global__ void __launch_bounds__(kSweepThreads)
 flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restrict__ expert_idx,
                     int32_t* __restrict__ cand, int T, int E, int k, int C, KeyGen g, int first,
                     int verify_only, long long theta_scale, int32_t* __restrict__ expert_load_out,
-                    void* stats_out, const unsigned* __restrict__ error_flag, int unbounded) {
+                    void* stats_out, const unsigned* __restrict__ error_flag, int unbounded, long long* __restrict__ Dg) {
   if (!verify_only && *(volatile int*)&st->converged) return;
+  if (Dg)   // the move-cost matrix the build kernel fills next starts out empty
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < E * (E | 1); i += gridDim.x * blockDim.x) Dg[i] = kInf;
   __shared__ long long sp[kMaxE];
   __shared__ float spf[kMaxE];
   __shared__ int sload[kMaxE];
@@ -830,6 +853,72 @@ constexpr int kMaxFix = 48;
 constexpr int kMaxArcs = 8192;      // finite arcs of D the Bellman-Ford search can list
 constexpr int kSortMax = 16384;     // candidate lists up to this length are sorted (they fit in D's space)
 
+// First build of D for a round, spread over the whole GPU: one warp per candidate token, results
+// merged into global memory with 64-bit atomicMin.  (Inside the exact phase's single CTA the same
+// work costs a quarter of a millisecond at 1 600 candidates.)
+__global__ void __launch_bounds__(256)
+flow_build_kernel(const float* __restrict__ M, const FlowState* st, const int32_t* __restrict__ expert_idx,
+                  const int32_t* __restrict__ cand, long long* __restrict__ Dg, int T, int E, int k, KeyGen g) {
+  if (*(volatile const int*)&st->converged) return;
+  __shared__ long long sp[kMaxE];
+  for (int e = threadIdx.x; e < E; e += blockDim.x) sp[e] = st->p[e];
+  __syncthreads();
+  const int n = min(st->ncand, T);
+  const int ES = E | 1;
+  const long long theta = st->theta_used;
+  const long long arc_window = theta >= (kInf >> 2) ? kInf : 2 * theta;
+  const int lane = threadIdx.x & 31;
+  const int nwarps = gridDim.x * (blockDim.x >> 5);
+  for (int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); c < n; c += nwarps) {
+    const int tok = cand[c];
+    int h[kMaxK];
+#pragma unroll
+    for (int j = 0; j < kMaxK; ++j) h[j] = j < k ? expert_idx[(size_t)tok * k + j] : -1;
+    const float* row = M + (size_t)tok * E;
+    const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+    long long key[kEPLf]; bool in[kEPLf];
+#pragma unroll
+    for (int q = 0; q < kEPLf; ++q) {
+      const int f = lane + 32 * q;
+      key[q] = f < E ? make_key(g, __ldg(row + f), flat + f) : 0;
+      bool hd = f >= E;
+#pragma unroll
+      for (int j = 0; j < kMaxK; ++j) hd |= (h[j] == f);
+      in[q] = hd;
+    }
+    long long vmax = -kInf;
+#pragma unroll
+    for (int q = 0; q < kEPLf; ++q) {
+      const int f = lane + 32 * q;
+      if (!in[q]) { const long long val = key[q] - sp[f]; vmax = val > vmax ? val : vmax; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const long long ov = __shfl_xor_sync(0xffffffffu, vmax, o);
+      vmax = ov > vmax ? ov : vmax;
+    }
+#pragma unroll
+    for (int j = 0; j < kMaxK; ++j) {
+      if (j >= k) continue;
+      const int e = h[j];
+      long long mine = 0;
+#pragma unroll
+      for (int q = 0; q < kEPLf; ++q) if ((e >> 5) == q) mine = key[q];
+      const long long we = __shfl_sync(0xffffffffu, mine, e & 31);
+      const long long pe = sp[e];
+      if (arc_window < kInf && (we - pe) - vmax > arc_window) continue;
+#pragma unroll
+      for (int q = 0; q < kEPLf; ++q) {
+        const int f = lane + 32 * q;
+        if (!in[q]) {
+          const long long cst = we - key[q];
+          if (cst - pe + sp[f] <= arc_window && cst < Dg[e * ES + f]) atomicMin(&Dg[e * ES + f], cst);
+        }
+      }
+    }
+  }
+}
+
 struct P2Shared {
   long long p[kMaxE + 1];        // potentials: prices of the experts, then Z
   long long p0[kMaxE + 1];       // potentials at the start of the round
@@ -847,7 +936,7 @@ struct P2Shared {
 
 __global__ void __launch_bounds__(kP2Threads)
 flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_idx, int32_t* cand, int T, int E,
-                  int k, int C, KeyGen g, int max_aug) {
+                  int k, int C, KeyGen g, int max_aug, const long long* __restrict__ Dg) {
   if (*(volatile int*)&st->converged) return;
   extern __shared__ __align__(16) unsigned char p2smem[];
   long long* D = reinterpret_cast<long long*>(p2smem);                              // [E][E] raw arc costs
@@ -902,8 +991,9 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
     s.p[e] = st->p[e]; s.p0[e] = s.p[e];
     const int load = st->load_cur[e];
     const int fl = s.p[e] > 0 ? C : min(load, C);
-    s.flow[e] = fl; s.imb[e] = load - fl; s.dirty[e] = 1;
+    s.flow[e] = fl; s.imb[e] = load - fl; s.dirty[e] = 0;
   }
+  for (int i = tid; i < E * ES; i += blockDim.x) D[i] = Dg[i];       // built by flow_build_kernel
   __syncthreads();
   if (tid == 0) {
     int tot = 0;
@@ -992,7 +1082,8 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
           const int f = lane + 32 * q;
           if (!in[q]) {
             const long long cst = we - key[q];
-            if (cst - pe + s.p[f] <= arc_window) atomicMin(&D[e * ES + f], cst);
+            // D only ever decreases, so a stale read can only let a useless atomic through
+            if (cst - pe + s.p[f] <= arc_window && cst < D[e * ES + f]) atomicMin(&D[e * ES + f], cst);
           }
         }
       }
@@ -1342,7 +1433,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
               if (!he || hf) continue;
               const long long cst = make_key(g, __ldg(M + (size_t)tok * E + e), flat + e) -
                                     make_key(g, __ldg(M + (size_t)tok * E + f), flat + f);
-              if (cst - s.p[e] + s.p[f] <= arc_window) atomicMin(&D[e * ES + f], cst);
+              if (cst - s.p[e] + s.p[f] <= arc_window && cst < D[e * ES + f]) atomicMin(&D[e * ES + f], cst);
             }
           }
           __syncthreads();

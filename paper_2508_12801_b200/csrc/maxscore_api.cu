@@ -50,7 +50,7 @@ int32_t capacity_of(const maxscore_params& p) {
 }
 
 struct Layout {          // byte offsets inside the workspace
-  size_t state, cand, cache_x, cache_id, cache_bound, block_counts, wt, error_flag, dls, wk, dwpart, total;
+  size_t state, cand, dmat, cache_x, cache_id, cache_bound, block_counts, wt, error_flag, dls, wk, dwpart, total;
   int Npad, n_idx_blocks;
   int Kpad, dw_splits, dw_tokens_per_split;   // tensor-core backward GEMMs (bf16 I/O)
 };
@@ -63,6 +63,7 @@ Layout layout_of(const maxscore_params& p) {
   l.state = off; off = align_up(off + sizeof(FlowState), 256);
   l.error_flag = off; off = align_up(off + 16, 256);
   l.cand = off; off = align_up(off + sizeof(int32_t) * (size_t)p.T, 256);
+  l.dmat = off; off = align_up(off + sizeof(long long) * (size_t)p.E * (p.E | 1), 256);
   l.cache_x = off; off = align_up(off + sizeof(float) * (size_t)kCacheN * p.T, 256);
   l.cache_id = off; off = align_up(off + (size_t)kCacheN * p.T, 256);
   l.cache_bound = off; off = align_up(off + sizeof(long long) * (size_t)p.T, 256);
@@ -234,15 +235,19 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
     MS_LAUNCH_CHECK("flow_sweep_kernel");
   }
   const size_t p2smem = sizeof(long long) * (size_t)p.E * (p.E | 1) + (size_t)kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache + 2 * kMaxArcs;
+  long long* Dg = reinterpret_cast<long long*>(c->ws + c->lay.dmat);
+  const int build_blocks = c->sm_count * 4;
   for (int r = 0; r < kRounds; ++r) {
     flow_collect_kernel<<<blocks, kSweepThreads, tile_smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, r == 0, 0,
-                                                         32LL, nullptr, nullptr, nullptr, r == kRounds - 1);
+                                                         32LL, nullptr, nullptr, nullptr, r == kRounds - 1, Dg);
     MS_LAUNCH_CHECK("flow_collect_kernel");
-    flow_exact_kernel<<<1, kP2Threads, p2smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, max_aug);
+    flow_build_kernel<<<build_blocks, 256, 0, st>>>(M, fs, expert_idx, cand, Dg, p.T, p.E, p.k, g);
+    MS_LAUNCH_CHECK("flow_build_kernel");
+    flow_exact_kernel<<<1, kP2Threads, p2smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, max_aug, Dg);
     MS_LAUNCH_CHECK("flow_exact_kernel");
   }
   flow_collect_kernel<<<blocks, kSweepThreads, tile_smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, 0, 1, 32LL,
-                                                       expert_load, stats, error_flag_of(c), 0);
+                                                       expert_load, stats, error_flag_of(c), 0, nullptr);
   MS_LAUNCH_CHECK("flow_collect_kernel(verify)");
   return MAXSCORE_OK;
 }
