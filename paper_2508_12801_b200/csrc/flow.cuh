@@ -849,7 +849,7 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
 // the smallest token index whatever order the collect pass appended the tokens in.
 constexpr int kP2Threads = 1024;
 constexpr int kHeldCache = 2048;
-constexpr int kMaxFix = 48;
+constexpr int kMaxFix = 256;
 constexpr int kMaxArcs = 8192;      // finite arcs of D the Bellman-Ford search can list
 constexpr int kSortMax = 16384;     // candidate lists up to this length are sorted (they fit in D's space)
 
@@ -928,8 +928,10 @@ struct P2Shared {
   int imb[kMaxE + 1];            // + excess, - deficit
   int flow[kMaxE];               // units on expert -> sink
   int dirty[kMaxE];
+  unsigned char fixrow[kMaxE];   // rows that have a stale entry to recompute
   int path[kMaxE + 2];
-  int npath, changed, who, target, stop, any_pos, qn, nfix, narc, bf_bad;
+  int npath, changed, who, target, stop, any_pos, qn, nfix, narc, bf_bad, dup;
+  int who_a[kMaxE + 2];          // per arc of the path: the candidate that moves
   int fix_e[kMaxFix], fix_f[kMaxFix];   // stale D entries to recompute after a move
   long long dt;
 };
@@ -1004,6 +1006,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
 
   int naug = 0;
   int bf_rounds = 0; long long q_total = 0, t_first = 0;
+  long long t_who = 0, t_patch = 0, t_fix = 0; int n_arcs = 0;
   long long t_rebuild = 0, t_bf = 0, t_move = 0, t0 = clock64();   // phase timers (thread 0), diagnostics
   for (;;) {
     // ---- rebuild the rows of D marked dirty: D[e][f] = min over candidates in e, not in f ----------
@@ -1309,9 +1312,206 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
     }
     __syncthreads();
     // ---- push one unit along the path (stored target first) ------------------------------------------
+    // All arcs of the path at once: (W) every thread looks up, for its candidates, which arcs they are
+    // the cheapest token of; (P) one warp per arc patches D from that token's keys and lists the entries
+    // that became stale; (F) one pass recomputes the listed entries.  The path's nodes are distinct, so
+    // arcs touch different (row, column) pairs except where a min-update is used.  If one token is the
+    // cheapest of two arcs the arcs are taken one by one instead (below).
+    auto fix_pass = [&]() {
+        if (s.nfix > 0 && n <= kHeldCache) {
+          // recompute the listed entries: candidates that hold one of the listed rows are queued by one
+          // thread each; a warp then takes a queued candidate with its lanes spread over the entries,
+          // so that the loads of one candidate are in flight together
+          const int nfix = s.nfix;
+          for (int e = tid; e < E; e += blockDim.x) s.fixrow[e] = 0;
+          if (tid == 0) s.qn = 0;
+          __syncthreads();
+          if (tid < nfix) s.fixrow[s.fix_e[tid]] = 1;
+          __syncthreads();
+          for (int c0 = 0; c0 < n; c0 += blockDim.x) {
+            const int c = c0 + tid;
+            bool any = false;
+            if (c < n)
+              for (int j = 0; j < k; ++j) any |= (s.fixrow[held_s[c * kMaxK + j]] != 0);
+            const unsigned mask = __ballot_sync(0xffffffffu, any);
+            int base = 0;
+            if (lane == 0 && mask) base = atomicAdd(&s.qn, __popc(mask));
+            base = __shfl_sync(0xffffffffu, base, 0);
+            if (any) queue_s[base + __popc(mask & ((1u << lane) - 1u))] = c;
+          }
+          __syncthreads();
+          const int qn = s.qn;
+          for (int qi = warp; qi < qn; qi += kP2Threads / 32) {
+            const int c = queue_s[qi];
+            const int tok = cand_s[c];
+            int h[kMaxK];
+#pragma unroll
+            for (int j = 0; j < kMaxK; ++j) h[j] = j < k ? (int)held_s[c * kMaxK + j] : -1;
+            const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+            for (int i = lane; i < nfix; i += 32) {
+              const int e = s.fix_e[i], f = s.fix_f[i];
+              bool he = false, hf = false;
+#pragma unroll
+              for (int j = 0; j < kMaxK; ++j) { he |= (h[j] == e); hf |= (h[j] == f); }
+              if (!he || hf) continue;
+              const long long cst = make_key(g, __ldg(M + (size_t)tok * E + e), flat + e) -
+                                    make_key(g, __ldg(M + (size_t)tok * E + f), flat + f);
+              if (cst - s.p[e] + s.p[f] <= arc_window && cst < D[e * ES + f]) atomicMin(&D[e * ES + f], cst);
+            }
+          }
+          __syncthreads();
+        } else if (s.nfix > 0) {
+          // one thread per candidate (lists longer than the shared-memory mirror)
+          for (int c = tid; c < n; c += blockDim.x) {
+            const int tok = tok_of(c);
+            int h[kMaxK];
+#pragma unroll
+            for (int j = 0; j < kMaxK; ++j) h[j] = j < k ? held_of(c, tok, j) : -1;
+            const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+            for (int i = 0; i < s.nfix; ++i) {
+              const int e = s.fix_e[i], f = s.fix_f[i];
+              bool he = false, hf = false;
+#pragma unroll
+              for (int j = 0; j < kMaxK; ++j) { he |= (h[j] == e); hf |= (h[j] == f); }
+              if (!he || hf) continue;
+              const long long cst = make_key(g, __ldg(M + (size_t)tok * E + e), flat + e) -
+                                    make_key(g, __ldg(M + (size_t)tok * E + f), flat + f);
+              if (cst - s.p[e] + s.p[f] <= arc_window && cst < D[e * ES + f]) atomicMin(&D[e * ES + f], cst);
+            }
+          }
+          __syncthreads();
+        }
+    };
+    bool batched = false;
+    {
+      const int L = s.npath - 1;
+      long long ta = clock64();
+      for (int a = tid; a <= L; a += blockDim.x) s.who_a[a] = 0x7fffffff;
+      if (tid == 0) { s.dup = 0; s.nfix = 0; }
+      __syncthreads();
+      for (int c = tid; c < n; c += blockDim.x) {
+        const int tok = tok_of(c);
+        unsigned hm[4] = {0, 0, 0, 0};
+        for (int j = 0; j < k; ++j) { const int e = held_of(c, tok, j); hm[e >> 5] |= 1u << (e & 31); }
+        const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+        for (int a = L; a >= 1; --a) {
+          const int u = s.path[a], v = s.path[a - 1];
+          if (u >= E || v >= E) continue;
+          if (!((hm[u >> 5] >> (u & 31)) & 1u) || ((hm[v >> 5] >> (v & 31)) & 1u)) continue;
+          const long long cost = make_key(g, __ldg(M + (size_t)tok * E + u), flat + u) -
+                                 make_key(g, __ldg(M + (size_t)tok * E + v), flat + v);
+          if (cost == D[u * ES + v]) atomicMin(&s.who_a[a], c);    // sorted list: smallest c = smallest token
+        }
+      }
+      __syncthreads();
+      for (int idx = tid; idx < L * L; idx += blockDim.x) {
+        const int i = idx / L + 1, j = idx - (i - 1) * L + 1;
+        if (i < j && s.who_a[i] != 0x7fffffff && s.who_a[i] == s.who_a[j]) s.dup = 1;
+      }
+      __syncthreads();
+      batched = !s.dup;
+      { const long long tb = clock64(); t_who += tb - ta; ta = tb; }
+      if (batched) {
+        n_arcs += L;
+        for (int a = L - warp; a >= 1; a -= kP2Threads / 32) {
+          const int u = s.path[a], v = s.path[a - 1];
+          if (u >= E || v >= E) continue;
+          const int c = s.who_a[a];
+          if (c == 0x7fffffff) { if (lane == 0) { atomicOr(&st->status, 4u); s.stop = 1; } continue; }
+          const int tok = tok_of(c);
+          int h[kMaxK];
+#pragma unroll
+          for (int j = 0; j < kMaxK; ++j) {
+            h[j] = j < k ? held_of(c, tok, j) : -1;
+            if (h[j] == u) h[j] = v;                   // experts after the move
+          }
+          const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+          long long key[kEPLf]; bool in[kEPLf];
+#pragma unroll
+          for (int q = 0; q < kEPLf; ++q) {
+            const int f = lane + 32 * q;
+            key[q] = f < E ? make_key(g, __ldg(M + (size_t)tok * E + f), flat + f) : 0;
+            bool hd = f >= E;
+#pragma unroll
+            for (int j = 0; j < kMaxK; ++j) hd |= (h[j] == f);
+            in[q] = hd;
+          }
+          auto key_of = [&](int e) -> long long {
+            long long mine = 0;
+#pragma unroll
+            for (int q = 0; q < kEPLf; ++q) if ((e >> 5) == q) mine = key[q];
+            return __shfl_sync(0xffffffffu, mine, e & 31);
+          };
+          const long long ku = key_of(u), kv = key_of(v);
+#pragma unroll
+          for (int q = 0; q < kEPLf; ++q) {
+            const int f = lane + 32 * q;
+            if (!in[q]) {                               // row v gains the token
+              const long long cst = kv - key[q];
+              if (cst - s.p[v] + s.p[f] <= arc_window && cst < D[v * ES + f]) atomicMin(&D[v * ES + f], cst);
+            }
+            const bool was_out = f < E && f != u && (!in[q] || f == v);
+            if (was_out && D[u * ES + f] == ku - key[q]) {      // the token's own offer from u is gone
+              const int slot = atomicAdd(&s.nfix, 1);
+              if (slot < kMaxFix) { s.fix_e[slot] = u; s.fix_f[slot] = f; }
+            }
+          }
+#pragma unroll
+          for (int j = 0; j < kMaxK; ++j) {
+            if (j >= k || h[j] == v) continue;
+            const int gg = h[j];
+            const long long kg = key_of(gg);
+            if (lane == 0) {
+              if (kg - ku - s.p[gg] + s.p[u] <= arc_window && kg - ku < D[gg * ES + u]) atomicMin(&D[gg * ES + u], kg - ku);
+              if (D[gg * ES + v] == kg - kv) {
+                const int slot = atomicAdd(&s.nfix, 1);
+                if (slot < kMaxFix) { s.fix_e[slot] = gg; s.fix_f[slot] = v; }
+              }
+            }
+          }
+          __syncwarp();
+          if (lane == 0)
+            for (int j = 0; j < k; ++j)
+              if (held_of(c, tok, j) == u) {
+                if (c < nc) held_s[c * kMaxK + j] = (unsigned char)v;
+                expert_idx[(size_t)tok * k + j] = v;
+              }
+        }
+        if (tid == 0)
+          for (int a = L; a >= 1; --a) {
+            const int u = s.path[a], v = s.path[a - 1];
+            if (u < E && v < E) continue;
+            if (v == nZ) s.flow[u] += 1; else s.flow[v] -= 1;
+          }
+        __syncthreads();
+        if (s.nfix > kMaxFix) {
+          // too many stale entries: rebuild the rows they sit in.  The tokens have moved already, so a
+          // token's other experts are what it holds now, minus the arc's target
+          for (int a = L - warp; a >= 1; a -= kP2Threads / 32) {
+            const int u = s.path[a], v = s.path[a - 1];
+            if (u >= E || v >= E || lane != 0) continue;
+            const int c = s.who_a[a];
+            if (c == 0x7fffffff) continue;
+            const int tok = tok_of(c);
+            s.dirty[u] = 1;
+            for (int j = 0; j < k; ++j) { const int e = held_of(c, tok, j); if (e != v) s.dirty[e] = 1; }
+          }
+          __syncthreads();
+          if (tid == 0) s.nfix = 0;
+        } else {
+          for (int i = tid; i < s.nfix; i += blockDim.x) D[s.fix_e[i] * ES + s.fix_f[i]] = kInf;
+        }
+        __syncthreads();
+        { const long long tb = clock64(); t_patch += tb - ta; ta = tb; }
+        fix_pass();
+        t_fix += clock64() - ta;
+      }
+    }
+    if (!batched)
     for (int a = s.npath - 1; a >= 1; --a) {
       const int u = s.path[a], v = s.path[a - 1];
       if (u < E && v < E) {
+        long long ta = clock64(); ++n_arcs;
         if (tid == 0) s.who = 0x7fffffff;
         __syncthreads();
         const long long want = D[u * ES + v];
@@ -1334,6 +1534,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
           __syncthreads();
           break;
         }
+        { const long long tb = clock64(); t_who += tb - ta; ta = tb; }
         if (warp == 0) {
           // the token leaves u for v: patch D from its own keys instead of rebuilding every row it touches
           const int c = s.who, tok = tok_of(c);
@@ -1417,27 +1618,9 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
           for (int i = lane; i < s.nfix; i += 32) D[s.fix_e[i] * ES + s.fix_f[i]] = kInf;
         }
         __syncthreads();
-        if (s.nfix > 0) {
-          // one thread per candidate: recompute the listed entries from the tokens that hold the row
-          for (int c = tid; c < n; c += blockDim.x) {
-            const int tok = tok_of(c);
-            int h[kMaxK];
-#pragma unroll
-            for (int j = 0; j < kMaxK; ++j) h[j] = j < k ? held_of(c, tok, j) : -1;
-            const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-            for (int i = 0; i < s.nfix; ++i) {
-              const int e = s.fix_e[i], f = s.fix_f[i];
-              bool he = false, hf = false;
-#pragma unroll
-              for (int j = 0; j < kMaxK; ++j) { he |= (h[j] == e); hf |= (h[j] == f); }
-              if (!he || hf) continue;
-              const long long cst = make_key(g, __ldg(M + (size_t)tok * E + e), flat + e) -
-                                    make_key(g, __ldg(M + (size_t)tok * E + f), flat + f);
-              if (cst - s.p[e] + s.p[f] <= arc_window && cst < D[e * ES + f]) atomicMin(&D[e * ES + f], cst);
-            }
-          }
-          __syncthreads();
-        }
+        { const long long tb = clock64(); t_patch += tb - ta; ta = tb; }
+        fix_pass();
+        t_fix += clock64() - ta;
       } else if (tid == 0) {
         if (v == nZ) s.flow[u] += 1; else s.flow[v] -= 1;
       }
@@ -1457,6 +1640,7 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
   if (tid == 0) {
     st->naug += naug; st->ncand_last = n; st->ncand = 0;
     st->trace[44] = (int)(t_rebuild >> 10); st->trace[45] = (int)(t_bf >> 10); st->trace[46] = (int)(t_move >> 10); st->trace[47] = bf_rounds; st->trace[41] = (int)q_total; st->trace[42] = (int)(t_first >> 10);   // kilo-cycles
+    st->trace[34] = (int)(t_who >> 10); st->trace[35] = (int)(t_patch >> 10); st->trace[36] = (int)(t_fix >> 10); st->trace[37] = n_arcs;
   }
 }
 

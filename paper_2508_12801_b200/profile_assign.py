@@ -34,7 +34,7 @@ def main():
               f"aug={st.augmentations} rounds={st.rounds} cand={st.candidates}")
         base = (ctx.workspace.data_ptr() + 255) // 256 * 256 - ctx.workspace.data_ptr()
         tr = ctx.workspace[base:base + 512].cpu().numpy().view("int32")
-        print("  exact-phase kilo-cycles (rebuild, path search, moves), path-search rounds, of the last round run:", tr[44:48].tolist(), "price-update tail cycles:", int(tr[40]) * 16, "queue entries:", int(tr[41]), "first rebuild kc:", int(tr[42]), "tail parts (arrive, prices, zero, rest):", tr[30:34].tolist())
+        print("  exact-phase kilo-cycles (rebuild, path search, moves), path-search rounds, of the last round run:", tr[44:48].tolist(), "queue entries:", int(tr[41]), "first rebuild kc:", int(tr[42]), "moves split (find token, patch, recompute) kc and arcs moved:", tr[34:38].tolist())
         print("  rows scanned in full per sweep:", tr[64:64 + st.sweeps].tolist())
 
 
