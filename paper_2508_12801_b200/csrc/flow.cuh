@@ -387,7 +387,9 @@ struct SweepShared {
 __device__ __forceinline__ void emit_margin(unsigned* hist, long long* mins, const int* caplog, int e, long long m) {
   if (m >= 0 && m < (1LL << caplog[e])) {
     atomicAdd(&hist[e * kNB + log_bin(m)], 1u);
-    atomicMin(&mins[e], m);                             // the exact smallest margin, for steps that move one token
+    // the exact smallest margin, for steps that move one token; it only ever drops, so a stale read
+    // can only let a useless atomic through
+    if (m < __ldcg(&mins[e])) atomicMin(&mins[e], m);
   }
 }
 
@@ -1093,10 +1095,9 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
     }
     __syncthreads();
     for (int e = tid; e < E; e += blockDim.x) s.dirty[e] = 0;
-    if (tid == 0) {
-      int any = 0;
-      for (int v = 0; v <= E; ++v) any |= (s.imb[v] > 0);
-      s.any_pos = any;
+    {
+      const int any = __syncthreads_or(tid <= E && s.imb[tid] > 0);
+      if (tid == 0) s.any_pos = any;
     }
     __syncthreads();
     { const long long t1 = clock64(); t_rebuild += t1 - t0; if (t_first == -1) t_first = t1 - t0; t0 = t1; }
@@ -1180,11 +1181,17 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
           __syncthreads();
           if (tid <= E) { s.dist[0][tid] = dv; s.pred[tid] = pv; }
           __syncthreads();
-          if (tid == 0) {
-            int t = -1; long long dt = kInf;
-            for (int v = 0; v <= E; ++v)
+          if (warp == 0) {
+            long long dt = kInf; int t = 0x7fffffff;
+            for (int v = lane; v <= E; v += 32)
               if (s.imb[v] < 0 && s.dist[0][v] < dt) { dt = s.dist[0][v]; t = v; }
-            s.target = t; s.dt = dt;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+              const long long od = __shfl_xor_sync(0xffffffffu, dt, o);
+              const int ot = __shfl_xor_sync(0xffffffffu, t, o);
+              if (od < dt || (od == dt && ot < t)) { dt = od; t = ot; }
+            }
+            if (lane == 0) { s.target = dt < kInf ? t : -1; s.dt = dt; }
           }
           __syncthreads();
           have_paths = s.target >= 0;
@@ -1287,20 +1294,28 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
     __syncthreads();
     const int cur = 0;
     // ---- nearest node with a deficit; would the price update stay within theta? -----------------------
-    if (tid == 0) {
+    if (warp == 0) {
       const int t = s.target; const long long dt = s.dt;
-      s.npath = 0;
+      if (lane == 0) s.npath = 0;
       if (t >= 0) {
-        int len = 0, v = t;
-        while (v >= 0 && len <= E + 1) { s.path[len++] = v; v = s.pred[v]; }
-        s.npath = len;
+        if (lane == 0) {
+          int len = 0, v = t;
+          while (v >= 0 && len <= E + 1) { s.path[len++] = v; v = s.pred[v]; }
+          s.npath = len;
+        }
         long long lo = kInf, hi = -kInf;
-        for (int e = 0; e < E; ++e) {
+        for (int e = lane; e < E; e += 32) {
           const long long d = s.dist[cur][e];
           const long long chg = s.p[e] - (d < dt ? d : dt) - s.p0[e];
           lo = chg < lo ? chg : lo; hi = chg > hi ? chg : hi;
         }
-        if (theta < kInf && hi - lo > theta) s.target = -2;   // stop here; the next round lists more tokens
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const long long ol = __shfl_xor_sync(0xffffffffu, lo, o), oh = __shfl_xor_sync(0xffffffffu, hi, o);
+          lo = ol < lo ? ol : lo; hi = oh > hi ? oh : hi;
+        }
+        __syncwarp();
+        if (lane == 0 && theta < kInf && hi - lo > theta) s.target = -2;   // stop here; the next round lists more tokens
       }
     }
     __syncthreads();
