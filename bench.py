@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 
 METRIC = "routed tokens/s per MoE layer (gate->flow->dispatch) on 1 B200; % of roofline"
 UNIT = "tokens/s"
-SWEEPS, ROUNDS = 24, 4
+SWEEPS, ROUNDS = 24, 6
 
 
 def launches_per_step():

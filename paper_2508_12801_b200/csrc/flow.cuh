@@ -683,6 +683,44 @@ flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every) {
   }
 }
 
+// Exact selection over one row held by a warp (lane l: entries l, l+32, ...).  Picks the `count`
+// largest values (larger value first, lower expert index first on equal values), sets sel[] for the first
+// `nsel` of them, and returns the values picked as number nsel (v_a) and nsel+1 (v_b), where reached.
+// A 64-bit maximum is taken as three 32-bit warp reductions: high word, low word among the lanes that
+// match the high word, lowest index among the entries that match both.
+__device__ __forceinline__ void warp_select(const long long (&val)[kEPLf], int E, int count, bool (&sel)[kEPLf],
+                                            long long& v_a, long long& v_b, int nsel) {
+  const int lane = threadIdx.x & 31;
+  unsigned hi[kEPLf], lo[kEPLf]; bool gone[kEPLf];
+#pragma unroll
+  for (int q = 0; q < kEPLf; ++q) {
+    const unsigned long long u = (unsigned long long)val[q] ^ 0x8000000000000000ULL;   // order-preserving
+    hi[q] = (unsigned)(u >> 32); lo[q] = (unsigned)u;
+    gone[q] = lane + 32 * q >= E;
+    sel[q] = false;
+  }
+  for (int r = 0; r < count && r < E; ++r) {
+    unsigned mh = 0;
+#pragma unroll
+    for (int q = 0; q < kEPLf; ++q) if (!gone[q]) mh = max(mh, hi[q]);
+    const unsigned bh = __reduce_max_sync(0xffffffffu, mh);
+    unsigned ml = 0;
+#pragma unroll
+    for (int q = 0; q < kEPLf; ++q) if (!gone[q] && hi[q] == bh) ml = max(ml, lo[q]);
+    const unsigned bl = __reduce_max_sync(0xffffffffu, ml);
+    unsigned me = 0xffffffffu;
+#pragma unroll
+    for (int q = 0; q < kEPLf; ++q) if (!gone[q] && hi[q] == bh && lo[q] == bl) me = min(me, (unsigned)(lane + 32 * q));
+    const unsigned be = __reduce_min_sync(0xffffffffu, me);
+    const long long v = (long long)((((unsigned long long)bh << 32) | bl) ^ 0x8000000000000000ULL);
+    if (r == nsel - 1) v_a = v;
+    if (r == nsel) v_b = v;
+#pragma unroll
+    for (int q = 0; q < kEPLf; ++q)
+      if ((unsigned)(lane + 32 * q) == be) { gone[q] = true; if (r < nsel) sel[q] = true; }
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Collect / verify pass.  round 0 picks every token's top-k under the sweep prices.  Later rounds
 // keep a token's experts when they still are a top-k under the current prices (ties included) and
@@ -705,83 +743,92 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
   if (threadIdx.x == 0) { s_viol = 0; s_rer = 0; s_score = 0.0; s_flags = 0; }
   __syncthreads();
   const long long theta = unbounded ? kInf : st->theta;   // the last round lists every token
-  extern __shared__ __align__(16) float collect_tile[];
-  const int tok0 = blockIdx.x * blockDim.x;
-  stage_rows(M, collect_tile, tok0, min((int)blockDim.x, T - tok0), E);
-  __syncthreads();
-  const int tok = tok0 + threadIdx.x;
-  if (tok < T) {
-    unsigned held[4] = {0, 0, 0, 0};
-    if (!first)
-      for (int c = 0; c < k; ++c) {
-        int e = expert_idx[(size_t)tok * k + c];
-        if (e >= 0 && e < E) held[e >> 5] |= 1u << (e & 31);
-      }
-    long long v[kTopN]; int id[kTopN];
-    long long min_held = kInf, max_non = -kInf;
-    const float* row = collect_tile + (size_t)threadIdx.x * E;
+  // One warp per token, lane l holds experts l, l+32, l+64, l+96: coalesced row loads, exact int64
+  // values in registers, every decision by warp votes and reductions.
+  const int lane = threadIdx.x & 31;
+  const int wid = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), nwarp = gridDim.x * (blockDim.x >> 5);
+  int w_viol = 0, w_rer = 0; double w_score = 0.0; bool w_bad = false;
+  for (int tok = wid; tok < T; tok += nwarp) {
+    const float* row = M + (size_t)tok * E;
     const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-    const int start = threadIdx.x % E;
-    bool bad = false;
-    if (!first) {                                     // exact check of the experts the token holds now
-      int e = start;
-      for (int jj = 0; jj < E; ++jj) {
-        const float x = row[e];
-        bad |= !isfinite(x);
-        const long long val = make_key(g, x, flat + e) - sp[e];
-        if (held[e >> 5] >> (e & 31) & 1u) min_held = val < min_held ? val : min_held;
-        else max_non = val > max_non ? val : max_non;
-        if (++e == E) e = 0;
-      }
-    }
-    const bool repick = !verify_only && (first || min_held < max_non);
-    if (repick) select_top(row, sp, spf, g, flat, E, start, true, v, id);
-    long long kth_raw = -kInf;                        // k-th largest raw key: the token's own top-k boundary
-    if (verify_only) {
-      long long rv[kTopN]; int rid[kTopN];
-      select_top(row, (const long long*)nullptr, (const float*)nullptr, g, flat, E, start, true, rv, rid);
+    float x[kEPLf]; long long key[kEPLf], val[kEPLf]; bool in[kEPLf];
+    int mine = -1;
+    if (!first && lane < k) mine = expert_idx[(size_t)tok * k + lane];
 #pragma unroll
-      for (int j = 0; j < kTopN; ++j) if (j == k - 1) kth_raw = rv[j];
+    for (int q = 0; q < kEPLf; ++q) {
+      const int e = lane + 32 * q;
+      x[q] = e < E ? __ldg(row + e) : 0.f;
+      w_bad |= !isfinite(x[q]);
+      key[q] = e < E ? make_key(g, x[q], flat + e) : -kInf;
+      val[q] = e < E ? key[q] - sp[e] : -kInf;
+      in[q] = false;
     }
-    if (bad) atomicOr(&s_flags, 2u);
+    if (!first)
+      for (int j = 0; j < k; ++j) {
+        const int ej = __shfl_sync(0xffffffffu, mine, j);
+#pragma unroll
+        for (int q = 0; q < kEPLf; ++q) in[q] |= (ej == lane + 32 * q);
+      }
+    // exact check of the experts the token holds now: the worst held value against the best other one
+    long long min_held = kInf, max_non = -kInf;
+#pragma unroll
+    for (int q = 0; q < kEPLf; ++q) {
+      if (lane + 32 * q >= E) continue;
+      if (in[q]) min_held = val[q] < min_held ? val[q] : min_held;
+      else max_non = val[q] > max_non ? val[q] : max_non;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const long long a = __shfl_xor_sync(0xffffffffu, min_held, o), c = __shfl_xor_sync(0xffffffffu, max_non, o);
+      min_held = a < min_held ? a : min_held; max_non = c > max_non ? c : max_non;
+    }
     const bool keep = !first && (min_held >= max_non);
-    long long gap;
-    if (!keep) {
-      if (!first) atomicAdd(&s_viol, 1);
-      if (!verify_only) {
-        held[0] = held[1] = held[2] = held[3] = 0;
+    const bool repick = !verify_only && !keep;
+    long long gap = keep ? ((E > k) ? min_held - max_non : kInf) : kInf;
+    if (!keep && !first) ++w_viol;
+    if (repick) {
+      long long vk = -kInf, vk1 = -kInf;
+      warp_select(val, E, k + 1, in, vk, vk1, k);
+      gap = (E > k) ? vk - vk1 : kInf;
+    }
+    // the experts in ascending order: word q of the held mask is the vote over in[q]
+    unsigned words[kEPLf]; int below = 0;
 #pragma unroll
-        for (int j = 0; j < kMaxK; ++j)
-          if (j < k) held[id[j] >> 5] |= 1u << (id[j] & 31);
-        // the k-th value sits at v[k-1], the best alternative at v[k]
-        long long vk = -kInf, vk1 = -kInf;
+    for (int q = 0; q < kEPLf; ++q) words[q] = __ballot_sync(0xffffffffu, in[q]);
 #pragma unroll
-        for (int j = 0; j < kTopN; ++j) { if (j == k - 1) vk = v[j]; if (j == k) vk1 = v[j]; }
-        gap = (E > k) ? vk - vk1 : kInf;
-      } else gap = kInf;
-    } else gap = (E > k) ? min_held - max_non : kInf;
-    // write the experts in ascending order (bit order of the mask)
-    int c = 0;
-    double sc = 0.0; int rer = 0;
-    for (int wd = 0; wd < 4; ++wd) {
-      unsigned m = held[wd];
-      while (m) {
-        int e = (wd << 5) + __ffs(m) - 1; m &= m - 1;
-        if (c < k) expert_idx[(size_t)tok * k + c] = e;
-        ++c;
-        atomicAdd(&sload[e], 1);
-        if (verify_only) {
-          const float x = row[e];
-          const long long key = make_key(g, x, flat + e);
-          sc += (g.mode == 0) ? (double)x : (double)key;
-          if (key < kth_raw) ++rer;
-        }
+    for (int q = 0; q < kEPLf; ++q) {
+      if (in[q]) {
+        const int rank = below + __popc(words[q] & ((1u << lane) - 1u));
+        if (rank < k) expert_idx[(size_t)tok * k + rank] = lane + 32 * q;
+        atomicAdd(&sload[lane + 32 * q], 1);
       }
+      below += __popc(words[q]);
     }
-    if (verify_only) { atomicAdd(&s_score, sc); if (rer) atomicAdd(&s_rer, rer); }
-    if (!verify_only && gap < kInf && gap <= theta) {
-      cand[atomicAdd(&st->ncand, 1)] = tok;   // the list has room for every token
+    if (verify_only) {
+      // statistics: the score of the held pairs, and how many of them are not in the token's own top-k
+      bool none[kEPLf];
+#pragma unroll
+      for (int q = 0; q < kEPLf; ++q) none[q] = false;
+      long long kth_raw = -kInf, next_raw = -kInf;
+      warp_select(key, E, k, none, kth_raw, next_raw, k);
+      double sc = 0.0; int rer = 0;
+#pragma unroll
+      for (int q = 0; q < kEPLf; ++q)
+        if (in[q]) {
+          sc += (g.mode == 0) ? (double)x[q] : (double)key[q];
+          if (key[q] < kth_raw) ++rer;
+        }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) { sc += __shfl_xor_sync(0xffffffffu, sc, o); rer += __shfl_xor_sync(0xffffffffu, rer, o); }
+      w_score += sc; w_rer += rer;
     }
+    if (!verify_only && gap < kInf && gap <= theta && lane == 0)
+      cand[atomicAdd(&st->ncand, 1)] = tok;     // the list has room for every token
+  }
+  if (__any_sync(0xffffffffu, w_bad) && lane == 0) atomicOr(&s_flags, 2u);
+  if (lane == 0) {
+    if (w_viol) atomicAdd(&s_viol, w_viol);
+    if (verify_only) { atomicAdd(&s_score, w_score); if (w_rer) atomicAdd(&s_rer, w_rer); }
   }
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += blockDim.x)

@@ -204,7 +204,7 @@ maxscore_status launch_softtopk_fwd(maxscore_ctx* c, const float* logits, float*
   return MAXSCORE_OK;
 }
 
-constexpr int kSweeps = 24, kRounds = 4, kDefaultAug = 4096;
+constexpr int kSweeps = 24, kRounds = 6, kDefaultAug = 4096;
 
 maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_idx, int32_t* expert_load,
                               maxscore_stats* stats, cudaStream_t st) {
@@ -216,7 +216,7 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   const long long eps0 = 1LL << (scale_bits - 10);
   const long long eps_min = p.score_mode == 0 ? (1LL << 20) : (1LL << 12);
   const int cap0 = kCapLogMax;   // the first sweep records every margin
-  const long long theta0 = 1LL << (scale_bits - 13);
+  const long long theta0 = 1LL << (scale_bits - 15);
   const int balanced = ((long long)p.E * c->C == (long long)p.T * p.k) ? 1 : 0;
   const int budget = p.max_sweeps > 0 ? p.max_sweeps : kSweeps + kDefaultAug;
   const int n_sweeps = budget < kSweeps ? budget : kSweeps;
@@ -225,7 +225,6 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   flow_init_kernel<<<1, 256, 0, st>>>(fs, eps0, eps_min, cap0, theta0, balanced, p.E);
   MS_LAUNCH_CHECK("flow_init_kernel");
   const int blocks = (p.T + kSweepThreads - 1) / kSweepThreads;
-  const size_t tile_smem = sizeof(float) * (size_t)kSweepThreads * p.E;
   SweepCache cache{reinterpret_cast<float*>(c->ws + c->lay.cache_x), reinterpret_cast<unsigned char*>(c->ws + c->lay.cache_id),
                    reinterpret_cast<long long*>(c->ws + c->lay.cache_bound)};
   for (int s = 0; s < n_sweeps; ++s) {
@@ -237,16 +236,17 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   const size_t p2smem = sizeof(long long) * (size_t)p.E * (p.E | 1) + (size_t)kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache + 2 * kMaxArcs;
   long long* Dg = reinterpret_cast<long long*>(c->ws + c->lay.dmat);
   const int build_blocks = c->sm_count * 4;
+  const int collect_blocks = std::min((p.T + kSweepThreads / 32 - 1) / (kSweepThreads / 32), c->sm_count * 16);   // one warp per token
   for (int r = 0; r < kRounds; ++r) {
-    flow_collect_kernel<<<blocks, kSweepThreads, tile_smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, r == 0, 0,
-                                                         32LL, nullptr, nullptr, nullptr, r == kRounds - 1, Dg);
+    flow_collect_kernel<<<collect_blocks, kSweepThreads, 0, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, r == 0, 0,
+                                                         8LL, nullptr, nullptr, nullptr, r == kRounds - 1, Dg);
     MS_LAUNCH_CHECK("flow_collect_kernel");
     flow_build_kernel<<<build_blocks, 256, 0, st>>>(M, fs, expert_idx, cand, Dg, p.T, p.E, p.k, g);
     MS_LAUNCH_CHECK("flow_build_kernel");
     flow_exact_kernel<<<1, kP2Threads, p2smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, max_aug, Dg);
     MS_LAUNCH_CHECK("flow_exact_kernel");
   }
-  flow_collect_kernel<<<blocks, kSweepThreads, tile_smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, 0, 1, 32LL,
+  flow_collect_kernel<<<collect_blocks, kSweepThreads, 0, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, 0, 1, 32LL,
                                                        expert_load, stats, error_flag_of(c), 0, nullptr);
   MS_LAUNCH_CHECK("flow_collect_kernel(verify)");
   return MAXSCORE_OK;
@@ -322,7 +322,6 @@ maxscore_status maxscore_create(maxscore_ctx** out, const maxscore_params* param
     return MAXSCORE_ERR_CUDA;
   }
   MS_CUDA(cudaFuncSetAttribute(gate_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGateSmemBytes));
-  MS_CUDA(cudaFuncSetAttribute(flow_collect_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * kSweepThreads * kMaxE)));
   MS_CUDA(cudaFuncSetAttribute(flow_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kP2SmemMax));
   MS_CUDA(cudaFuncSetAttribute(dispatch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDispatchSmem));
   MS_CUDA(cudaFuncSetAttribute(gate_bwd_dh_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDhSmemMax));
