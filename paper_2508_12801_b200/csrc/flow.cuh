@@ -6,17 +6,22 @@
 // the E prices, never on the T x E arcs:
 //
 //   sweeps    (data parallel, one thread per token)  every token re-picks its top-k under the
-//             current prices; per expert a load count and two small histograms of margins (how much
-//             a price rise makes a holder leave / how much a price cut makes an outsider join) are
-//             collected; the last CTA to finish moves each over- or under-loaded expert's price to
-//             the histogram quantile that balances it, plus a step eps that is halved as the sweeps
-//             go on.  This is an epsilon-scaled simultaneous price adjustment (auction-style); it
-//             ends a few dozen token moves away from the optimum.
+//             current prices; per expert a load count, two histograms of margins (how much a price
+//             rise makes a holder leave / how much a price cut makes an outsider join) and the exact
+//             smallest margin are collected.  The first sweep scans whole rows and caches each
+//             token's 16 best experts with a bound on everything else; later sweeps re-evaluate the
+//             cached entries only, and rescan a row (one warp) when the bound no longer vouches for
+//             them.  A one-CTA kernel then moves each over- or under-loaded expert's price to the
+//             histogram quantile that balances it, plus a step eps that is halved as the sweeps go
+//             on; small imbalances move one exact margin at a time.  This is an epsilon-scaled
+//             simultaneous price adjustment (auction-style); it ends a few dozen token moves away
+//             from the optimum and stops early once a small imbalance has stopped shrinking.
 //   collect   every token's top-k under the final prices is written out; tokens whose k-th and
 //             (k+1)-th values differ by at most theta are listed as candidates.
+//   build     the cost matrix D[e][f] = cheapest move of one candidate token from e to f is built by
+//             the whole GPU (one warp per candidate, 64-bit atomicMin).
 //   exact     one CTA runs successive shortest augmenting paths on the expert-level residual graph
-//             (E experts + one node Z for the sink side), arcs e->f costing the cheapest candidate
-//             token move; node potentials keep reduced costs non-negative, so each search is a
+//             (E experts + one node Z for the sink side) with D as arc costs; node potentials keep reduced costs non-negative, so each search is a
 //             Bellman-Ford over E+1 nodes held in shared memory.  It ends with every expert within
 //             capacity and complementary slackness satisfied for the candidates.
 //   verify    a last data-parallel pass checks complementary slackness for EVERY token under the
@@ -109,24 +114,7 @@ __global__ void flow_init_kernel(FlowState* st, long long eps0, long long eps_mi
   }
 }
 
-// Insert (val, id) into a list sorted by descending value; on equal values the earlier (lower id,
-// because ids arrive ascending) entry stays in front.
-template <int N>
-__device__ __forceinline__ void top_insert(long long (&v)[N], int (&id)[N], long long val, int e) {
-  if (val > v[N - 1]) {
-    v[N - 1] = val; id[N - 1] = e;
-#pragma unroll
-    for (int j = N - 1; j > 0; --j) {
-      if (v[j] > v[j - 1]) {
-        long long tv = v[j]; v[j] = v[j - 1]; v[j - 1] = tv;
-        int ti = id[j]; id[j] = id[j - 1]; id[j - 1] = ti;
-      }
-    }
-  }
-}
-
-// Same, but with the order made explicit: larger value first, lower expert index first on equal values.
-// Needed where entries do not arrive in ascending index order.
+// Insert (val, id) into a list sorted by descending value, lower expert index first on equal values.
 template <int N>
 __device__ __forceinline__ void top_insert_tb(long long (&v)[N], int (&id)[N], long long val, int e) {
   if (val > v[N - 1] || (val == v[N - 1] && e < id[N - 1])) {
@@ -221,21 +209,6 @@ __device__ __forceinline__ void select_top(const float* row, const long long* sp
   for (e = 0; e < E; ++e) top_insert_tb(v, id, make_key(g, row[e], flat + e) - (sp ? sp[e] : 0), e);
 }
 
-// Copy the score rows of this CTA's tokens (contiguous in memory) into shared memory with coalesced
-// loads.  A thread then walks its own row starting at a column rotated by its index, so that the lanes
-// of a warp hit different banks although the rows are E floats apart.
-__device__ __forceinline__ void stage_rows(const float* __restrict__ M, float* tile, int tok0, int ntok, int E) {
-  const long long n = (long long)ntok * E;
-  const float* src = M + (size_t)tok0 * E;
-  if ((E & 3) == 0) {
-    const float4* s4 = reinterpret_cast<const float4*>(src);
-    float4* d4 = reinterpret_cast<float4*>(tile);
-    for (int i = threadIdx.x; i < n / 4; i += blockDim.x) d4[i] = __ldg(s4 + i);
-  } else {
-    for (int i = threadIdx.x; i < n; i += blockDim.x) tile[i] = __ldg(src + i);
-  }
-}
-
 __device__ __forceinline__ bool last_block_arrives(unsigned* ticket) {
   __shared__ bool is_last;
   __threadfence();
@@ -258,7 +231,6 @@ __device__ __forceinline__ int log_bin(long long m) {
   const int o = 63 - __clzll(m);
   return 4 * (o - 1) + (int)((m >> (o - 2)) & 3);
 }
-__device__ __forceinline__ int rel_bin(long long m, int) { return log_bin(m); }
 __device__ __forceinline__ long long bin_lower_edge(int b) {
   if (b < 4) return b;
   const int o = b / 4 + 1, sub = b & 3;
@@ -271,45 +243,7 @@ __device__ __forceinline__ long long bin_lower_edge(int b) {
 // Otherwise the step goes to the bin's upper edge plus eps (capped by the bin width).  `cut` is the
 // log2 of the largest margin the tokens were asked to record; if fewer than `need` lie below it the
 // step goes to 2^cut and the cut-off is lifted for the next sweep.
-__device__ __forceinline__ long long price_step(const unsigned* hist, int need, long long eps, int& cut,
-                                                bool& window_short, int cut_max) {
-  window_short = false;
-  const int base = 0;
-  const int nb = min(kNB, 4 * cut);                   // bins at or above 2^cut are empty
-  unsigned cum = 0, before = 0; int pos = -1, last = -1;
-  for (int b0 = 0; b0 < nb && pos < 0; b0 += 16) {
-    uint4 h[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) h[q] = __ldcg(reinterpret_cast<const uint4*>(hist + b0) + q);
-    const unsigned* hv = reinterpret_cast<const unsigned*>(h);
-#pragma unroll
-    for (int q = 0; q < 16; ++q) {
-      if (pos < 0) {
-        if (cum + hv[q] >= (unsigned)need) { pos = b0 + q; before = cum; }
-        if (hv[q]) last = b0 + q;
-        cum += hv[q];
-      }
-    }
-  }
-  if (pos < 0) {
-    // fewer than `need` margins were recorded.  Under a cut-off, everything below it may move; with
-    // no cut-off, move what was recorded (an outsider list can be incomplete) and ask for a full scan.
-    const long long step = cut < cut_max ? (1LL << cut) : (last >= 0 ? bin_lower_edge(last + 1 + base) : 0);
-    cut = cut_max;
-    window_short = true;
-    return step;
-  }
-  const long long lo = pos == 0 ? 0 : bin_lower_edge(pos + base), hi = bin_lower_edge(pos + 1 + base);
-  cut = min(cut_max, max(12, ((pos + base) >> 2) + 5));   // next sweep: record up to ~16x this margin
-  (void)before;
-  if (cum <= 2u * (unsigned)need || lo == 0) {
-    const long long w = hi - lo;
-    return hi + (eps < w ? eps : w);
-  }
-  return lo;                                          // conservative: moves `before` < need tokens
-}
-
-// The same step computed by a whole warp: lane l holds bins 8l .. 8l+7 of the expert's histogram.
+// Computed by a whole warp: lane l holds bins 8l .. 8l+7 of the expert's histogram.
 __device__ __forceinline__ long long price_step_warp(const uint4& ha, const uint4& hb, int need, long long eps, int& cut,
                                                      bool& window_short, int cut_max, long long m1) {
   const int lane = threadIdx.x & 31;
@@ -734,12 +668,11 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
   if (Dg)   // the move-cost matrix the build kernel fills next starts out empty
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < E * (E | 1); i += gridDim.x * blockDim.x) Dg[i] = kInf;
   __shared__ long long sp[kMaxE];
-  __shared__ float spf[kMaxE];
   __shared__ int sload[kMaxE];
   __shared__ int s_viol, s_rer;
   __shared__ double s_score;
   __shared__ unsigned s_flags;
-  for (int e = threadIdx.x; e < E; e += blockDim.x) { sp[e] = st->p[e]; spf[e] = (float)sp[e]; sload[e] = 0; }
+  for (int e = threadIdx.x; e < E; e += blockDim.x) { sp[e] = st->p[e]; sload[e] = 0; }
   if (threadIdx.x == 0) { s_viol = 0; s_rer = 0; s_score = 0.0; s_flags = 0; }
   __syncthreads();
   const long long theta = unbounded ? kInf : st->theta;   // the last round lists every token

@@ -116,7 +116,6 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 constexpr int kP2SmemMax = (int)(sizeof(long long) * kMaxE * (kMaxE | 1) + kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache + 2 * kMaxArcs);
-constexpr int kDispatchSmem = 64 * 1024;
 constexpr int kDhSmemMax = 2 * 2 * 16384 + kDhStages * 2 * 16384 + 2 * 128 * kDhOutStride + 1024;     // Kpad = 128
 constexpr int kDwSmemMax = kDwStages * (16384 + 2 * 2 * 8192) + 1024;
 
@@ -323,7 +322,6 @@ maxscore_status maxscore_create(maxscore_ctx** out, const maxscore_params* param
   }
   MS_CUDA(cudaFuncSetAttribute(gate_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGateSmemBytes));
   MS_CUDA(cudaFuncSetAttribute(flow_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kP2SmemMax));
-  MS_CUDA(cudaFuncSetAttribute(dispatch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDispatchSmem));
   MS_CUDA(cudaFuncSetAttribute(gate_bwd_dh_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDhSmemMax));
   MS_CUDA(cudaFuncSetAttribute(gate_bwd_dw_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDwSmemMax));
   MS_CUDA(cudaMemsetAsync(workspace, 0, lay.cand, 0));
@@ -404,17 +402,8 @@ maxscore_status maxscore_dispatch(maxscore_ctx* c, const void* src, const int32_
   if (!aligned16(src) || !aligned16(dst)) return MAXSCORE_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   const maxscore_params& p = c->p;
-  DispatchArgs a{};
-  a.src = (const char*)src; a.dst = (char*)dst; a.expert_idx = expert_idx; a.slot_idx = slot_idx;
-  a.T = p.T; a.k = p.k; a.C = c->C;
-  a.row_bytes = (uint32_t)(p.d_model * elem_bytes(c));
-  a.chunk_bytes = a.row_bytes < 8192 ? (uint32_t)align_up(a.row_bytes, 128) : 8192;
-  a.chunks_per_row = (a.row_bytes + a.chunk_bytes - 1) / a.chunk_bytes;
-  a.stages = (int)(kDispatchSmem / a.chunk_bytes); if (a.stages > 16) a.stages = 16;
-  a.error_flag = error_flag_of(c);
-  const long long units = (long long)p.T * a.chunks_per_row;
-  long long grid = c->sm_count * 3; if (grid > units) grid = units;
-  dispatch_kernel<<<(int)grid, 32, (size_t)a.stages * a.chunk_bytes, st>>>(a);
+  const uint32_t row_bytes = (uint32_t)(p.d_model * elem_bytes(c));
+  dispatch_kernel<<<c->sm_count * 8, 256, 0, st>>>((const char*)src, expert_idx, slot_idx, (char*)dst, p.T, row_bytes, p.k, c->C);
   MS_LAUNCH_CHECK("dispatch_kernel");
   return launch_zero_padding(c, slot_token, dst, st);
 }
