@@ -83,8 +83,9 @@ index_fill_kernel(const int32_t* __restrict__ expert_idx, const int32_t* __restr
 // every row is read once and written k times.  (A variant that staged rows through a shared-memory
 // ring of 1-D bulk copies driven by one thread per CTA measured 0.86 of the HBM copy peak on the
 // write-heavy stress shape; this one measures 0.91.)
-// One warp per token, a lane owns 16-byte column groups, four groups are loaded (streaming loads)
-// before their 4*k copies are stored (streaming stores).
+// One warp per token, a lane owns 16-byte column groups, kDispatchBatch groups are loaded (streaming
+// loads) before their copies are stored (streaming stores).
+constexpr int kDispatchBatch = 4;     // 16-byte groups a lane loads before it stores their copies
 __global__ void __launch_bounds__(256)
 dispatch_kernel(const char* __restrict__ src, const int32_t* __restrict__ expert_idx,
                      const int32_t* __restrict__ slot_idx, char* __restrict__ dst, int Tn, uint32_t row_bytes,
@@ -102,16 +103,16 @@ dispatch_kernel(const char* __restrict__ src, const int32_t* __restrict__ expert
 #pragma unroll
     for (int c = 0; c < kMaxK; ++c) off[c] = __shfl_sync(0xffffffffu, my_off, c);
     const uint4* srow = reinterpret_cast<const uint4*>(src + (size_t)tok * row_bytes);
-    for (uint32_t v0 = lane; v0 < nvec; v0 += 128) {
-      uint4 x[4];
+    for (uint32_t v0 = lane; v0 < nvec; v0 += 32 * kDispatchBatch) {
+      uint4 x[kDispatchBatch];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) if (v0 + 32 * u < nvec) x[u] = __ldcs(srow + v0 + 32 * u);
+      for (int u = 0; u < kDispatchBatch; ++u) if (v0 + 32 * u < nvec) x[u] = __ldcs(srow + v0 + 32 * u);
 #pragma unroll
       for (int c = 0; c < kMaxK; ++c) {
         if (c >= k || off[c] < 0) continue;
         uint4* drow = reinterpret_cast<uint4*>(dst + off[c]);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) if (v0 + 32 * u < nvec) __stcs(drow + v0 + 32 * u, x[u]);
+        for (int u = 0; u < kDispatchBatch; ++u) if (v0 + 32 * u < nvec) __stcs(drow + v0 + 32 * u, x[u]);
       }
     }
   }
