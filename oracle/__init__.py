@@ -281,6 +281,14 @@ def aux_loss(A, expert_idx, lam: float) -> float:
     return float(lib().mso_aux_loss(I64(T), I64(E), I64(idx.shape[1]), C.c_double(lam), _p(A), _p(idx)))
 
 
+def aux_loss_grad(expert_idx, T: int, E: int, lam: float) -> np.ndarray:
+    """dL_aux/dA_ij (Eq. 9, P constant): one value per expert j, the same for every token."""
+    idx = _i32(expert_idx)
+    out = np.empty(E, np.float64)
+    lib().mso_aux_loss_grad(I64(T), I64(E), I64(idx.shape[1]), C.c_double(lam), _p(idx), _p(out))
+    return out
+
+
 def gate_weights(A, expert_idx) -> np.ndarray:
     """R(x)_e = P_ie * A_ie at the assigned pairs, not renormalised (Eq. 1-2)."""
     A = np.asarray(A)

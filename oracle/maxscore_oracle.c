@@ -663,3 +663,16 @@ double mso_aux_loss(int64_t T, int64_t E, int64_t k, double lambda, const double
   }
   return lambda * tot / (double)E;
 }
+
+/* Gradient of Eq. 9 with respect to the affinities, P held constant (it is  */
+/* binary): dL_aux/dA_ij = lambda / (e n^2) * sum_i' P_i'j, the same for     */
+/* every token i, so one value per expert is returned.                       */
+void mso_aux_loss_grad(int64_t T, int64_t E, int64_t k, double lambda, const int32_t *expert_idx,
+                       double *dA_col) {
+  for (int64_t j = 0; j < E; ++j) {
+    double sp = 0.0;
+    for (int64_t i = 0; i < T; ++i)
+      for (int64_t c = 0; c < k; ++c) if (expert_idx[i * k + c] == j) sp += 1.0;
+    dA_col[j] = lambda * sp / ((double)E * (double)T * (double)T);
+  }
+}

@@ -149,3 +149,22 @@ def test_aux_loss_eq9(orc):
     P = np.zeros((T, E)); np.put_along_axis(P, idx.astype(np.int64), 1.0, axis=1)
     want = lam / E * (A.mean(0) * P.mean(0)).sum()
     assert abs(orc.aux_loss(A, idx, lam) - want) < 1e-15
+
+
+def test_aux_loss_grad_matches_finite_differences(orc):
+    """Eq. 9 is linear in A, so a central difference of the loss itself is exact up to rounding."""
+    rng = np.random.default_rng(5)
+    T, E, k, lam = 24, 6, 2, 3e-2
+    A = rng.random((T, E))
+    idx = np.sort(np.argsort(-A, axis=1)[:, :k], axis=1).astype(np.int32)
+    g = orc.aux_loss_grad(idx, T, E, lam)
+    assert g.shape == (E,)
+    h = 1e-3
+    for (i, j) in [(0, 0), (5, 3), (23, 5), (11, 1)]:
+        Ap, Am = A.copy(), A.copy()
+        Ap[i, j] += h; Am[i, j] -= h
+        fd = (orc.aux_loss(Ap, idx, lam) - orc.aux_loss(Am, idx, lam)) / (2 * h)
+        assert abs(fd - g[j]) < 1e-12
+    # closed form: lambda / (E T^2) * load_j
+    load = np.bincount(idx.ravel(), minlength=E)
+    np.testing.assert_allclose(g, lam * load / (E * T * T), rtol=1e-14)
