@@ -170,6 +170,23 @@ maxscore_status maxscore_softtopk_bwd(maxscore_ctx* ctx, const float* logits,
                                       const int32_t* expert_idx, const float* dgate_w,
                                       float* dlogits, void* cuda_stream);
 
+/* Auxiliary load-balance loss, Eq. 9: loss = lambda / (E T^2) * sum_j (sum_i scores[i, j]) * expert_load[j]
+ * (the column sum of the binary P is the expert's load), and its gradient with respect to the scores with
+ * P held constant, which is the same for every token: dscores_col[j] = lambda * expert_load[j] / (E T^2).
+ * scores [T, E] fp32, expert_load [E] int32, loss: one double, dscores_col [E] fp32; all device memory,
+ * caller-owned.  Uses the context's workspace (calls on one context must not overlap).  Column sums are
+ * accumulated in double with atomics, so the loss is reproducible to rounding (about 1e-15 relative), not
+ * bit for bit.  Errors: NULL arguments -> MAXSCORE_ERR_INVALID_ARG. */
+maxscore_status maxscore_aux_loss(maxscore_ctx* ctx, const float* scores, const int32_t* expert_load,
+                                  float lambda, double* loss, float* dscores_col, void* cuda_stream);
+
+/* maxscore_softtopk_bwd with the auxiliary loss folded in: g[i, j] = dscores_col[j] for every expert j, plus
+ * dgate_w[i, c] at j = expert_idx[i, c]; dlogits = J^T g (derivative of Eq. 6 applied to the sum of the
+ * gradients of Eq. 1 and Eq. 9). */
+maxscore_status maxscore_softtopk_bwd_aux(maxscore_ctx* ctx, const float* logits, const int32_t* expert_idx,
+                                          const float* dgate_w, const float* dscores_col, float* dlogits,
+                                          void* cuda_stream);
+
 /* Eq. 7-8 only: the solver on a caller-supplied [T, E] fp32 matrix (affinities in score_mode 0,
  * logits in score_mode 1).  Writes expert_idx [T, k], expert_load [E] and stats. */
 maxscore_status maxscore_assign(maxscore_ctx* ctx, const float* matrix, int32_t* expert_idx,

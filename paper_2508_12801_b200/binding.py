@@ -45,7 +45,8 @@ EXPORTS = ["maxscore_capacity", "maxscore_workspace_bytes", "maxscore_create", "
            "maxscore_last_cuda_error", "maxscore_route_fwd", "maxscore_dispatch", "maxscore_combine",
            "maxscore_route_bwd", "maxscore_gate", "maxscore_softtopk_fwd", "maxscore_softtopk_bwd",
            "maxscore_assign", "maxscore_index_build", "maxscore_combine_bwd", "maxscore_gate_bwd",
-           "maxscore_route_dispatch_host", "maxscore_index_build_noalloc"]
+           "maxscore_route_dispatch_host", "maxscore_index_build_noalloc", "maxscore_aux_loss",
+           "maxscore_softtopk_bwd_aux"]
 
 
 def _load():
@@ -182,6 +183,17 @@ def softtopk_fwd(ctx, logits, scores, stream=None):
 def softtopk_bwd(ctx, logits, expert_idx, dgate_w, dlogits, stream=None):
     _check(_lib.maxscore_softtopk_bwd(ctx.handle, _ptr(logits), _ptr(expert_idx), _ptr(dgate_w), _ptr(dlogits),
                                       _stream(stream)), "maxscore_softtopk_bwd")
+
+
+def softtopk_bwd_aux(ctx, logits, expert_idx, dgate_w, dscores_col, dlogits, stream=None):
+    _check(_lib.maxscore_softtopk_bwd_aux(ctx.handle, _ptr(logits), _ptr(expert_idx), _ptr(dgate_w), _ptr(dscores_col),
+                                          _ptr(dlogits), _stream(stream)), "maxscore_softtopk_bwd_aux")
+
+
+def aux_loss(ctx, scores, expert_load, lam, loss, dscores_col, stream=None):
+    """Eq. 9 and its gradient: loss is a 1-element float64 device tensor, dscores_col an [E] float32 one."""
+    _check(_lib.maxscore_aux_loss(ctx.handle, _ptr(scores), _ptr(expert_load), C.c_float(lam), _ptr(loss),
+                                  _ptr(dscores_col), _stream(stream)), "maxscore_aux_loss")
 
 
 def assign(ctx, matrix, expert_idx, expert_load, stats, stream=None):

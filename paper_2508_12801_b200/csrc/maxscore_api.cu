@@ -50,7 +50,7 @@ int32_t capacity_of(const maxscore_params& p) {
 }
 
 struct Layout {          // byte offsets inside the workspace
-  size_t state, cand, dmat, cache_x, cache_id, cache_bound, block_counts, wt, error_flag, dls, wk, dwpart, total;
+  size_t state, aux, cand, dmat, cache_x, cache_id, cache_bound, block_counts, wt, error_flag, dls, wk, dwpart, total;
   int Npad, n_idx_blocks;
   int Kpad, dw_splits, dw_tokens_per_split;   // tensor-core backward GEMMs (bf16 I/O)
 };
@@ -62,6 +62,7 @@ Layout layout_of(const maxscore_params& p) {
   size_t off = 0;
   l.state = off; off = align_up(off + sizeof(FlowState), 256);
   l.error_flag = off; off = align_up(off + 16, 256);
+  l.aux = off; off = align_up(off + sizeof(double) * kMaxE + 16, 256);     // column sums + ticket of the auxiliary loss
   l.cand = off; off = align_up(off + sizeof(int32_t) * (size_t)p.T, 256);
   l.dmat = off; off = align_up(off + sizeof(long long) * (size_t)p.E * (p.E | 1), 256);
   l.cache_x = off; off = align_up(off + sizeof(float) * (size_t)kCacheN * p.T, 256);
@@ -353,8 +354,30 @@ maxscore_status maxscore_softtopk_bwd(maxscore_ctx* c, const float* logits, cons
   if (!c || !logits || !expert_idx || !dgate_w || !dlogits) return MAXSCORE_ERR_INVALID_ARG;
   const maxscore_params& p = c->p;
   int blocks = (p.T + 7) / 8; if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
-  softtopk_bwd_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, dlogits, p.T, p.E, p.k, p.t);
+  softtopk_bwd_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, nullptr, dlogits, p.T, p.E, p.k, p.t);
   MS_LAUNCH_CHECK("softtopk_bwd_kernel");
+  return MAXSCORE_OK;
+}
+
+maxscore_status maxscore_softtopk_bwd_aux(maxscore_ctx* c, const float* logits, const int32_t* expert_idx,
+                                          const float* dgate_w, const float* dscores_col, float* dlogits, void* stream) {
+  if (!c || !logits || !expert_idx || !dgate_w || !dscores_col || !dlogits) return MAXSCORE_ERR_INVALID_ARG;
+  const maxscore_params& p = c->p;
+  int blocks = (p.T + 7) / 8; if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
+  softtopk_bwd_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, dscores_col, dlogits, p.T, p.E, p.k, p.t);
+  MS_LAUNCH_CHECK("softtopk_bwd_kernel");
+  return MAXSCORE_OK;
+}
+
+maxscore_status maxscore_aux_loss(maxscore_ctx* c, const float* scores, const int32_t* expert_load, float lambda,
+                                  double* loss, float* dscores_col, void* stream) {
+  if (!c || !scores || !expert_load || !loss || !dscores_col) return MAXSCORE_ERR_INVALID_ARG;
+  const maxscore_params& p = c->p;
+  double* colsum = reinterpret_cast<double*>(c->ws + c->lay.aux);
+  unsigned* ticket = reinterpret_cast<unsigned*>(c->ws + c->lay.aux + sizeof(double) * kMaxE);
+  int blocks = (p.T + 7) / 8; if (blocks > c->sm_count * 4) blocks = c->sm_count * 4;
+  aux_loss_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>(scores, expert_load, colsum, ticket, loss, dscores_col, p.T, p.E, lambda);
+  MS_LAUNCH_CHECK("aux_loss_kernel");
   return MAXSCORE_OK;
 }
 

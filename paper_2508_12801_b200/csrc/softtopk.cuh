@@ -74,12 +74,13 @@ softtopk_fwd_kernel(const float* __restrict__ logits, float* __restrict__ scores
   }
 }
 
-// dlogits = J^T g with g non-zero only at the token's k assigned experts.  The masks are constants.
+// dlogits = J^T g with g = the k gradients of the token's assigned experts plus, if given, a per-expert
+// term shared by all tokens (the gradient of the auxiliary loss, Eq. 9).  The masks are constants.
 //   da_l = (1/t) * sum_{levels j with l unmasked} q_l * (g_l - sum_i g_i q_i),  q = level-j softmax
 __global__ void __launch_bounds__(256)
 softtopk_bwd_kernel(const float* __restrict__ logits, const int32_t* __restrict__ expert_idx,
-                    const float* __restrict__ dgate_w, float* __restrict__ dlogits, int T, int E, int k,
-                    float t) {
+                    const float* __restrict__ dgate_w, const float* __restrict__ dscores_col,
+                    float* __restrict__ dlogits, int T, int E, int k, float t) {
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
   for (int tok = blockIdx.x * warps_per_block + (threadIdx.x >> 5); tok < T;
@@ -92,14 +93,14 @@ softtopk_bwd_kernel(const float* __restrict__ logits, const int32_t* __restrict_
       int e = lane + 32 * j;
       live[j] = e < E;
       a[j] = live[j] ? __ldg(row + e) : 0.f;
-      g[j] = 0.f; da[j] = 0.f;
+      g[j] = (live[j] && dscores_col) ? __ldg(dscores_col + e) : 0.f; da[j] = 0.f;
     }
     for (int c = 0; c < k; ++c) {
       int e = __ldg(expert_idx + (size_t)tok * k + c);
       float gv = __ldg(dgate_w + (size_t)tok * k + c);
 #pragma unroll
       for (int j = 0; j < kEPL; ++j)
-        if (lane + 32 * j == e) g[j] = gv;
+        if (lane + 32 * j == e) g[j] += gv;
     }
     float z[kEPL];
     float ref = 0.f;
@@ -134,6 +135,60 @@ softtopk_bwd_kernel(const float* __restrict__ logits, const int32_t* __restrict_
       int e = lane + 32 * j;
       if (e < E) out[e] = da[j];
     }
+  }
+}
+
+// Auxiliary load-balance loss, Eq. 9: L = lambda / (E T^2) * sum_j (sum_i A_ij) * load_j, and its
+// gradient with respect to A (P is a constant): dL/dA_ij = lambda * load_j / (E T^2) for every token i.
+// Column sums are taken by warps over rows (lane l owns columns l, l+32, ...) in double precision and
+// merged with one atomic per column and CTA; the last CTA to finish forms the loss and clears the scratch.
+__global__ void __launch_bounds__(256)
+aux_loss_kernel(const float* __restrict__ scores, const int32_t* __restrict__ expert_load, double* colsum,
+                unsigned* ticket, double* __restrict__ loss, float* __restrict__ dscores_col, int T, int E,
+                float lambda) {
+  __shared__ double ssum[kMaxE];
+  __shared__ bool is_last;
+  for (int e = threadIdx.x; e < E; e += blockDim.x) ssum[e] = 0.0;
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  double acc[kEPL];
+#pragma unroll
+  for (int j = 0; j < kEPL; ++j) acc[j] = 0.0;
+  for (int tok = blockIdx.x * warps_per_block + (threadIdx.x >> 5); tok < T; tok += gridDim.x * warps_per_block) {
+    const float* row = scores + (size_t)tok * E;
+#pragma unroll
+    for (int j = 0; j < kEPL; ++j) {
+      const int e = lane + 32 * j;
+      if (e < E) acc[j] += (double)__ldg(row + e);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < kEPL; ++j) {
+    const int e = lane + 32 * j;
+    if (e < E) atomicAdd(&ssum[e], acc[j]);
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x) atomicAdd(&colsum[e], ssum[e]);
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const double coef = (double)lambda / ((double)E * (double)T * (double)T);
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    const double load = (double)__ldg(expert_load + e);
+    ssum[e] = __ldcg(&colsum[e]) * load;
+    dscores_col[e] = (float)(coef * load);
+    colsum[e] = 0.0;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot = 0.0;
+    for (int e = 0; e < E; ++e) tot += ssum[e];      // fixed order
+    *loss = coef * tot;
+    *ticket = 0;
   }
 }
 

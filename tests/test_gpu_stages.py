@@ -84,6 +84,41 @@ def test_softtopk_fwd_bwd(ms, orc, synth, T, E, k, t):
     assert (np.abs(got - refb) <= 1e-5 * rowmax + 1e-9).all()
 
 
+@pytest.mark.parametrize("T,E,k,lam", [(512, 8, 2, 1e-2), (1000, 16, 2, 1e-2), (4099, 64, 8, 3e-3), (777, 128, 8, 1.0),
+                                        (33, 5, 5, 0.5)])
+def test_aux_loss_and_its_gradient_through_softtopk(ms, orc, synth, T, E, k, lam):
+    """Eq. 9 on the GPU's own scores, and dlogits with its gradient folded into the SoftTopk backward."""
+    lam = float(np.float32(lam))                         # the C ABI takes lambda as a float
+    L = synth.logits_like(T, E, seed=7)
+    ctx = _ctx(ms, T, 64, E, k, cf=float(E), t=1.0)
+    Ld = L.to(DEV)
+    A = torch.empty_like(Ld)
+    ms.softtopk_fwd(ctx, Ld, A)
+    g = torch.Generator().manual_seed(9)
+    idx = torch.stack([torch.randperm(E, generator=g)[:k].sort().values for _ in range(T)]).to(torch.int32)
+    load = torch.bincount(idx.flatten().long(), minlength=E).to(torch.int32)
+    loss = torch.zeros(1, dtype=torch.float64, device=DEV)
+    col = torch.empty(E, dtype=torch.float32, device=DEV)
+    for _ in range(2):                                   # twice: the scratch must come back clean
+        ms.aux_loss(ctx, A, load.to(DEV), lam, loss, col)
+    torch.cuda.synchronize()
+    An = np32(A).astype(np.float64)
+    want = orc.aux_loss(An, idx.numpy(), lam)
+    assert abs(loss.item() - want) <= 1e-12 * abs(want)          # double accumulation of the same fp32 scores
+    gref = orc.aux_loss_grad(idx.numpy(), T, E, lam)
+    np.testing.assert_allclose(np32(col), gref, rtol=1e-6, atol=0)
+    # backward: dense per-expert term plus the sparse combine-weight gradients
+    dg = torch.randn(T, k, generator=g)
+    dL = torch.empty_like(Ld)
+    ms.softtopk_bwd_aux(ctx, Ld, idx.to(DEV), dg.to(DEV), col, dL)
+    G = np.tile(np32(col).astype(np.float64), (T, 1))
+    G[np.arange(T)[:, None], idx.numpy().astype(np.int64)] += f64(dg)
+    refb = orc.softtopk_bwd(f64(L), G, k, 1.0)
+    got = np32(dL)
+    scale = (np.abs(G).max(axis=1, keepdims=True))               # |J^T g| <= k/t * max|g| per row
+    assert (np.abs(got - refb) <= 1e-5 * scale + 1e-12).all()
+
+
 # ------------------------------------------------------------------------------------------- assignment
 def _run_assign(ms, M, T, E, k, cf, **kw):
     ctx = _ctx(ms, T, 64, E, k, cf=cf, **kw)
