@@ -830,7 +830,7 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
 // (expert_idx itself is edited in place as well); the list is sorted first, so ties are broken by
 // the smallest token index whatever order the collect pass appended the tokens in.
 constexpr int kP2Threads = 1024;
-constexpr int kHeldCache = 2048;
+constexpr int kHeldCache = 4096;
 constexpr int kMaxFix = 256;
 constexpr int kMaxArcs = 8192;      // finite arcs of D the Bellman-Ford search can list
 constexpr int kSortMax = 16384;     // candidate lists up to this length are sorted (they fit in D's space)
@@ -1295,7 +1295,10 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
           lo = ol < lo ? ol : lo; hi = oh > hi ? oh : hi;
         }
         __syncwarp();
-        if (lane == 0 && theta < kInf && hi - lo > theta) s.target = -2;   // stop here; the next round lists more tokens
+        if (lane == 0 && theta < kInf && hi - lo > theta) {
+          s.target = -2;                                // stop here; the next round lists more tokens:
+          if (st->theta < 2 * (hi - lo)) st->theta = 2 * (hi - lo);   // enough of them for this price update
+        }
       }
     }
     __syncthreads();

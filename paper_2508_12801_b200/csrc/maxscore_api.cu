@@ -239,7 +239,7 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   const int collect_blocks = std::min((p.T + kSweepThreads / 32 - 1) / (kSweepThreads / 32), c->sm_count * 16);   // one warp per token
   for (int r = 0; r < kRounds; ++r) {
     flow_collect_kernel<<<collect_blocks, kSweepThreads, 0, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, r == 0, 0,
-                                                         8LL, nullptr, nullptr, nullptr, r == kRounds - 1, Dg);
+                                                         4LL, nullptr, nullptr, nullptr, r == kRounds - 1, Dg);
     MS_LAUNCH_CHECK("flow_collect_kernel");
     flow_build_kernel<<<build_blocks, 256, 0, st>>>(M, fs, expert_idx, cand, Dg, p.T, p.E, p.k, g);
     MS_LAUNCH_CHECK("flow_build_kernel");
