@@ -617,6 +617,44 @@ flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every) {
   }
 }
 
+// fp32 <-> unsigned integers that order the same way (for the integer warp reductions)
+__device__ __forceinline__ unsigned flip_f32(float f) {
+  const unsigned b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float unflip_f32(unsigned u) {
+  return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
+}
+
+// Approximate selection over one row held by a warp: the `count` largest fp32 values, one warp reduction
+// each (the expert index rides in the low 7 mantissa bits, so values are distinct and the winner's
+// owner is known).  sel[] marks the first `nsel`; v_a / v_b are the values picked as number nsel and
+// nsel+1 (-inf where there is none).  The caller decides whether v_a - v_b is large enough to trust.
+__device__ __forceinline__ void warp_select_f32(const float (&val)[kEPLf], int E, int count, bool (&sel)[kEPLf],
+                                                float& v_a, float& v_b, int nsel) {
+  const int lane = threadIdx.x & 31;
+  unsigned u[kEPLf];
+#pragma unroll
+  for (int q = 0; q < kEPLf; ++q) {
+    const int e = lane + 32 * q;
+    u[q] = e < E ? flip_f32(__uint_as_float((__float_as_uint(val[q]) & ~127u) | (unsigned)e)) : 0u;
+    sel[q] = false;
+  }
+  v_a = -INFINITY; v_b = -INFINITY;
+  for (int r = 0; r < count && r < E; ++r) {
+    unsigned m = u[0];
+#pragma unroll
+    for (int q = 1; q < kEPLf; ++q) m = max(m, u[q]);
+    const unsigned w = __reduce_max_sync(0xffffffffu, m);
+    const float v = unflip_f32(w);
+    if (r == nsel - 1) v_a = v;
+    if (r == nsel) v_b = v;
+#pragma unroll
+    for (int q = 0; q < kEPLf; ++q)
+      if (u[q] == w) { u[q] = 0u; if (r < nsel) sel[q] = true; }
+  }
+}
+
 // Exact selection over one row held by a warp (lane l: entries l, l+32, ...).  Picks the `count`
 // largest values (larger value first, lower expert index first on equal values), sets sel[] for the first
 // `nsel` of them, and returns the values picked as number nsel (v_a) and nsel+1 (v_b), where reached.
@@ -668,62 +706,112 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
   if (Dg)   // the move-cost matrix the build kernel fills next starts out empty
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < E * (E | 1); i += gridDim.x * blockDim.x) Dg[i] = kInf;
   __shared__ long long sp[kMaxE];
+  __shared__ float spf[kMaxE];
   __shared__ int sload[kMaxE];
   __shared__ int s_viol, s_rer;
   __shared__ double s_score;
   __shared__ unsigned s_flags;
-  for (int e = threadIdx.x; e < E; e += blockDim.x) { sp[e] = st->p[e]; sload[e] = 0; }
+  for (int e = threadIdx.x; e < E; e += blockDim.x) { sp[e] = st->p[e]; spf[e] = (float)sp[e]; sload[e] = 0; }
   if (threadIdx.x == 0) { s_viol = 0; s_rer = 0; s_score = 0.0; s_flags = 0; }
   __syncthreads();
   const long long theta = unbounded ? kInf : st->theta;   // the last round lists every token
-  // One warp per token, lane l holds experts l, l+32, l+64, l+96: coalesced row loads, exact int64
-  // values in registers, every decision by warp votes and reductions.
+  // One warp per token, lane l holds experts l, l+32, l+64, l+96: coalesced row loads, every decision
+  // by warp votes and reductions.  Decisions are first tried on fp32 approximations of key - price with
+  // a rigorous error bound; only a token whose decision the bound cannot settle (a near-tie) is redone
+  // on the exact int64 values.  A token may be listed as a candidate on the approximate gap: the list
+  // only has to be a superset.
   const int lane = threadIdx.x & 31;
   const int wid = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), nwarp = gridDim.x * (blockDim.x >> 5);
+  const float hash_bound = g.mode == 0 ? 4096.f : 1048576.f;      // key - approx_key lies in [-0.5, this)
+  const float thetaf = theta >= kInf ? INFINITY : (float)theta * 1.0000005f;
   int w_viol = 0, w_rer = 0; double w_score = 0.0; bool w_bad = false;
   for (int tok = wid; tok < T; tok += nwarp) {
     const float* row = M + (size_t)tok * E;
     const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-    float x[kEPLf]; long long key[kEPLf], val[kEPLf]; bool in[kEPLf];
+    float x[kEPLf], kf[kEPLf], vf[kEPLf]; bool in[kEPLf];
     int mine = -1;
     if (!first && lane < k) mine = expert_idx[(size_t)tok * k + lane];
+    float mag = 0.f;
 #pragma unroll
     for (int q = 0; q < kEPLf; ++q) {
       const int e = lane + 32 * q;
       x[q] = e < E ? __ldg(row + e) : 0.f;
       w_bad |= !isfinite(x[q]);
-      key[q] = e < E ? make_key(g, x[q], flat + e) : -kInf;
-      val[q] = e < E ? key[q] - sp[e] : -kInf;
+      kf[q] = e < E ? approx_key(g, x[q]) : -INFINITY;
+      const float pf = e < E ? spf[e] : 0.f;
+      vf[q] = kf[q] - pf;
+      if (e < E) mag = fmaxf(mag, fabsf(kf[q]) + fabsf(pf));
       in[q] = false;
     }
+    // |approximation - exact| <= hash_bound + 2^-15 * (|key| + |price|): float conversion of the price,
+    // one rounding of the difference, and the 7 mantissa bits that carry the expert index in selections
+    mag = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mag)));
+    const float err3 = 3.f * (hash_bound + mag * (1.f / 32768.f));
     if (!first)
       for (int j = 0; j < k; ++j) {
         const int ej = __shfl_sync(0xffffffffu, mine, j);
 #pragma unroll
         for (int q = 0; q < kEPLf; ++q) in[q] |= (ej == lane + 32 * q);
       }
-    // exact check of the experts the token holds now: the worst held value against the best other one
-    long long min_held = kInf, max_non = -kInf;
+    bool settled = false, list = false, keep = false;
+    if (!first) {
+      float mh = INFINITY, mn = -INFINITY;
 #pragma unroll
-    for (int q = 0; q < kEPLf; ++q) {
-      if (lane + 32 * q >= E) continue;
-      if (in[q]) min_held = val[q] < min_held ? val[q] : min_held;
-      else max_non = val[q] > max_non ? val[q] : max_non;
-    }
+      for (int q = 0; q < kEPLf; ++q) {
+        if (lane + 32 * q >= E) continue;
+        if (in[q]) mh = fminf(mh, vf[q]); else mn = fmaxf(mn, vf[q]);
+      }
+      mh = unflip_f32(__reduce_min_sync(0xffffffffu, flip_f32(mh)));
+      mn = unflip_f32(__reduce_max_sync(0xffffffffu, flip_f32(mn)));
+      const float diff = mh - mn;
+      if (diff > err3) {                                // certainly still a top-k (E == k: diff = inf)
+        settled = true; keep = true;
+        list = E > k && (diff - err3 <= thetaf);
+      }
+    } else {
+      float vkf, vk1f; bool sel[kEPLf];
+      warp_select_f32(vf, E, k + 1, sel, vkf, vk1f, k);
+      if (vkf - vk1f > err3) {                          // the approximate top-k is certainly the exact one
+        settled = true;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const long long a = __shfl_xor_sync(0xffffffffu, min_held, o), c = __shfl_xor_sync(0xffffffffu, max_non, o);
-      min_held = a < min_held ? a : min_held; max_non = c > max_non ? c : max_non;
+        for (int q = 0; q < kEPLf; ++q) in[q] = sel[q];
+        list = E > k && (vkf - vk1f - err3 <= thetaf);
+      }
     }
-    const bool keep = !first && (min_held >= max_non);
-    const bool repick = !verify_only && !keep;
-    long long gap = keep ? ((E > k) ? min_held - max_non : kInf) : kInf;
+    long long key[kEPLf];
+    bool have_keys = false;
+    if (!settled) {
+      long long val[kEPLf];
+#pragma unroll
+      for (int q = 0; q < kEPLf; ++q) {
+        const int e = lane + 32 * q;
+        key[q] = e < E ? make_key(g, x[q], flat + e) : -kInf;
+        val[q] = e < E ? key[q] - sp[e] : -kInf;
+      }
+      have_keys = true;
+      // exact check of the experts the token holds now: the worst held value against the best other one
+      long long min_held = kInf, max_non = -kInf;
+#pragma unroll
+      for (int q = 0; q < kEPLf; ++q) {
+        if (lane + 32 * q >= E) continue;
+        if (in[q]) min_held = val[q] < min_held ? val[q] : min_held;
+        else max_non = val[q] > max_non ? val[q] : max_non;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const long long a = __shfl_xor_sync(0xffffffffu, min_held, o), c = __shfl_xor_sync(0xffffffffu, max_non, o);
+        min_held = a < min_held ? a : min_held; max_non = c > max_non ? c : max_non;
+      }
+      keep = !first && (min_held >= max_non);
+      long long gap = keep ? ((E > k) ? min_held - max_non : kInf) : kInf;
+      if (!verify_only && !keep) {
+        long long vk = -kInf, vk1 = -kInf;
+        warp_select(val, E, k + 1, in, vk, vk1, k);
+        gap = (E > k) ? vk - vk1 : kInf;
+      }
+      list = gap < kInf && gap <= theta;
+    }
     if (!keep && !first) ++w_viol;
-    if (repick) {
-      long long vk = -kInf, vk1 = -kInf;
-      warp_select(val, E, k + 1, in, vk, vk1, k);
-      gap = (E > k) ? vk - vk1 : kInf;
-    }
     // the experts in ascending order: word q of the held mask is the vote over in[q]
     unsigned words[kEPLf]; int below = 0;
 #pragma unroll
@@ -739,23 +827,32 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
     }
     if (verify_only) {
       // statistics: the score of the held pairs, and how many of them are not in the token's own top-k
-      bool none[kEPLf];
+      // of raw keys (the k-th and (k+1)-th raw keys must be told apart for certain, else exact keys decide)
+      float rkf, rk1f; bool rsel[kEPLf];
+      warp_select_f32(kf, E, k + 1, rsel, rkf, rk1f, k);
+      int rer = 0; double sc = 0.0;
+      if (rkf - rk1f > err3) {
 #pragma unroll
-      for (int q = 0; q < kEPLf; ++q) none[q] = false;
-      long long kth_raw = -kInf, next_raw = -kInf;
-      warp_select(key, E, k, none, kth_raw, next_raw, k);
-      double sc = 0.0; int rer = 0;
+        for (int q = 0; q < kEPLf; ++q) rer += (in[q] && !rsel[q]) ? 1 : 0;
+      } else {
+        if (!have_keys) {
+#pragma unroll
+          for (int q = 0; q < kEPLf; ++q) { const int e = lane + 32 * q; key[q] = e < E ? make_key(g, x[q], flat + e) : -kInf; }
+          have_keys = true;
+        }
+        long long kth_raw = -kInf, next_raw = -kInf;
+        warp_select(key, E, k, rsel, kth_raw, next_raw, k);
+#pragma unroll
+        for (int q = 0; q < kEPLf; ++q) rer += (in[q] && key[q] < kth_raw) ? 1 : 0;
+      }
 #pragma unroll
       for (int q = 0; q < kEPLf; ++q)
-        if (in[q]) {
-          sc += (g.mode == 0) ? (double)x[q] : (double)key[q];
-          if (key[q] < kth_raw) ++rer;
-        }
+        if (in[q]) sc += (g.mode == 0) ? (double)x[q] : (double)(have_keys ? key[q] : make_key(g, x[q], flat + lane + 32 * q));
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) { sc += __shfl_xor_sync(0xffffffffu, sc, o); rer += __shfl_xor_sync(0xffffffffu, rer, o); }
       w_score += sc; w_rer += rer;
     }
-    if (!verify_only && gap < kInf && gap <= theta && lane == 0)
+    if (!verify_only && list && lane == 0)
       cand[atomicAdd(&st->ncand, 1)] = tok;     // the list has room for every token
   }
   if (__any_sync(0xffffffffu, w_bad) && lane == 0) atomicOr(&s_flags, 2u);
