@@ -330,11 +330,11 @@ __device__ __forceinline__ void emit_margin(unsigned* hist, long long* mins, con
 template <bool kFirst>   // the first sweep scans every row (one thread per token) and fills the cache
 __global__ void __launch_bounds__(kSweepThreads)
 flow_sweep_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, int T, int E, int k, int C,
-                  KeyGen g) {
+                  KeyGen g, int sweep_index) {
   if (*(volatile int*)&st->p1_done) return;
   // histograms alternate between two buffers: this sweep fills one while every CTA clears a slice of
   // the other for the next sweep (its last reader, the previous price update, has finished)
-  const int sweep0 = st->sweep;
+  const int sweep0 = sweep_index;                     // sweeps run in launch order; a finished phase returns above
   const long long cumdrop = st->cumdrop;
   const int par = sweep0 & 1;
   unsigned* hup = st->hist_up[par]; unsigned* hdn = st->hist_dn[par];
@@ -530,32 +530,45 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, 
 // histograms in flight at once).
 constexpr int kPriceThreads = 1024;
 __global__ void __launch_bounds__(kPriceThreads)
-flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every) {
-  if (*(volatile int*)&st->p1_done) return;
+flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every, int sweep_index) {
+  // every input is loaded up front, independently of the others, so that the kernel pays two global
+  // round trips (state, then the histogram rows picked by the sign of the imbalance), not one per field
   __shared__ long long sp[kMaxE];
   __shared__ int s_imb;
   __shared__ long long pmin, s_drop;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   constexpr int kWarps = kPriceThreads / 32, kBatch = kMaxE / kWarps;
-  const int par = st->sweep & 1;
+  const int par = sweep_index & 1;                    // the sweep this update closes filled these buffers
   const unsigned* hup = st->hist_up[par]; const unsigned* hdn = st->hist_dn[par];
-  const long long eps = st->eps;
-  const bool balanced = st->balanced != 0;
-  const int cut_max = st->cut_max;
-  if (threadIdx.x == 0) { s_imb = 0; s_drop = 0; }
-  uint4 ha[kBatch], hb[kBatch]; int xs[kBatch]; long long ps[kBatch], m1[kBatch];
+  const int done_before = __ldcg(&st->p1_done);
+  const long long eps = __ldcg(&st->eps), eps_min = __ldcg(&st->eps_min);
+  const bool balanced = __ldcg(&st->balanced) != 0;
+  const int cut_max = __ldcg(&st->cut_max), best_imb = __ldcg(&st->best_imb), stall_before = __ldcg(&st->stall);
+  int xs[kBatch], cup[kBatch], cdn[kBatch]; long long ps[kBatch], mu[kBatch], md[kBatch];
 #pragma unroll
   for (int b = 0; b < kBatch; ++b) {
     const int e = warp + b * kWarps;
-    xs[b] = 0; ps[b] = 0; m1[b] = kInf; ha[b] = make_uint4(0, 0, 0, 0); hb[b] = ha[b];
+    xs[b] = 0; ps[b] = 0; mu[b] = kInf; md[b] = kInf; cup[b] = 0; cdn[b] = 0;
     if (e < E) {
-      const int x = st->load[e] - C;
-      xs[b] = x; ps[b] = st->p[e];
+      xs[b] = __ldcg(&st->load[e]) - C; ps[b] = __ldcg(&st->p[e]);
+      cup[b] = __ldcg(&st->cap_up[e]); cdn[b] = __ldcg(&st->cap_dn[e]);
+      mu[b] = __ldcg(&st->min_up[e]); md[b] = __ldcg(&st->min_dn[e]);
+    }
+  }
+  if (done_before) return;
+  if (threadIdx.x == 0) { s_imb = 0; s_drop = 0; }
+  uint4 ha[kBatch], hb[kBatch]; long long m1[kBatch];
+#pragma unroll
+  for (int b = 0; b < kBatch; ++b) {
+    const int e = warp + b * kWarps;
+    m1[b] = kInf; ha[b] = make_uint4(0, 0, 0, 0); hb[b] = ha[b];
+    if (e < E) {
+      const int x = xs[b];
       const bool up = x > 0, dn = x < 0 && (balanced || ps[b] > 0);
       if (up || dn) {
         const uint4* h = reinterpret_cast<const uint4*>((up ? hup : hdn) + e * kNB) + 2 * lane;
-        ha[b] = h[0]; hb[b] = h[1];
-        m1[b] = up ? st->min_up[e] : st->min_dn[e];
+        ha[b] = __ldcg(h); hb[b] = __ldcg(h + 1);
+        m1[b] = up ? mu[b] : md[b];
       }
     }
   }
@@ -569,12 +582,12 @@ flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every) {
     long long p = ps[b];
     int flag = 0;
     if (x > 0) {
-      int cl = st->cap_up[e]; bool shortw;
+      int cl = cup[b]; bool shortw;
       p += price_step_warp(ha[b], hb[b], x, eps, cl, shortw, cut_max, m1[b]);
       if (lane == 0) st->cap_up[e] = cl;
       imb += x;
     } else if (x < 0 && (balanced || p > 0)) {
-      int cl = st->cap_dn[e]; bool shortw;
+      int cl = cdn[b]; bool shortw;
       p -= price_step_warp(ha[b], hb[b], -x, eps, cl, shortw, cut_max, m1[b]);
       if (!balanced && p < 0) p = 0;
       if (lane == 0) st->cap_dn[e] = cl;
@@ -594,10 +607,10 @@ flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every) {
   }
   if (lane == 0) { if (imb) atomicAdd(&s_imb, imb); if (drop > 0) atomicMax(&s_drop, drop); }
   __syncthreads();
-  const int sweep = st->sweep + 1;
+  const int sweep = sweep_index + 1;
   // a small imbalance that has stopped shrinking is a price war between a few experts: the exact phase
   // ends it faster than more sweeps would
-  const int stall = s_imb < st->best_imb ? 0 : st->stall + 1;
+  const int stall = s_imb < best_imb ? 0 : stall_before + 1;
   const bool done = (s_imb == 0) || sweep >= n_sweeps || (stall >= kStallSweeps && s_imb <= kStallImbalance);
   if (threadIdx.x == 0) {
     // prices are only defined up to a shift when every expert must be full; anchor the minimum at 0
@@ -612,7 +625,7 @@ flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every) {
     st->sweep = sweep;
     st->stall = stall; if (stall == 0) st->best_imb = s_imb;
     st->cumdrop += s_drop;
-    if (sweep % decay_every == 0) { long long ne = eps >> 1; st->eps = ne < st->eps_min ? st->eps_min : ne; }
+    if (sweep % decay_every == 0) { long long ne = eps >> 1; st->eps = ne < eps_min ? eps_min : ne; }
     if (done) st->p1_done = 1;
   }
 }

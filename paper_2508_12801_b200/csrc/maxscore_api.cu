@@ -228,9 +228,9 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   SweepCache cache{reinterpret_cast<float*>(c->ws + c->lay.cache_x), reinterpret_cast<unsigned char*>(c->ws + c->lay.cache_id),
                    reinterpret_cast<long long*>(c->ws + c->lay.cache_bound)};
   for (int s = 0; s < n_sweeps; ++s) {
-    if (s == 0) flow_sweep_kernel<true><<<blocks, kSweepThreads, 0, st>>>(M, fs, cache, p.T, p.E, p.k, c->C, g);
-    else flow_sweep_kernel<false><<<blocks, kSweepThreads, 0, st>>>(M, fs, cache, p.T, p.E, p.k, c->C, g);
-    flow_price_kernel<<<1, kPriceThreads, 0, st>>>(fs, p.E, c->C, n_sweeps, 1);
+    if (s == 0) flow_sweep_kernel<true><<<blocks, kSweepThreads, 0, st>>>(M, fs, cache, p.T, p.E, p.k, c->C, g, s);
+    else flow_sweep_kernel<false><<<blocks, kSweepThreads, 0, st>>>(M, fs, cache, p.T, p.E, p.k, c->C, g, s);
+    flow_price_kernel<<<1, kPriceThreads, 0, st>>>(fs, p.E, c->C, n_sweeps, 1, s);
     MS_LAUNCH_CHECK("flow_sweep_kernel");
   }
   const size_t p2smem = sizeof(long long) * (size_t)p.E * (p.E | 1) + (size_t)kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache + 2 * kMaxArcs;
