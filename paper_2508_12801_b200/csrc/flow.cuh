@@ -738,17 +738,27 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
   const float hash_bound = g.mode == 0 ? 4096.f : 1048576.f;      // key - approx_key lies in [-0.5, this)
   const float thetaf = theta >= kInf ? INFINITY : (float)theta * 1.0000005f;
   int w_viol = 0, w_rer = 0; double w_score = 0.0; bool w_bad = false;
+  // the next token's row and experts are fetched while the current token is worked on
+  float nx[kEPLf]; int nmine = -1;
+  auto fetch = [&](int t) {
+    if (t >= T) return;
+    const float* r = M + (size_t)t * E;
+#pragma unroll
+    for (int q = 0; q < kEPLf; ++q) { const int e = lane + 32 * q; nx[q] = e < E ? __ldg(r + e) : 0.f; }
+    nmine = (!first && lane < k) ? expert_idx[(size_t)t * k + lane] : -1;
+  };
+  fetch(wid);
   for (int tok = wid; tok < T; tok += nwarp) {
-    const float* row = M + (size_t)tok * E;
     const uint32_t flat = (uint32_t)tok * (uint32_t)E;
     float x[kEPLf], kf[kEPLf], vf[kEPLf]; bool in[kEPLf];
-    int mine = -1;
-    if (!first && lane < k) mine = expert_idx[(size_t)tok * k + lane];
+    const int mine = nmine;
+#pragma unroll
+    for (int q = 0; q < kEPLf; ++q) x[q] = nx[q];
+    fetch(tok + nwarp);
     float mag = 0.f;
 #pragma unroll
     for (int q = 0; q < kEPLf; ++q) {
       const int e = lane + 32 * q;
-      x[q] = e < E ? __ldg(row + e) : 0.f;
       w_bad |= !isfinite(x[q]);
       kf[q] = e < E ? approx_key(g, x[q]) : -INFINITY;
       const float pf = e < E ? spf[e] : 0.f;
