@@ -306,7 +306,7 @@ def run_ours(args, wl):
     if world == 1 and not args.no_cpu_baseline:
         import oracle
         oracle.build()
-        Ts = args.ref_tokens
+        Ts = args.cpu_tokens
         oracle_step(wl, 128)
         dt_cpu, _ = oracle_step(wl, Ts)
         cpu = {"value": Ts / dt_cpu, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
@@ -347,7 +347,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="stress")
     ap.add_argument("--tokens", type=int, default=0, help="override T (profiling on a smaller case)")
-    ap.add_argument("--ref-tokens", type=int, default=4096, help="tokens per step of the CPU checker's sample")
+    ap.add_argument("--ref-tokens", type=int, default=4096, help="tokens per step of the CPU checker's sample (--impl reference)")
+    ap.add_argument("--cpu-tokens", type=int, default=16384, help="tokens of the one-off cpu_baseline sample (10-30 s of CPU work)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     from paper_2508_12801_b200 import synth
