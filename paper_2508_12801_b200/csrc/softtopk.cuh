@@ -14,14 +14,16 @@ namespace msr {
 
 constexpr int kEPL = kMaxE / 32;  // experts per lane
 
-// arg-max over the warp of (value, index) pairs, lowest index on equal values
+// arg-max over the warp of (value, index) pairs, lowest index on equal values: two integer warp
+// reductions (the largest value through an order-preserving map to unsigned, then the lowest index
+// among the lanes that hold it) instead of five shuffle rounds.  Adding +0.0 first turns -0.0 into +0.0,
+// so the two zeros tie as they do in a floating-point comparison.
 __device__ __forceinline__ void warp_argmax(float& v, int& idx) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    float ov = __shfl_xor_sync(0xffffffffu, v, o);
-    int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-    if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
-  }
+  const unsigned b = __float_as_uint(v + 0.f);
+  const unsigned u = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+  const unsigned best = __reduce_max_sync(0xffffffffu, u);
+  idx = (int)__reduce_min_sync(0xffffffffu, u == best ? (unsigned)idx : 0x7fffffffu);
+  v = __uint_as_float((best & 0x80000000u) ? (best & 0x7fffffffu) : ~best);
 }
 
 __global__ void __launch_bounds__(256)
