@@ -149,23 +149,21 @@ def run_reference(args, wl):
 # ------------------------------------------------------------------------------------------------ our arm
 def run_ours(args, wl):
     import torch
-    import torch.distributed as dist
 
     from paper_2508_12801_b200 import binding as ms
     from paper_2508_12801_b200 import synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2508_12801_b200 import replicas
+    info = replicas.rank_info()
+    world, rank, local = info.world, info.rank, info.local_rank
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the router has no CPU path")
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    replicas.init_group(info, "nccl", device_id=torch.device(dev))
 
     T, d, E, k = wl.T, wl.d_model, wl.E, wl.k
-    seed = rank                                           # replicas route different batches
+    seed = replicas.replica_seed(info)                    # replicas route different batches
     H_host = synth.hidden(wl, seed).pin_memory()
     W_host = synth.w_gate(wl, seed).pin_memory()
     b = synth.expert_bias(wl, seed)
@@ -213,7 +211,7 @@ def run_ours(args, wl):
     def sync_all():
         torch.cuda.synchronize()
         if world > 1:
-            dist.barrier()
+            replicas.barrier(info)
             torch.cuda.synchronize()
 
     for _ in range(max(args.warmup, 3)):
@@ -237,10 +235,7 @@ def run_ours(args, wl):
     clocks = sampler.stop() if rank == 0 else None
     ms_total = e0.elapsed_time(e1)
     stage_ms = [sum(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(args.steps)) / args.steps for j in range(7)]
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
+    ms_step = replicas.max_over_ranks(info, ms_total, dev) / args.steps
     st2 = ms.read_stats(buf.stats)
 
     # ---- end to end: the same step, batch coming from pinned host memory through the C ABI ---------------
@@ -258,17 +253,13 @@ def run_ours(args, wl):
     sync_all()
     e2e_ms = g0.elapsed_time(g1) / args.steps
     wall_ms = (time.perf_counter() - t0) * 1e3 / args.steps
-    te = torch.tensor([max(e2e_ms, wall_ms)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_ms = float(te.item())
+    e2e_ms = replicas.max_over_ranks(info, max(e2e_ms, wall_ms), dev)
     eb = H_host.element_size()
     h2d = eb * (T * d + d * E)
     d2h = 3 * 4 * T * k + 40
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        replicas.shutdown(info)
         return
 
     # ---- roofline of the dominant kernel -------------------------------------------------------------
@@ -313,7 +304,7 @@ def run_ours(args, wl):
                "sample": f"first {Ts} tokens of the workload, whole path fwd+bwd, {dt_cpu:.1f} s"}
 
     out = {
-        "metric": METRIC, "value": world * T / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": replicas.aggregate_tokens_per_s(info, T, ms_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
         "config": {"workload": wl.name, "T": T, "d_model": d, "E": E, "k": k, "capacity_factor": wl.capacity_factor,
@@ -328,15 +319,14 @@ def run_ours(args, wl):
         "roofline": {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src},
         "cpu_baseline": cpu,
-        "e2e": {"value": world * T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": replicas.aggregate_tokens_per_s(info, T, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                 "covers": "maxscore_route_dispatch_host (pinned host batch in, indices out) + rest of the step on device"},
         "gpu_launches": launches_per_step() * args.steps,
         "clocks": clocks,
     }
     print(json.dumps(out))
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.shutdown(info)
 
 
 def main():
