@@ -57,6 +57,16 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&r)[16]) {
   for (int i = 0; i < 16; ++i) r[i] = __uint_as_float(u[i]);
 }
 
+// Issue only: the registers may be read after tmem_ld_wait().  Several loads can be in flight.
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&u)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+        "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 // Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64 elements) and
 // were written by TMA with the 128-byte swizzle: groups of 8 rows are 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_k128(uint32_t saddr) {
@@ -417,17 +427,23 @@ gate_bwd_dh_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       // the staged copy of this buffer from two tiles ago must have been read by its bulk store
       if (nt >= 2) bulk_wait_read<1>();
       unsigned char* my_row = out_stage + ((size_t)buf * 128 + quarter * 32 + lane) * kDhOutStride;
-      for (int c0 = 0; c0 < kDhBN; c0 += 16) {
-        float r[16];
-        tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kDhBN + c0), r);
-        uint32_t w[8];
+      for (int c0 = 0; c0 < kDhBN; c0 += 64) {          // four TMEM loads in flight, one wait
+        uint32_t u[4][16];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          __nv_bfloat162 h = __floats2bfloat162_rn(r[2 * j], r[2 * j + 1]);
-          w[j] = *reinterpret_cast<uint32_t*>(&h);
+        for (int q = 0; q < 4; ++q)
+          tmem_ld16_issue(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kDhBN + c0 + 16 * q), u[q]);
+        tmem_ld_wait();
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t w[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(u[q][2 * j]), __uint_as_float(u[q][2 * j + 1]));
+            w[j] = *reinterpret_cast<uint32_t*>(&h);
+          }
+          reinterpret_cast<uint4*>(my_row + (c0 + 16 * q) * 2)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+          reinterpret_cast<uint4*>(my_row + (c0 + 16 * q) * 2)[1] = make_uint4(w[4], w[5], w[6], w[7]);
         }
-        reinterpret_cast<uint4*>(my_row + c0 * 2)[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        reinterpret_cast<uint4*>(my_row + c0 * 2)[1] = make_uint4(w[4], w[5], w[6], w[7]);
       }
       // each lane ships its own row: one 256-byte bulk store instead of sixteen scattered 16-byte ones
       fence_proxy_async();
