@@ -22,6 +22,12 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* t
       ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(x), "r"(y)
       : "memory");
 }
+// 2-D tile store shared -> global (clipped at the tensor's bounds), tracked by bulk async-groups
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tmap, int x, int y, const void* smem_src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tmap),
+               "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+               : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_slot, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_slot)),
                "r"(ncols)
@@ -338,9 +344,9 @@ __host__ __device__ constexpr uint32_t idesc_bf16_m128_mn(int n) {   // both ope
 // ---- dH[T, d] = dL[T, E] . W_g^T -------------------------------------------------------------------
 // One CTA per 128-token tile.  The dL tile (hi and lo) is loaded once; 128-column tiles of W_g stream
 // through a 2-stage ring; two TMEM accumulators alternate so that the four epilogue warps convert and
-// stage tile n in shared memory (one bulk store per row) while the MMA warp works on tile n+1.
+// stage tile n in shared memory (two TMA tile stores per warp) while the MMA warp works on tile n+1.
 constexpr int kDhBN = 128, kDhStages = 2;
-constexpr int kDhOutStride = kDhBN * 2 + 16;     // bytes per staged output row (padded against bank conflicts)
+constexpr int kDhOutBytes = 2 * 4 * 2 * 4096;     // output staging: [2 buffers][4 warps][2 column halves][32 rows x 128 B]
 struct DhSmem {
   uint64_t a_full, b_full[kDhStages], b_empty[kDhStages], acc_full[2], acc_empty[2];
   uint32_t tmem_base;
@@ -349,7 +355,7 @@ struct DhSmem {
 
 __global__ void __launch_bounds__(192)
 gate_bwd_dh_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                      __nv_bfloat16* __restrict__ dH, int T, int d, int Kpad, unsigned* error_flag) {
+                      const __grid_constant__ CUtensorMap tmOut, int T, int d, int Kpad, unsigned* error_flag) {
   extern __shared__ unsigned char dsm_raw[];
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(dsm_raw) + 1023) & ~(uintptr_t)1023);
   __shared__ DhSmem sm;
@@ -360,7 +366,7 @@ gate_bwd_dh_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   const uint32_t b_bytes = kboxes * 16384u;
   unsigned char* a_tile = base;                       // [2*kboxes][128 rows][128 B]
   unsigned char* b_ring = base + a_bytes;             // [stage][kboxes][128 rows][128 B]
-  unsigned char* out_stage = b_ring + (size_t)kDhStages * b_bytes;   // [2][128 rows][kDhOutStride]
+  unsigned char* out_stage = b_ring + (size_t)kDhStages * b_bytes;   // kDhOutBytes, 1024-byte aligned pieces
   const int n_tiles = (d + kDhBN - 1) / kDhBN;
 
   if (threadIdx.x == 0) {
@@ -417,22 +423,25 @@ gate_bwd_dh_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     if (!ok) sm.failed = 1;
   } else if (warp >= 2) {
     const int quarter = warp & 3;                      // TMEM lanes this warp may read
-    const int row = m0 + quarter * 32 + lane;
     bool ok = true;
     for (int nt = 0; nt < n_tiles && ok; ++nt) {
       const int buf = nt & 1;
       ok = mbar_wait_bounded(&sm.acc_full[buf], (uint32_t)((nt >> 1) & 1));
       if (!ok) break;
       tc_fence_after();
-      // the staged copy of this buffer from two tiles ago must have been read by its bulk store
-      if (nt >= 2) bulk_wait_read<1>();
-      unsigned char* my_row = out_stage + ((size_t)buf * 128 + quarter * 32 + lane) * kDhOutStride;
+      // Staging for the TMA tile store: per warp and column half a 32-row x 128-byte box in the 128-byte
+      // swizzle (16-byte chunk c of row r sits at chunk c ^ (r & 7)), which also spreads the lanes' writes
+      // over the banks.  The buffer used two tiles ago must have been read by its store first.
+      if (lane == 0 && nt >= 2) bulk_wait_read<1>();
+      __syncwarp();
+      unsigned char* my_box = out_stage + ((size_t)buf * 4 + quarter) * 8192;
       for (int c0 = 0; c0 < kDhBN; c0 += 64) {          // four TMEM loads in flight, one wait
         uint32_t u[4][16];
 #pragma unroll
         for (int q = 0; q < 4; ++q)
           tmem_ld16_issue(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kDhBN + c0 + 16 * q), u[q]);
         tmem_ld_wait();
+        unsigned char* my_row = my_box + (c0 >> 6) * 4096 + lane * 128;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           uint32_t w[8];
@@ -441,23 +450,27 @@ gate_bwd_dh_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(u[q][2 * j]), __uint_as_float(u[q][2 * j + 1]));
             w[j] = *reinterpret_cast<uint32_t*>(&h);
           }
-          reinterpret_cast<uint4*>(my_row + (c0 + 16 * q) * 2)[0] = make_uint4(w[0], w[1], w[2], w[3]);
-          reinterpret_cast<uint4*>(my_row + (c0 + 16 * q) * 2)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+          *reinterpret_cast<uint4*>(my_row + (((2 * q) ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(my_row + (((2 * q + 1) ^ (lane & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
         }
       }
-      // each lane ships its own row: one 256-byte bulk store instead of sixteen scattered 16-byte ones
       fence_proxy_async();
-      {
-        const int col0 = nt * kDhBN;
-        const int ncol = min(kDhBN, d - col0);
-        if (row < T && ncol > 0) bulk_s2g(dH + (size_t)row * d + col0, my_row, (uint32_t)ncol * 2);
+      __syncwarp();
+      if (lane == 0) {
+        // two tile stores per warp and tile (rows beyond T and columns beyond d are clipped by the copy)
+        const int y = m0 + quarter * 32;
+        if (y < T) {
+          const int col0 = nt * kDhBN;
+          tma_store_2d(&tmOut, col0, y, my_box);
+          if (col0 + 64 < d) tma_store_2d(&tmOut, col0 + 64, y, my_box + 4096);
+        }
         bulk_commit();
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);
     }
-    bulk_wait_all<0>();
+    if (lane == 0) bulk_wait_all<0>();
     if (!ok && lane == 0) sm.failed = 1;
   }
   __syncthreads();

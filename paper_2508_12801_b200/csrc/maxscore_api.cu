@@ -117,7 +117,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 constexpr int kP2SmemMax = (int)(sizeof(long long) * kMaxE * (kMaxE | 1) + kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache + 2 * kMaxArcs);
-constexpr int kDhSmemMax = 2 * 2 * 16384 + kDhStages * 2 * 16384 + 2 * 128 * kDhOutStride + 1024;     // Kpad = 128
+constexpr int kDhSmemMax = 2 * 2 * 16384 + kDhStages * 2 * 16384 + kDhOutBytes + 1024;     // Kpad = 128
 constexpr int kDwSmemMax = kDwStages * (16384 + 2 * 2 * 8192) + 1024;
 
 }  // namespace
@@ -499,9 +499,11 @@ maxscore_status maxscore_gate_bwd(maxscore_ctx* c, const void* hidden, const voi
     if (!s2) s2 = make_tmap_bf16(c, &tmL2, dls, (uint64_t)2 * Kpad, (uint64_t)p.T, 64, 64);
     if (s2) return s2;
     const int kboxes = Kpad / 64;
-    const size_t dh_smem = (size_t)2 * kboxes * 16384 + (size_t)kDhStages * kboxes * 16384 + (size_t)2 * 128 * kDhOutStride + 1024;
-    gate_bwd_dh_tc_kernel<<<(p.T + 127) / 128, 192, dh_smem, st>>>(tmA, tmB, (__nv_bfloat16*)dH, p.T, p.d_model, Kpad,
-                                                                  error_flag_of(c));
+    const size_t dh_smem = (size_t)2 * kboxes * 16384 + (size_t)kDhStages * kboxes * 16384 + (size_t)kDhOutBytes + 1024;
+    CUtensorMap tmOut;
+    s2 = make_tmap_bf16(c, &tmOut, dH, (uint64_t)p.d_model, (uint64_t)p.T, 64, 32);
+    if (s2) return s2;
+    gate_bwd_dh_tc_kernel<<<(p.T + 127) / 128, 192, dh_smem, st>>>(tmA, tmB, tmOut, p.T, p.d_model, Kpad, error_flag_of(c));
     MS_LAUNCH_CHECK("gate_bwd_dh_tc_kernel");
     const size_t dw_smem = (size_t)kDwStages * (16384 + (size_t)2 * kboxes * 8192) + 1024;
     dim3 gdw((p.d_model + 127) / 128, l.dw_splits);
