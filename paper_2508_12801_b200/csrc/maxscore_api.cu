@@ -74,7 +74,7 @@ Layout layout_of(const maxscore_params& p) {
   l.Kpad = (int)align_up((size_t)p.E, 64);
   {   // split the token dimension of dW so that about two CTAs per SM are busy
     const int mtiles = (p.d_model + 127) / 128;
-    int splits = (296 + mtiles - 1) / mtiles;
+    int splits = 296 / mtiles;     // one CTA per SM (192 KB of shared memory): at most two full waves on 148 SMs
     const int max_splits = (p.T + 255) / 256;
     if (splits > max_splits) splits = max_splits;
     if (splits > 64) splits = 64;
