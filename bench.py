@@ -282,9 +282,9 @@ def run_ours(args, wl):
     achieved = alg_bytes[dom_name] / (stage_ms[dom] * 1e-3) / 1e9
     # DRAM bytes per token from the ncu capture summarised in profiles/ncu_data_movement_and_gate_T16384.md
     # (bf16, d_model=4096, k=8; traffic is proportional to T).  None for any other shape.
-    ncu_bytes_per_token = {"dispatch": (0.1353e9 + 1.0146e9) / 16384, "combine": (1.0756e9 + 0.1287e9) / 16384,
-                           "combine_bwd": (1.2095e9 + 1.0308e9) / 16384,
-                           "dispatch_bwd": (1.2103e9 + 0.1313e9) / 16384}
+    ncu_bytes_per_token = {"dispatch": (0.1354e9 + 1.0151e9) / 16384, "combine": (1.0756e9 + 0.1285e9) / 16384,
+                           "combine_bwd": (1.2095e9 + 1.0316e9) / 16384,
+                           "dispatch_bwd": (1.2103e9 + 0.1285e9) / 16384}
     traffic = ncu_bytes_per_token[dom_name] * T if (d == 4096 and k == 8 and eb == 2) else None
     stages = {n: {"ms": round(stage_ms[j], 4), "alg_GB": round(alg_bytes[n] / 1e9, 4),
                   "GBps": round(alg_bytes[n] / (stage_ms[j] * 1e-3) / 1e9, 1),
