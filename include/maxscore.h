@@ -22,6 +22,11 @@
  *     after synchronising.  Nothing aborts, throws or traps.
  *   - expert_idx[i, :] is ascending.  slot_idx[i, c] is the rank of token i among the tokens of expert
  *     expert_idx[i, c], in ascending token order.  Unused slots of slot_token hold -1.
+ *   - If the solver runs out of its budget (MAXSCORE_STAT_NOT_CONVERGED; never seen with the default
+ *     budget on the documented workloads) every token still has k distinct experts, but an expert may
+ *     hold more than C tokens.  The surplus pairs then have slot_idx >= C: index build leaves them out of
+ *     slot_token, dispatch does not write them, combine and the backward passes skip them (they contribute
+ *     zero), so nothing is read or written out of bounds.
  *   - Limits of this build: 1 <= k <= 8, k <= E <= 128, bf16 I/O needs d_model % 8 == 0, fp32 I/O
  *     needs d_model % 4 == 0, T * k < 2^31.
  */
