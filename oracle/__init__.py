@@ -117,6 +117,30 @@ def softtopk_bwd(L, G, k: int, t: float) -> np.ndarray:
     return dL
 
 
+def softtopk_rankscale_fwd(L, k: int, t: float, beta: float, delta: int) -> np.ndarray:
+    """The literal readings of Eq. 6: y = softmax(a) * (beta + t * min(rank - delta, k)).  Parity unpinned
+    against the paper (it prints no value that separates the readings)."""
+    L = _f64(L)
+    T, E = L.shape
+    A = np.empty_like(L)
+    rc = lib().mso_softtopk_rankscale_fwd(I64(T), I64(E), I64(k), C.c_double(t), C.c_double(beta), I64(delta),
+                                          _p(L), _p(A))
+    if rc:
+        raise ValueError("softtopk_rankscale_fwd: bad arguments")
+    return A
+
+
+def softtopk_rankscale_bwd(L, G, k: int, t: float, beta: float, delta: int) -> np.ndarray:
+    L, G = _f64(L), _f64(G)
+    T, E = L.shape
+    dL = np.empty_like(L)
+    rc = lib().mso_softtopk_rankscale_bwd(I64(T), I64(E), I64(k), C.c_double(t), C.c_double(beta), I64(delta),
+                                          _p(L), _p(G), _p(dL))
+    if rc:
+        raise ValueError("softtopk_rankscale_bwd: bad arguments")
+    return dL
+
+
 def keys_from_scores(A) -> np.ndarray:
     """Fixed-point keys rne(A * 2^40) as int64."""
     A = _f64(A)

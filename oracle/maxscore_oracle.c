@@ -676,3 +676,73 @@ void mso_aux_loss_grad(int64_t T, int64_t E, int64_t k, double lambda, const int
     dA_col[j] = lambda * sp / ((double)E * (double)T * (double)T);
   }
 }
+
+/* ------------------------------------------------------------------ */
+/* The literal readings of Eq. 6 ("RANKSCALE").  Read as printed, the   */
+/* recursion adds t * Softmax(a)_i (softmax over ALL experts, t a       */
+/* factor) at every level at which entry i is not masked, so an entry   */
+/* of rank r (1 = largest, ties: lowest index first) ends up with       */
+/*     y_i = p_i * (beta + t * min(r_i - delta, k)),  p = Softmax(a).    */
+/* (beta, delta) = (0, 0): base 0, level j masks the j-1 largest;       */
+/* (beta, delta) = (1, 1): base Softmax(a), level j masks the j largest. */
+/* The paper prints no value that tells these readings (or ITERMASK)    */
+/* apart: parity unpinned against the paper; the pins are the formula's */
+/* own special cases (tests/test_oracle_softtopk.py).                   */
+static void rank_of_row(int64_t E, const double *a, int64_t *rank) {
+  for (int64_t i = 0; i < E; ++i) {
+    int64_t r = 1;
+    for (int64_t j = 0; j < E; ++j)
+      if (a[j] > a[i] || (a[j] == a[i] && j < i)) ++r;
+    rank[i] = r;
+  }
+}
+
+int mso_softtopk_rankscale_fwd(int64_t T, int64_t E, int64_t k, double t, double beta, int64_t delta,
+                               const double *L, double *A) {
+  if (k < 1 || k > E) return MSO_ERR_ARG;
+  int64_t *rank = (int64_t *)malloc(sizeof(int64_t) * (size_t)E);
+  if (!rank) return MSO_ERR_ALLOC;
+  for (int64_t r = 0; r < T; ++r) {
+    const double *a = L + r * E;
+    double m = a[0], Z = 0.0;
+    for (int64_t i = 1; i < E; ++i) if (a[i] > m) m = a[i];
+    for (int64_t i = 0; i < E; ++i) Z += exp(a[i] - m);
+    rank_of_row(E, a, rank);
+    for (int64_t i = 0; i < E; ++i) {
+      int64_t c = rank[i] - delta; if (c > k) c = k;
+      A[r * E + i] = exp(a[i] - m) / Z * (beta + t * (double)c);
+    }
+  }
+  free(rank);
+  return MSO_OK;
+}
+
+/* Backward with the ranks held constant: y = s (.) p with s fixed, so   */
+/* da_l = p_l * (g_l s_l - sum_i g_i s_i p_i), the softmax Jacobian      */
+/* applied to g (.) s.                                                   */
+int mso_softtopk_rankscale_bwd(int64_t T, int64_t E, int64_t k, double t, double beta, int64_t delta,
+                               const double *L, const double *G, double *dL) {
+  if (k < 1 || k > E) return MSO_ERR_ARG;
+  int64_t *rank = (int64_t *)malloc(sizeof(int64_t) * (size_t)E);
+  double *p = (double *)malloc(sizeof(double) * (size_t)E);
+  if (!rank || !p) { free(rank); free(p); return MSO_ERR_ALLOC; }
+  for (int64_t r = 0; r < T; ++r) {
+    const double *a = L + r * E, *g = G + r * E;
+    double m = a[0], Z = 0.0;
+    for (int64_t i = 1; i < E; ++i) if (a[i] > m) m = a[i];
+    for (int64_t i = 0; i < E; ++i) Z += exp(a[i] - m);
+    rank_of_row(E, a, rank);
+    double dot = 0.0;
+    for (int64_t i = 0; i < E; ++i) {
+      int64_t c = rank[i] - delta; if (c > k) c = k;
+      p[i] = exp(a[i] - m) / Z;
+      dot += g[i] * (beta + t * (double)c) * p[i];
+    }
+    for (int64_t i = 0; i < E; ++i) {
+      int64_t c = rank[i] - delta; if (c > k) c = k;
+      dL[r * E + i] = p[i] * (g[i] * (beta + t * (double)c) - dot);
+    }
+  }
+  free(rank); free(p);
+  return MSO_OK;
+}

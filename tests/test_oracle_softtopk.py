@@ -168,3 +168,47 @@ def test_aux_loss_grad_matches_finite_differences(orc):
     # closed form: lambda / (E T^2) * load_j
     load = np.bincount(idx.ravel(), minlength=E)
     np.testing.assert_allclose(g, lam * load / (E * T * T), rtol=1e-14)
+
+
+# ---- the literal readings of Eq. 6 ("RANKSCALE"); parity unpinned against the paper ---------------------
+def test_rankscale_hand_cases(orc):
+    """Worked by hand from y_i = p_i * (beta + t * min(rank_i - delta, k)), ranks from 1, ties lowest index first."""
+    p = np.array([[0.8, 0.05, 0.1, 0.05]])
+    a = np.log(p)
+    np.testing.assert_allclose(orc.softtopk_rankscale_fwd(a, 2, 1.0, 0.0, 0), [[0.8, 0.1, 0.2, 0.1]], rtol=1e-14)
+    np.testing.assert_allclose(orc.softtopk_rankscale_fwd(a, 2, 1.0, 1.0, 1), [[0.8, 0.15, 0.2, 0.15]], rtol=1e-14)
+    np.testing.assert_allclose(orc.softtopk_rankscale_fwd(a, 2, 0.5, 1.0, 1), [[0.8, 0.1, 0.15, 0.1]], rtol=1e-14)
+    # the tie rule: equal logits, the lower index ranks first
+    q = np.log(np.array([[0.4, 0.4, 0.2]]))
+    np.testing.assert_allclose(orc.softtopk_rankscale_fwd(q, 2, 1.0, 0.0, 0), [[0.4, 0.8, 0.4]], rtol=1e-14)
+
+
+def test_rankscale_special_cases(orc):
+    from scipy.special import softmax
+    rng = np.random.default_rng(6)
+    a = rng.normal(size=(7, 12))
+    # t = 0 with base Softmax is the softmax itself (library routine)
+    np.testing.assert_allclose(orc.softtopk_rankscale_fwd(a, 3, 0.0, 1.0, 1), softmax(a, axis=1), rtol=1e-13)
+    # shift invariance and permutation equivariance
+    y = orc.softtopk_rankscale_fwd(a, 3, 0.7, 0.0, 0)
+    np.testing.assert_allclose(orc.softtopk_rankscale_fwd(a + 5.0, 3, 0.7, 0.0, 0), y, rtol=1e-12)
+    perm = rng.permutation(12)
+    np.testing.assert_allclose(orc.softtopk_rankscale_fwd(a[:, perm], 3, 0.7, 0.0, 0), y[:, perm], rtol=1e-12)
+    # k = E, (0, 0): every entry is scaled by t * its rank
+    ranks = (-a).argsort(1).argsort(1) + 1
+    np.testing.assert_allclose(orc.softtopk_rankscale_fwd(a, 12, 2.0, 0.0, 0), softmax(a, axis=1) * 2.0 * ranks, rtol=1e-13)
+
+
+@pytest.mark.parametrize("beta,delta", [(0.0, 0), (1.0, 1)])
+def test_rankscale_bwd_finite_differences(orc, beta, delta):
+    rng = np.random.default_rng(8)
+    a = rng.normal(size=(3, 9)); g = rng.normal(size=(3, 9))
+    k, t, h = 3, 0.8, 1e-6
+    got = orc.softtopk_rankscale_bwd(a, g, k, t, beta, delta)
+    for (r, l) in [(0, 0), (1, 4), (2, 8), (0, 5)]:
+        ap, am = a.copy(), a.copy()
+        ap[r, l] += h; am[r, l] -= h
+        fd = ((orc.softtopk_rankscale_fwd(ap, k, t, beta, delta) - orc.softtopk_rankscale_fwd(am, k, t, beta, delta)) * g).sum() / (2 * h)
+        assert abs(fd - got[r, l]) < 1e-7
+    # a softmax Jacobian applied to anything sums to zero over the logits
+    np.testing.assert_allclose(got.sum(1), 0.0, atol=1e-14)
