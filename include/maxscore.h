@@ -80,6 +80,13 @@ typedef struct {
   int32_t max_sweeps;      /* bound on price sweeps + augmentations of the solver; 0 = default     */
   int32_t io_dtype;        /* maxscore_dtype of hidden, w_gate, xdisp, yexp, y, dY, dH             */
   int32_t w_gate_layout;   /* 0: w_gate is [d_model, E] as in Eq. 2; 1: [E, d_model]               */
+  int32_t softtopk_mode;   /* 0: Eq. 6 read as k masked softmaxes with temperature t (level j runs  */
+                           /*    over the entries that are not among the j-1 largest); the default */
+                           /* 1: Eq. 6 read literally: y_i = p_i * (beta + t * min(rank_i - delta, */
+                           /*    k)), p = Softmax over all experts, rank 1 = largest, ties: lowest */
+                           /*    index first                                                       */
+  float rankscale_beta;    /* mode 1: 0 = the recursion starts from 0, 1 = it starts from Softmax  */
+  int32_t rankscale_delta; /* mode 1: 0 = level j masks the j-1 largest, 1 = the j largest         */
 } maxscore_params;
 
 typedef struct {           /* lives in DEVICE memory; written by route_fwd / assign                */

@@ -26,7 +26,8 @@ class Params(C.Structure):
     _fields_ = [("T", C.c_int32), ("d_model", C.c_int32), ("E", C.c_int32), ("k", C.c_int32),
                 ("capacity_factor", C.c_float), ("capacity", C.c_int32), ("t", C.c_float),
                 ("score_mode", C.c_int32), ("quant_shift", C.c_int32), ("tiebreak_seed", C.c_uint32),
-                ("max_sweeps", C.c_int32), ("io_dtype", C.c_int32), ("w_gate_layout", C.c_int32)]
+                ("max_sweeps", C.c_int32), ("io_dtype", C.c_int32), ("w_gate_layout", C.c_int32),
+                ("softtopk_mode", C.c_int32), ("rankscale_beta", C.c_float), ("rankscale_delta", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -95,9 +96,10 @@ def _stream(stream):
 
 
 def make_params(T, d_model, E, k, capacity_factor=1.0, capacity=0, t=1.0, score_mode=0, quant_shift=11,
-                tiebreak_seed=0, max_sweeps=0, io_dtype=BF16, w_gate_layout=0) -> Params:
+                tiebreak_seed=0, max_sweeps=0, io_dtype=BF16, w_gate_layout=0, softtopk_mode=0, rankscale_beta=0.0,
+                rankscale_delta=0) -> Params:
     return Params(T, d_model, E, k, capacity_factor, capacity, t, score_mode, quant_shift, tiebreak_seed,
-                  max_sweeps, io_dtype, w_gate_layout)
+                  max_sweeps, io_dtype, w_gate_layout, softtopk_mode, rankscale_beta, rankscale_delta)
 
 
 def capacity(params: Params) -> int:

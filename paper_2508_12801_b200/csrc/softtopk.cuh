@@ -140,6 +140,74 @@ softtopk_bwd_kernel(const float* __restrict__ logits, const int32_t* __restrict_
   }
 }
 
+// The literal readings of Eq. 6 ("rank-scaled softmax"): y_i = p_i * (beta + t * min(rank_i - delta, k)) with
+// p = Softmax(a) over all experts and rank 1 = largest (ties: lowest index first).  Only the k + delta - 1
+// largest entries have a count below k, so that many arg-max rounds give every entry its scale.  The same
+// routine serves the backward pass, where the ranks are constants:
+//   da_l = p_l * (g_l s_l - sum_i g_i s_i p_i),   s_i = beta + t * min(rank_i - delta, k).
+template <bool kBackward>
+__global__ void __launch_bounds__(256)
+softtopk_rankscale_kernel(const float* __restrict__ logits, const int32_t* __restrict__ expert_idx,
+                          const float* __restrict__ dgate_w, const float* __restrict__ dscores_col,
+                          float* __restrict__ out, int T, int E, int k, float t, float beta, int delta) {
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  for (int tok = blockIdx.x * warps_per_block + (threadIdx.x >> 5); tok < T; tok += gridDim.x * warps_per_block) {
+    const float* row = logits + (size_t)tok * E;
+    float a[kEPL], sc[kEPL]; bool live[kEPL];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < kEPL; ++j) {
+      const int e = lane + 32 * j;
+      live[j] = e < E;
+      a[j] = live[j] ? __ldg(row + e) : -INFINITY;
+      mx = fmaxf(mx, a[j]);
+      sc[j] = beta + t * (float)k;                      // every entry of rank >= k + delta
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float p[kEPL], zs = 0.f;
+#pragma unroll
+    for (int j = 0; j < kEPL; ++j) { p[j] = live[j] ? expf(a[j] - mx) : 0.f; zs += p[j]; }
+    zs = warp_sum(zs);
+    const float inv = 1.f / zs;
+    for (int r = 1; r < k + delta && r <= E; ++r) {     // the entry of rank r
+      float best = -INFINITY; int bidx = 0x7fffffff;
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j)
+        if (live[j] && (a[j] > best || bidx == 0x7fffffff)) { best = a[j]; bidx = lane + 32 * j; }
+      warp_argmax(best, bidx);
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j)
+        if (lane + 32 * j == bidx) { live[j] = false; sc[j] = beta + t * (float)(r - delta); }
+    }
+    float* o = out + (size_t)tok * E;
+    if (!kBackward) {
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j) { const int e = lane + 32 * j; if (e < E) o[e] = p[j] * inv * sc[j]; }
+    } else {
+      float g[kEPL];
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j) {
+        const int e = lane + 32 * j;
+        g[j] = (e < E && dscores_col) ? __ldg(dscores_col + e) : 0.f;
+      }
+      for (int c = 0; c < k; ++c) {
+        const int e = __ldg(expert_idx + (size_t)tok * k + c);
+        const float gv = __ldg(dgate_w + (size_t)tok * k + c);
+#pragma unroll
+        for (int j = 0; j < kEPL; ++j) if (lane + 32 * j == e) g[j] += gv;
+      }
+      float dot = 0.f;
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j) dot += g[j] * sc[j] * p[j] * inv;
+      dot = warp_sum(dot);
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j) { const int e = lane + 32 * j; if (e < E) o[e] = p[j] * inv * (g[j] * sc[j] - dot); }
+    }
+  }
+}
+
 // Auxiliary load-balance loss, Eq. 9: L = lambda / (E T^2) * sum_j (sum_i A_ij) * load_j, and its
 // gradient with respect to A (P is a constant): dL/dA_ij = lambda * load_j / (E T^2) for every token i.
 // Column sums are taken by warps over rows (lane l owns columns l, l+32, ...) in double precision and

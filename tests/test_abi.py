@@ -26,7 +26,7 @@ def test_header_symbols_are_exported(ms):
 
 
 def test_struct_layouts_match_header(ms):
-    assert C.sizeof(ms.Params) == 13 * 4
+    assert C.sizeof(ms.Params) == 16 * 4 and ms.Params.softtopk_mode.offset == 13 * 4
     assert C.sizeof(ms.Stats) == 40 and ms.Stats.total_score.offset == 32
     assert C.sizeof(ms.DeviceBuffers) == 12 * 8
 

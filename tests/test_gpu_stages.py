@@ -119,6 +119,50 @@ def test_aux_loss_and_its_gradient_through_softtopk(ms, orc, synth, T, E, k, lam
     assert (np.abs(got - refb) <= 1e-5 * scale + 1e-12).all()
 
 
+@pytest.mark.parametrize("T,E,k,t,beta,delta", [(512, 8, 2, 1.0, 0.0, 0), (1000, 16, 2, 0.5, 1.0, 1), (777, 64, 8, 1.0, 1.0, 1),
+                                                 (515, 128, 8, 0.25, 0.0, 0), (33, 5, 5, 1.0, 0.0, 0), (64, 20, 3, 2.0, 1.0, 1)])
+def test_softtopk_literal_readings_fwd_bwd(ms, orc, synth, T, E, k, t, beta, delta):
+    """softtopk_mode 1: y = softmax(a) * (beta + t * min(rank - delta, k)) and its backward (ranks constant)."""
+    L = synth.logits_like(T, E, seed=4)
+    ctx = _ctx(ms, T, 64, E, k, cf=float(E), t=t, softtopk_mode=1, rankscale_beta=beta, rankscale_delta=delta)
+    Ld = L.to(DEV)
+    A = torch.empty_like(Ld)
+    ms.softtopk_fwd(ctx, Ld, A)
+    assert_rel(np32(A), orc.softtopk_rankscale_fwd(f64(L), k, t, beta, delta), 1e-5, "rank-scaled softmax fwd")
+    g = torch.Generator().manual_seed(6)
+    idx = torch.stack([torch.randperm(E, generator=g)[:k].sort().values for _ in range(T)]).to(torch.int32)
+    dg = torch.randn(T, k, generator=g)
+    col = torch.randn(E, generator=g) * 0.1
+    dL = torch.empty_like(Ld)
+    ms.softtopk_bwd_aux(ctx, Ld, idx.to(DEV), dg.to(DEV), col.to(DEV), dL)
+    G = np.tile(f64(col), (T, 1))
+    G[np.arange(T)[:, None], idx.numpy().astype(np.int64)] += f64(dg)
+    ref = orc.softtopk_rankscale_bwd(f64(L), G, k, t, beta, delta)
+    scale = np.abs(G).max(axis=1, keepdims=True) * (abs(beta) + t * k)      # |da| <= 2 * max|g s| per row
+    assert (np.abs(np32(dL) - ref) <= 1e-5 * scale + 1e-12).all()
+    ms.softtopk_bwd(ctx, Ld, idx.to(DEV), dg.to(DEV), dL)                    # without the dense term
+    G2 = np.zeros((T, E)); np.put_along_axis(G2, idx.numpy().astype(np.int64), f64(dg), axis=1)
+    ref2 = orc.softtopk_rankscale_bwd(f64(L), G2, k, t, beta, delta)
+    assert (np.abs(np32(dL) - ref2) <= 1e-5 * scale + 1e-12).all()
+
+
+def test_route_fwd_with_the_literal_reading(ms, orc, synth):
+    """The solver does not care which reading produced the affinities: optimal for the scores it is given."""
+    wl = synth.scaled(synth.WORKLOADS["k2e16"], T=2048, d_model=256)
+    H, W = synth.hidden(wl), synth.w_gate(wl)
+    ctx = ms.create(ms.make_params(wl.T, wl.d_model, wl.E, wl.k, 1.0, softtopk_mode=1, rankscale_beta=1.0,
+                                   rankscale_delta=1), DEV)
+    buf = ms.RouterBuffers(ctx)
+    ms.route_fwd(ctx, H.to(DEV), W.to(DEV), None, *buf.args())
+    torch.cuda.synchronize()
+    assert ms.read_stats(buf.stats).status == 0
+    L = np32(buf.logits); A = np32(buf.scores)
+    assert_rel(A, orc.softtopk_rankscale_fwd(L.astype(np.float64), wl.k, 1.0, 1.0, 1), 1e-5, "scores")
+    idx = buf.expert_idx.cpu().numpy()
+    res, _ = orc.flow_certificate(float_keys(A), idx, ctx.capacity)
+    assert res >= 1
+
+
 # ------------------------------------------------------------------------------------------- assignment
 def _run_assign(ms, M, T, E, k, cf, **kw):
     ctx = _ctx(ms, T, 64, E, k, cf=cf, **kw)
