@@ -31,8 +31,12 @@
  * largest; ties go to the lowest expert index.
  *
  * Every function here is pinned by tests/test_oracle_*.py against closed
- * forms, library routines, brute force or invariants; none is "parity
- * unpinned".
+ * forms, library routines, brute force or invariants.  One pair is "parity
+ * unpinned" against the paper: mso_softtopk_rankscale_fwd/bwd, the literal
+ * readings of Eq. 6 (pinned by the formula's own special cases only: the
+ * paper prints no value that tells the readings of Eq. 6 apart).
+ *   mso_softtopk_rankscale_fwd/bwd   Eq. 6 read literally (rank-scaled softmax)
+ *   mso_aux_loss_grad                derivative of Eq. 9 with respect to A
  */
 #include <math.h>
 #include <stdint.h>
