@@ -307,6 +307,35 @@ namespace msr {
 
 __global__ void split_dlogits_kernel(const float* __restrict__ dL, __nv_bfloat16* __restrict__ dLs, int T, int E,
                                      int Kpad) {
+  if ((E & 7) == 0) {
+    // eight columns per thread: two 16-byte loads, one 16-byte store each for the hi and the lo part
+    const int g8 = Kpad >> 3;
+    const long long n = (long long)T * g8;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+      const long long t = i / g8; const int j = (int)(i - t * g8) << 3;
+      float x[8];
+      if (j < E) {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(dL + t * E + j));
+        const float4 b = __ldg(reinterpret_cast<const float4*>(dL + t * E + j) + 1);
+        x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+      } else {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) x[q] = 0.f;
+      }
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const __nv_bfloat16 h0 = __float2bfloat16(x[2 * q]), h1 = __float2bfloat16(x[2 * q + 1]);
+        const __nv_bfloat16 l0 = __float2bfloat16(x[2 * q] - __bfloat162float(h0));
+        const __nv_bfloat16 l1 = __float2bfloat16(x[2 * q + 1] - __bfloat162float(h1));
+        hi[q] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+        lo[q] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+      }
+      *reinterpret_cast<uint4*>(dLs + t * 2 * Kpad + j) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      *reinterpret_cast<uint4*>(dLs + t * 2 * Kpad + Kpad + j) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    }
+    return;
+  }
   const long long n = (long long)T * Kpad;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
     const long long t = i / Kpad; const int j = (int)(i - t * Kpad);

@@ -486,6 +486,8 @@ maxscore_status maxscore_combine_bwd(maxscore_ctx* c, const void* dY, const void
 maxscore_status maxscore_gate_bwd(maxscore_ctx* c, const void* hidden, const void* w_gate, const float* dlogits,
                                   float* dw_gate, void* dH, void* stream) {
   if (!c || !hidden || !w_gate || !dlogits || !dw_gate || !dH) return MAXSCORE_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(w_gate) || !aligned16(dlogits) || !aligned16(dw_gate) || !aligned16(dH))
+    return MAXSCORE_ERR_INVALID_ARG;
   const maxscore_params& p = c->p;
   cudaStream_t st = (cudaStream_t)stream;
   if (p.io_dtype != MAXSCORE_BF16) MS_CUDA(cudaMemsetAsync(dw_gate, 0, sizeof(float) * (size_t)p.d_model * p.E, st));
