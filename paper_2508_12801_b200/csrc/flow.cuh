@@ -101,7 +101,13 @@ static_assert(offsetof(FlowState, hist_up) % 16 == 0 && offsetof(FlowState, hist
 // ---------------------------------------------------------------------------------------------
 __global__ void flow_init_kernel(FlowState* st, long long eps0, long long eps_min, int cap0,
                                  long long theta0, int balanced, int E) {
-  for (int i = threadIdx.x; i < 2 * kMaxE * kNB; i += blockDim.x) { st->hist_up[0][i] = 0; st->hist_dn[0][i] = 0; }
+  {   // both histogram buffers, by all CTAs of the launch
+    uint4* zu = reinterpret_cast<uint4*>(st->hist_up[0]); uint4* zd = reinterpret_cast<uint4*>(st->hist_dn[0]);
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 2 * kMaxE * kNB / 4; i += gridDim.x * blockDim.x) {
+      zu[i] = make_uint4(0, 0, 0, 0); zd[i] = make_uint4(0, 0, 0, 0);
+    }
+  }
+  if (blockIdx.x != 0) return;
   for (int e = threadIdx.x; e < kMaxE; e += blockDim.x) {
     st->p[e] = 0; st->load[e] = 0; st->load_cur[e] = 0; st->min_up[e] = kInf; st->min_dn[e] = kInf; st->cap_up[e] = cap0; st->cap_dn[e] = cap0; st->flag_dn[e] = 0;
   }

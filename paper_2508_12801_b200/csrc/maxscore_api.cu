@@ -229,7 +229,7 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   const int n_sweeps = budget < kSweeps ? budget : kSweeps;
   const int max_aug = budget - n_sweeps;
 
-  flow_init_kernel<<<1, 256, 0, st>>>(fs, eps0, eps_min, cap0, theta0, balanced, p.E);
+  flow_init_kernel<<<32, 256, 0, st>>>(fs, eps0, eps_min, cap0, theta0, balanced, p.E);
   MS_LAUNCH_CHECK("flow_init_kernel");
   const int blocks = (p.T + kSweepThreads - 1) / kSweepThreads;
   SweepCache cache{reinterpret_cast<float*>(c->ws + c->lay.cache_x), reinterpret_cast<unsigned char*>(c->ws + c->lay.cache_id),

@@ -37,18 +37,31 @@ index_fill_kernel(const int32_t* __restrict__ expert_idx, const int32_t* __restr
   __shared__ int wcnt[kIdxTok / 32][kMaxE + 1];     // per-warp counts, then exclusive offsets
   __shared__ unsigned bits[kIdxTok / 32][kMaxE];    // lanes of the warp that hold the expert
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int e = threadIdx.x; e < E; e += blockDim.x) {
-    int b = 0, total = 0;
-    for (int blk = 0; blk < (int)gridDim.x; ++blk) {
-      int v = __ldg(block_counts + (size_t)blk * E + e);
-      if (blk < (int)blockIdx.x) b += v;
-      total += v;
-    }
-    base[e] = b;
-    if (blockIdx.x == 0) expert_load[e] = total;
-  }
+  // first slot of this block per expert = the counts of all earlier blocks; the sums are split over
+  // the threads (part p of an expert takes blocks p, p + parts, ...) so that the loads overlap.  Integer
+  // sums: the order of the additions does not matter.
+  __shared__ int total[kMaxE];
+  for (int e = threadIdx.x; e < E; e += blockDim.x) { base[e] = 0; total[e] = 0; }
   for (int e = lane; e < E; e += 32) bits[warp][e] = 0u;
   __syncthreads();
+  {
+    const int parts = max(1, (int)blockDim.x / E);
+    const int e = threadIdx.x % E, part = threadIdx.x / E;
+    if (part < parts) {
+      int b = 0, tot = 0;
+#pragma unroll 4
+      for (int blk = part; blk < (int)gridDim.x; blk += parts) {
+        const int v = __ldg(block_counts + (size_t)blk * E + e);
+        if (blk < (int)blockIdx.x) b += v;
+        tot += v;
+      }
+      if (b) atomicAdd(&base[e], b);
+      if (tot) atomicAdd(&total[e], tot);
+    }
+  }
+  __syncthreads();
+  if (blockIdx.x == 0)
+    for (int e = threadIdx.x; e < E; e += blockDim.x) expert_load[e] = total[e];
   const int tok = blockIdx.x * kIdxTok + threadIdx.x;
   int mine[kMaxK];
 #pragma unroll
