@@ -713,7 +713,7 @@ __device__ __forceinline__ void warp_select(const long long (&val)[kEPLf], int E
 }
 
 // ---------------------------------------------------------------------------------------------
-// Collect / verify pass.  round 0 picks every token's top-k under the sweep prices.  Later rounds
+// Collect / verify pass.  The first pass picks every token's top-k under the sweep prices.  Later ones
 // keep a token's experts when they still are a top-k under the current prices (ties included) and
 // re-pick otherwise.  verify_only never re-picks: it only counts violations and gathers statistics.
 __global__ void __launch_bounds__(kSweepThreads)
