@@ -369,3 +369,49 @@ def test_route_fwd_end_to_end(ms, orc, synth, name, T):
     np.testing.assert_array_equal(buf.slot_token.cpu().numpy(), o_tok)
     np.testing.assert_array_equal(load, o_load)
     np.testing.assert_array_equal(np32(buf.gate_w), np.take_along_axis(A, idx.astype(np.int64), axis=1))
+
+
+@pytest.mark.parametrize("name,T,bias", [("tiny", None, False), ("k2e16", 1000, False), ("skew", 2048, True)])
+def test_route_dispatch_from_host_buffers(ms, orc, synth, name, T, bias):
+    """The end-to-end entry point: batch in host memory in, indices and combine weights back in host memory,
+    dispatched rows on the device.  Same kernels as route_fwd + dispatch, so the results are bit-identical to
+    that path, and the dispatched rows are checked against the oracle."""
+    wl = synth.WORKLOADS[name]
+    wl = synth.scaled(wl, T=T, d_model=min(wl.d_model, 512)) if T else wl
+    T, d, E, k = wl.T, wl.d_model, wl.E, wl.k
+    H, W = synth.hidden(wl), synth.w_gate(wl)
+    b = synth.expert_bias(wl) if bias else None
+    dt = H.dtype
+    ctx = ms.create(ms.make_params(T, d, E, k, wl.capacity_factor, io_dtype=ms.BF16 if wl.dtype == "bf16" else ms.F32), DEV)
+    C_ = ctx.capacity
+    # device path
+    buf = ms.RouterBuffers(ctx)
+    Hd, Wd = H.to(DEV), W.to(DEV)
+    bd = b.to(DEV) if b is not None else None
+    ms.route_fwd(ctx, Hd, Wd, bd, *buf.args())
+    xd = torch.empty(E, C_, d, dtype=dt, device=DEV)
+    ms.dispatch(ctx, Hd, buf.expert_idx, buf.slot_idx, buf.slot_token, xd)
+    torch.cuda.synchronize()
+    want = [t.cpu().clone() for t in (buf.expert_idx, buf.slot_idx, buf.gate_w, buf.slot_token, buf.expert_load, xd)]
+    # host path, fresh device staging buffers
+    buf2 = ms.RouterBuffers(ctx)
+    Hs, Ws = torch.empty_like(Hd), torch.empty_like(Wd)
+    bs = torch.empty_like(bd) if bd is not None else None
+    xd2 = torch.full((E, C_, d), 3.0, dtype=dt, device=DEV)
+    dev = buf2.device_buffers(Hs, Ws, bs, xd2)
+    idx_h = torch.empty(T, k, dtype=torch.int32).pin_memory()
+    slot_h = torch.empty(T, k, dtype=torch.int32).pin_memory()
+    gw_h = torch.empty(T, k, dtype=torch.float32).pin_memory()
+    st_h = torch.zeros(40, dtype=torch.uint8).pin_memory()
+    ms.route_dispatch_host(ctx, H.pin_memory(), W.pin_memory(), b.pin_memory() if b is not None else None, dev,
+                           idx_h, slot_h, gw_h, st_h)
+    torch.cuda.synchronize()
+    assert ms.read_stats(st_h).status == 0
+    assert torch.equal(idx_h, want[0]) and torch.equal(slot_h, want[1]) and torch.equal(gw_h, want[2])
+    assert torch.equal(buf2.slot_token.cpu(), want[3]) and torch.equal(buf2.expert_load.cpu(), want[4])
+    as_int = torch.int16 if dt == torch.bfloat16 else torch.int32
+    assert torch.equal(xd2.cpu().view(as_int), want[5].view(as_int))
+    o_slot, o_tok, _ = orc.index_build(idx_h.numpy(), E, C_)
+    np.testing.assert_array_equal(slot_h.numpy(), o_slot)
+    ref = orc.dispatch(H.view(as_int).numpy(), o_tok)
+    np.testing.assert_array_equal(xd2.cpu().view(as_int).numpy(), ref)
