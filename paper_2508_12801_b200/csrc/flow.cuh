@@ -337,6 +337,20 @@ template <bool kFirst>   // the first sweep scans every row (one thread per toke
 __global__ void __launch_bounds__(kSweepThreads)
 flow_sweep_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, int T, int E, int k, int C,
                   KeyGen g, int sweep_index) {
+  // the token's cache entries do not depend on anything the prologue reads: fetch them first, so that
+  // their latency overlaps the state loads and barriers below
+  uint4 pre_id = make_uint4(0, 0, 0, 0); float pre_x[kCacheN]; long long pre_bound = kInf;
+  {
+    const int tok = blockIdx.x * blockDim.x + threadIdx.x;
+#pragma unroll
+    for (int j = 0; j < kCacheN; ++j) pre_x[j] = 0.f;
+    if (!kFirst && sweep_index > 0 && tok < T) {
+      pre_id = *reinterpret_cast<const uint4*>(cache.id + (size_t)tok * kCacheN);
+#pragma unroll
+      for (int j = 0; j < kCacheN; ++j) pre_x[j] = cache.x[(size_t)j * T + tok];
+      pre_bound = cache.bound[tok];
+    }
+  }
   if (*(volatile int*)&st->p1_done) return;
   // histograms alternate between two buffers: this sweep fills one while every CTA clears a slice of
   // the other for the next sweep (its last reader, the previous price update, has finished)
@@ -398,13 +412,12 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, 
         valid = true;                                   // no expert is flagged before the first sweep
       } else if (sweep0 > 0) {
         const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-        const uint4 idw = *reinterpret_cast<const uint4*>(cache.id + (size_t)tok * kCacheN);
-        const unsigned idws[4] = {idw.x, idw.y, idw.z, idw.w};
+        const unsigned idws[4] = {pre_id.x, pre_id.y, pre_id.z, pre_id.w};
         long long v[kCacheN]; int rank[kCacheN];
 #pragma unroll
         for (int j = 0; j < kCacheN; ++j) {
           const int e = (int)((idws[j >> 2] >> (8 * (j & 3))) & 255u);
-          const float x = cache.x[(size_t)j * T + tok];
+          const float x = pre_x[j];
           v[j] = e < E ? make_key(g, x, flat + e) - sp[e] : -kInf;
           rank[j] = 0;
         }
@@ -422,7 +435,7 @@ flow_sweep_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, 
           if (rank[j] == k) vk1 = v[j];
           if (rank[j] == need - 1) vneed = v[j];
         }
-        const long long bound = cache.bound[tok];
+        const long long bound = pre_bound;
         valid = bound <= -kInf || vneed >= bound + cumdrop;
         if (valid) {
           const bool has_alt = E > k;
