@@ -27,17 +27,6 @@ if ROOT not in sys.path:
 
 METRIC = "routed tokens/s per MoE layer (gate->flow->dispatch) on 1 B200; % of roofline"
 UNIT = "tokens/s"
-SWEEPS, ROUNDS = 24, 6
-
-
-def launches_per_step():
-    """Kernels of this library launched by one step (memsets not counted)."""
-    gate = 2                       # W_g transpose/pad + tcgen05 GEMM
-    assign = 1 + 2 * SWEEPS + 3 * ROUNDS + 1      # init, (sweep + price update) x SWEEPS, (collect + build + exact) x ROUNDS, verify
-    route_fwd = gate + 1 + assign + 2 + 1          # + SoftTopk + index (count, fill) + gate_w gather
-    dispatch, combine = 2, 1
-    route_bwd = 2 + 1 + 5                          # combine-bwd (+padding), SoftTopk-bwd, gate-bwd (split, W_g, dH, dW, reduce)
-    return route_fwd + dispatch + combine + route_bwd + combine   # last combine = dispatch backward
 
 
 class ClockSampler:
@@ -89,6 +78,55 @@ def measured_peak_gbs():
             return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     except Exception:
         return 6650.0, "fallback (6.65 TB/s)"
+
+
+def measured_peak_tflops():
+    """Dense bf16 peak for a kernel timed alone (burst figure)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured (MEASURED_PEAKS.json bf16_tflops)"
+    except Exception:
+        return 1590.0, "fallback (1.59 PFLOP/s)"
+
+
+def time_call(torch, fn, reps=5, flush=None):
+    """Median CUDA-event time of fn() in ms, with an L2 flush (a write larger than L2) before each repetition."""
+    ts = []
+    for _ in range(reps):
+        if flush is not None:
+            flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); fn(); e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    return sorted(ts)[len(ts) // 2]
+
+
+def run_stage_assign(args, wl):
+    """The solver alone on SoftTopk scores of N(0,1) logits shaped like the workload (for ncu captures of its
+    kernels: 4*T*E bytes of scores plus the workspace on the device)."""
+    import torch
+
+    from paper_2508_12801_b200 import binding as ms
+    from paper_2508_12801_b200 import synth
+    dev = "cuda:0"
+    T, E, k = wl.T, wl.E, wl.k
+    ctx = ms.create(ms.make_params(T, 64, E, k, wl.capacity_factor, t=wl.temperature), dev)
+    logits = synth.logits_like(T, E, 0, bias=synth.expert_bias(wl, 0)).to(dev)
+    scores = torch.empty_like(logits)
+    ms.softtopk_fwd(ctx, logits, scores)
+    idx = torch.empty(T, k, dtype=torch.int32, device=dev)
+    load = torch.empty(E, dtype=torch.int32, device=dev)
+    stats = ms.new_stats(dev)
+    for _ in range(max(args.warmup, 1)):
+        ms.assign(ctx, scores, idx, load, stats)
+    torch.cuda.synchronize()
+    t = time_call(torch, lambda: ms.assign(ctx, scores, idx, load, stats), reps=max(args.steps, 1))
+    st = ms.read_stats(stats)
+    print(json.dumps({"stage": "assign", "workload": wl.name, "T": T, "E": E, "k": k, "ms": t, "status": st.status,
+                      "sweeps": st.sweeps, "augmentations": st.augmentations, "rounds": st.rounds,
+                      "candidates": st.candidates, "rerouted": st.rerouted}))
 
 
 # ------------------------------------------------------------------------------------------------ reference arm
@@ -227,11 +265,13 @@ def run_ours(args, wl):
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(8)] for _ in range(args.steps)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sync_all()
+    launches0 = ms.launch_count(ctx)
     e0.record()
     for i in range(args.steps):
         step(evs[i])
     e1.record()
     sync_all()
+    launches = ms.launch_count(ctx) - launches0           # counted by the library at every launch site
     clocks = sampler.stop() if rank == 0 else None
     ms_total = e0.elapsed_time(e1)
     stage_ms = [sum(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(args.steps)) / args.steps for j in range(7)]
@@ -262,10 +302,39 @@ def run_ours(args, wl):
         replicas.shutdown(info)
         return
 
-    # ---- roofline of the dominant kernel -------------------------------------------------------------
+    # ---- the stages of route_fwd one by one (the same kernels through the single-stage entry points), each
+    # timed after an L2 flush; and the solver on the skewed workload's shape, where it has to reroute heavily
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    sub_ms = {
+        "gate": time_call(torch, lambda: ms.gate(ctx, Hd, Wd, bd, buf.logits), flush=flush),
+        "softtopk_fwd": time_call(torch, lambda: ms.softtopk_fwd(ctx, buf.logits, buf.scores), flush=flush),
+        "assign": time_call(torch, lambda: ms.assign(ctx, buf.scores, buf.expert_idx, buf.expert_load, buf.stats), flush=flush),
+        "index_build": time_call(torch, lambda: ms.index_build(ctx, buf.expert_idx, buf.slot_idx, buf.slot_token,
+                                                                buf.expert_load), flush=flush),
+    }
+    st_a = ms.read_stats(buf.stats)
+    skew = synth.WORKLOADS["skew"]
+    ctx_s = ms.create(ms.make_params(skew.T, 64, skew.E, skew.k, skew.capacity_factor), dev)
+    Ls = synth.logits_like(skew.T, skew.E, 0, bias=synth.expert_bias(skew, 0)).to(dev)
+    As = torch.empty_like(Ls)
+    ms.softtopk_fwd(ctx_s, Ls, As)
+    idx_s = torch.empty(skew.T, skew.k, dtype=torch.int32, device=dev)
+    load_s = torch.empty(skew.E, dtype=torch.int32, device=dev)
+    stats_s = ms.new_stats(dev)
+    skew_ms = time_call(torch, lambda: ms.assign(ctx_s, As, idx_s, load_s, stats_s), reps=7, flush=flush)
+    st_s = ms.read_stats(stats_s)
+    del flush
+
+    # ---- rooflines ----------------------------------------------------------------------------------------
     peak, peak_src = measured_peak_gbs()
+    tpeak, tpeak_src = measured_peak_tflops()
     row = d * eb
-    alg_bytes = {   # algorithmic bytes per launch
+    passes = st_a.sweeps + 1 + max(st_a.rounds, 1)              # score-matrix passes the solver's budget allows: scan, sweeps, checks
+    alg_bytes = {   # algorithmic bytes per launch (bytes per token x T tokens)
+        "gate": T * (row + 4 * E) + d * E * eb,                    # read H once and W_g, write the logits
+        "softtopk_fwd": T * 8 * E,                                 # read the logits, write the scores
+        "assign": T * 4 * E * passes,                              # 4E bytes per token and pass over the scores
+        "index_build": T * 12 * k,
         "route_fwd": T * row + T * E * 4 * 4,                      # read H once; logits and scores written and read
         "dispatch": T * row + T * k * row,                         # read each row once, write it k times
         "combine": T * k * row + T * row,
@@ -274,23 +343,36 @@ def run_ours(args, wl):
         "gate_bwd": 2 * T * row + T * E * 4,                       # read H (dW) and dL, write dH
         "dispatch_bwd": T * k * row + 2 * T * row,                 # read k rows, read-modify-write dH
     }
-    # dominant single kernel: the slowest of the four data movers (each stage is that kernel plus the small
-    # padding-zero kernel); route_fwd and gate_bwd are chains of kernels and are reported in "stages"
-    movers = [1, 2, 3, 6]
-    dom = max(movers, key=lambda j: stage_ms[j])
-    dom_name = stage_names[dom]
-    achieved = alg_bytes[dom_name] / (stage_ms[dom] * 1e-3) / 1e9
-    # DRAM bytes per token from the ncu capture summarised in profiles/ncu_data_movement_and_gate_T16384.md
-    # (bf16, d_model=4096, k=8; traffic is proportional to T).  None for any other shape.
+    all_ms = dict(zip(stage_names, stage_ms))
+    all_ms.update(sub_ms)
+    def frac_of(n):
+        return alg_bytes[n] / (all_ms[n] * 1e-3) / 1e9 / peak
+    # the kernel (or chain of kernels) furthest from its roofline among those that take at least 5 % of the step
+    parts = ["gate", "softtopk_fwd", "assign", "index_build", "dispatch", "combine", "combine_bwd", "softtopk_bwd",
+             "gate_bwd", "dispatch_bwd"]
+    heavy = [n for n in parts if all_ms[n] >= 0.05 * ms_step]
+    dom_name = min(heavy, key=frac_of)
+    achieved = alg_bytes[dom_name] / (all_ms[dom_name] * 1e-3) / 1e9
+    # DRAM bytes per launch from the ncu captures summarised under profiles/ (data movers: T=16384 capture, traffic
+    # proportional to T; solver: capture of the solver alone at this size).  None for any other shape.
     ncu_bytes_per_token = {"dispatch": (0.1354e9 + 1.0151e9) / 16384, "combine": (1.0756e9 + 0.1285e9) / 16384,
                            "combine_bwd": (1.2095e9 + 1.0316e9) / 16384,
                            "dispatch_bwd": (1.2103e9 + 0.1285e9) / 16384}
-    traffic = ncu_bytes_per_token[dom_name] * T if (d == 4096 and k == 8 and eb == 2) else None
-    stages = {n: {"ms": round(stage_ms[j], 4), "alg_GB": round(alg_bytes[n] / 1e9, 4),
-                  "GBps": round(alg_bytes[n] / (stage_ms[j] * 1e-3) / 1e9, 1),
-                  "frac_of_hbm_peak": round(alg_bytes[n] / (stage_ms[j] * 1e-3) / 1e9 / peak, 4)}
-              for j, n in enumerate(stage_names)}
+    traffic = None
+    if d == 4096 and k == 8 and eb == 2 and dom_name in ncu_bytes_per_token:
+        traffic = ncu_bytes_per_token[dom_name] * T
+    stages = {n: {"ms": round(all_ms[n], 4), "alg_GB": round(alg_bytes[n] / 1e9, 4),
+                  "GBps": round(alg_bytes[n] / (all_ms[n] * 1e-3) / 1e9, 1),
+                  "frac_of_hbm_peak": round(frac_of(n), 4)}
+              for n in stage_names + list(sub_ms)}
+    gate_tflops = 2.0 * T * d * E / (sub_ms["gate"] * 1e-3) / 1e12
+    stages["gate"]["TFLOPs"] = round(gate_tflops, 1)
+    stages["gate"]["frac_of_bf16_peak"] = round(gate_tflops / tpeak, 4)     # tensor pipe beside HBM: the GEMM is HBM-bound
     fwd_ms = stage_ms[0] + stage_ms[1]
+    span_bytes = alg_bytes["gate"] + alg_bytes["softtopk_fwd"] + alg_bytes["dispatch"]      # the metric's span without the solver
+    roofline_span = {"covers": "gate -> SoftTopk -> flow -> index -> dispatch", "alg_GB": round(span_bytes / 1e9, 3),
+                     "ms": round(fwd_ms, 4), "floor_ms": round(span_bytes / peak / 1e6, 4),
+                     "frac": round(span_bytes / peak / 1e6 / fwd_ms, 4)}
 
     # ---- the CPU checker on the host cores, bounded sample ------------------------------------------------
     cpu = None
@@ -316,13 +398,19 @@ def run_ours(args, wl):
         "solver": {"status": st2.status, "sweeps": st2.sweeps, "augmentations": st2.augmentations,
                    "rounds": st2.rounds, "candidates": st2.candidates, "rerouted": st2.rerouted,
                    "total_score": st2.total_score},
+        "solver_skew": {"workload": "skew (T=16384, E=64, k=8, cf=1.25, Zipf bias)", "ms": round(skew_ms, 4),
+                        "status": st_s.status, "sweeps": st_s.sweeps, "augmentations": st_s.augmentations,
+                        "rounds": st_s.rounds, "candidates": st_s.candidates, "rerouted": st_s.rerouted},
         "roofline": {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src},
+                     "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                     "rule": "lowest fraction among the stages that take at least 5 % of the step",
+                     "tensor_peak_TFLOPs": tpeak, "tensor_peak_source": tpeak_src},
+        "roofline_span": roofline_span,
         "cpu_baseline": cpu,
         "e2e": {"value": replicas.aggregate_tokens_per_s(info, T, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                 "covers": "maxscore_route_dispatch_host (pinned host batch in, indices out) + rest of the step on device"},
-        "gpu_launches": launches_per_step() * args.steps,
+        "gpu_launches": launches,
         "clocks": clocks,
     }
     print(json.dumps(out))
@@ -340,12 +428,15 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=4096, help="tokens per step of the CPU checker's sample (--impl reference)")
     ap.add_argument("--cpu-tokens", type=int, default=16384, help="tokens of the one-off cpu_baseline sample (10-30 s of CPU work)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stage", default="", choices=["", "assign"], help="run one stage alone (for profiler captures)")
     args = ap.parse_args()
     from paper_2508_12801_b200 import synth
     wl = synth.WORKLOADS[args.workload]
     if args.tokens:
         wl = synth.scaled(wl, T=args.tokens)
-    if args.impl == "reference":
+    if args.stage == "assign":
+        run_stage_assign(args, wl)
+    elif args.impl == "reference":
         run_reference(args, wl)
     else:
         run_ours(args, wl)

@@ -20,6 +20,10 @@
  *     short workspace) return a status before anything is launched.  Conditions only the device sees
  *     (solver gave up, non-finite input) set bits in maxscore_stats.status, which the caller reads
  *     after synchronising.  Nothing aborts, throws or traps.
+ *   - Every wait inside a kernel is bounded.  A wait that runs out raises the context's internal-error
+ *     flag and the kernel returns with its output incomplete.  maxscore_route_fwd and maxscore_assign
+ *     report the flag as MAXSCORE_STAT_INTERNAL in stats.status and clear it; after the calls that write
+ *     no stats (maxscore_gate, maxscore_gate_bwd, maxscore_route_bwd) read it with maxscore_check_internal.
  *   - expert_idx[i, :] is ascending.  slot_idx[i, c] is the rank of token i among the tokens of expert
  *     expert_idx[i, c], in ascending token order.  Unused slots of slot_token hold -1.
  *   - If the solver runs out of its budget (MAXSCORE_STAT_NOT_CONVERGED; never seen with the default
@@ -217,6 +221,20 @@ maxscore_status maxscore_combine_bwd(maxscore_ctx* ctx, const void* dY, const vo
 /* Derivative of Eq. 2 alone (last two outputs of route_bwd). */
 maxscore_status maxscore_gate_bwd(maxscore_ctx* ctx, const void* hidden, const void* w_gate,
                                   const float* dlogits, float* dw_gate, void* dH, void* cuda_stream);
+
+/* ---- housekeeping (no counterpart in the paper) --------------------------------------------------- */
+
+/* Reads and clears the context's internal-error flag: *flag_out != 0 means that a bounded wait inside one of
+ * the tensor-core kernels (gate, gate backward) or the solver's grid barrier gave up since the flag was last
+ * cleared, so some output of that call is incomplete.  Synchronises cuda_stream.  flag_out is HOST memory. */
+maxscore_status maxscore_check_internal(maxscore_ctx* ctx, uint32_t* flag_out, void* cuda_stream);
+
+/* Kernels launched through this context since maxscore_create (memsets and copies not counted).  Host only. */
+long long maxscore_launch_count(const maxscore_ctx* ctx);
+
+/* For tests of the error plumbing only: raises the internal-error flag from the host (one cudaMemsetAsync on
+ * cuda_stream), as if a bounded wait had run out.  Nothing waits, hangs or faults. */
+maxscore_status maxscore_test_raise_internal(maxscore_ctx* ctx, void* cuda_stream);
 
 /* ---- end-to-end from host memory ---------------------------------------------------------------- */
 

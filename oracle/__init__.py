@@ -149,6 +149,16 @@ def keys_from_scores(A) -> np.ndarray:
     return w
 
 
+def keys_from_scores_hashed(A) -> np.ndarray:
+    """Float-mode keys as the library documents them: rne(A * 2^40) plus the 12-bit position hash
+    ((i*E + j) * 2654435761 mod 2^32) >> 20."""
+    A = _f64(A)
+    T, E = A.shape
+    w = np.empty(A.shape, np.int64)
+    lib().mso_keys_from_scores_hashed(I64(T), I64(E), _p(A), _p(w))
+    return w
+
+
 def tiebreak_shift(T: int, k: int) -> int:
     return int(lib().mso_tiebreak_shift(I64(T), I64(k)))
 

@@ -15,6 +15,7 @@
  *   mso_gate                Eq. 2, x . W_g  (plus the optional expert bias)
  *   mso_softtopk_fwd/bwd    Eq. 6 (reading "ITERMASK", see below) and its derivative
  *   mso_keys_from_scores    fixed-point keys of the affinities A (Eq. 8 objective)
+ *   mso_keys_from_scores_hashed   the same plus the 12-bit position hash the library documents
  *   mso_keys_from_logits    int16-quantised logits with a hashed tie-break
  *   mso_flow_ssp            Eq. 7-8 on the network of Table 1, solved by
  *                           successive shortest augmenting paths (SPFA), Sec. 3.2
@@ -157,6 +158,18 @@ int mso_softtopk_bwd(int64_t T, int64_t E, int64_t k, double t, const double *L,
 /* Float mode: fixed-point image of the affinities, w = rne(A * 2^40).  */
 void mso_keys_from_scores(int64_t n, const double *A, int64_t *w) {
   for (int64_t i = 0; i < n; ++i) w[i] = llrint(ldexp(A[i], 40));
+}
+
+/* Float mode as the library solves it: the same fixed-point image plus a 12-bit  */
+/* multiplicative hash of the entry's position (i*E + j) * 2654435761 mod 2^32,   */
+/* top 12 bits.  The hash only separates exact ties between equal scores; it adds */
+/* less than 2^12 units of 2^-40 (under 4e-9) to any key.                          */
+void mso_keys_from_scores_hashed(int64_t T, int64_t E, const double *A, int64_t *w) {
+  for (int64_t i = 0; i < T; ++i)
+    for (int64_t j = 0; j < E; ++j) {
+      uint32_t pos = (uint32_t)(i * E + j);
+      w[i * E + j] = llrint(ldexp(A[i * E + j], 40)) + (int64_t)((pos * 2654435761u) >> 20);
+    }
 }
 
 /* 32-bit finaliser of MurmurHash3 (Appleby, public domain). */

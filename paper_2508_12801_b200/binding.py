@@ -47,7 +47,8 @@ EXPORTS = ["maxscore_capacity", "maxscore_workspace_bytes", "maxscore_create", "
            "maxscore_route_bwd", "maxscore_gate", "maxscore_softtopk_fwd", "maxscore_softtopk_bwd",
            "maxscore_assign", "maxscore_index_build", "maxscore_combine_bwd", "maxscore_gate_bwd",
            "maxscore_route_dispatch_host", "maxscore_index_build_noalloc", "maxscore_aux_loss",
-           "maxscore_softtopk_bwd_aux"]
+           "maxscore_softtopk_bwd_aux", "maxscore_check_internal", "maxscore_launch_count",
+           "maxscore_test_raise_internal"]
 
 
 def _load():
@@ -59,8 +60,9 @@ def _load():
     lib.maxscore_capacity.restype = C.c_int32
     lib.maxscore_last_cuda_error.restype = C.c_char_p
     lib.maxscore_destroy.restype = None
+    lib.maxscore_launch_count.restype = C.c_longlong
     for name in EXPORTS:
-        if name not in ("maxscore_capacity", "maxscore_last_cuda_error", "maxscore_destroy"):
+        if name not in ("maxscore_capacity", "maxscore_last_cuda_error", "maxscore_destroy", "maxscore_launch_count"):
             getattr(lib, name).restype = C.c_int
     return lib
 
@@ -217,6 +219,21 @@ def combine_bwd(ctx, dY, yexp, expert_idx, slot_idx, gate_w, slot_token, dyexp, 
 def gate_bwd(ctx, hidden, w_gate, dlogits, dw_gate, dH, stream=None):
     _check(_lib.maxscore_gate_bwd(ctx.handle, _ptr(hidden), _ptr(w_gate), _ptr(dlogits), _ptr(dw_gate), _ptr(dH),
                                   _stream(stream)), "maxscore_gate_bwd")
+
+
+def check_internal(ctx, stream=None) -> int:
+    """Reads and clears the context's internal-error flag (synchronises the stream); non-zero = a bounded wait gave up."""
+    flag = C.c_uint32(0)
+    _check(_lib.maxscore_check_internal(ctx.handle, C.byref(flag), _stream(stream)), "maxscore_check_internal")
+    return int(flag.value)
+
+
+def launch_count(ctx) -> int:
+    return int(_lib.maxscore_launch_count(ctx.handle))
+
+
+def test_raise_internal(ctx, stream=None):
+    _check(_lib.maxscore_test_raise_internal(ctx.handle, _stream(stream)), "maxscore_test_raise_internal")
 
 
 def route_dispatch_host(ctx, hidden_host, w_gate_host, expert_bias_host, dev: DeviceBuffers, expert_idx_host,

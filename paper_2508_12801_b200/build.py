@@ -29,6 +29,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-shared", "-Xcompiler", "-fPIC", "--cudart", "static", "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("MAXSCORE_NVCC_FLAGS", "").split()
     cmd += [os.path.join(CSRC, f) for f in SOURCES]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)

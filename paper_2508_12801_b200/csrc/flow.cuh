@@ -5,41 +5,42 @@
 // token independently holds its k largest values of key(i, e) - p_e.  The solver therefore works on
 // the E prices, never on the T x E arcs:
 //
-//   sweeps    (data parallel, one thread per token)  every token re-picks its top-k under the
-//             current prices; per expert a load count, two histograms of margins (how much a price
-//             rise makes a holder leave / how much a price cut makes an outsider join) and the exact
-//             smallest margin are collected.  The first sweep scans whole rows and caches each
-//             token's 16 best experts with a bound on everything else; later sweeps re-evaluate the
-//             cached entries only, and rescan a row (one warp) when the bound no longer vouches for
-//             them.  A one-CTA kernel then moves each over- or under-loaded expert's price to the
-//             histogram quantile that balances it, plus a step eps that is halved as the sweeps go
-//             on; small imbalances move one exact margin at a time.  This is an epsilon-scaled
-//             simultaneous price adjustment (auction-style); it ends a few dozen token moves away
-//             from the optimum and stops early once a small imbalance has stopped shrinking.
-//   collect   every token's top-k under the final prices is written out; tokens whose k-th and
-//             (k+1)-th values differ by at most theta are listed as candidates.
-//   build     the cost matrix D[e][f] = cheapest move of one candidate token from e to f is built by
-//             the whole GPU (one warp per candidate, 64-bit atomicMin).
+//   scan      (one warp per token) reads the score matrix once and keeps, per token, its 16 best experts
+//             (score and index) with a rigorous bound on everything else: the token's candidate cache.
+//   sweeps    (one persistent cooperative kernel, one thread per token) every token re-picks its top-k
+//             under the current prices from its cache; per expert a load count, two histograms of margins
+//             (how much a price rise makes a holder leave / how much a price cut makes an outsider join)
+//             and the exact smallest margin are collected.  After a grid-wide barrier one warp per expert
+//             moves the price of an over- or under-loaded expert to the histogram quantile that balances
+//             it, plus a step eps that is halved as the sweeps go on; small imbalances move one exact
+//             margin at a time.  This is an epsilon-scaled simultaneous price adjustment (auction-style);
+//             it ends a few dozen token moves away from the optimum and stops early once a small imbalance
+//             has stopped shrinking.  A token whose cache can no longer vouch for its top-(k+2) (the bound
+//             on the uncached experts has come too close) is rescanned by a warp.  The kernel ends by
+//             writing every token's top-k under the final prices and listing the tokens whose k-th and
+//             (k+1)-th values differ by at most theta as candidates.
+//   records   per candidate, the experts it could give up or take within the arc window (whole GPU).
 //   exact     one CTA runs successive shortest augmenting paths on the expert-level residual graph
-//             (E experts + one node Z for the sink side) with D as arc costs; node potentials keep reduced costs non-negative, so each search is a
-//             Bellman-Ford over E+1 nodes held in shared memory.  It ends with every expert within
-//             capacity and complementary slackness satisfied for the candidates.
-//   verify    a last data-parallel pass checks complementary slackness for EVERY token under the
-//             final prices.  If a non-candidate token is violated, theta grows and collect/exact run
-//             again.  Passing this check is a proof of optimality (LP duality of Eq. 7-8).
+//             (E experts + one node Z for the sink side); node potentials keep reduced costs
+//             non-negative, so each search is a Bellman-Ford over E+1 nodes whose arcs are read off the
+//             candidate records.  It ends with every expert within capacity and complementary slackness
+//             satisfied for the candidates.
+//   check     a data-parallel pass checks complementary slackness for EVERY token under the final prices
+//             (from the cache where its bound allows, from the full row otherwise).  If a token is
+//             violated it re-picks, theta grows and records/exact run again.  Passing this check is a
+//             proof of optimality (LP duality of Eq. 7-8); the same pass gathers the statistics.
 //
 // All arithmetic is on int64 keys: key = rne(A * 2^40) (+ a 12-bit position hash) for float
 // affinities, or the quantised logit with a hashed tie-break.
 #pragma once
 #include <cstddef>
+#include <type_traits>
 #include "common.cuh"
 
 namespace msr {
 
 constexpr int kNB = 256;                  // histogram bins per expert: 4 per octave of the margin
-constexpr int kTopN = kMaxK + 2;          // sorted values kept per token in a sweep
 constexpr long long kInf = 1LL << 62;
-constexpr long long kArcLimit = 1LL << 58; // arcs with a larger reduced cost are ignored by the exact phase
 constexpr long long kPriceLimit = 1LL << 56; // sweeps keep |price| below this
 constexpr int kCapLogMax = 60;
 constexpr int kStallSweeps = 3, kStallImbalance = 256;
@@ -60,7 +61,7 @@ __device__ __forceinline__ uint32_t fmix32(uint32_t h) {   // 32-bit finaliser o
 }
 
 __device__ __forceinline__ long long make_key(const KeyGen& g, float x, uint32_t flat_idx) {
-  if (!isfinite(x)) x = 0.f;   // reported separately by the collect pass
+  if (!isfinite(x)) x = 0.f;   // reported separately by the scan
   // x * 2^40 is exact in fp32; the low 12 bits carry a multiplicative hash of the entry's position so
   // that identical rows do not tie exactly (it moves the optimum by less than 4e-9 per chosen pair)
   if (g.mode == 0) return __float2ll_rn(x * 1099511627776.0f) + (long long)((flat_idx * 2654435761u) >> 20);
@@ -71,36 +72,44 @@ __device__ __forceinline__ long long make_key(const KeyGen& g, float x, uint32_t
   return q * (1LL << g.S) + (long long)r;
 }
 
+// Key in fp32 (24 significant bits): good enough to FIND the largest few entries of a row cheaply.
+// key - approx_key lies in [-0.5, 4096.5) for float affinities and in [0, 2^20) for quantised logits.
+__device__ __forceinline__ float approx_key(const KeyGen& g, float x) {
+  if (!isfinite(x)) x = 0.f;
+  if (g.mode == 0) return x * 1099511627776.0f;
+  return fminf(fmaxf(rintf(x * g.fshift), -32768.f), 32767.f) * g.fS;
+}
+
+
 struct FlowState {
-  int trace[128];            // diagnostics: [0..23] imbalance per sweep, [64..] rows scanned in full per sweep
   long long p[kMaxE];        // expert prices
-  long long eps, eps_min;
-  long long theta;           // candidate threshold of the next collect pass
+  long long theta;           // candidate threshold of the next listing
   long long theta_used;      // threshold the current candidate list was collected with
+  long long cumdrop;         // bound on how much any expert's price has dropped since the caches were built
   double total_score;
-  int load[kMaxE];           // accumulated by the running pass, consumed by its last CTA
+  int load[kMaxE];           // accumulated by the running pass, consumed by its price step / last CTA
   int load_cur[kMaxE];       // loads of the assignment currently written in expert_idx
   alignas(16) unsigned hist_up[2][kMaxE * kNB];   // [sweep parity]; read and cleared with 16-byte accesses
   alignas(16) unsigned hist_dn[2][kMaxE * kNB];
-  long long cumdrop;                              // sum over sweeps of the largest price decrease of that sweep
-  int cut_max;                                    // log2 of the largest margin worth recording at all
-  long long min_up[kMaxE], min_dn[kMaxE];   // smallest margin recorded by the running sweep (reset by the price update)
+  long long min_up[kMaxE], min_dn[kMaxE];   // smallest margin recorded by the running sweep (reset by the price step)
   int cap_up[kMaxE], cap_dn[kMaxE];   // log2 of the largest margin worth recording
   int flag_dn[kMaxE];                 // expert whose join-histogram came out short: scan it in full next sweep
+  int imb_e[kMaxE];                   // |load - C| of the experts that moved their price in the last price step
+  long long drop_e[kMaxE];            // by how much the last price step lowered each price
+  unsigned bar_count, bar_abort;      // grid-wide barrier of the sweeps kernel
   unsigned ticket;
-  int sweep, p1_done, balanced;
-  int best_imb, stall;                // smallest imbalance seen so far; sweeps since it last improved
-  int round, converged, ncand, violations, naug, rerouted;
+  int sweep, balanced;
+  int round, converged, done, ncand, violations, naug, rerouted;
   unsigned status;
   int ncand_last;
+  int nrec, rec_overflow;             // entries of the exact phase's candidate records in use; set when they ran out
 };
 
 static_assert(offsetof(FlowState, hist_up) % 16 == 0 && offsetof(FlowState, hist_dn) % 16 == 0 && (kMaxE * kNB * 4) % 16 == 0,
               "histograms are accessed as uint4");
 
 // ---------------------------------------------------------------------------------------------
-__global__ void flow_init_kernel(FlowState* st, long long eps0, long long eps_min, int cap0,
-                                 long long theta0, int balanced, int E) {
+__global__ void flow_init_kernel(FlowState* st, int cap0, long long theta0, int balanced, int E) {
   {   // both histogram buffers, by all CTAs of the launch
     uint4* zu = reinterpret_cast<uint4*>(st->hist_up[0]); uint4* zd = reinterpret_cast<uint4*>(st->hist_dn[0]);
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 2 * kMaxE * kNB / 4; i += gridDim.x * blockDim.x) {
@@ -109,110 +118,16 @@ __global__ void flow_init_kernel(FlowState* st, long long eps0, long long eps_mi
   }
   if (blockIdx.x != 0) return;
   for (int e = threadIdx.x; e < kMaxE; e += blockDim.x) {
-    st->p[e] = 0; st->load[e] = 0; st->load_cur[e] = 0; st->min_up[e] = kInf; st->min_dn[e] = kInf; st->cap_up[e] = cap0; st->cap_dn[e] = cap0; st->flag_dn[e] = 0;
+    st->p[e] = 0; st->load[e] = 0; st->load_cur[e] = 0; st->min_up[e] = kInf; st->min_dn[e] = kInf;
+    st->cap_up[e] = cap0; st->cap_dn[e] = cap0; st->flag_dn[e] = 0; st->imb_e[e] = 0; st->drop_e[e] = 0;
   }
   if (threadIdx.x == 0) {
-    st->eps = eps0; st->eps_min = eps_min; st->theta = theta0; st->total_score = 0.0;
-    st->ticket = 0; st->sweep = 0; st->p1_done = 0; st->balanced = balanced; st->best_imb = 0x7fffffff; st->stall = 0;
-    for (int i = 64; i < 128; ++i) st->trace[i] = 0;
-    st->round = 0; st->converged = 0; st->ncand = 0; st->violations = 0; st->naug = 0;
-    st->rerouted = 0; st->status = 0; st->ncand_last = 0; st->cut_max = cap0; st->cumdrop = 0;
+    st->theta = theta0; st->theta_used = theta0; st->total_score = 0.0; st->cumdrop = 0;
+    st->bar_count = 0; st->bar_abort = 0;
+    st->ticket = 0; st->sweep = 0; st->balanced = balanced;
+    st->round = 0; st->converged = 0; st->done = 0; st->ncand = 0; st->violations = 0; st->naug = 0;
+    st->rerouted = 0; st->status = 0; st->ncand_last = 0; st->nrec = 0; st->rec_overflow = 0;
   }
-}
-
-// Insert (val, id) into a list sorted by descending value, lower expert index first on equal values.
-template <int N>
-__device__ __forceinline__ void top_insert_tb(long long (&v)[N], int (&id)[N], long long val, int e) {
-  if (val > v[N - 1] || (val == v[N - 1] && e < id[N - 1])) {
-    v[N - 1] = val; id[N - 1] = e;
-#pragma unroll
-    for (int j = N - 1; j > 0; --j) {
-      if (v[j] > v[j - 1] || (v[j] == v[j - 1] && id[j] < id[j - 1])) {
-        long long tv = v[j]; v[j] = v[j - 1]; v[j - 1] = tv;
-        int ti = id[j]; id[j] = id[j - 1]; id[j - 1] = ti;
-      }
-    }
-  }
-}
-
-// Key in fp32 (24 significant bits): good enough to FIND the largest few entries of a row cheaply.
-__device__ __forceinline__ float approx_key(const KeyGen& g, float x) {
-  if (!isfinite(x)) x = 0.f;
-  if (g.mode == 0) return x * 1099511627776.0f;
-  return fminf(fmaxf(rintf(x * g.fshift), -32768.f), 32767.f) * g.fS;
-}
-
-// The N largest entries of key(e) - price(e) over one row, exact and sorted (value descending, lower
-// expert index first on equal values).
-//   1. a branch-free pass keeps the N largest fp32 approximations; the expert index rides in the low
-//      7 mantissa bits, so each slot costs one max and one min;
-//   2. the exact int64 values of those N experts are computed and sorted;
-//   3. if `exact`, a second pass checks that no other expert beats the N-th one exactly; in the rare
-//      case one does (values closer than fp32 resolves), the row is redone by exact insertion.
-// Without `exact` the result may miss an entry that differs from the N-th by less than ~2^-17 relative.
-template <int N>
-__device__ __forceinline__ void select_top(const float* row, const long long* sp, const float* spf, const KeyGen& g,
-                                           uint32_t flat, int E, int start, bool exact, long long (&v)[N],
-                                           int (&id)[N]) {
-  float pk[N];
-#pragma unroll
-  for (int j = 0; j < N; ++j) pk[j] = -INFINITY;
-  int e = start;
-  auto feed = [&](float val, int ee) {
-    const float vf = approx_key(g, val) - (spf ? spf[ee] : 0.f);
-    float x = __uint_as_float((__float_as_uint(vf) & ~127u) | (unsigned)ee);
-#pragma unroll
-    for (int j = 0; j < N; ++j) { const float hi = fmaxf(pk[j], x); x = fminf(pk[j], x); pk[j] = hi; }
-  };
-  if (start < 0) {
-    // row in global memory: 16-byte loads, so that each 32-byte sector is fetched by two adjacent
-    // instructions instead of eight that the L1 may not keep apart
-    for (int e4 = 0; e4 < E; e4 += 4) {
-      const float4 x4 = __ldg(reinterpret_cast<const float4*>(row + e4));
-      feed(x4.x, e4); feed(x4.y, e4 + 1); feed(x4.z, e4 + 2); feed(x4.w, e4 + 3);
-    }
-    start = 0;
-  } else {
-    for (int jj = 0; jj < E; ++jj) {
-      feed(row[e], e);
-      if (++e == E) e = 0;
-    }
-  }
-#pragma unroll
-  for (int j = 0; j < N; ++j) {
-    const bool ok = pk[j] != -INFINITY;
-    const int ee = (int)(__float_as_uint(pk[j]) & 127u);
-    id[j] = ok ? ee : -1;
-    v[j] = ok ? make_key(g, row[ee], flat + ee) - (sp ? sp[ee] : 0) : -kInf;
-  }
-#pragma unroll
-  for (int pass = 0; pass < N; ++pass) {
-#pragma unroll
-    for (int j = (pass & 1); j + 1 < N; j += 2) {
-      if (v[j + 1] > v[j] || (v[j + 1] == v[j] && id[j + 1] >= 0 && id[j + 1] < id[j])) {
-        const long long tv = v[j]; v[j] = v[j + 1]; v[j + 1] = tv;
-        const int ti = id[j]; id[j] = id[j + 1]; id[j + 1] = ti;
-      }
-    }
-  }
-  if (!exact || id[N - 1] < 0) return;                 // E <= N: every expert is in the list
-  const long long tv = v[N - 1]; const int ti = id[N - 1];
-  bool missed = false;
-  e = start;
-  for (int jj = 0; jj < E; ++jj) {
-    const long long val = make_key(g, row[e], flat + e) - (sp ? sp[e] : 0);
-    if (val > tv || (val == tv && e < ti)) {
-      bool in = false;
-#pragma unroll
-      for (int j = 0; j < N; ++j) in |= (id[j] == e);
-      missed |= !in;
-    }
-    if (++e == E) e = 0;
-  }
-  if (!missed) return;
-#pragma unroll
-  for (int j = 0; j < N; ++j) { v[j] = -kInf; id[j] = -1; }
-  for (e = 0; e < E; ++e) top_insert_tb(v, id, make_key(g, row[e], flat + e) - (sp ? sp[e] : 0), e);
 }
 
 __device__ __forceinline__ bool last_block_arrives(unsigned* ticket) {
@@ -300,355 +215,6 @@ __device__ __forceinline__ long long price_step_warp(const uint4& ha, const uint
   return lo;
 }
 
-// ---------------------------------------------------------------------------------------------
-// One price sweep.
-constexpr int kSweepThreads = 128;
-
-// Per-token candidate cache of the sweeps.  A full scan of a token's row keeps its kCacheN best experts
-// (score and index) and `bound` = the smallest of their values minus the total price drop so far.  A
-// later sweep re-evaluates only those kCacheN entries; every other expert is worth at most
-// bound + (total price drop now), so while the (k+2)-th cached value stays at or above that, the cached
-// entries still contain the token's k+2 best experts and the row need not be read again.
-constexpr int kCacheN = 16;
-struct SweepCache {
-  float* x;              // [kCacheN][T] scores of the cached experts
-  unsigned char* id;     // [T][kCacheN] their indices (255 = none)
-  long long* bound;      // [T]
-};
-
-struct SweepShared {
-  long long sp[kMaxE];
-  float spf[kMaxE];
-  int sload[kMaxE], scu[kMaxE], scd[kMaxE], sflag[kMaxE];
-  int nflag, nslow;
-  unsigned short slow[kSweepThreads];
-};
-
-__device__ __forceinline__ void emit_margin(unsigned* hist, long long* mins, const int* caplog, int e, long long m) {
-  if (m >= 0 && m < (1LL << caplog[e])) {
-    atomicAdd(&hist[e * kNB + log_bin(m)], 1u);
-    // the exact smallest margin, for steps that move one token; it only ever drops, so a stale read
-    // can only let a useless atomic through
-    if (m < __ldcg(&mins[e])) atomicMin(&mins[e], m);
-  }
-}
-
-template <bool kFirst>   // the first sweep scans every row (one thread per token) and fills the cache
-__global__ void __launch_bounds__(kSweepThreads)
-flow_sweep_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, int T, int E, int k, int C,
-                  KeyGen g, int sweep_index) {
-  // the token's cache entries do not depend on anything the prologue reads: fetch them first, so that
-  // their latency overlaps the state loads and barriers below
-  uint4 pre_id = make_uint4(0, 0, 0, 0); float pre_x[kCacheN]; long long pre_bound = kInf;
-  {
-    const int tok = blockIdx.x * blockDim.x + threadIdx.x;
-#pragma unroll
-    for (int j = 0; j < kCacheN; ++j) pre_x[j] = 0.f;
-    if (!kFirst && sweep_index > 0 && tok < T) {
-      pre_id = *reinterpret_cast<const uint4*>(cache.id + (size_t)tok * kCacheN);
-#pragma unroll
-      for (int j = 0; j < kCacheN; ++j) pre_x[j] = cache.x[(size_t)j * T + tok];
-      pre_bound = cache.bound[tok];
-    }
-  }
-  if (*(volatile int*)&st->p1_done) return;
-  // histograms alternate between two buffers: this sweep fills one while every CTA clears a slice of
-  // the other for the next sweep (its last reader, the previous price update, has finished)
-  const int sweep0 = sweep_index;                     // sweeps run in launch order; a finished phase returns above
-  const long long cumdrop = st->cumdrop;
-  const int par = sweep0 & 1;
-  unsigned* hup = st->hist_up[par]; unsigned* hdn = st->hist_dn[par];
-  long long* mup = st->min_up; long long* mdn = st->min_dn;
-  {
-    uint4* zu = reinterpret_cast<uint4*>(st->hist_up[par ^ 1]); uint4* zd = reinterpret_cast<uint4*>(st->hist_dn[par ^ 1]);
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < kMaxE * kNB / 4; i += gridDim.x * blockDim.x) {
-      zu[i] = make_uint4(0, 0, 0, 0); zd[i] = make_uint4(0, 0, 0, 0);
-    }
-  }
-  __shared__ SweepShared sh;
-  long long (&sp)[kMaxE] = sh.sp;
-  int (&sload)[kMaxE] = sh.sload; int (&scu)[kMaxE] = sh.scu; int (&scd)[kMaxE] = sh.scd;
-  if (threadIdx.x == 0) { sh.nflag = 0; sh.nslow = 0; }
-  __syncthreads();
-  for (int e = threadIdx.x; e < E; e += blockDim.x) {
-    sp[e] = st->p[e]; sh.spf[e] = (float)sp[e]; sload[e] = 0; scu[e] = st->cap_up[e]; scd[e] = st->cap_dn[e];
-    if (st->flag_dn[e]) sh.sflag[atomicAdd(&sh.nflag, 1)] = e;
-  }
-  __syncthreads();
-  const int tok0 = blockIdx.x * blockDim.x;
-  const int need = min(k + 2, E);                       // sorted values a token has to know
-  const int nflag = sh.nflag;
-  // ---- pass A, one thread per token: re-evaluate the cached experts -----------------------------
-  {
-    const int tok = tok0 + threadIdx.x;
-    if (tok < T) {
-      bool valid = false;
-      if (kFirst) {
-        const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-        const float* row = M + (size_t)tok * E;
-        long long v[kCacheN]; int id[kCacheN];
-        select_top(row, sp, sh.spf, g, flat, E, (E & 3) == 0 ? -1 : 0, false, v, id);
-        unsigned idws[4] = {0, 0, 0, 0};
-#pragma unroll
-        for (int j = 0; j < kCacheN; ++j) {
-          cache.x[(size_t)j * T + tok] = id[j] >= 0 ? __ldg(row + id[j]) : 0.f;
-          idws[j >> 2] |= (unsigned)(id[j] >= 0 ? id[j] : 255) << (8 * (j & 3));
-        }
-        *reinterpret_cast<uint4*>(cache.id + (size_t)tok * kCacheN) = make_uint4(idws[0], idws[1], idws[2], idws[3]);
-        cache.bound[tok] = id[kCacheN - 1] >= 0 ? v[kCacheN - 1] - cumdrop : -kInf;
-        long long vk = -kInf, vk1 = -kInf;
-#pragma unroll
-        for (int j = 0; j < kCacheN; ++j) { if (j == k - 1) vk = v[j]; if (j == k) vk1 = v[j]; }
-#pragma unroll
-        for (int j = 0; j < kMaxK + 2; ++j) {
-          const int e = id[j];
-          if (j < k) {
-            atomicAdd(&sload[e], 1);
-            if (E > k) emit_margin(hup, mup, scu, e, v[j] - vk1);
-          } else if (j <= k + 1 && e >= 0) {
-            emit_margin(hdn, mdn, scd, e, vk - v[j]);
-          }
-        }
-        valid = true;                                   // no expert is flagged before the first sweep
-      } else if (sweep0 > 0) {
-        const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-        const unsigned idws[4] = {pre_id.x, pre_id.y, pre_id.z, pre_id.w};
-        long long v[kCacheN]; int rank[kCacheN];
-#pragma unroll
-        for (int j = 0; j < kCacheN; ++j) {
-          const int e = (int)((idws[j >> 2] >> (8 * (j & 3))) & 255u);
-          const float x = pre_x[j];
-          v[j] = e < E ? make_key(g, x, flat + e) - sp[e] : -kInf;
-          rank[j] = 0;
-        }
-#pragma unroll
-        for (int j = 1; j < kCacheN; ++j)
-#pragma unroll
-          for (int i = 0; i < j; ++i) {
-            const bool first = v[i] >= v[j];            // the earlier entry wins a tie
-            rank[j] += first ? 1 : 0; rank[i] += first ? 0 : 1;
-          }
-        long long vk = -kInf, vk1 = -kInf, vneed = -kInf;
-#pragma unroll
-        for (int j = 0; j < kCacheN; ++j) {
-          if (rank[j] == k - 1) vk = v[j];
-          if (rank[j] == k) vk1 = v[j];
-          if (rank[j] == need - 1) vneed = v[j];
-        }
-        const long long bound = pre_bound;
-        valid = bound <= -kInf || vneed >= bound + cumdrop;
-        if (valid) {
-          const bool has_alt = E > k;
-#pragma unroll
-          for (int j = 0; j < kCacheN; ++j) {
-            const int e = (int)((idws[j >> 2] >> (8 * (j & 3))) & 255u);
-            if (rank[j] < k) {
-              atomicAdd(&sload[e], 1);
-              if (has_alt) emit_margin(hup, mup, scu, e, v[j] - vk1);        // price rise at which the token leaves e
-            } else if (rank[j] <= k + 1 && e < E) {
-              emit_margin(hdn, mdn, scd, e, vk - v[j]);                      // price cut at which the token joins e
-            }
-          }
-          // experts whose join-histogram was short last time: count this token even if the expert is
-          // not among its best alternatives
-          for (int q = 0; q < nflag; ++q) {
-            const int e = sh.sflag[q];
-            bool seen = false;
-#pragma unroll
-            for (int j = 0; j < kCacheN; ++j)
-              seen |= (rank[j] <= k + 1) && ((int)((idws[j >> 2] >> (8 * (j & 3))) & 255u) == e);
-            if (seen) continue;
-            emit_margin(hdn, mdn, scd, e, vk - (make_key(g, __ldg(M + (size_t)tok * E + e), flat + e) - sp[e]));
-          }
-        }
-      }
-      if (!valid) sh.slow[atomicAdd(&sh.nslow, 1)] = (unsigned short)threadIdx.x;
-    }
-  }
-  __syncthreads();
-  if (threadIdx.x == 0 && sweep0 < 64 && sh.nslow) atomicAdd(&st->trace[64 + sweep0], sh.nslow);
-  // ---- pass B, one warp per token whose cache no longer vouches for itself: scan the whole row ----
-  {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int nslow = sh.nslow;
-    for (int s = warp; s < nslow; s += kSweepThreads / 32) {
-      const int tok = tok0 + sh.slow[s];
-      const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-      const float* row = M + (size_t)tok * E;
-      // lane l looks at experts l, l+32, l+64, l+96.  fp32 approximations, the expert index in the low
-      // 7 mantissa bits, mapped to unsigned integers that order the same way; 0 = absent
-      unsigned u[kEPLf];
-#pragma unroll
-      for (int q = 0; q < kEPLf; ++q) {
-        const int e = lane + 32 * q;
-        u[q] = 0;
-        if (e < E) {
-          const float vf = approx_key(g, __ldg(row + e)) - sh.spf[e];
-          const unsigned bits = (__float_as_uint(vf) & ~127u) | (unsigned)e;
-          u[q] = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
-        }
-      }
-      unsigned mine = 0;
-      for (int r = 0; r < kCacheN; ++r) {
-        unsigned m = u[0];
-#pragma unroll
-        for (int q = 1; q < kEPLf; ++q) m = max(m, u[q]);
-        const unsigned w = __reduce_max_sync(0xffffffffu, m);
-        if (lane == r) mine = w;
-#pragma unroll
-        for (int q = 0; q < kEPLf; ++q) u[q] = (u[q] == w) ? 0u : u[q];
-      }
-      // lanes 0..kCacheN-1 now hold the winners in descending approximate order; make them exact
-      int ee = 255; float xv = 0.f; long long val = -kInf;
-      if (lane < kCacheN && mine != 0) {
-        const unsigned bits = (mine & 0x80000000u) ? (mine & 0x7fffffffu) : ~mine;
-        ee = (int)(bits & 127u);
-        xv = __ldg(row + ee);
-        val = make_key(g, xv, flat + ee) - sp[ee];
-      }
-      if (lane < kCacheN) {
-        cache.x[(size_t)lane * T + tok] = xv;
-        cache.id[(size_t)tok * kCacheN + lane] = (unsigned char)ee;
-      }
-      // every expert outside the cache is worth no more than the last winner (none if E <= kCacheN)
-      const long long vlast = __shfl_sync(0xffffffffu, val, kCacheN - 1);
-      if (lane == 0) cache.bound[tok] = (vlast <= -kInf) ? -kInf : vlast - cumdrop;
-      int rank = 0;
-#pragma unroll
-      for (int i = 0; i < kCacheN; ++i) {
-        const long long vi = __shfl_sync(0xffffffffu, val, i);
-        rank += (vi > val || (vi == val && i < lane)) ? 1 : 0;
-      }
-      const bool listed = lane < kCacheN && ee < E;
-      const unsigned bk = __ballot_sync(0xffffffffu, listed && rank == k - 1);
-      const unsigned bk1 = __ballot_sync(0xffffffffu, listed && rank == k);
-      const long long vk = __shfl_sync(0xffffffffu, val, bk ? __ffs(bk) - 1 : 0);
-      const long long vk1 = bk1 ? __shfl_sync(0xffffffffu, val, __ffs(bk1) - 1) : -kInf;
-      if (listed) {
-        if (rank < k) {
-          atomicAdd(&sload[ee], 1);
-          if (E > k) emit_margin(hup, mup, scu, ee, val - vk1);
-        } else if (rank <= k + 1) {
-          emit_margin(hdn, mdn, scd, ee, vk - val);
-        }
-      }
-      for (int q = 0; q < nflag; ++q) {
-        const int e = sh.sflag[q];
-        const unsigned seen = __ballot_sync(0xffffffffu, listed && rank <= k + 1 && ee == e);
-        if (!seen && lane == 0) emit_margin(hdn, mdn, scd, e, vk - (make_key(g, __ldg(row + e), flat + e) - sp[e]));
-      }
-    }
-  }
-  __syncthreads();
-  for (int e = threadIdx.x; e < E; e += blockDim.x)
-    if (sload[e]) atomicAdd(&st->load[e], sload[e]);
-
-}
-
-// Price update that closes a sweep: one CTA, one warp per expert (four experts per warp, all their
-// histograms in flight at once).
-constexpr int kPriceThreads = 1024;
-__global__ void __launch_bounds__(kPriceThreads)
-flow_price_kernel(FlowState* st, int E, int C, int n_sweeps, int decay_every, int sweep_index) {
-  // every input is loaded up front, independently of the others, so that the kernel pays two global
-  // round trips (state, then the histogram rows picked by the sign of the imbalance), not one per field
-  __shared__ long long sp[kMaxE];
-  __shared__ int s_imb;
-  __shared__ long long pmin, s_drop;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  constexpr int kWarps = kPriceThreads / 32, kBatch = kMaxE / kWarps;
-  const int par = sweep_index & 1;                    // the sweep this update closes filled these buffers
-  const unsigned* hup = st->hist_up[par]; const unsigned* hdn = st->hist_dn[par];
-  const int done_before = __ldcg(&st->p1_done);
-  const long long eps = __ldcg(&st->eps), eps_min = __ldcg(&st->eps_min);
-  const bool balanced = __ldcg(&st->balanced) != 0;
-  const int cut_max = __ldcg(&st->cut_max), best_imb = __ldcg(&st->best_imb), stall_before = __ldcg(&st->stall);
-  int xs[kBatch], cup[kBatch], cdn[kBatch]; long long ps[kBatch], mu[kBatch], md[kBatch];
-#pragma unroll
-  for (int b = 0; b < kBatch; ++b) {
-    const int e = warp + b * kWarps;
-    xs[b] = 0; ps[b] = 0; mu[b] = kInf; md[b] = kInf; cup[b] = 0; cdn[b] = 0;
-    if (e < E) {
-      xs[b] = __ldcg(&st->load[e]) - C; ps[b] = __ldcg(&st->p[e]);
-      cup[b] = __ldcg(&st->cap_up[e]); cdn[b] = __ldcg(&st->cap_dn[e]);
-      mu[b] = __ldcg(&st->min_up[e]); md[b] = __ldcg(&st->min_dn[e]);
-    }
-  }
-  if (done_before) return;
-  if (threadIdx.x == 0) { s_imb = 0; s_drop = 0; }
-  uint4 ha[kBatch], hb[kBatch]; long long m1[kBatch];
-#pragma unroll
-  for (int b = 0; b < kBatch; ++b) {
-    const int e = warp + b * kWarps;
-    m1[b] = kInf; ha[b] = make_uint4(0, 0, 0, 0); hb[b] = ha[b];
-    if (e < E) {
-      const int x = xs[b];
-      const bool up = x > 0, dn = x < 0 && (balanced || ps[b] > 0);
-      if (up || dn) {
-        const uint4* h = reinterpret_cast<const uint4*>((up ? hup : hdn) + e * kNB) + 2 * lane;
-        ha[b] = __ldcg(h); hb[b] = __ldcg(h + 1);
-        m1[b] = up ? mu[b] : md[b];
-      }
-    }
-  }
-  __syncthreads();
-  int imb = 0; long long drop = 0;
-#pragma unroll
-  for (int b = 0; b < kBatch; ++b) {
-    const int e = warp + b * kWarps;
-    if (e >= E) continue;
-    const int x = xs[b];
-    long long p = ps[b];
-    int flag = 0;
-    if (x > 0) {
-      int cl = cup[b]; bool shortw;
-      p += price_step_warp(ha[b], hb[b], x, eps, cl, shortw, cut_max, m1[b]);
-      if (lane == 0) st->cap_up[e] = cl;
-      imb += x;
-    } else if (x < 0 && (balanced || p > 0)) {
-      int cl = cdn[b]; bool shortw;
-      p -= price_step_warp(ha[b], hb[b], -x, eps, cl, shortw, cut_max, m1[b]);
-      if (!balanced && p < 0) p = 0;
-      if (lane == 0) st->cap_dn[e] = cl;
-      flag = shortw ? 1 : 0;
-      imb += -x;
-    }
-    p = p > kPriceLimit ? kPriceLimit : (p < -kPriceLimit ? -kPriceLimit : p);
-    // when nothing was out of balance the prices stay put and the collect pass reproduces this state
-    if (x == 0) p = ps[b];
-    if (lane == 0) {
-      st->flag_dn[e] = flag;
-      st->load[e] = 0;
-      st->min_up[e] = kInf; st->min_dn[e] = kInf;
-      if (ps[b] - p > drop) drop = ps[b] - p;
-      sp[e] = p;
-    }
-  }
-  if (lane == 0) { if (imb) atomicAdd(&s_imb, imb); if (drop > 0) atomicMax(&s_drop, drop); }
-  __syncthreads();
-  const int sweep = sweep_index + 1;
-  // a small imbalance that has stopped shrinking is a price war between a few experts: the exact phase
-  // ends it faster than more sweeps would
-  const int stall = s_imb < best_imb ? 0 : stall_before + 1;
-  const bool done = (s_imb == 0) || sweep >= n_sweeps || (stall >= kStallSweeps && s_imb <= kStallImbalance);
-  if (threadIdx.x == 0) {
-    // prices are only defined up to a shift when every expert must be full; anchor the minimum at 0
-    long long m = 0;
-    if (done && balanced) { m = sp[0]; for (int e = 1; e < E; ++e) m = sp[e] < m ? sp[e] : m; }
-    pmin = m;
-  }
-  __syncthreads();
-  for (int e = threadIdx.x; e < E; e += blockDim.x) st->p[e] = sp[e] - pmin;
-  if (threadIdx.x == 0) {
-    if (sweep <= 40) st->trace[sweep - 1] = s_imb;
-    st->sweep = sweep;
-    st->stall = stall; if (stall == 0) st->best_imb = s_imb;
-    st->cumdrop += s_drop;
-    if (sweep % decay_every == 0) { long long ne = eps >> 1; st->eps = ne < eps_min ? eps_min : ne; }
-    if (done) st->p1_done = 1;
-  }
-}
-
 // fp32 <-> unsigned integers that order the same way (for the integer warp reductions)
 __device__ __forceinline__ unsigned flip_f32(float f) {
   const unsigned b = __float_as_uint(f);
@@ -656,35 +222,6 @@ __device__ __forceinline__ unsigned flip_f32(float f) {
 }
 __device__ __forceinline__ float unflip_f32(unsigned u) {
   return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
-}
-
-// Approximate selection over one row held by a warp: the `count` largest fp32 values, one warp reduction
-// each (the expert index rides in the low 7 mantissa bits, so values are distinct and the winner's
-// owner is known).  sel[] marks the first `nsel`; v_a / v_b are the values picked as number nsel and
-// nsel+1 (-inf where there is none).  The caller decides whether v_a - v_b is large enough to trust.
-__device__ __forceinline__ void warp_select_f32(const float (&val)[kEPLf], int E, int count, bool (&sel)[kEPLf],
-                                                float& v_a, float& v_b, int nsel) {
-  const int lane = threadIdx.x & 31;
-  unsigned u[kEPLf];
-#pragma unroll
-  for (int q = 0; q < kEPLf; ++q) {
-    const int e = lane + 32 * q;
-    u[q] = e < E ? flip_f32(__uint_as_float((__float_as_uint(val[q]) & ~127u) | (unsigned)e)) : 0u;
-    sel[q] = false;
-  }
-  v_a = -INFINITY; v_b = -INFINITY;
-  for (int r = 0; r < count && r < E; ++r) {
-    unsigned m = u[0];
-#pragma unroll
-    for (int q = 1; q < kEPLf; ++q) m = max(m, u[q]);
-    const unsigned w = __reduce_max_sync(0xffffffffu, m);
-    const float v = unflip_f32(w);
-    if (r == nsel - 1) v_a = v;
-    if (r == nsel) v_b = v;
-#pragma unroll
-    for (int q = 0; q < kEPLf; ++q)
-      if (u[q] == w) { u[q] = 0u; if (r < nsel) sel[q] = true; }
-  }
 }
 
 // Exact selection over one row held by a warp (lane l: entries l, l+32, ...).  Picks the `count`
@@ -726,112 +263,600 @@ __device__ __forceinline__ void warp_select(const long long (&val)[kEPLf], int E
 }
 
 // ---------------------------------------------------------------------------------------------
-// Collect / verify pass.  The first pass picks every token's top-k under the sweep prices.  Later ones
-// keep a token's experts when they still are a top-k under the current prices (ties included) and
-// re-pick otherwise.  verify_only never re-picks: it only counts violations and gathers statistics.
-__global__ void __launch_bounds__(kSweepThreads)
-flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restrict__ expert_idx,
-                    int32_t* __restrict__ cand, int T, int E, int k, int C, KeyGen g, int first,
-                    int verify_only, long long theta_scale, int32_t* __restrict__ expert_load_out,
-                    void* stats_out, const unsigned* __restrict__ error_flag, int unbounded, long long* __restrict__ Dg) {
-  if (!verify_only && *(volatile int*)&st->converged) return;
-  if (Dg)   // the move-cost matrix the build kernel fills next starts out empty
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < E * (E | 1); i += gridDim.x * blockDim.x) Dg[i] = kInf;
+// Per-token candidate cache.  A full scan of a token's row keeps its kCacheN best experts (score and
+// index) and `bound` = an upper bound on key - price of every other expert at scan time, minus the
+// total price drop up to then.  Later, every uncached expert is worth at most bound + (total price
+// drop now), so while the (k+2)-th cached value stays at or above that, the cached entries still
+// contain the token's k+2 best experts and the row need not be read again.
+constexpr int kCacheN = 16;
+struct SweepCache {
+  float* x;              // [kCacheN][T] scores of the cached experts
+  unsigned char* id;     // [T][kCacheN] their indices (255 = none)
+  long long* bound;      // [T]
+  unsigned char* raw;    // [T] 1 = scanned at zero prices: the cache also holds the token's best raw keys
+};
+
+// One warp rebuilds the cache of one token from its row under the prices sp (spf = the same as floats).
+// Lane l looks at experts l, l+32, l+64, l+96: fp32 approximations of key - price, the expert index in
+// the low 7 mantissa bits, mapped to unsigned integers that order the same way (0 = absent); kCacheN
+// rounds of one warp reduction each pick the winners.  |approximation - exact| <= hash_bound +
+// 2^-15 (|key| + |price|) (float conversion of the price, one rounding of the difference, the 7 index
+// bits), which turns the last winner's approximate value into a rigorous bound on every loser.
+__device__ __forceinline__ void rescan_row(const float* __restrict__ row, uint32_t flat, int tok, int T, int E,
+                                           const KeyGen& g, const long long* sp, const float* spf, long long cumdrop,
+                                           bool raw, const SweepCache& cache, bool& bad) {
+  const int lane = threadIdx.x & 31;
+  unsigned u[kEPLf]; float mag = 0.f;
+#pragma unroll
+  for (int q = 0; q < kEPLf; ++q) {
+    const int e = lane + 32 * q;
+    u[q] = 0;
+    if (e < E) {
+      const float x = __ldg(row + e);
+      bad |= !isfinite(x);
+      const float kf = approx_key(g, x), pf = spf[e];
+      const float vf = kf - pf;
+      mag = fmaxf(mag, fabsf(kf) + fabsf(pf));
+      const unsigned bits = (__float_as_uint(vf) & ~127u) | (unsigned)e;
+      u[q] = (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+    }
+  }
+  unsigned mine = 0;
+  for (int r = 0; r < kCacheN; ++r) {
+    unsigned m = u[0];
+#pragma unroll
+    for (int q = 1; q < kEPLf; ++q) m = max(m, u[q]);
+    const unsigned w = __reduce_max_sync(0xffffffffu, m);
+    if (lane == r) mine = w;
+#pragma unroll
+    for (int q = 0; q < kEPLf; ++q) u[q] = (u[q] == w) ? 0u : u[q];
+  }
+  // lanes 0..kCacheN-1 now hold the winners in descending approximate order
+  int ee = 255; float xv = 0.f;
+  if (lane < kCacheN && mine != 0) {
+    const unsigned bits = (mine & 0x80000000u) ? (mine & 0x7fffffffu) : ~mine;
+    ee = (int)(bits & 127u);
+    xv = __ldg(row + ee);
+  }
+  if (lane < kCacheN) {
+    cache.x[(size_t)lane * T + tok] = xv;
+    cache.id[(size_t)tok * kCacheN + lane] = (unsigned char)ee;
+  }
+  mag = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mag)));
+  const unsigned wlast = __shfl_sync(0xffffffffu, mine, kCacheN - 1);
+  if (lane == 0) {
+    long long b = -kInf;                                // fewer than kCacheN experts: nothing is left out
+    if (wlast != 0) {
+      const float a = __uint_as_float((wlast & 0x80000000u) ? (wlast & 0x7fffffffu) : ~wlast);
+      const double ub = (double)a + (double)(g.mode == 0 ? 4097.f : 1048577.f) + (double)mag * (1.0 / 32768.0) + 1.0;
+      b = ub >= 4.0e18 ? kInf : (ub <= -4.0e18 ? -kInf : (long long)ceil(ub));
+      if (b < kInf && b > -kInf) b -= cumdrop;
+    }
+    cache.bound[tok] = b;
+    cache.raw[tok] = raw ? 1 : 0;
+  }
+}
+
+// First pass over the score matrix: the cache of every token at zero prices, one warp per token.
+__global__ void __launch_bounds__(256)
+flow_scan_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, int T, int E, KeyGen g) {
   __shared__ long long sp[kMaxE];
   __shared__ float spf[kMaxE];
-  __shared__ int sload[kMaxE];
-  __shared__ int s_viol, s_rer;
-  __shared__ double s_score;
-  __shared__ unsigned s_flags;
-  for (int e = threadIdx.x; e < E; e += blockDim.x) { sp[e] = st->p[e]; spf[e] = (float)sp[e]; sload[e] = 0; }
-  if (threadIdx.x == 0) { s_viol = 0; s_rer = 0; s_score = 0.0; s_flags = 0; }
+  for (int e = threadIdx.x; e < kMaxE; e += blockDim.x) { sp[e] = 0; spf[e] = 0.f; }
   __syncthreads();
-  const long long theta = unbounded ? kInf : st->theta;   // the last round lists every token
-  // One warp per token, lane l holds experts l, l+32, l+64, l+96: coalesced row loads, every decision
-  // by warp votes and reductions.  Decisions are first tried on fp32 approximations of key - price with
-  // a rigorous error bound; only a token whose decision the bound cannot settle (a near-tie) is redone
-  // on the exact int64 values.  A token may be listed as a candidate on the approximate gap: the list
-  // only has to be a superset.
-  const int lane = threadIdx.x & 31;
   const int wid = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), nwarp = gridDim.x * (blockDim.x >> 5);
-  const float hash_bound = g.mode == 0 ? 4096.f : 1048576.f;      // key - approx_key lies in [-0.5, this)
-  const float thetaf = theta >= kInf ? INFINITY : (float)theta * 1.0000005f;
-  int w_viol = 0, w_rer = 0; double w_score = 0.0; bool w_bad = false;
-  // the next token's row and experts are fetched while the current token is worked on
-  float nx[kEPLf]; int nmine = -1;
-  auto fetch = [&](int t) {
-    if (t >= T) return;
-    const float* r = M + (size_t)t * E;
+  bool bad = false;
+  for (int tok = wid; tok < T; tok += nwarp)
+    rescan_row(M + (size_t)tok * E, (uint32_t)tok * (uint32_t)E, tok, T, E, g, sp, spf, 0, true, cache, bad);
+  if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicOr(&st->status, 2u);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Grid-wide barrier of the cooperative sweeps kernel: a monotone arrival counter in global memory.
+// Every wait is bounded: a CTA that gives up raises the abort flag, which releases all the others,
+// and the kernel then returns with the internal-error status set.
+constexpr unsigned kBarrierSpinLimit = 1u << 22;
+__device__ __forceinline__ bool grid_barrier(FlowState* st, unsigned& epoch) {
+  __syncthreads();
+  __shared__ int s_bar_ok;
+  if (threadIdx.x == 0) {
+    epoch += gridDim.x;
+    __threadfence();
+    atomicAdd(&st->bar_count, 1u);
+    bool ok = true;
+    for (unsigned spins = 0;; ++spins) {
+      unsigned c;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(c) : "l"(&st->bar_count) : "memory");
+      if ((int)(c - epoch) >= 0) break;
+      if (spins > kBarrierSpinLimit || *(volatile unsigned*)&st->bar_abort) {
+        atomicExch(&st->bar_abort, 1u); atomicOr(&st->status, 4u); ok = false; break;
+      }
+      if (spins > 64) __nanosleep(20);
+    }
+    s_bar_ok = ok ? 1 : 0;
+  }
+  __syncthreads();
+  return s_bar_ok != 0;
+}
+
+// Bin of a non-negative margin held as a float: the same bins as log_bin (exponent and two mantissa bits).
+__device__ __forceinline__ int float_bin(float m) {
+  if (m < 4.f) return (int)m;
+  const unsigned b = __float_as_uint(m);
+  return 4 * ((int)(b >> 23) - 128) + (int)((b >> 21) & 3u);
+}
+
+// A margin goes into the expert's global histogram (fire-and-forget) and, for the steps that move one token
+// exactly, into the CTA's running minimum in shared memory (merged into global memory after the pass;
+// non-negative floats order like their bit patterns).
+__device__ __forceinline__ void emit_margin(unsigned* hist, unsigned* smin, const float* capf, int e, float m) {
+  if (m >= 0.f && m < capf[e]) {
+    atomicAdd(&hist[e * kNB + float_bin(m)], 1u);
+    const unsigned mb = __float_as_uint(m);
+    if (mb < smin[e]) atomicMin(&smin[e], mb);
+  }
+}
+
+// The experts of a 128-bit mask in ascending order, as a token's row of expert_idx.
+__device__ __forceinline__ void write_sorted_experts(int32_t* __restrict__ out, const unsigned (&hm)[4], int k) {
+  int n = 0;
 #pragma unroll
-    for (int q = 0; q < kEPLf; ++q) { const int e = lane + 32 * q; nx[q] = e < E ? __ldg(r + e) : 0.f; }
-    nmine = (!first && lane < k) ? expert_idx[(size_t)t * k + lane] : -1;
+  for (int w = 0; w < 4; ++w) {
+    unsigned m = hm[w];
+    while (m && n < k) { const int b = __ffs(m) - 1; m &= m - 1; out[n++] = 32 * w + b; }
+  }
+}
+
+constexpr int kSwThreads = 512;
+
+struct SweepShared {
+  long long sp[kMaxE];
+  float spf[kMaxE];
+  unsigned smin_up[kMaxE], smin_dn[kMaxE];   // smallest margins of the pass, as float bit patterns
+  float capu[kMaxE], capd[kMaxE];            // margins at or above these are not recorded
+  int sload[kMaxE], sflag[kMaxE];
+  int nflag, nslow, s_imb;
+  long long s_drop, s_pmin;
+  int slow[kSwThreads];
+};
+
+struct SweepArgs {
+  int T, E, k, C, n_sweeps, balanced;
+  long long eps0, eps_min, theta0;
+};
+
+struct TokCache {          // one token's cache entries in registers
+  unsigned idws[4]; float x[kCacheN]; long long bound;
+};
+__device__ __forceinline__ void load_tok_cache(TokCache& c, const SweepCache& cache, int tok, int T) {
+  const uint4 idv = __ldcg(reinterpret_cast<const uint4*>(cache.id + (size_t)tok * kCacheN));
+  c.idws[0] = idv.x; c.idws[1] = idv.y; c.idws[2] = idv.z; c.idws[3] = idv.w;
+#pragma unroll
+  for (int j = 0; j < kCacheN; ++j) c.x[j] = __ldcg(cache.x + (size_t)j * T + tok);
+  c.bound = __ldcg(cache.bound + tok);
+}
+
+// One token of a sweep, from its cache, in fp32: the sweeps only steer the prices, so approximate values
+// do (what they leave undone the exact phase repairs, and the first pick and the check pass are exact).
+// Returns false when the cache cannot vouch for the token's k+2 best experts any more (the caller then has
+// the row rescanned and calls again).
+__device__ __forceinline__ bool sweep_token(int tok, const TokCache& c, SweepShared& sh, const SweepArgs& a,
+                                            const KeyGen& g, float cumdropf, unsigned* hup, unsigned* hdn) {
+  const int E = a.E, k = a.k;
+  const int need = min(k + 2, E);                       // sorted values a token has to know
+  float v[kCacheN]; int rank[kCacheN];
+#pragma unroll
+  for (int j = 0; j < kCacheN; ++j) {
+    const int e = (int)((c.idws[j >> 2] >> (8 * (j & 3))) & 255u);
+    v[j] = e < E ? approx_key(g, c.x[j]) - sh.spf[e] : -INFINITY;
+    rank[j] = 0;
+  }
+#pragma unroll
+  for (int j = 1; j < kCacheN; ++j)
+#pragma unroll
+    for (int i = 0; i < j; ++i) {
+      const bool first = v[i] >= v[j];                  // the earlier entry wins a tie
+      rank[j] += first ? 1 : 0; rank[i] += first ? 0 : 1;
+    }
+  float vk = -INFINITY, vk1 = -INFINITY, vneed = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < kCacheN; ++j) {
+    if (rank[j] == k - 1) vk = v[j];
+    if (rank[j] == k) vk1 = v[j];
+    if (rank[j] == need - 1) vneed = v[j];
+  }
+  if (!(c.bound <= -kInf || vneed >= (float)c.bound + cumdropf)) return false;
+  const bool has_alt = E > k;
+  const int nflag = sh.nflag;
+#pragma unroll
+  for (int j = 0; j < kCacheN; ++j) {
+    const int e = (int)((c.idws[j >> 2] >> (8 * (j & 3))) & 255u);
+    if (rank[j] < k) {
+      atomicAdd(&sh.sload[e], 1);
+      if (has_alt) emit_margin(hup, sh.smin_up, sh.capu, e, v[j] - vk1);        // price rise at which the token leaves e
+    } else if (e < E) {
+      bool rec = rank[j] <= k + 1;                                             // price cut at which the token joins e
+      // experts whose join-histogram was short last time: count this token even if the expert is not among
+      // its best alternatives
+      for (int q = 0; q < nflag; ++q) rec |= sh.sflag[q] == e;
+      if (rec) emit_margin(hdn, sh.smin_dn, sh.capd, e, vk - v[j]);
+    }
+  }
+  return true;
+}
+
+// One token of the first pick, from its cache, exact: the token's k best experts under the final prices go
+// to expert_idx in ascending order, and the token is listed as a candidate when its k-th and (k+1)-th values
+// are within theta.  Returns false when the cache cannot vouch for the token's k+1 best experts.
+__device__ __forceinline__ bool pick_token(int tok, const TokCache& c, FlowState* st, SweepShared& sh, const SweepArgs& a,
+                                           const KeyGen& g, long long cumdrop, int32_t* __restrict__ expert_idx,
+                                           int32_t* __restrict__ cand) {
+  const int E = a.E, k = a.k;
+  const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+  const int need = min(k + 1, E);
+  long long v[kCacheN]; int rank[kCacheN];
+#pragma unroll
+  for (int j = 0; j < kCacheN; ++j) {
+    const int e = (int)((c.idws[j >> 2] >> (8 * (j & 3))) & 255u);
+    v[j] = e < E ? make_key(g, c.x[j], flat + e) - sh.sp[e] : -kInf;
+    rank[j] = 0;
+  }
+#pragma unroll
+  for (int j = 1; j < kCacheN; ++j)
+#pragma unroll
+    for (int i = 0; i < j; ++i) {
+      const bool first = v[i] >= v[j];                  // the earlier entry wins a tie
+      rank[j] += first ? 1 : 0; rank[i] += first ? 0 : 1;
+    }
+  long long vk = -kInf, vk1 = -kInf, vneed = -kInf;
+#pragma unroll
+  for (int j = 0; j < kCacheN; ++j) {
+    if (rank[j] == k - 1) vk = v[j];
+    if (rank[j] == k) vk1 = v[j];
+    if (rank[j] == need - 1) vneed = v[j];
+  }
+  if (!(c.bound <= -kInf || vneed >= c.bound + cumdrop)) return false;
+  unsigned hm[4] = {0, 0, 0, 0};
+#pragma unroll
+  for (int j = 0; j < kCacheN; ++j) {
+    const int e = (int)((c.idws[j >> 2] >> (8 * (j & 3))) & 255u);
+    if (rank[j] < k && e < E) { hm[e >> 5] |= 1u << (e & 31); atomicAdd(&sh.sload[e], 1); }
+  }
+  write_sorted_experts(expert_idx + (size_t)tok * k, hm, k);
+  if (E > k && vk - vk1 <= a.theta0) cand[atomicAdd(&st->ncand, 1)] = tok;     // the list has room for every token
+  return true;
+}
+
+// All price sweeps and the first pick in one cooperative launch (every CTA resident, one thread per token
+// and pass; the price step of expert e is taken by one warp of CTA e mod grid).  When the grid has a
+// thread for every token, a token's cache entries stay in its thread's registers from sweep to sweep.
+__global__ void __launch_bounds__(kSwThreads, 1)
+flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, int32_t* __restrict__ expert_idx,
+                   int32_t* __restrict__ cand, SweepArgs a, KeyGen g) {
+  __shared__ SweepShared sh;
+  const int T = a.T, E = a.E, C = a.C;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gtid = blockIdx.x * blockDim.x + tid, gsize = gridDim.x * blockDim.x;
+  const bool resident = T <= gsize;
+  unsigned epoch = 0;
+  long long cumdrop = 0, eps = a.eps0;
+  int best_imb = 0x7fffffff, stall = 0, sweep = 0;
+  bool done = a.n_sweeps <= 0;
+  TokCache mine;
+  if (resident && gtid < T) load_tok_cache(mine, cache, gtid, T);
+
+  // a pass over this CTA's tokens: one thread per token from the caches, then one warp per token whose
+  // cache had to be rebuilt
+  auto token_pass = [&](auto pick_tag, unsigned* hup, unsigned* hdn) {
+    constexpr bool kPick = decltype(pick_tag)::value;
+    for (int base = blockIdx.x * blockDim.x; base < T; base += gsize) {
+      if (tid == 0) sh.nslow = 0;
+      __syncthreads();
+      const int tok = base + tid;
+      bool was_slow = false;
+      if (tok < T) {
+        if (!resident) load_tok_cache(mine, cache, tok, T);
+        const bool ok = kPick ? pick_token(tok, mine, st, sh, a, g, cumdrop, expert_idx, cand)
+                              : sweep_token(tok, mine, sh, a, g, (float)cumdrop, hup, hdn);
+        if (!ok) { sh.slow[atomicAdd(&sh.nslow, 1)] = tok; was_slow = true; }
+      }
+      __syncthreads();
+      const int nslow = sh.nslow;
+      if (nslow) {
+        for (int s = warp; s < nslow; s += kSwThreads / 32) {
+          const int t2 = sh.slow[s];
+          bool bad = false;
+          rescan_row(M + (size_t)t2 * E, (uint32_t)t2 * (uint32_t)E, t2, T, E, g, sh.sp, sh.spf, cumdrop, false, cache, bad);
+          __syncwarp();
+          if (lane == 0) {
+            TokCache fresh;
+            load_tok_cache(fresh, cache, t2, T);
+            if (kPick) pick_token(t2, fresh, st, sh, a, g, cumdrop, expert_idx, cand);
+            else sweep_token(t2, fresh, sh, a, g, (float)cumdrop, hup, hdn);
+          }
+        }
+        __syncthreads();
+        if (resident && was_slow) load_tok_cache(mine, cache, tok, T);
+      }
+    }
   };
-  fetch(wid);
-  for (int tok = wid; tok < T; tok += nwarp) {
-    const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-    float x[kEPLf], kf[kEPLf], vf[kEPLf]; bool in[kEPLf];
-    const int mine = nmine;
-#pragma unroll
-    for (int q = 0; q < kEPLf; ++q) x[q] = nx[q];
-    fetch(tok + nwarp);
-    float mag = 0.f;
-#pragma unroll
-    for (int q = 0; q < kEPLf; ++q) {
-      const int e = lane + 32 * q;
-      w_bad |= !isfinite(x[q]);
-      kf[q] = e < E ? approx_key(g, x[q]) : -INFINITY;
-      const float pf = e < E ? spf[e] : 0.f;
-      vf[q] = kf[q] - pf;
-      if (e < E) mag = fmaxf(mag, fabsf(kf[q]) + fabsf(pf));
-      in[q] = false;
+  // prices, caps and flags for the next pass; on the way, what the last price step left behind
+  auto load_state = [&]() {
+    if (tid == 0) { sh.nflag = 0; sh.s_imb = 0; sh.s_drop = 0; }
+    __syncthreads();
+    for (int e = tid; e < E; e += blockDim.x) {
+      const long long pe = __ldcg(&st->p[e]);
+      const int cu = __ldcg(&st->cap_up[e]), cd = __ldcg(&st->cap_dn[e]), fl = __ldcg(&st->flag_dn[e]);
+      const int im = __ldcg(&st->imb_e[e]); const long long dr = __ldcg(&st->drop_e[e]);
+      sh.sp[e] = pe; sh.spf[e] = (float)pe; sh.sload[e] = 0; sh.capu[e] = ldexpf(1.f, cu); sh.capd[e] = ldexpf(1.f, cd);
+      sh.smin_up[e] = 0x7f800000u; sh.smin_dn[e] = 0x7f800000u;
+      if (fl) sh.sflag[atomicAdd(&sh.nflag, 1)] = e;
+      if (im) atomicAdd(&sh.s_imb, im);
+      if (dr > 0) atomicMax(&sh.s_drop, dr);
     }
-    // |approximation - exact| <= hash_bound + 2^-15 * (|key| + |price|): float conversion of the price,
-    // one rounding of the difference, and the 7 mantissa bits that carry the expert index in selections
-    mag = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mag)));
-    const float err3 = 3.f * (hash_bound + mag * (1.f / 32768.f));
-    if (!first)
+    __syncthreads();
+  };
+
+  load_state();
+  while (!done) {
+    const int par = sweep & 1;
+    unsigned* hup = st->hist_up[par]; unsigned* hdn = st->hist_dn[par];
+    {   // every CTA clears a slice of the other pair of histograms for the next sweep (its last reader,
+        // the previous price step, finished before the barrier that let this sweep start)
+      uint4* zu = reinterpret_cast<uint4*>(st->hist_up[par ^ 1]); uint4* zd = reinterpret_cast<uint4*>(st->hist_dn[par ^ 1]);
+      for (int i = gtid; i < kMaxE * kNB / 4; i += gsize) { zu[i] = make_uint4(0, 0, 0, 0); zd[i] = make_uint4(0, 0, 0, 0); }
+    }
+    token_pass(std::false_type{}, hup, hdn);
+    for (int e = tid; e < E; e += blockDim.x) {
+      if (sh.sload[e]) atomicAdd(&st->load[e], sh.sload[e]);
+      if (sh.smin_up[e] < 0x7f800000u) atomicMin(&st->min_up[e], (long long)__uint_as_float(sh.smin_up[e]));
+      if (sh.smin_dn[e] < 0x7f800000u) atomicMin(&st->min_dn[e], (long long)__uint_as_float(sh.smin_dn[e]));
+    }
+    if (!grid_barrier(st, epoch)) return;
+
+    // ---- price step: one warp per expert, every input fetched in one round trip -------------------------
+    for (int e = blockIdx.x + warp * gridDim.x; e < E; e += gridDim.x * (kSwThreads / 32)) {
+      const int xs = __ldcg(&st->load[e]) - C;
+      const long long ps = __ldcg(&st->p[e]);
+      const int cup = __ldcg(&st->cap_up[e]), cdn = __ldcg(&st->cap_dn[e]);
+      const long long mu = __ldcg(&st->min_up[e]), md = __ldcg(&st->min_dn[e]);
+      const uint4* hu = reinterpret_cast<const uint4*>(hup + e * kNB) + 2 * lane;
+      const uint4* hd = reinterpret_cast<const uint4*>(hdn + e * kNB) + 2 * lane;
+      const uint4 hau = __ldcg(hu), hbu = __ldcg(hu + 1), had = __ldcg(hd), hbd = __ldcg(hd + 1);
+      const bool up = xs > 0, dn = xs < 0 && (a.balanced || ps > 0);
+      long long p = ps; int flag = 0, imb = 0;
+      if (up) {
+        int cl = cup; bool shortw;
+        p += price_step_warp(hau, hbu, xs, eps, cl, shortw, kCapLogMax, mu);
+        if (lane == 0) st->cap_up[e] = cl;
+        imb = xs;
+      } else if (dn) {
+        int cl = cdn; bool shortw;
+        p -= price_step_warp(had, hbd, -xs, eps, cl, shortw, kCapLogMax, md);
+        if (!a.balanced && p < 0) p = 0;
+        if (lane == 0) st->cap_dn[e] = cl;
+        flag = shortw ? 1 : 0;
+        imb = -xs;
+      }
+      p = p > kPriceLimit ? kPriceLimit : (p < -kPriceLimit ? -kPriceLimit : p);
+      // when nothing was out of balance the prices stay put and the pick reproduces this state
+      if (xs == 0) p = ps;
+      if (lane == 0) {
+        st->flag_dn[e] = flag; st->load[e] = 0; st->min_up[e] = kInf; st->min_dn[e] = kInf;
+        st->imb_e[e] = imb; st->drop_e[e] = ps - p > 0 ? ps - p : 0;
+        st->p[e] = p;
+      }
+    }
+    if (!grid_barrier(st, epoch)) return;
+
+    // ---- every CTA draws the same conclusions from the same numbers ----------------------------------
+    load_state();
+    ++sweep;
+    // a small imbalance that has stopped shrinking is a price war between a few experts: the exact phase
+    // ends it faster than more sweeps would
+    stall = sh.s_imb < best_imb ? 0 : stall + 1;
+    if (stall == 0) best_imb = sh.s_imb;
+    done = (sh.s_imb == 0) || sweep >= a.n_sweeps || (stall >= kStallSweeps && sh.s_imb <= kStallImbalance);
+    cumdrop += sh.s_drop;
+    { const long long ne = eps >> 1; eps = ne < a.eps_min ? a.eps_min : ne; }
+  }
+
+  // ---- first pick: every token's top-k under the final prices, candidates listed ----------------------
+  if (a.balanced) {
+    // prices are only defined up to a shift when every expert must be full; anchor the minimum at 0.
+    // A uniform shift moves every value of a token alike, the bound on its uncached experts included.
+    __syncthreads();
+    if (tid == 0) { long long m = sh.sp[0]; for (int e = 1; e < E; ++e) m = sh.sp[e] < m ? sh.sp[e] : m; sh.s_pmin = m; }
+    __syncthreads();
+    const long long pmin = sh.s_pmin;
+    for (int e = tid; e < E; e += blockDim.x) { sh.sp[e] -= pmin; sh.spf[e] = (float)sh.sp[e]; }
+    cumdrop += pmin;
+    __syncthreads();
+  }
+  token_pass(std::true_type{}, nullptr, nullptr);
+  for (int e = tid; e < E; e += blockDim.x)
+    if (sh.sload[e]) atomicAdd(&st->load[e], sh.sload[e]);
+  if (!grid_barrier(st, epoch)) return;
+  if (blockIdx.x != 0) return;
+  // ---- CTA 0: is the state already a certificate? -------------------------------------------------------
+  __shared__ int s_badload;
+  if (tid == 0) s_badload = 0;
+  __syncthreads();
+  for (int e = tid; e < E; e += blockDim.x) {
+    const int load = __ldcg(&st->load[e]);
+    st->load_cur[e] = load; st->load[e] = 0;
+    st->p[e] = sh.sp[e];
+    // primal feasibility and complementary slackness on the expert -> sink arcs
+    if (load > C || (sh.sp[e] > 0 && load < C)) atomicAdd(&s_badload, 1);
+  }
+  __syncthreads();
+  if (tid == 0) {
+    st->sweep = sweep; st->cumdrop = cumdrop;
+    st->round = 1; st->theta_used = a.theta0; st->theta = a.theta0 * 4;
+    st->converged = s_badload == 0 ? 1 : 0;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Check pass.  Every token's experts must still be a top-k under the current prices (ties included).
+// A token that fails re-picks (unless this is the last pass); tokens within theta of a tie are listed
+// as the next round's candidates; loads, violations and the statistics are gathered on the way.  The last
+// CTA decides: no violation and every expert within capacity with complementary slackness = optimal.
+//   fast path  one thread per token, from the cache, when the cache's bound settles every question;
+//   slow path  one warp per token over the full row, exact int64 throughout.
+struct CheckShared {
+  long long sp[kMaxE];
+  int sload[kMaxE];
+  int nslow, viol, rer;
+  unsigned flags;
+  double score;
+  int slow[256];
+};
+
+__global__ void __launch_bounds__(256)
+flow_check_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, int32_t* __restrict__ expert_idx,
+                  int32_t* __restrict__ cand, int T, int E, int k, int C, KeyGen g, int final_pass, int unbounded,
+                  int32_t* __restrict__ expert_load_out, void* stats_out, const unsigned* __restrict__ error_flag) {
+  if (*(volatile int*)&st->done) return;
+  __shared__ CheckShared sh;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int e = tid; e < E; e += blockDim.x) { sh.sp[e] = st->p[e]; sh.sload[e] = 0; }
+  if (tid == 0) { sh.viol = 0; sh.rer = 0; sh.flags = 0; sh.score = 0.0; }
+  __syncthreads();
+  const long long cumdrop = st->cumdrop;
+  const long long theta = final_pass ? -1 : (unbounded ? kInf : st->theta);      // the last pass lists nothing, the one before every token
+  const int gsize = gridDim.x * blockDim.x;
+  int t_viol = 0, t_rer = 0; double t_score = 0.0;
+  for (int base = blockIdx.x * blockDim.x; base < T; base += gsize) {
+    if (tid == 0) sh.nslow = 0;
+    __syncthreads();
+    const int tok = base + tid;
+    if (tok < T) {
+      bool slow = false;
+      const uint4 idv = *reinterpret_cast<const uint4*>(cache.id + (size_t)tok * kCacheN);
+      const unsigned idws[4] = {idv.x, idv.y, idv.z, idv.w};
+      float x[kCacheN];
+#pragma unroll
+      for (int j = 0; j < kCacheN; ++j) x[j] = cache.x[(size_t)j * T + tok];
+      const long long bound = cache.bound[tok];
+      const bool raw = cache.raw[tok] != 0;
+      const uint32_t flat = (uint32_t)tok * (uint32_t)E;
+      unsigned hm[4] = {0, 0, 0, 0}; bool sorted = true; int prev = -1;
       for (int j = 0; j < k; ++j) {
-        const int ej = __shfl_sync(0xffffffffu, mine, j);
-#pragma unroll
-        for (int q = 0; q < kEPLf; ++q) in[q] |= (ej == lane + 32 * q);
+        const int h = expert_idx[(size_t)tok * k + j];
+        if ((unsigned)h >= (unsigned)E) { slow = true; break; }
+        if (hm[h >> 5] & (1u << (h & 31))) { slow = true; break; }
+        hm[h >> 5] |= 1u << (h & 31);
+        sorted &= h > prev; prev = h;
       }
-    bool settled = false, list = false, keep = false;
-    if (!first) {
-      float mh = INFINITY, mn = -INFINITY;
+      long long key[kCacheN], v[kCacheN]; unsigned heldbits = 0;
+      long long min_held = kInf, max_non = -kInf;
+      if (!slow) {
 #pragma unroll
-      for (int q = 0; q < kEPLf; ++q) {
-        if (lane + 32 * q >= E) continue;
-        if (in[q]) mh = fminf(mh, vf[q]); else mn = fmaxf(mn, vf[q]);
+        for (int j = 0; j < kCacheN; ++j) {
+          const int e = (int)((idws[j >> 2] >> (8 * (j & 3))) & 255u);
+          const bool ok = e < E;
+          key[j] = ok ? make_key(g, x[j], flat + e) : -kInf;
+          v[j] = ok ? key[j] - sh.sp[e] : -kInf;
+          const bool held = ok && ((hm[e >> 5] >> (e & 31)) & 1u);
+          if (held) { heldbits |= 1u << j; min_held = v[j] < min_held ? v[j] : min_held; }
+          else if (ok) max_non = v[j] > max_non ? v[j] : max_non;
+        }
+        if (__popc(heldbits) != k) slow = true;           // an expert the token holds is not in its cache
       }
-      mh = unflip_f32(__reduce_min_sync(0xffffffffu, flip_f32(mh)));
-      mn = unflip_f32(__reduce_max_sync(0xffffffffu, flip_f32(mn)));
-      const float diff = mh - mn;
-      if (diff > err3) {                                // certainly still a top-k (E == k: diff = inf)
-        settled = true; keep = true;
-        list = E > k && (diff - err3 <= thetaf);
-      }
-    } else {
-      float vkf, vk1f; bool sel[kEPLf];
-      warp_select_f32(vf, E, k + 1, sel, vkf, vk1f, k);
-      if (vkf - vk1f > err3) {                          // the approximate top-k is certainly the exact one
-        settled = true;
+      const long long ob = bound <= -kInf ? -kInf : (bound >= kInf ? kInf : bound + cumdrop);   // uncached experts
+      bool list = false;
+      if (!slow) {
+        if (min_held >= max_non && min_held >= ob) {
+          const long long other = max_non > ob ? max_non : ob;
+          list = E > k && other > -kInf && min_held - other <= theta;
+        } else if (max_non > min_held) {
+          // a cached expert beats a held one: a violation for certain.  Re-pick from the cache if it still
+          // holds the token's k+1 best experts for certain.
+          int rank[kCacheN];
 #pragma unroll
-        for (int q = 0; q < kEPLf; ++q) in[q] = sel[q];
-        list = E > k && (vkf - vk1f - err3 <= thetaf);
+          for (int j = 0; j < kCacheN; ++j) rank[j] = 0;
+#pragma unroll
+          for (int j = 1; j < kCacheN; ++j)
+#pragma unroll
+            for (int i = 0; i < j; ++i) {
+              const bool first = v[i] >= v[j];
+              rank[j] += first ? 1 : 0; rank[i] += first ? 0 : 1;
+            }
+          long long vk = -kInf, vk1 = -kInf;
+#pragma unroll
+          for (int j = 0; j < kCacheN; ++j) { if (rank[j] == k - 1) vk = v[j]; if (rank[j] == k) vk1 = v[j]; }
+          if (final_pass) {
+            ++t_viol;                                     // reported, not repaired
+          } else if (vk1 >= ob && vk1 > -kInf) {
+            ++t_viol;
+            heldbits = 0; hm[0] = hm[1] = hm[2] = hm[3] = 0;
+#pragma unroll
+            for (int j = 0; j < kCacheN; ++j) {
+              const int e = (int)((idws[j >> 2] >> (8 * (j & 3))) & 255u);
+              if (rank[j] < k && e < E) { heldbits |= 1u << j; hm[e >> 5] |= 1u << (e & 31); }
+            }
+            sorted = false;
+            list = vk - vk1 <= theta;
+          } else {
+            slow = true;
+          }
+        } else {
+          slow = true;                                    // only the bound on the uncached experts is in the way
+        }
+      }
+      // statistics: the score of the held pairs and how many of them are not among the token's k best raw keys
+      if (!slow) {
+        int rer = 0; double sc = 0.0;
+#pragma unroll
+        for (int j = 0; j < kCacheN; ++j) {
+          if (!((heldbits >> j) & 1u)) continue;
+          int above = 0;
+#pragma unroll
+          for (int i = 0; i < kCacheN; ++i) above += key[i] > key[j] ? 1 : 0;
+          if (above >= k) ++rer;
+          else if (bound > -kInf && (!raw || key[j] <= bound)) slow = true;   // an uncached raw key might be larger
+          sc += g.mode == 0 ? (double)x[j] : (double)key[j];
+        }
+        if (!slow) { t_rer += rer; t_score += sc; }
+      }
+      if (!slow) {
+        if (!sorted) write_sorted_experts(expert_idx + (size_t)tok * k, hm, k);
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          unsigned m = hm[w];
+          while (m) { const int b = __ffs(m) - 1; m &= m - 1; atomicAdd(&sh.sload[32 * w + b], 1); }
+        }
+        if (list) cand[atomicAdd(&st->ncand, 1)] = tok;
+      } else {
+        sh.slow[atomicAdd(&sh.nslow, 1)] = tok;
       }
     }
-    long long key[kEPLf];
-    bool have_keys = false;
-    if (!settled) {
-      long long val[kEPLf];
+    __syncthreads();
+    // ---- slow path: one warp per token over the full row --------------------------------------------
+    const int nslow = sh.nslow;
+    for (int s = warp; s < nslow; s += 8) {
+      const int t2 = sh.slow[s];
+      const uint32_t flat = (uint32_t)t2 * (uint32_t)E;
+      const float* row = M + (size_t)t2 * E;
+      const int mine = lane < k ? expert_idx[(size_t)t2 * k + lane] : -1;
+      long long key[kEPLf], val[kEPLf]; bool in[kEPLf]; float xr[kEPLf];
 #pragma unroll
       for (int q = 0; q < kEPLf; ++q) {
         const int e = lane + 32 * q;
-        key[q] = e < E ? make_key(g, x[q], flat + e) : -kInf;
-        val[q] = e < E ? key[q] - sp[e] : -kInf;
+        xr[q] = e < E ? __ldg(row + e) : 0.f;
+        key[q] = e < E ? make_key(g, xr[q], flat + e) : -kInf;
+        val[q] = e < E ? key[q] - sh.sp[e] : -kInf;
+        in[q] = false;
       }
-      have_keys = true;
-      // exact check of the experts the token holds now: the worst held value against the best other one
+      for (int j = 0; j < k; ++j) {
+        const int ej = __shfl_sync(0xffffffffu, mine, j);
+#pragma unroll
+        for (int q = 0; q < kEPLf; ++q) in[q] |= (ej == lane + 32 * q) && (ej < E);
+      }
+      int cnt = 0;
+#pragma unroll
+      for (int q = 0; q < kEPLf; ++q) cnt += __popc(__ballot_sync(0xffffffffu, in[q]));
       long long min_held = kInf, max_non = -kInf;
 #pragma unroll
       for (int q = 0; q < kEPLf; ++q) {
@@ -844,148 +869,150 @@ flow_collect_kernel(const float* __restrict__ M, FlowState* st, int32_t* __restr
         const long long a = __shfl_xor_sync(0xffffffffu, min_held, o), c = __shfl_xor_sync(0xffffffffu, max_non, o);
         min_held = a < min_held ? a : min_held; max_non = c > max_non ? c : max_non;
       }
-      keep = !first && (min_held >= max_non);
+      const bool keep = cnt == k && min_held >= max_non;
       long long gap = keep ? ((E > k) ? min_held - max_non : kInf) : kInf;
-      if (!verify_only && !keep) {
-        long long vk = -kInf, vk1 = -kInf;
-        warp_select(val, E, k + 1, in, vk, vk1, k);
-        gap = (E > k) ? vk - vk1 : kInf;
-      }
-      list = gap < kInf && gap <= theta;
-    }
-    if (!keep && !first) ++w_viol;
-    // the experts in ascending order: word q of the held mask is the vote over in[q]
-    unsigned words[kEPLf]; int below = 0;
-#pragma unroll
-    for (int q = 0; q < kEPLf; ++q) words[q] = __ballot_sync(0xffffffffu, in[q]);
-#pragma unroll
-    for (int q = 0; q < kEPLf; ++q) {
-      if (in[q]) {
-        const int rank = below + __popc(words[q] & ((1u << lane) - 1u));
-        if (rank < k) expert_idx[(size_t)tok * k + rank] = lane + 32 * q;
-        atomicAdd(&sload[lane + 32 * q], 1);
-      }
-      below += __popc(words[q]);
-    }
-    if (verify_only) {
-      // statistics: the score of the held pairs, and how many of them are not in the token's own top-k
-      // of raw keys (the k-th and (k+1)-th raw keys must be told apart for certain, else exact keys decide)
-      float rkf, rk1f; bool rsel[kEPLf];
-      warp_select_f32(kf, E, k + 1, rsel, rkf, rk1f, k);
-      int rer = 0; double sc = 0.0;
-      if (rkf - rk1f > err3) {
-#pragma unroll
-        for (int q = 0; q < kEPLf; ++q) rer += (in[q] && !rsel[q]) ? 1 : 0;
-      } else {
-        if (!have_keys) {
-#pragma unroll
-          for (int q = 0; q < kEPLf; ++q) { const int e = lane + 32 * q; key[q] = e < E ? make_key(g, x[q], flat + e) : -kInf; }
-          have_keys = true;
+      if (!keep) {
+        if (lane == 0) ++t_viol;
+        if (!final_pass) {
+          long long vk = -kInf, vk1 = -kInf;
+          warp_select(val, E, k + 1, in, vk, vk1, k);
+          gap = (E > k) ? vk - vk1 : kInf;
         }
-        long long kth_raw = -kInf, next_raw = -kInf;
-        warp_select(key, E, k, rsel, kth_raw, next_raw, k);
+      }
+      // the experts in ascending order: word q of the held mask is the vote over in[q]
+      unsigned words[kEPLf]; int below = 0;
 #pragma unroll
-        for (int q = 0; q < kEPLf; ++q) rer += (in[q] && key[q] < kth_raw) ? 1 : 0;
+      for (int q = 0; q < kEPLf; ++q) words[q] = __ballot_sync(0xffffffffu, in[q]);
+      if (keep || !final_pass) {
+#pragma unroll
+        for (int q = 0; q < kEPLf; ++q) {
+          if (in[q]) {
+            const int rank = below + __popc(words[q] & ((1u << lane) - 1u));
+            if (rank < k) expert_idx[(size_t)t2 * k + rank] = lane + 32 * q;
+          }
+          below += __popc(words[q]);
+        }
       }
 #pragma unroll
-      for (int q = 0; q < kEPLf; ++q)
-        if (in[q]) sc += (g.mode == 0) ? (double)x[q] : (double)(have_keys ? key[q] : make_key(g, x[q], flat + lane + 32 * q));
+      for (int q = 0; q < kEPLf; ++q) if (in[q]) atomicAdd(&sh.sload[lane + 32 * q], 1);
+      {
+        bool rsel[kEPLf]; long long kth_raw = -kInf, next_raw = -kInf;
+        warp_select(key, E, k, rsel, kth_raw, next_raw, k);
+        int rer = 0; double sc = 0.0;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) { sc += __shfl_xor_sync(0xffffffffu, sc, o); rer += __shfl_xor_sync(0xffffffffu, rer, o); }
-      w_score += sc; w_rer += rer;
+        for (int q = 0; q < kEPLf; ++q) {
+          rer += (in[q] && key[q] < kth_raw) ? 1 : 0;
+          if (in[q]) sc += g.mode == 0 ? (double)xr[q] : (double)key[q];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { sc += __shfl_xor_sync(0xffffffffu, sc, o); rer += __shfl_xor_sync(0xffffffffu, rer, o); }
+        if (lane == 0) { t_rer += rer; t_score += sc; }
+      }
+      if (gap < kInf && gap <= theta && lane == 0) cand[atomicAdd(&st->ncand, 1)] = t2;
     }
-    if (!verify_only && list && lane == 0)
-      cand[atomicAdd(&st->ncand, 1)] = tok;     // the list has room for every token
+    __syncthreads();
   }
-  if (__any_sync(0xffffffffu, w_bad) && lane == 0) atomicOr(&s_flags, 2u);
-  if (lane == 0) {
-    if (w_viol) atomicAdd(&s_viol, w_viol);
-    if (verify_only) { atomicAdd(&s_score, w_score); if (w_rer) atomicAdd(&s_rer, w_rer); }
-  }
+  if (t_viol) atomicAdd(&sh.viol, t_viol);
+  if (t_rer) atomicAdd(&sh.rer, t_rer);
+  if (t_score != 0.0) atomicAdd(&sh.score, t_score);
   __syncthreads();
-  for (int e = threadIdx.x; e < E; e += blockDim.x)
-    if (sload[e]) atomicAdd(&st->load[e], sload[e]);
-  if (threadIdx.x == 0) {
-    if (s_viol) atomicAdd(&st->violations, s_viol);
-    if (s_flags) atomicOr(&st->status, s_flags);
-    if (verify_only) { atomicAdd(&st->total_score, s_score); if (s_rer) atomicAdd(&st->rerouted, s_rer); }
+  for (int e = tid; e < E; e += blockDim.x)
+    if (sh.sload[e]) atomicAdd(&st->load[e], sh.sload[e]);
+  if (tid == 0) {
+    if (sh.viol) atomicAdd(&st->violations, sh.viol);
+    if (sh.rer) atomicAdd(&st->rerouted, sh.rer);
+    if (sh.score != 0.0) atomicAdd(&st->total_score, sh.score);
   }
   if (!last_block_arrives(&st->ticket)) return;
   // ---- last CTA: is the state a certificate? ---------------------------------------------------
   __shared__ int s_badload;
-  if (threadIdx.x == 0) s_badload = 0;
+  if (tid == 0) s_badload = 0;
   __syncthreads();
-  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+  for (int e = tid; e < E; e += blockDim.x) {
     const int load = __ldcg(&st->load[e]);
     st->load_cur[e] = load;
     st->load[e] = 0;
-    if (verify_only && expert_load_out) expert_load_out[e] = load;
+    if (expert_load_out) expert_load_out[e] = load;
     // primal feasibility and complementary slackness on the expert -> sink arcs
-    if (load > C || (sp[e] > 0 && load < C)) atomicAdd(&s_badload, 1);
+    if (load > C || (sh.sp[e] > 0 && load < C)) atomicAdd(&s_badload, 1);
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (tid == 0) {
     const int viol = *(volatile int*)&st->violations;
-    const bool ok = (first || viol == 0) && s_badload == 0;
-    {   // diagnostics: per round, violations / experts out of balance / augmentations so far / candidates
-      const int r = st->round < 4 ? st->round : 3;
-      st->trace[48 + 4 * r] = viol; st->trace[49 + 4 * r] = s_badload; st->trace[50 + 4 * r] = st->naug;
-      st->trace[51 + 4 * r] = st->ncand;
-    }
+    const bool ok = viol == 0 && s_badload == 0;
     st->violations = 0;
     st->ticket = 0;
-    if (!verify_only) {
-      st->round = st->round + 1;
-      st->theta_used = theta;
-      st->theta = (theta > (kInf >> 8)) ? kInf : theta * theta_scale;   // next round looks further
-    }
-    if (verify_only && !ok) atomicOr(&st->status, 1u);
-    if (verify_only && error_flag && *error_flag) atomicOr(&st->status, 4u);
-    __threadfence();
-    if (ok) st->converged = 1;
-    if (verify_only && stats_out) {
+    if (ok || final_pass) {
+      unsigned status = *(volatile unsigned*)&st->status;
+      if (!ok) status |= 1u;
+      if (error_flag && *error_flag) status |= 4u;
       // layout of maxscore_stats: status, capacity, sweeps, augmentations, rounds, candidates,
       // rerouted, reserved, total_score
       int* so = reinterpret_cast<int*>(stats_out);
-      so[0] = (int)(*(volatile unsigned*)&st->status & 7u);
+      so[0] = (int)(status & 7u);
       so[1] = C; so[2] = st->sweep; so[3] = st->naug; so[4] = st->round;
       so[5] = st->ncand_last; so[6] = *(volatile int*)&st->rerouted; so[7] = 0;
       *reinterpret_cast<double*>(so + 8) = *(volatile double*)&st->total_score;
+      st->converged = 1;
+      __threadfence();
+      st->done = 1;
+    } else {
+      // the next round looks further: its candidates were listed with this pass's theta
+      const long long th = theta;
+      st->round = st->round + 1;
+      st->theta_used = th;
+      st->theta = (th > (kInf >> 8)) ? kInf : th * 4;
+      st->rerouted = 0; st->total_score = 0.0;
+      st->converged = 0;
     }
   }
 }
 
 // ---------------------------------------------------------------------------------------------
-// Exact phase: successive shortest augmenting paths on the expert-level residual graph, one CTA.
+// Exact phase: successive shortest augmenting paths on the expert-level residual graph of Table 1's
+// network (E experts + one node Z for the sink side).
 //
 // Only candidate tokens (gap <= theta) are in the graph.  A round stops BEFORE an augmentation whose
 // price update would spread the experts' price changes of this round by more than theta: up to that
-// point no token outside the list can have lost its top-k, so the state handed to the next collect
+// point no token outside the list can have lost its top-k, so the state handed to the next check
 // pass is consistent, and that pass only has to list more tokens.
 //
-// D[e][f] (shared memory) is the cheapest move of one candidate token from e to f.  After a token
-// moves u -> v only row u is rebuilt; the rows of its other experts and of v are patched from the
-// token's own keys.  The experts of the first kHeldCache candidates are mirrored in shared memory
-// (expert_idx itself is edited in place as well); the list is sorted first, so ties are broken by
-// the smallest token index whatever order the collect pass appended the tokens in.
-constexpr int kP2Threads = 1024;
-constexpr int kHeldCache = 4096;
-constexpr int kMaxFix = 256;
-constexpr int kMaxArcs = 8192;      // finite arcs of D the Bellman-Ford search can list
-constexpr int kSortMax = 16384;     // candidate lists up to this length are sorted (they fit in D's space)
+// The graph is never materialised as an E x E matrix.  Each candidate carries a short record: the
+// experts it holds that could be given up within the arc window, and the experts it does not hold
+// that could be taken within it, each with value0 = key - price at the start of the round.  A token
+// that holds e and not f is a residual arc e -> f of reduced cost value(e) - value(f) >= 0, where
+// value = value0 - (price now - price at round start).  One round of the Bellman-Ford search is then
+// one pass over the records: A = min over held entries of dist[e] + value(e), and every entry f not
+// held is offered A - value(f).  Moving a token flips two flags of its record; nothing is rebuilt.
+constexpr int kP2Group = 4;                // threads that share one node of the graph in a search round
+constexpr int kP2Threads = kP2Group * kMaxE + 32;   // a group per expert node and one warp for node Z
+constexpr int kP2Own = 2;                  // candidates per thread whose records stay in registers during a search
+constexpr int kRecSmemBytes = 96 * 1024;   // records up to this size are mirrored in shared memory
+constexpr long long kDistLimit = 1LL << 58;  // distances stay below this, so that sums cannot overflow
+constexpr long long kExactCycleBudget = 4000000000LL;   // about two seconds: the exact phase gives up beyond this
 
-// First build of D for a round, spread over the whole GPU: one warp per candidate token, results
-// merged into global memory with 64-bit atomicMin.  (Inside the exact phase's single CTA the same
-// work costs a quarter of a millisecond at 1 600 candidates.)
+struct Records {
+  long long* val;          // [cap] value0 of each entry
+  unsigned short* meta;    // [cap] expert index | held << 8
+  int* off;                // [T] first entry of candidate c
+  int* cnt;                // [T] number of its entries
+  // scratch of the exact phase when the records do not fit in shared memory
+  int* pos;                // [cap] position of the entry in the by-expert order
+  int* bxc;                // [cap] by-expert order: position in the candidate list of the entry's token
+  long long* ndv;          // [cap] by-expert order: the offer the entry makes to its expert in this search round
+  int* aarg;               // [T] the held expert through which the candidate is reached most cheaply
+  int cap;
+};
+
+// Records of one round, built by the whole GPU: one warp per candidate token reads the token's row once.
 __global__ void __launch_bounds__(256)
-flow_build_kernel(const float* __restrict__ M, const FlowState* st, const int32_t* __restrict__ expert_idx,
-                  const int32_t* __restrict__ cand, long long* __restrict__ Dg, int T, int E, int k, KeyGen g) {
+flow_records_kernel(const float* __restrict__ M, FlowState* st, const int32_t* __restrict__ expert_idx,
+                    const int32_t* __restrict__ cand, Records rec, int T, int E, int k, KeyGen g) {
   if (*(volatile const int*)&st->converged) return;
   __shared__ long long sp[kMaxE];
   for (int e = threadIdx.x; e < E; e += blockDim.x) sp[e] = st->p[e];
   __syncthreads();
   const int n = min(st->ncand, T);
-  const int ES = E | 1;
   const long long theta = st->theta_used;
   const long long arc_window = theta >= (kInf >> 2) ? kInf : 2 * theta;
   const int lane = threadIdx.x & 31;
@@ -997,435 +1024,329 @@ flow_build_kernel(const float* __restrict__ M, const FlowState* st, const int32_
     for (int j = 0; j < kMaxK; ++j) h[j] = j < k ? expert_idx[(size_t)tok * k + j] : -1;
     const float* row = M + (size_t)tok * E;
     const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-    long long key[kEPLf]; bool in[kEPLf];
+    long long val[kEPLf]; bool in[kEPLf];
 #pragma unroll
     for (int q = 0; q < kEPLf; ++q) {
       const int f = lane + 32 * q;
-      key[q] = f < E ? make_key(g, __ldg(row + f), flat + f) : 0;
-      bool hd = f >= E;
+      val[q] = f < E ? make_key(g, __ldg(row + f), flat + f) - sp[f] : -kInf;
+      bool hd = false;
 #pragma unroll
       for (int j = 0; j < kMaxK; ++j) hd |= (h[j] == f);
       in[q] = hd;
     }
-    long long vmax = -kInf;
+    long long best_out = -kInf;                         // best value among the experts the token does not hold
+#pragma unroll
+    for (int q = 0; q < kEPLf; ++q)
+      if (!in[q] && lane + 32 * q < E) best_out = val[q] > best_out ? val[q] : best_out;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const long long ov = __shfl_xor_sync(0xffffffffu, best_out, o);
+      best_out = ov > best_out ? ov : best_out;
+    }
+    // a held expert further than the arc window above every alternative cannot be given up this round
+    bool inc[kEPLf];
+    long long low_held = kInf;
 #pragma unroll
     for (int q = 0; q < kEPLf; ++q) {
-      const int f = lane + 32 * q;
-      if (!in[q]) { const long long val = key[q] - sp[f]; vmax = val > vmax ? val : vmax; }
+      inc[q] = in[q] && best_out > -kInf && (arc_window >= kInf || val[q] - best_out <= arc_window);
+      if (inc[q]) low_held = val[q] < low_held ? val[q] : low_held;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-      const long long ov = __shfl_xor_sync(0xffffffffu, vmax, o);
-      vmax = ov > vmax ? ov : vmax;
+      const long long ov = __shfl_xor_sync(0xffffffffu, low_held, o);
+      low_held = ov < low_held ? ov : low_held;
     }
+    // an expert not held further than the window below every held one that can move cannot be taken
 #pragma unroll
-    for (int j = 0; j < kMaxK; ++j) {
-      if (j >= k) continue;
-      const int e = h[j];
-      long long mine = 0;
+    for (int q = 0; q < kEPLf; ++q)
+      if (!in[q]) inc[q] = lane + 32 * q < E && low_held < kInf && (arc_window >= kInf || low_held - val[q] <= arc_window);
+    unsigned words[kEPLf]; int total = 0;
 #pragma unroll
-      for (int q = 0; q < kEPLf; ++q) if ((e >> 5) == q) mine = key[q];
-      const long long we = __shfl_sync(0xffffffffu, mine, e & 31);
-      const long long pe = sp[e];
-      if (arc_window < kInf && (we - pe) - vmax > arc_window) continue;
+    for (int q = 0; q < kEPLf; ++q) { words[q] = __ballot_sync(0xffffffffu, inc[q]); total += __popc(words[q]); }
+    int base = 0;
+    if (lane == 0) {
+      base = atomicAdd(&st->nrec, total);
+      if (base + total > rec.cap) { base = -1; st->rec_overflow = 1; }     // no room: the token stays out of the graph
+      rec.off[c] = base < 0 ? 0 : base;
+      rec.cnt[c] = base < 0 ? 0 : total;
+    }
+    base = __shfl_sync(0xffffffffu, base, 0);
+    if (base < 0) continue;
+    int before = 0;
 #pragma unroll
-      for (int q = 0; q < kEPLf; ++q) {
-        const int f = lane + 32 * q;
-        if (!in[q]) {
-          const long long cst = we - key[q];
-          if (cst - pe + sp[f] <= arc_window && cst < Dg[e * ES + f]) atomicMin(&Dg[e * ES + f], cst);
-        }
+    for (int q = 0; q < kEPLf; ++q) {
+      if (inc[q]) {
+        const int pos = base + before + __popc(words[q] & ((1u << lane) - 1u));
+        rec.val[pos] = val[q];
+        rec.meta[pos] = (unsigned short)((lane + 32 * q) | (in[q] ? 256 : 0));
       }
+      before += __popc(words[q]);
     }
   }
 }
 
+constexpr int kRecUnroll = 6;      // records up to this many entries are handled with all loads in flight
+
 struct P2Shared {
   long long p[kMaxE + 1];        // potentials: prices of the experts, then Z
-  long long p0[kMaxE + 1];       // potentials at the start of the round
-  long long dist[2][kMaxE + 1];  // [0] current, [1] snapshot of the previous round
-  int pred[kMaxE + 1];
-  unsigned char act[2][kMaxE + 4];   // nodes whose distance changed in the last round
+  long long dp[kMaxE + 1];       // potentials now minus potentials at the start of the round
+  long long p0[kMaxE + 1];
+  long long dist[2][kMaxE + 1];  // distances as of the last search round / of the running one
+  int lvl[kMaxE + 1];            // search round in which the node's distance became final
   int imb[kMaxE + 1];            // + excess, - deficit
   int flow[kMaxE];               // units on expert -> sink
-  int dirty[kMaxE];
-  unsigned char fixrow[kMaxE];   // rows that have a stale entry to recompute
-  int path[kMaxE + 2];
-  int npath, changed, who, target, stop, any_pos, qn, nfix, narc, bf_bad, dup;
-  int who_a[kMaxE + 2];          // per arc of the path: the candidate that moves
-  int fix_e[kMaxFix], fix_f[kMaxFix];   // stale D entries to recompute after a move
-  long long dt;
+  int estart[kMaxE + 2], efill[kMaxE + 1];   // entries grouped by expert: first position, fill counter
+  int path_v[kMaxE + 2], path_u[kMaxE + 2], path_tok[kMaxE + 2], path_c[kMaxE + 2];
+  int npath, target, stop;
+  long long dt, dtb;             // distance of the chosen target; best distance of any node with a deficit so far
 };
 
+// kSmem = true: the records are mirrored in shared memory (the kernel returns at once if they do not fit);
+// kSmem = false: they stay in global memory (the kernel returns at once if they would have fitted).  The
+// host launches both, one after the other; exactly one of them does the work.
+template <bool kSmem>
 __global__ void __launch_bounds__(kP2Threads)
-flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_idx, int32_t* cand, int T, int E,
-                  int k, int C, KeyGen g, int max_aug, const long long* __restrict__ Dg) {
-  if (*(volatile int*)&st->converged) return;
+flow_exact_kernel(FlowState* st, int32_t* expert_idx, const int32_t* __restrict__ cand, Records rec, int T, int E,
+                  int k, int C, int max_aug) {
+  if (*(volatile int*)&st->done) return;
+  if (*(volatile int*)&st->converged) {             // nothing to repair; the check pass starts a fresh list
+    if (threadIdx.x == 0) { st->ncand = 0; st->nrec = 0; }
+    return;
+  }
   extern __shared__ __align__(16) unsigned char p2smem[];
-  long long* D = reinterpret_cast<long long*>(p2smem);                              // [E][E] raw arc costs
-  unsigned char* held_s = reinterpret_cast<unsigned char*>(D + (size_t)E * (E | 1));       // [kHeldCache][kMaxK]
-  int* cand_s = reinterpret_cast<int*>(held_s + (size_t)kHeldCache * kMaxK);          // [kHeldCache]
-  int* queue_s = cand_s + kHeldCache;                                                // [kHeldCache]
-  unsigned short* arcs_s = reinterpret_cast<unsigned short*>(queue_s + kHeldCache);  // [kMaxArcs] (u << 8 | v)
   __shared__ P2Shared s;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = min(st->ncand, T);
-  const int nZ = E;   // index of Z
-  const int ES = E | 1;   // odd row stride of D: a warp walking down a column hits different banks
+  const int nent = min(st->nrec, rec.cap);
+  const int nZ = E;
   const long long theta = st->theta_used;
-  const long long arc_window = theta >= (kInf >> 2) ? kInf : 2 * theta;
+  const long long t_start = clock64();
 
-  // ---- sort the candidate list (in D's space, not yet in use) ----------------------------------------
-  if (n > 1 && n <= kSortMax && (size_t)n * 4 <= (size_t)E * (E | 1) * 8) {
-    int* buf = reinterpret_cast<int*>(D);
-    int npow = 1; while (npow < n) npow <<= 1;
-    if ((size_t)npow * 4 <= (size_t)E * (E | 1) * 8) {
-      for (int i = tid; i < npow; i += blockDim.x) buf[i] = i < n ? cand[i] : 0x7fffffff;
-      __syncthreads();
-      for (int size = 2; size <= npow; size <<= 1)
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-          for (int i = tid; i < npow; i += blockDim.x) {
-            const int j = i ^ stride;
-            if (j > i) {
-              const bool up = (i & size) == 0;
-              const int a = buf[i], b = buf[j];
-              if ((a > b) == up) { buf[i] = b; buf[j] = a; }
-            }
-          }
-          __syncthreads();
-        }
-      for (int i = tid; i < n; i += blockDim.x) cand[i] = buf[i];
-      __syncthreads();
-    }
+  if ((((size_t)nent * 26 + (size_t)n * 16 + 64) <= (size_t)kRecSmemBytes) != kSmem) return;
+  // ---- mirror the records in shared memory when they fit ------------------------------------------
+  long long* v_s = reinterpret_cast<long long*>(p2smem);
+  long long* nd_s = v_s + nent;
+  int* off_s = reinterpret_cast<int*>(nd_s + nent);
+  int* cnt_s = off_s + n;
+  int* tok_s = cnt_s + n;
+  int* aarg_s = tok_s + n;
+  int* pos_s = aarg_s + n;
+  int* bxc_s = pos_s + nent;
+  unsigned short* m_s = reinterpret_cast<unsigned short*>(bxc_s + nent);
+  if (kSmem) {
+    for (int i = tid; i < nent; i += blockDim.x) { v_s[i] = rec.val[i]; m_s[i] = rec.meta[i]; }
+    for (int i = tid; i < n; i += blockDim.x) { off_s[i] = rec.off[i]; cnt_s[i] = rec.cnt[i]; tok_s[i] = cand[i]; }
   }
-  const int nc = min(n, kHeldCache);
-  for (int i = tid; i < nc; i += blockDim.x) cand_s[i] = cand[i];
-  __syncthreads();
-  for (int i = tid; i < nc * k; i += blockDim.x) {
-    const int c = i / k, j = i - c * k;
-    held_s[c * kMaxK + j] = (unsigned char)expert_idx[(size_t)cand_s[c] * k + j];
-  }
-  auto tok_of = [&](int c) -> int { return c < nc ? cand_s[c] : cand[c]; };
-  auto held_of = [&](int c, int tok, int j) -> int {
-    return c < nc ? (int)held_s[c * kMaxK + j] : expert_idx[(size_t)tok * k + j];
-  };
-
+  const long long* rval = kSmem ? v_s : rec.val; unsigned short* rmeta = kSmem ? m_s : rec.meta;
+  const int* roff = kSmem ? off_s : rec.off; const int* rcnt = kSmem ? cnt_s : rec.cnt; const int* rtok = kSmem ? tok_s : cand;
+  int* rpos = kSmem ? pos_s : rec.pos; int* bxc = kSmem ? bxc_s : rec.bxc; long long* ndv = kSmem ? nd_s : rec.ndv;
+  int* aarg = kSmem ? aarg_s : rec.aarg;
+  for (int e = tid; e <= E + 1; e += blockDim.x) { s.estart[e] = 0; if (e <= E) s.efill[e] = 0; }
   for (int e = tid; e < E; e += blockDim.x) {
-    s.p[e] = st->p[e]; s.p0[e] = s.p[e];
+    s.p[e] = st->p[e]; s.p0[e] = s.p[e]; s.dp[e] = 0;
     const int load = st->load_cur[e];
     const int fl = s.p[e] > 0 ? C : min(load, C);
-    s.flow[e] = fl; s.imb[e] = load - fl; s.dirty[e] = 0;
+    s.flow[e] = fl; s.imb[e] = load - fl;
   }
-  for (int i = tid; i < E * ES; i += blockDim.x) D[i] = Dg[i];       // built by flow_build_kernel
+  __syncthreads();
+  // ---- the entries grouped by expert (counting sort over the candidates' records) ---------------------
+  for (int c = tid; c < n; c += blockDim.x) {
+    const int o = roff[c], m = rcnt[c];
+    for (int i = o; i < o + m; ++i) atomicAdd(&s.estart[(rmeta[i] & 255) + 1], 1);
+  }
   __syncthreads();
   if (tid == 0) {
     int tot = 0;
     for (int e = 0; e < E; ++e) tot += s.imb[e];
-    s.imb[nZ] = -tot; s.p[nZ] = 0; s.p0[nZ] = 0; s.stop = 0;
+    s.imb[nZ] = -tot; s.p[nZ] = 0; s.p0[nZ] = 0; s.dp[nZ] = 0; s.stop = 0;
+    for (int e = 0; e <= E; ++e) s.estart[e + 1] += s.estart[e];
+  }
+  __syncthreads();
+  for (int c = tid; c < n; c += blockDim.x) {
+    const int o = roff[c], m = rcnt[c];
+    for (int i = o; i < o + m; ++i) {
+      const int e = rmeta[i] & 255;
+      const int ps = s.estart[e] + atomicAdd(&s.efill[e], 1);
+      rpos[i] = ps; bxc[ps] = c;
+    }
   }
   __syncthreads();
 
   int naug = 0;
-  int bf_rounds = 0; long long q_total = 0, t_first = 0;
-  long long t_who = 0, t_patch = 0, t_fix = 0; int n_arcs = 0;
-  long long t_rebuild = 0, t_bf = 0, t_move = 0, t0 = clock64();   // phase timers (thread 0), diagnostics
+  const int naug_before = st->naug;
+  long long* d0 = s.dist[0]; long long* dn = s.dist[1];
   for (;;) {
-    // ---- rebuild the rows of D marked dirty: D[e][f] = min over candidates in e, not in f ----------
-    for (int i = tid; i < E * ES; i += blockDim.x)
-      if (s.dirty[i / ES]) D[i] = kInf;
-    __syncthreads();
-    // cached candidates that hold a dirty row are queued first (one thread each, shared memory only);
-    // the warps then work through the queue and through the uncached tail of the list
-    if (tid == 0) s.qn = 0;
-    __syncthreads();
-    for (int c0 = 0; c0 < nc; c0 += blockDim.x) {
-      const int c = c0 + tid;
-      bool any = false;
-      if (c < nc)
-        for (int j = 0; j < k; ++j) any |= (s.dirty[held_s[c * kMaxK + j]] != 0);
-      const unsigned mask = __ballot_sync(0xffffffffu, any);
-      int base = 0;
-      if (lane == 0 && mask) base = atomicAdd(&s.qn, __popc(mask));
-      base = __shfl_sync(0xffffffffu, base, 0);
-      if (any) queue_s[base + __popc(mask & ((1u << lane) - 1u))] = c;
+    {
+      if (tid == 0 && clock64() - t_start > kExactCycleBudget) s.stop = 1;
+      const int any = __syncthreads_or(tid <= E && s.imb[tid] > 0);
+      if (s.stop) { if (tid == 0) atomicOr(&st->status, 4u); break; }
+      if (!any || naug_before + naug >= max_aug) break;
     }
+    // ---- shortest paths from every node with excess: synchronous Bellman-Ford ---------------------------
+    // A round has two halves.  (A) One thread per candidate: A = the cheapest way to reach the token through
+    // an expert it holds; every entry it does not hold is offered A - value, written where the entry sits in
+    // the by-expert order.  (B) A group of threads per node: the best offer over the node's stretch of that
+    // order, and the arcs through Z.  No atomics on distances, and distances only ever come from the previous
+    // round's, so the round in which a node's distance became final orders the nodes.
+    // Offers that cannot beat the nearest node with a deficit found so far are dropped: all costs are
+    // non-negative, and beyond that distance the price update only needs to know "at least that far".
+    for (int v = tid; v <= E; v += blockDim.x) { d0[v] = s.imb[v] > 0 ? 0 : kInf; s.lvl[v] = 0; }
+    if (tid == 0) s.dtb = kDistLimit;
     __syncthreads();
-    const int work = s.qn + (n - nc);
-    q_total += work; if (naug == 0 && t_first == 0) t_first = -1;
-    for (int i = warp; i < work; i += kP2Threads / 32) {
-      const int c = i < s.qn ? queue_s[i] : nc + (i - s.qn);
-      const int tok = tok_of(c);
-      int h[kMaxK];
-      bool any = false;
+    // this thread's candidates: entries, flags and current values in registers for the whole search
+    int om[kP2Own], oex[kP2Own][kRecUnroll], ops[kP2Own][kRecUnroll]; unsigned oheld[kP2Own]; long long ovc[kP2Own][kRecUnroll];
 #pragma unroll
-      for (int j = 0; j < kMaxK; ++j) {
-        h[j] = j < k ? held_of(c, tok, j) : -1;
-        if (j < k) any |= (s.dirty[h[j]] != 0);
+    for (int r = 0; r < kP2Own; ++r) {
+      const int c = tid + r * kP2Threads;
+      om[r] = c < n ? rcnt[c] : 0;
+      oheld[r] = 0;
+      if (om[r] > kRecUnroll) om[r] = -1;               // too long for registers: handled from memory below
+      const int o = c < n ? roff[c] : 0;
+#pragma unroll
+      for (int j = 0; j < kRecUnroll; ++j) {
+        const int i = j < om[r] ? o + j : o;
+        const int mt = om[r] > 0 ? rmeta[i] : 0;
+        oex[r][j] = mt & 255; ops[r][j] = om[r] > 0 ? rpos[i] : 0;
+        if (j < om[r] && (mt & 256)) oheld[r] |= 1u << j;
+        ovc[r][j] = om[r] > 0 ? rval[i] - s.dp[oex[r][j]] : 0;
       }
-      if (!any) continue;
-      const float* row = M + (size_t)tok * E;
-      const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-      long long key[kEPLf];
-      bool in[kEPLf];
+    }
+    int more = 1;
+    for (int round = 1; round <= E + 2 && more; ++round) {
 #pragma unroll
-      for (int q = 0; q < kEPLf; ++q) {
-        const int f = lane + 32 * q;
-        key[q] = f < E ? make_key(g, __ldg(row + f), flat + f) : 0;
-        bool hd = f >= E;
+      for (int r = 0; r < kP2Own; ++r) {
+        if (om[r] <= 0) continue;
+        long long x[kRecUnroll];
 #pragma unroll
-        for (int j = 0; j < kMaxK; ++j) hd |= (h[j] == f);
-        in[q] = hd;
+        for (int j = 0; j < kRecUnroll; ++j) {
+          const long long dv = d0[oex[r][j]];
+          x[j] = (j < om[r] && ((oheld[r] >> j) & 1u) && dv < kInf) ? dv + ovc[r][j] : kInf;
+        }
+        long long A = kInf; int ae = 0;
+#pragma unroll
+        for (int j = 0; j < kRecUnroll; ++j)
+          if (x[j] < A || (x[j] == A && x[j] < kInf && oex[r][j] < ae)) { A = x[j]; ae = oex[r][j]; }
+#pragma unroll
+        for (int j = 0; j < kRecUnroll; ++j)
+          if (j < om[r]) ndv[ops[r][j]] = (!((oheld[r] >> j) & 1u) && A < kInf) ? A - ovc[r][j] : kInf;
+        aarg[tid + r * kP2Threads] = ae;
       }
-      // best value among the experts the token does not hold: a held expert further than the arc
-      // window above it has no usable move at all
-      long long vmax = -kInf;
-#pragma unroll
-      for (int q = 0; q < kEPLf; ++q) {
-        const int f = lane + 32 * q;
-        if (!in[q]) { const long long val = key[q] - s.p[f]; vmax = val > vmax ? val : vmax; }
+      for (int c = tid; c < n; c += blockDim.x) {
+        if (c < kP2Own * kP2Threads && rcnt[c] <= kRecUnroll) continue;      // done from registers above
+        const int o = roff[c], m = rcnt[c];
+        if (m == 0) continue;
+        long long A = kInf; int ae = 0;
+        for (int i = o; i < o + m; ++i) {
+          const int mt = rmeta[i];
+          if (!(mt & 256)) continue;
+          const int e = mt & 255;
+          const long long du = d0[e];
+          if (du >= kInf) continue;
+          const long long x = du + (rval[i] - s.dp[e]);
+          if (x < A || (x == A && e < ae)) { A = x; ae = e; }
+        }
+        for (int i = o; i < o + m; ++i) {
+          const int mt = rmeta[i];
+          ndv[rpos[i]] = (!(mt & 256) && A < kInf) ? A - (rval[i] - s.dp[mt & 255]) : kInf;
+        }
+        aarg[c] = ae;
       }
+      __syncthreads();
+      bool changed = false;
+      const long long dtb = s.dtb;
+      {
+        const int f = tid / kP2Group, sub = tid % kP2Group;      // every thread takes part in the group shuffles
+        long long best = kInf;
+        if (f < E) {
+          const int hi = s.estart[f + 1];
+          for (int idx = s.estart[f] + sub; idx < hi; idx += 4 * kP2Group) {
+            long long a[4];
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const long long ov = __shfl_xor_sync(0xffffffffu, vmax, o);
-        vmax = ov > vmax ? ov : vmax;
+            for (int u = 0; u < 4; ++u) a[u] = idx + u * kP2Group < hi ? ndv[idx + u * kP2Group] : kInf;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) best = a[u] < best ? a[u] : best;
+          }
+          if (sub == 0) {                                 // one unit less on f -> sink
+            const long long dz = d0[nZ];
+            if (dz < kInf && s.flow[f] > 0) {
+              long long rc = -s.p[nZ] + s.p[f]; if (rc < 0) rc = 0;
+              best = dz + rc < best ? dz + rc : best;
+            }
+          }
+        }
+#pragma unroll
+        for (int o = kP2Group / 2; o > 0; o >>= 1) {
+          const long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+          best = ob < best ? ob : best;
+        }
+        if (f < E && sub == 0) {
+          const long long old = d0[f];
+          if (best < old && best < dtb) {
+            dn[f] = best; s.lvl[f] = round; changed = true;
+            if (s.imb[f] < 0) atomicMin(&s.dtb, best);
+          } else {
+            dn[f] = old;
+          }
+        }
       }
-#pragma unroll
-      for (int j = 0; j < kMaxK; ++j) {
-        if (j >= k) continue;
-        const int e = h[j];
-        if (!s.dirty[e]) continue;
-        long long mine = 0;
-#pragma unroll
-        for (int q = 0; q < kEPLf; ++q) if ((e >> 5) == q) mine = key[q];
-        const long long we = __shfl_sync(0xffffffffu, mine, e & 31);
-        // only moves whose reduced cost is within 2*theta can be used before this round ends
-        const long long pe = s.p[e];
-        if (arc_window < kInf && (we - pe) - vmax > arc_window) continue;
+      if (warp == kP2Threads / 32 - 1) {                  // node Z: one more unit on e -> sink, for any expert with room
+        long long off[kEPLf];
 #pragma unroll
         for (int q = 0; q < kEPLf; ++q) {
-          const int f = lane + 32 * q;
-          if (!in[q]) {
-            const long long cst = we - key[q];
-            // D only ever decreases, so a stale read can only let a useless atomic through
-            if (cst - pe + s.p[f] <= arc_window && cst < D[e * ES + f]) atomicMin(&D[e * ES + f], cst);
+          const int e = lane + 32 * q;
+          off[q] = kInf;
+          if (e < E) {
+            const long long de = d0[e]; const int fl = s.flow[e];
+            long long rc = -s.p[e] + s.p[nZ]; if (rc < 0) rc = 0;
+            if (de < kInf && fl < C) off[q] = de + rc;
           }
         }
-      }
-    }
-    __syncthreads();
-    for (int e = tid; e < E; e += blockDim.x) s.dirty[e] = 0;
-    {
-      const int any = __syncthreads_or(tid <= E && s.imb[tid] > 0);
-      if (tid == 0) s.any_pos = any;
-    }
-    __syncthreads();
-    { const long long t1 = clock64(); t_rebuild += t1 - t0; if (t_first == -1) t_first = t1 - t0; t0 = t1; }
-    if (!s.any_pos || naug >= max_aug) break;
-
-    // ---- shortest paths from every node with excess ---------------------------------------------------
-    // First choice: synchronous Bellman-Ford over the list of finite arcs of D (a few thousand after the
-    // window filter), all threads, distance and predecessor packed in one word (dist << 8 | pred) so
-    // that one atomicMin keeps them consistent.  A node is only updated when its distance strictly
-    // drops against the previous round, so the predecessor graph has no cycle.  If the arc list does
-    // not fit, or distances leave the packed range, the single-warp Dijkstra below takes over.
-    bool have_paths = false;
-    {
-      if (tid == 0) s.narc = 0;
-      __syncthreads();
-      for (int i0 = 0; i0 < E * ES; i0 += blockDim.x) {      // one counter update per warp, not per arc
-        const int i = i0 + tid;
-        const int u = i / ES, v = i - u * ES;
-        const bool finite = i < E * ES && v < E && D[i] < kInf;
-        const unsigned mask = __ballot_sync(0xffffffffu, finite);
-        int base = 0;
-        if (lane == 0 && mask) base = atomicAdd(&s.narc, __popc(mask));
-        base = __shfl_sync(0xffffffffu, base, 0);
-        const int slot = base + __popc(mask & ((1u << lane) - 1u));
-        if (finite && slot < kMaxArcs) arcs_s[slot] = (unsigned short)((u << 8) | v);
-      }
-      __syncthreads();
-      if (s.narc <= kMaxArcs) {
-        const int narc = s.narc;
-        constexpr long long kPInf = 0x7fffffffffffffffLL;
-        constexpr long long kBfLimit = 1LL << 46;     // arcs and distances beyond this leave the packed range
-        long long* pd0 = s.dist[0]; long long* pd1 = s.dist[1];
-        for (int v = tid; v <= E; v += blockDim.x) pd0[v] = s.imb[v] > 0 ? 255LL : kPInf;   // dist 0, no pred
-        if (tid == 0) s.bf_bad = 0;
-        __syncthreads();
-        for (int round = 0; round <= E + 1; ++round) {
-          for (int v = tid; v <= E; v += blockDim.x) pd1[v] = pd0[v];
-          if (tid == 0) s.changed = 0;
-          __syncthreads();
-          for (int a = tid; a < narc; a += blockDim.x) {
-            const int u = arcs_s[a] >> 8, v = arcs_s[a] & 255;
-            const long long pu = pd0[u];
-            if (pu == kPInf) continue;
-            long long rc = D[u * ES + v] - s.p[u] + s.p[v];
-            if (rc < 0) rc = 0;
-            if (rc >= kBfLimit) { s.bf_bad = 1; continue; }
-            const long long nd = (pu >> 8) + rc;
-            if (nd >= kBfLimit) { s.bf_bad = 1; continue; }
-            const long long old = pd0[v];
-            if (old == kPInf || nd < (old >> 8)) { atomicMin(&pd1[v], (nd << 8) | u); s.changed = 1; }
-          }
-          for (int e = tid; e < E; e += blockDim.x) {      // the arcs through Z
-            const long long pe = pd0[e], pz = pd0[nZ];
-            if (pe != kPInf && s.flow[e] < C) {
-              long long rc = -s.p[e] + s.p[nZ]; if (rc < 0) rc = 0;
-              const long long nd = (pe >> 8) + rc;
-              if (rc >= kBfLimit || nd >= kBfLimit) s.bf_bad = 1;
-              else if (pz == kPInf || nd < (pz >> 8)) { atomicMin(&pd1[nZ], (nd << 8) | e); s.changed = 1; }
-            }
-            if (pz != kPInf && s.flow[e] > 0) {
-              long long rc = -s.p[nZ] + s.p[e]; if (rc < 0) rc = 0;
-              const long long nd = (pz >> 8) + rc;
-              if (rc >= kBfLimit || nd >= kBfLimit) s.bf_bad = 1;
-              else if (pe == kPInf || nd < (pe >> 8)) { atomicMin(&pd1[e], (nd << 8) | nZ); s.changed = 1; }
-            }
-          }
-          __syncthreads();
-          long long* t = pd0; pd0 = pd1; pd1 = t;
-          ++bf_rounds;
-          const bool more = s.changed != 0;
-          __syncthreads();
-          if (!more) break;
-        }
-        if (!s.bf_bad) {
-          // unpack; nearest node with a deficit (lowest index on ties)
-          long long dv = kInf; int pv = -1;
-          if (tid <= E) {
-            const long long w = pd0[tid];
-            if (w != kPInf) { dv = w >> 8; pv = (int)(w & 255); if (pv == 255) pv = -1; }
-          }
-          __syncthreads();
-          if (tid <= E) { s.dist[0][tid] = dv; s.pred[tid] = pv; }
-          __syncthreads();
-          if (warp == 0) {
-            long long dt = kInf; int t = 0x7fffffff;
-            for (int v = lane; v <= E; v += 32)
-              if (s.imb[v] < 0 && s.dist[0][v] < dt) { dt = s.dist[0][v]; t = v; }
+        long long best = kInf;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-              const long long od = __shfl_xor_sync(0xffffffffu, dt, o);
-              const int ot = __shfl_xor_sync(0xffffffffu, t, o);
-              if (od < dt || (od == dt && ot < t)) { dt = od; t = ot; }
-            }
-            if (lane == 0) { s.target = dt < kInf ? t : -1; s.dt = dt; }
-          }
-          __syncthreads();
-          have_paths = s.target >= 0;
-        }
-      }
-    }
-    // ---- Dijkstra from every node with excess (reduced costs rc = cost - p[u] + p[v] are >= 0) ---------
-    if (!have_paths)
-
-    // One warp, nodes spread over its lanes; it stops when the first node with a deficit is settled:
-    // every node still open is at least that far away, which is all the price update needs to know.
-    if (warp == 0) {
-      constexpr int NQ = (kMaxE + 1 + 31) / 32;
-      long long d[NQ]; int pr[NQ]; bool open[NQ];
-#pragma unroll
-      for (int q = 0; q < NQ; ++q) {
-        const int v = lane + 32 * q;
-        open[q] = v <= E;
-        d[q] = (v <= E && s.imb[v] > 0) ? 0 : kInf;
-        pr[q] = -1;
-      }
-      int target = -1; long long dt = kInf;
-      // all nodes with excess start at distance 0: settle them together and relax their arcs in one go
-#pragma unroll
-      for (int q = 0; q < NQ; ++q) if (open[q] && d[q] == 0) open[q] = false;
-      for (int u = 0; u <= E; ++u) {
-        if (s.imb[u] <= 0) continue;
-        const long long pu = s.p[u];
-#pragma unroll
-        for (int q = 0; q < NQ; ++q) {
-          const int v = lane + 32 * q;
-          if (!open[q]) continue;
-          long long rc;
-          if (u < E && v < E) {
-            const long long c = D[u * ES + v];
-            if (c >= kInf) continue;
-            rc = c - pu + s.p[v];
-          } else if (v == nZ) {
-            if (s.flow[u] >= C) continue;
-            rc = -pu + s.p[nZ];
-          } else {
-            if (s.flow[v] <= 0) continue;
-            rc = -pu + s.p[v];
-          }
-          if (rc < 0) rc = 0;
-          if (rc >= kArcLimit) continue;
-          if (rc < d[q]) { d[q] = rc; pr[q] = u; }
-        }
-      }
-      for (int it = 0; it <= E; ++it) {
-        long long best = kInf; int bv = 0x7fffffff;
-#pragma unroll
-        for (int q = 0; q < NQ; ++q)
-          if (open[q] && d[q] < best) { best = d[q]; bv = lane + 32 * q; }
+        for (int q = 0; q < kEPLf; ++q) best = off[q] < best ? off[q] : best;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
           const long long ob = __shfl_xor_sync(0xffffffffu, best, o);
-          const int ov = __shfl_xor_sync(0xffffffffu, bv, o);
-          if (ob < best || (ob == best && ov < bv)) { best = ob; bv = ov; }
+          best = ob < best ? ob : best;
         }
-        if (best >= kInf) break;                       // nothing reachable is left
-        const int u = bv; const long long du = best;
-#pragma unroll
-        for (int q = 0; q < NQ; ++q) if (lane + 32 * q == u) open[q] = false;
-        ++bf_rounds;
-        if (s.imb[u] < 0) { target = u; dt = du; break; }
-        const long long pu = s.p[u];
-#pragma unroll
-        for (int q = 0; q < NQ; ++q) {
-          const int v = lane + 32 * q;
-          if (!open[q]) continue;
-          long long rc;
-          if (u < E && v < E) {
-            const long long c = D[u * ES + v];
-            if (c >= kInf) continue;
-            rc = c - pu + s.p[v];
-          } else if (v == nZ) {          // expert u -> Z: one more unit on u -> sink
-            if (s.flow[u] >= C) continue;
-            rc = -pu + s.p[nZ];
-          } else {                       // Z -> expert v: one unit less on v -> sink
-            if (s.flow[v] <= 0) continue;
-            rc = -pu + s.p[v];
-          }
-          if (rc < 0) rc = 0;            // cannot happen while the potentials are valid
-          if (rc >= kArcLimit) continue;
-          if (du + rc < d[q]) { d[q] = du + rc; pr[q] = u; }
-        }
-      }
-#pragma unroll
-      for (int q = 0; q < NQ; ++q) {
-        const int v = lane + 32 * q;
-        if (v <= E) {
-          // settled nodes keep their distance; open ones are at least dt away
-          s.dist[0][v] = open[q] ? kInf : d[q];
-          s.pred[v] = pr[q];
-        }
-      }
-      if (lane == 0) { s.target = target; s.dt = dt; }
-    }
-    __syncthreads();
-    const int cur = 0;
-    // ---- nearest node with a deficit; would the price update stay within theta? -----------------------
-    if (warp == 0) {
-      const int t = s.target; const long long dt = s.dt;
-      if (lane == 0) s.npath = 0;
-      if (t >= 0) {
         if (lane == 0) {
-          int len = 0, v = t;
-          while (v >= 0 && len <= E + 1) { s.path[len++] = v; v = s.pred[v]; }
-          s.npath = len;
+          const long long old = d0[nZ];
+          if (best < old && best < dtb) {
+            dn[nZ] = best; s.lvl[nZ] = round; changed = true;
+            if (s.imb[nZ] < 0) atomicMin(&s.dtb, best);
+          } else {
+            dn[nZ] = old;
+          }
         }
+      }
+      more = __syncthreads_or(changed);
+      { long long* t = d0; d0 = dn; dn = t; }
+    }
+    // ---- nearest node with a deficit (lowest index on ties); would the price update stay within theta? --
+    // Then the walk back from it, by one warp.  An arc u -> v is eligible when dist[u] + cost == dist[v] and
+    // u's distance was final before v's: such an arc exists for every reached node, and following them
+    // strictly lowers the level, so the walk ends at a node with excess without repeating a node.  Among the
+    // eligible arcs the Z arc wins, then the smallest token index, then the smallest tail: the choice does
+    // not depend on the order of the candidate list.  The offers of the last search round (which changed
+    // nothing) are still in place: an entry whose offer equals its node's distance is a tight arc from the
+    // expert its candidate is reached through; only if that expert's level does not fit are the candidate's
+    // other experts looked at.
+    if (warp == 0) {
+      long long dt = kInf; int t = 0x7fffffff;
+      for (int v = lane; v <= E; v += 32)
+        if (s.imb[v] < 0 && d0[v] < dt) { dt = d0[v]; t = v; }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const long long od = __shfl_xor_sync(0xffffffffu, dt, o);
+        const int ot = __shfl_xor_sync(0xffffffffu, t, o);
+        if (od < dt || (od == dt && ot < t)) { dt = od; t = ot; }
+      }
+      int target = dt < kInf ? t : -1;
+      if (target >= 0) {
         long long lo = kInf, hi = -kInf;
         for (int e = lane; e < E; e += 32) {
-          const long long d = s.dist[cur][e];
-          const long long chg = s.p[e] - (d < dt ? d : dt) - s.p0[e];
+          const long long d = d0[e];
+          const long long chg = s.dp[e] - (d < dt ? d : dt);
           lo = chg < lo ? chg : lo; hi = chg > hi ? chg : hi;
         }
 #pragma unroll
@@ -1433,352 +1354,128 @@ flow_exact_kernel(const float* __restrict__ M, FlowState* st, int32_t* expert_id
           const long long ol = __shfl_xor_sync(0xffffffffu, lo, o), oh = __shfl_xor_sync(0xffffffffu, hi, o);
           lo = ol < lo ? ol : lo; hi = oh > hi ? oh : hi;
         }
-        __syncwarp();
-        if (lane == 0 && theta < kInf && hi - lo > theta) {
-          s.target = -2;                                // stop here; the next round lists more tokens:
-          if (st->theta < 2 * (hi - lo)) st->theta = 2 * (hi - lo);   // enough of them for this price update
+        if (theta < kInf && hi - lo > theta) {
+          target = -2;                                  // stop here; the next round lists more tokens:
+          if (lane == 0 && st->theta < 2 * (hi - lo)) st->theta = 2 * (hi - lo);   // enough of them for this price update
         }
       }
+      int len = 0; bool broken = more != 0;             // a search that never settled is not trusted
+      if (target >= 0 && !broken) {
+        int v = target;
+        while (s.lvl[v] > 0 && len <= E + 1) {
+          unsigned long long code = ~0ULL; int cc = -1;
+          const long long dv = d0[v]; const int lv = s.lvl[v];
+          if (v == nZ) {
+            for (int e = lane; e < E; e += 32) {
+              const long long de = d0[e];
+              if (de < kInf && s.flow[e] < C && s.lvl[e] < lv) {
+                long long rc = -s.p[e] + s.p[nZ]; if (rc < 0) rc = 0;
+                if (de + rc == dv && (unsigned long long)e < code) code = (unsigned long long)e;
+              }
+            }
+          } else {
+            const long long dz = d0[nZ];
+            bool zarc = false;
+            if (dz < kInf && s.flow[v] > 0 && s.lvl[nZ] < lv) {
+              long long rc = -s.p[nZ] + s.p[v]; if (rc < 0) rc = 0;
+              zarc = dz + rc == dv;
+            }
+            if (zarc) {
+              code = (unsigned long long)nZ;
+            } else {
+              for (int idx = s.estart[v] + lane; idx < s.estart[v + 1]; idx += 32) {
+                if (ndv[idx] != dv) continue;
+                const int c = bxc[idx];
+                const unsigned long long tk = ((unsigned long long)(unsigned)rtok[c] + 1ULL) << 8;
+                const int e1 = aarg[c];
+                if (s.lvl[e1] < lv) {
+                  if ((tk | (unsigned long long)e1) < code) { code = tk | (unsigned long long)e1; cc = c; }
+                  continue;
+                }
+                // the offer came through A = min over the candidate's held experts; any of them that attains A
+                // gives a tight arc as well
+                const int o = roff[c], m = rcnt[c];
+                long long Ac = kInf;
+                for (int j = o; j < o + m; ++j) {
+                  const int mj = rmeta[j];
+                  if (!(mj & 256)) continue;
+                  const long long de = d0[mj & 255];
+                  if (de >= kInf) continue;
+                  const long long x = de + (rval[j] - s.dp[mj & 255]);
+                  Ac = x < Ac ? x : Ac;
+                }
+                for (int j = o; j < o + m; ++j) {
+                  const int mj = rmeta[j];
+                  if (!(mj & 256)) continue;
+                  const int e = mj & 255;
+                  const long long de = d0[e];
+                  if (de >= kInf || s.lvl[e] >= lv) continue;
+                  if (de + (rval[j] - s.dp[e]) == Ac && (tk | (unsigned long long)e) < code) { code = tk | (unsigned long long)e; cc = c; }
+                }
+              }
+            }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long oc = __shfl_xor_sync(0xffffffffu, code, o);
+            const int occ = __shfl_xor_sync(0xffffffffu, cc, o);
+            if (oc < code) { code = oc; cc = occ; }
+          }
+          if (code == ~0ULL) { broken = true; break; }    // internal inconsistency: stop, the check pass will report it
+          const int u = (int)(code & 255ULL);
+          if (lane == 0) { s.path_v[len] = v; s.path_u[len] = u; s.path_tok[len] = (int)(code >> 8) - 1; s.path_c[len] = cc; }
+          ++len; v = u;
+        }
+        if (!broken && (s.lvl[v] > 0 || s.imb[v] <= 0)) broken = true;
+        if (!broken && lane == 0) { s.imb[v] -= 1; s.imb[target] += 1; }
+      }
+      if (lane == 0) { s.target = target; s.dt = dt; s.npath = len; if (broken) s.stop = 1; }
     }
     __syncthreads();
-    { const long long t1 = clock64(); t_bf += t1 - t0; t0 = t1; }
+    if (s.stop) { if (tid == 0) atomicOr(&st->status, 4u); break; }
     if (s.target < 0) break;        // -1: no augmenting path inside the candidate graph
+    const long long dt = s.dt;
+    // ---- move one unit along the path ------------------------------------------------------------------
+    const int L = s.npath;
     for (int v = tid; v <= E; v += blockDim.x) {
-      const long long d = s.dist[cur][v];
-      s.p[v] -= (d < s.dt ? d : s.dt);
+      const long long d = d0[v];
+      const long long step = d < dt ? d : dt;
+      s.p[v] -= step; s.dp[v] -= step;
     }
-    __syncthreads();
-    // ---- push one unit along the path (stored target first) ------------------------------------------
-    // All arcs of the path at once: (W) every thread looks up, for its candidates, which arcs they are
-    // the cheapest token of; (P) one warp per arc patches D from that token's keys and lists the entries
-    // that became stale; (F) one pass recomputes the listed entries.  The path's nodes are distinct, so
-    // arcs touch different (row, column) pairs except where a min-update is used.  If one token is the
-    // cheapest of two arcs the arcs are taken one by one instead (below).
-    auto fix_pass = [&]() {
-        if (s.nfix > 0 && n <= kHeldCache) {
-          // recompute the listed entries: candidates that hold one of the listed rows are queued by one
-          // thread each; a warp then takes a queued candidate with its lanes spread over the entries,
-          // so that the loads of one candidate are in flight together
-          const int nfix = s.nfix;
-          for (int e = tid; e < E; e += blockDim.x) s.fixrow[e] = 0;
-          if (tid == 0) s.qn = 0;
-          __syncthreads();
-          if (tid < nfix) s.fixrow[s.fix_e[tid]] = 1;
-          __syncthreads();
-          for (int c0 = 0; c0 < n; c0 += blockDim.x) {
-            const int c = c0 + tid;
-            bool any = false;
-            if (c < n)
-              for (int j = 0; j < k; ++j) any |= (s.fixrow[held_s[c * kMaxK + j]] != 0);
-            const unsigned mask = __ballot_sync(0xffffffffu, any);
-            int base = 0;
-            if (lane == 0 && mask) base = atomicAdd(&s.qn, __popc(mask));
-            base = __shfl_sync(0xffffffffu, base, 0);
-            if (any) queue_s[base + __popc(mask & ((1u << lane) - 1u))] = c;
-          }
-          __syncthreads();
-          const int qn = s.qn;
-          for (int qi = warp; qi < qn; qi += kP2Threads / 32) {
-            const int c = queue_s[qi];
-            const int tok = cand_s[c];
-            int h[kMaxK];
-#pragma unroll
-            for (int j = 0; j < kMaxK; ++j) h[j] = j < k ? (int)held_s[c * kMaxK + j] : -1;
-            const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-            for (int i = lane; i < nfix; i += 32) {
-              const int e = s.fix_e[i], f = s.fix_f[i];
-              bool he = false, hf = false;
-#pragma unroll
-              for (int j = 0; j < kMaxK; ++j) { he |= (h[j] == e); hf |= (h[j] == f); }
-              if (!he || hf) continue;
-              const long long cst = make_key(g, __ldg(M + (size_t)tok * E + e), flat + e) -
-                                    make_key(g, __ldg(M + (size_t)tok * E + f), flat + f);
-              if (cst - s.p[e] + s.p[f] <= arc_window && cst < D[e * ES + f]) atomicMin(&D[e * ES + f], cst);
-            }
-          }
-          __syncthreads();
-        } else if (s.nfix > 0) {
-          // one thread per candidate (lists longer than the shared-memory mirror)
-          for (int c = tid; c < n; c += blockDim.x) {
-            const int tok = tok_of(c);
-            int h[kMaxK];
-#pragma unroll
-            for (int j = 0; j < kMaxK; ++j) h[j] = j < k ? held_of(c, tok, j) : -1;
-            const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-            for (int i = 0; i < s.nfix; ++i) {
-              const int e = s.fix_e[i], f = s.fix_f[i];
-              bool he = false, hf = false;
-#pragma unroll
-              for (int j = 0; j < kMaxK; ++j) { he |= (h[j] == e); hf |= (h[j] == f); }
-              if (!he || hf) continue;
-              const long long cst = make_key(g, __ldg(M + (size_t)tok * E + e), flat + e) -
-                                    make_key(g, __ldg(M + (size_t)tok * E + f), flat + f);
-              if (cst - s.p[e] + s.p[f] <= arc_window && cst < D[e * ES + f]) atomicMin(&D[e * ES + f], cst);
-            }
-          }
-          __syncthreads();
+    for (int a = tid; a < L; a += blockDim.x) {
+      const int u = s.path_u[a], v = s.path_v[a], tok = s.path_tok[a];
+      if (tok >= 0) {
+        const int c = s.path_c[a];
+        const int o = roff[c], m = rcnt[c];
+        for (int i = o; i < o + m; ++i) {
+          const int e = rmeta[i] & 255;
+          if (e == u) rmeta[i] = (unsigned short)u;             // given up
+          if (e == v) rmeta[i] = (unsigned short)(v | 256);     // taken
         }
-    };
-    bool batched = false;
-    {
-      const int L = s.npath - 1;
-      long long ta = clock64();
-      for (int a = tid; a <= L; a += blockDim.x) s.who_a[a] = 0x7fffffff;
-      if (tid == 0) { s.dup = 0; s.nfix = 0; }
-      __syncthreads();
-      for (int c = tid; c < n; c += blockDim.x) {
-        const int tok = tok_of(c);
-        unsigned hm[4] = {0, 0, 0, 0};
-        for (int j = 0; j < k; ++j) { const int e = held_of(c, tok, j); hm[e >> 5] |= 1u << (e & 31); }
-        const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-        for (int a = L; a >= 1; --a) {
-          const int u = s.path[a], v = s.path[a - 1];
-          if (u >= E || v >= E) continue;
-          if (!((hm[u >> 5] >> (u & 31)) & 1u) || ((hm[v >> 5] >> (v & 31)) & 1u)) continue;
-          const long long cost = make_key(g, __ldg(M + (size_t)tok * E + u), flat + u) -
-                                 make_key(g, __ldg(M + (size_t)tok * E + v), flat + v);
-          if (cost == D[u * ES + v]) atomicMin(&s.who_a[a], c);    // sorted list: smallest c = smallest token
-        }
-      }
-      __syncthreads();
-      for (int idx = tid; idx < L * L; idx += blockDim.x) {
-        const int i = idx / L + 1, j = idx - (i - 1) * L + 1;
-        if (i < j && s.who_a[i] != 0x7fffffff && s.who_a[i] == s.who_a[j]) s.dup = 1;
-      }
-      __syncthreads();
-      batched = !s.dup;
-      { const long long tb = clock64(); t_who += tb - ta; ta = tb; }
-      if (batched) {
-        n_arcs += L;
-        for (int a = L - warp; a >= 1; a -= kP2Threads / 32) {
-          const int u = s.path[a], v = s.path[a - 1];
-          if (u >= E || v >= E) continue;
-          const int c = s.who_a[a];
-          if (c == 0x7fffffff) { if (lane == 0) { atomicOr(&st->status, 4u); s.stop = 1; } continue; }
-          const int tok = tok_of(c);
-          int h[kMaxK];
-#pragma unroll
-          for (int j = 0; j < kMaxK; ++j) {
-            h[j] = j < k ? held_of(c, tok, j) : -1;
-            if (h[j] == u) h[j] = v;                   // experts after the move
-          }
-          const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-          long long key[kEPLf]; bool in[kEPLf];
-#pragma unroll
-          for (int q = 0; q < kEPLf; ++q) {
-            const int f = lane + 32 * q;
-            key[q] = f < E ? make_key(g, __ldg(M + (size_t)tok * E + f), flat + f) : 0;
-            bool hd = f >= E;
-#pragma unroll
-            for (int j = 0; j < kMaxK; ++j) hd |= (h[j] == f);
-            in[q] = hd;
-          }
-          auto key_of = [&](int e) -> long long {
-            long long mine = 0;
-#pragma unroll
-            for (int q = 0; q < kEPLf; ++q) if ((e >> 5) == q) mine = key[q];
-            return __shfl_sync(0xffffffffu, mine, e & 31);
-          };
-          const long long ku = key_of(u), kv = key_of(v);
-#pragma unroll
-          for (int q = 0; q < kEPLf; ++q) {
-            const int f = lane + 32 * q;
-            if (!in[q]) {                               // row v gains the token
-              const long long cst = kv - key[q];
-              if (cst - s.p[v] + s.p[f] <= arc_window && cst < D[v * ES + f]) atomicMin(&D[v * ES + f], cst);
-            }
-            const bool was_out = f < E && f != u && (!in[q] || f == v);
-            if (was_out && D[u * ES + f] == ku - key[q]) {      // the token's own offer from u is gone
-              const int slot = atomicAdd(&s.nfix, 1);
-              if (slot < kMaxFix) { s.fix_e[slot] = u; s.fix_f[slot] = f; }
-            }
-          }
-#pragma unroll
-          for (int j = 0; j < kMaxK; ++j) {
-            if (j >= k || h[j] == v) continue;
-            const int gg = h[j];
-            const long long kg = key_of(gg);
-            if (lane == 0) {
-              if (kg - ku - s.p[gg] + s.p[u] <= arc_window && kg - ku < D[gg * ES + u]) atomicMin(&D[gg * ES + u], kg - ku);
-              if (D[gg * ES + v] == kg - kv) {
-                const int slot = atomicAdd(&s.nfix, 1);
-                if (slot < kMaxFix) { s.fix_e[slot] = gg; s.fix_f[slot] = v; }
-              }
-            }
-          }
-          __syncwarp();
-          if (lane == 0)
-            for (int j = 0; j < k; ++j)
-              if (held_of(c, tok, j) == u) {
-                if (c < nc) held_s[c * kMaxK + j] = (unsigned char)v;
-                expert_idx[(size_t)tok * k + j] = v;
-              }
-        }
-        if (tid == 0)
-          for (int a = L; a >= 1; --a) {
-            const int u = s.path[a], v = s.path[a - 1];
-            if (u < E && v < E) continue;
-            if (v == nZ) s.flow[u] += 1; else s.flow[v] -= 1;
-          }
-        __syncthreads();
-        if (s.nfix > kMaxFix) {
-          // too many stale entries: rebuild the rows they sit in.  The tokens have moved already, so a
-          // token's other experts are what it holds now, minus the arc's target
-          for (int a = L - warp; a >= 1; a -= kP2Threads / 32) {
-            const int u = s.path[a], v = s.path[a - 1];
-            if (u >= E || v >= E || lane != 0) continue;
-            const int c = s.who_a[a];
-            if (c == 0x7fffffff) continue;
-            const int tok = tok_of(c);
-            s.dirty[u] = 1;
-            for (int j = 0; j < k; ++j) { const int e = held_of(c, tok, j); if (e != v) s.dirty[e] = 1; }
-          }
-          __syncthreads();
-          if (tid == 0) s.nfix = 0;
-        } else {
-          for (int i = tid; i < s.nfix; i += blockDim.x) D[s.fix_e[i] * ES + s.fix_f[i]] = kInf;
-        }
-        __syncthreads();
-        { const long long tb = clock64(); t_patch += tb - ta; ta = tb; }
-        fix_pass();
-        t_fix += clock64() - ta;
+        for (int j = 0; j < k; ++j)
+          if (expert_idx[(size_t)tok * k + j] == u) expert_idx[(size_t)tok * k + j] = v;
+      } else if (v == nZ) {
+        atomicAdd(&s.flow[u], 1);
+      } else {
+        atomicAdd(&s.flow[v], -1);
       }
     }
-    if (!batched)
-    for (int a = s.npath - 1; a >= 1; --a) {
-      const int u = s.path[a], v = s.path[a - 1];
-      if (u < E && v < E) {
-        long long ta = clock64(); ++n_arcs;
-        if (tid == 0) s.who = 0x7fffffff;
-        __syncthreads();
-        const long long want = D[u * ES + v];
-        for (int c = tid; c < n; c += blockDim.x) {
-          const int tok = tok_of(c);
-          bool hu = false, hv = false;
-          for (int j = 0; j < k; ++j) {
-            const int e = held_of(c, tok, j);
-            hu |= (e == u); hv |= (e == v);
-          }
-          if (!hu || hv) continue;
-          const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-          const long long cost = make_key(g, __ldg(M + (size_t)tok * E + u), flat + u) -
-                                 make_key(g, __ldg(M + (size_t)tok * E + v), flat + v);
-          if (cost == want) atomicMin(&s.who, c);      // the list is sorted: smallest c = smallest token
-        }
-        __syncthreads();
-        if (s.who == 0x7fffffff) {   // internal inconsistency: stop, the verify pass will report it
-          if (tid == 0) { atomicOr(&st->status, 4u); s.stop = 1; }
-          __syncthreads();
-          break;
-        }
-        { const long long tb = clock64(); t_who += tb - ta; ta = tb; }
-        if (warp == 0) {
-          // the token leaves u for v: patch D from its own keys instead of rebuilding every row it touches
-          const int c = s.who, tok = tok_of(c);
-          int h[kMaxK];
-#pragma unroll
-          for (int j = 0; j < kMaxK; ++j) {
-            h[j] = j < k ? held_of(c, tok, j) : -1;
-            if (h[j] == u) h[j] = v;                   // experts after the move
-          }
-          const uint32_t flat = (uint32_t)tok * (uint32_t)E;
-          long long key[kEPLf]; bool in[kEPLf];
-#pragma unroll
-          for (int q = 0; q < kEPLf; ++q) {
-            const int f = lane + 32 * q;
-            key[q] = f < E ? make_key(g, __ldg(M + (size_t)tok * E + f), flat + f) : 0;
-            bool hd = f >= E;
-#pragma unroll
-            for (int j = 0; j < kMaxK; ++j) hd |= (h[j] == f);
-            in[q] = hd;
-          }
-          auto key_of = [&](int e) -> long long {
-            long long mine = 0;
-#pragma unroll
-            for (int q = 0; q < kEPLf; ++q) if ((e >> 5) == q) mine = key[q];
-            return __shfl_sync(0xffffffffu, mine, e & 31);
-          };
-          const long long ku = key_of(u), kv = key_of(v);
-          // row v gains the token: new moves v -> f for every expert f it does not hold
-#pragma unroll
-          for (int q = 0; q < kEPLf; ++q) {
-            const int f = lane + 32 * q;
-            if (!in[q]) {
-              const long long cst = kv - key[q];
-              if (cst - s.p[v] + s.p[f] <= arc_window && cst < D[v * ES + f]) D[v * ES + f] = cst;
-            }
-          }
-          // D entries whose cheapest move was this token's become stale: (u, f) for the experts f it
-          // offered from u, and (g, v) for its other experts g.  They are listed and recomputed below
-          // from the candidates that hold the row's expert; a full row rebuild is the fallback.
-          if (lane == 0) s.nfix = 0;
-          __syncwarp();
-#pragma unroll
-          for (int q = 0; q < kEPLf; ++q) {
-            const int f = lane + 32 * q;
-            // before the move the token held u and not f (f != v is covered by in[], v itself is the used arc)
-            const bool was_out = f < E && f != u && (!in[q] || f == v);
-            if (was_out && D[u * ES + f] == ku - key[q]) {
-              const int slot = atomicAdd(&s.nfix, 1);
-              if (slot < kMaxFix) { s.fix_e[slot] = u; s.fix_f[slot] = f; }
-            }
-          }
-#pragma unroll
-          for (int j = 0; j < kMaxK; ++j) {
-            if (j >= k || h[j] == v) continue;
-            const int gg = h[j];
-            const long long kg = key_of(gg);
-            if (lane == 0) {
-              if (kg - ku - s.p[gg] + s.p[u] <= arc_window && kg - ku < D[gg * ES + u]) D[gg * ES + u] = kg - ku;   // g -> u is a new move
-              if (D[gg * ES + v] == kg - kv) {                            // g -> v is gone
-                const int slot = atomicAdd(&s.nfix, 1);
-                if (slot < kMaxFix) { s.fix_e[slot] = gg; s.fix_f[slot] = v; }
-              }
-            }
-          }
-          __syncwarp();
-          if (lane == 0) {
-            if (s.nfix > kMaxFix) {                    // too many: rebuild the rows instead
-              s.dirty[u] = 1;
-              for (int j = 0; j < k; ++j) if (h[j] != v) s.dirty[h[j]] = 1;
-              s.nfix = 0;
-            }
-            for (int j = 0; j < k; ++j) {
-              const int e = held_of(c, tok, j);
-              if (e == u) {
-                if (c < nc) held_s[c * kMaxK + j] = (unsigned char)v;
-                expert_idx[(size_t)tok * k + j] = v;
-              }
-            }
-          }
-          __syncwarp();
-          for (int i = lane; i < s.nfix; i += 32) D[s.fix_e[i] * ES + s.fix_f[i]] = kInf;
-        }
-        __syncthreads();
-        { const long long tb = clock64(); t_patch += tb - ta; ta = tb; }
-        fix_pass();
-        t_fix += clock64() - ta;
-      } else if (tid == 0) {
-        if (v == nZ) s.flow[u] += 1; else s.flow[v] -= 1;
-      }
-    }
-    if (s.stop) break;
-    if (tid == 0) { s.imb[s.path[s.npath - 1]] -= 1; s.imb[s.target] += 1; }
     ++naug;
     __syncthreads();
-    { const long long t1 = clock64(); t_move += t1 - t0; t0 = t1; }
   }
   // ---- write back ---------------------------------------------------------------------------------
   __syncthreads();
+  if (tid == 0) s.dt = 0;
+  __syncthreads();
   for (int e = tid; e < E; e += blockDim.x) {
     long long pe = s.p[e] - s.p[nZ];
-    st->p[e] = pe < 0 ? 0 : pe;     // only an expert that holds nothing can come out negative
+    pe = pe < 0 ? 0 : pe;           // only an expert that holds nothing can come out negative
+    st->p[e] = pe;
+    if (s.p0[e] - pe > 0) atomicMax(&s.dt, s.p0[e] - pe);
   }
-  if (tid == 0) {
-    st->naug += naug; st->ncand_last = n; st->ncand = 0;
-    st->trace[44] = (int)(t_rebuild >> 10); st->trace[45] = (int)(t_bf >> 10); st->trace[46] = (int)(t_move >> 10); st->trace[47] = bf_rounds; st->trace[41] = (int)q_total; st->trace[42] = (int)(t_first >> 10);   // kilo-cycles
-    st->trace[34] = (int)(t_who >> 10); st->trace[35] = (int)(t_patch >> 10); st->trace[36] = (int)(t_fix >> 10); st->trace[37] = n_arcs;
-  }
+  __syncthreads();
+  // the caches' bounds on uncached experts must keep up with prices that fell during this round
+  if (tid == 0) { st->cumdrop += s.dt; st->naug += naug; st->ncand_last = n; st->ncand = 0; st->nrec = 0; }
 }
 
 }  // namespace msr

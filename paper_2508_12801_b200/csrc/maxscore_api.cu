@@ -50,8 +50,9 @@ int32_t capacity_of(const maxscore_params& p) {
 }
 
 struct Layout {          // byte offsets inside the workspace
-  size_t state, aux, cand, dmat, cache_x, cache_id, cache_bound, block_counts, wt, error_flag, dls, wk, dwpart, total;
+  size_t state, aux, cand, rec_val, rec_meta, rec_pos, rec_bxc, rec_ndv, rec_off, rec_cnt, rec_aarg, cache_x, cache_id, cache_bound, cache_raw, block_counts, wt, error_flag, dls, wk, dwpart, total;
   int Npad, n_idx_blocks;
+  int rec_cap;                                // entries of the exact phase's candidate records
   int Kpad, dw_splits, dw_tokens_per_split;   // tensor-core backward GEMMs (bf16 I/O)
 };
 
@@ -64,10 +65,24 @@ Layout layout_of(const maxscore_params& p) {
   l.error_flag = off; off = align_up(off + 16, 256);
   l.aux = off; off = align_up(off + sizeof(double) * kMaxE + 16, 256);     // column sums + ticket of the auxiliary loss
   l.cand = off; off = align_up(off + sizeof(int32_t) * (size_t)p.T, 256);
-  l.dmat = off; off = align_up(off + sizeof(long long) * (size_t)p.E * (p.E | 1), 256);
+  {   // candidate records of the exact phase: room for every (token, expert) pair, which the last, unbounded round
+      // of a heavily tied problem can need (26 bytes each); beyond 2^21 entries the list is cut short
+    long long cap = (long long)p.T * p.E;
+    if (cap > (1LL << 21)) cap = 1LL << 21;
+    l.rec_cap = (int)cap;
+  }
+  l.rec_val = off; off = align_up(off + sizeof(long long) * (size_t)l.rec_cap, 256);
+  l.rec_meta = off; off = align_up(off + sizeof(unsigned short) * (size_t)l.rec_cap, 256);
+  l.rec_pos = off; off = align_up(off + sizeof(int32_t) * (size_t)l.rec_cap, 256);
+  l.rec_bxc = off; off = align_up(off + sizeof(int32_t) * (size_t)l.rec_cap, 256);
+  l.rec_ndv = off; off = align_up(off + sizeof(long long) * (size_t)l.rec_cap, 256);
+  l.rec_off = off; off = align_up(off + sizeof(int32_t) * (size_t)p.T, 256);
+  l.rec_cnt = off; off = align_up(off + sizeof(int32_t) * (size_t)p.T, 256);
+  l.rec_aarg = off; off = align_up(off + sizeof(int32_t) * (size_t)p.T, 256);
   l.cache_x = off; off = align_up(off + sizeof(float) * (size_t)kCacheN * p.T, 256);
   l.cache_id = off; off = align_up(off + (size_t)kCacheN * p.T, 256);
   l.cache_bound = off; off = align_up(off + sizeof(long long) * (size_t)p.T, 256);
+  l.cache_raw = off; off = align_up(off + (size_t)p.T, 256);
   l.block_counts = off; off = align_up(off + sizeof(int32_t) * (size_t)l.n_idx_blocks * p.E, 1024);
   l.wt = off;
   off = align_up(off + (p.io_dtype == MAXSCORE_BF16 ? sizeof(__nv_bfloat16) * (size_t)l.Npad * p.d_model : 0), 1024);
@@ -119,7 +134,6 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-constexpr int kP2SmemMax = (int)(sizeof(long long) * kMaxE * (kMaxE | 1) + kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache + 2 * kMaxArcs);
 constexpr int kDhSmemMax = 2 * 2 * 16384 + kDhStages * 2 * 16384 + kDhOutBytes + 1024;     // Kpad = 128
 constexpr int kDwSmemMax = kDwStages * (16384 + 2 * 2 * 8192) + 1024;
 
@@ -132,6 +146,8 @@ struct maxscore_ctx {
   char* ws;
   EncodeTiledFn encode;
   int sm_count;
+  int sweep_grid_max;   // CTAs of the sweeps kernel that are resident at once
+  long long launches;   // kernels launched through this context so far
 };
 
 namespace {
@@ -177,6 +193,7 @@ maxscore_status launch_gate(maxscore_ctx* c, const void* hidden, const void* w_g
     gate_gemm_simt_kernel<float><<<grid, 256, 0, st>>>((const float*)hidden, (const float*)w_gate, bias, logits,
                                                         p.T, p.d_model, p.E, p.w_gate_layout);
     MS_LAUNCH_CHECK("gate_gemm_simt_kernel");
+    c->launches += 1;
     return MAXSCORE_OK;
   }
   __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(c->ws + c->lay.wt);
@@ -196,6 +213,7 @@ maxscore_status launch_gate(maxscore_ctx* c, const void* hidden, const void* w_g
   gate_gemm_tc_kernel<<<(p.T + kGateBM - 1) / kGateBM, 128, kGateSmemBytes, st>>>(tmH, tmW, bias, logits, p.T, p.E,
                                                                                    Npad, num_kb, error_flag_of(c));
   MS_LAUNCH_CHECK("gate_gemm_tc_kernel");
+  c->launches += 2;
   return MAXSCORE_OK;
 }
 
@@ -208,6 +226,7 @@ maxscore_status launch_softtopk_fwd(maxscore_ctx* c, const float* logits, float*
   else
     softtopk_fwd_kernel<<<blocks, 256, 0, st>>>(logits, scores, p.T, p.E, p.k, p.t);
   MS_LAUNCH_CHECK("softtopk_fwd_kernel");
+  c->launches += 1;
   return MAXSCORE_OK;
 }
 
@@ -218,44 +237,51 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   const maxscore_params& p = c->p;
   FlowState* fs = reinterpret_cast<FlowState*>(c->ws + c->lay.state);
   int32_t* cand = reinterpret_cast<int32_t*>(c->ws + c->lay.cand);
-  const KeyGen g = keygen_of(c);
+  KeyGen g = keygen_of(c);
   const int scale_bits = p.score_mode == 0 ? 40 : g.S + p.quant_shift;   // log2 of one unit of score
-  const long long eps0 = 1LL << (scale_bits - 10);
-  const long long eps_min = p.score_mode == 0 ? (1LL << 20) : (1LL << 12);
-  const int cap0 = kCapLogMax;   // the first sweep records every margin
-  const long long theta0 = 1LL << (scale_bits - 15);
-  const int balanced = ((long long)p.E * c->C == (long long)p.T * p.k) ? 1 : 0;
   const int budget = p.max_sweeps > 0 ? p.max_sweeps : kSweeps + kDefaultAug;
-  const int n_sweeps = budget < kSweeps ? budget : kSweeps;
-  const int max_aug = budget - n_sweeps;
+  SweepArgs a{};
+  a.T = p.T; a.E = p.E; a.k = p.k; a.C = c->C;
+  a.n_sweeps = budget < kSweeps ? budget : kSweeps;
+  a.balanced = ((long long)p.E * c->C == (long long)p.T * p.k) ? 1 : 0;
+  a.eps0 = 1LL << (scale_bits - 10);
+  a.eps_min = p.score_mode == 0 ? (1LL << 20) : (1LL << 12);
+  a.theta0 = 1LL << (scale_bits - 15);
+  int max_aug = budget - a.n_sweeps;
 
-  flow_init_kernel<<<32, 256, 0, st>>>(fs, eps0, eps_min, cap0, theta0, balanced, p.E);
+  flow_init_kernel<<<32, 256, 0, st>>>(fs, kCapLogMax, a.theta0, a.balanced, p.E);
   MS_LAUNCH_CHECK("flow_init_kernel");
-  const int blocks = (p.T + kSweepThreads - 1) / kSweepThreads;
   SweepCache cache{reinterpret_cast<float*>(c->ws + c->lay.cache_x), reinterpret_cast<unsigned char*>(c->ws + c->lay.cache_id),
-                   reinterpret_cast<long long*>(c->ws + c->lay.cache_bound)};
-  for (int s = 0; s < n_sweeps; ++s) {
-    if (s == 0) flow_sweep_kernel<true><<<blocks, kSweepThreads, 0, st>>>(M, fs, cache, p.T, p.E, p.k, c->C, g, s);
-    else flow_sweep_kernel<false><<<blocks, kSweepThreads, 0, st>>>(M, fs, cache, p.T, p.E, p.k, c->C, g, s);
-    flow_price_kernel<<<1, kPriceThreads, 0, st>>>(fs, p.E, c->C, n_sweeps, 1, s);
-    MS_LAUNCH_CHECK("flow_sweep_kernel");
+                   reinterpret_cast<long long*>(c->ws + c->lay.cache_bound), reinterpret_cast<unsigned char*>(c->ws + c->lay.cache_raw)};
+  const int warp_blocks = std::min((p.T + 7) / 8, c->sm_count * 8);       // kernels that give a warp to each token
+  flow_scan_kernel<<<warp_blocks, 256, 0, st>>>(M, fs, cache, p.T, p.E, g);
+  MS_LAUNCH_CHECK("flow_scan_kernel");
+  {
+    // cooperative launch: every CTA of the grid is resident, which the grid-wide barriers rely on
+    int grid = std::min((p.T + kSwThreads - 1) / kSwThreads, c->sweep_grid_max);
+    if (grid < 1) grid = 1;
+    void* args[] = {(void*)&M, (void*)&fs, (void*)&cache, (void*)&expert_idx, (void*)&cand, (void*)&a, (void*)&g};
+    MS_CUDA(cudaLaunchCooperativeKernel((const void*)flow_sweeps_kernel, dim3(grid), dim3(kSwThreads), args, 0, st));
   }
-  const size_t p2smem = sizeof(long long) * (size_t)p.E * (p.E | 1) + (size_t)kHeldCache * kMaxK + 2 * sizeof(int) * kHeldCache + 2 * kMaxArcs;
-  long long* Dg = reinterpret_cast<long long*>(c->ws + c->lay.dmat);
+  Records rec{reinterpret_cast<long long*>(c->ws + c->lay.rec_val), reinterpret_cast<unsigned short*>(c->ws + c->lay.rec_meta),
+              reinterpret_cast<int*>(c->ws + c->lay.rec_off), reinterpret_cast<int*>(c->ws + c->lay.rec_cnt),
+              reinterpret_cast<int*>(c->ws + c->lay.rec_pos), reinterpret_cast<int*>(c->ws + c->lay.rec_bxc),
+              reinterpret_cast<long long*>(c->ws + c->lay.rec_ndv), reinterpret_cast<int*>(c->ws + c->lay.rec_aarg), c->lay.rec_cap};
   const int build_blocks = c->sm_count * 4;
-  const int collect_blocks = std::min((p.T + kSweepThreads / 32 - 1) / (kSweepThreads / 32), c->sm_count * 16);   // one warp per token
+  const int check_blocks = std::min((p.T + 255) / 256, c->sm_count * 8);
   for (int r = 0; r < kRounds; ++r) {
-    flow_collect_kernel<<<collect_blocks, kSweepThreads, 0, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, r == 0, 0,
-                                                         4LL, nullptr, nullptr, nullptr, r == kRounds - 1, Dg);
-    MS_LAUNCH_CHECK("flow_collect_kernel");
-    flow_build_kernel<<<build_blocks, 256, 0, st>>>(M, fs, expert_idx, cand, Dg, p.T, p.E, p.k, g);
-    MS_LAUNCH_CHECK("flow_build_kernel");
-    flow_exact_kernel<<<1, kP2Threads, p2smem, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, max_aug, Dg);
+    flow_records_kernel<<<build_blocks, 256, 0, st>>>(M, fs, expert_idx, cand, rec, p.T, p.E, p.k, g);
+    MS_LAUNCH_CHECK("flow_records_kernel");
+    flow_exact_kernel<true><<<1, kP2Threads, kRecSmemBytes, st>>>(fs, expert_idx, cand, rec, p.T, p.E, p.k, c->C, max_aug);
+    flow_exact_kernel<false><<<1, kP2Threads, 0, st>>>(fs, expert_idx, cand, rec, p.T, p.E, p.k, c->C, max_aug);
     MS_LAUNCH_CHECK("flow_exact_kernel");
+    flow_check_kernel<<<check_blocks, 256, 0, st>>>(M, fs, cache, expert_idx, cand, p.T, p.E, p.k, c->C, g, r == kRounds - 1,
+                                                   r == kRounds - 2, expert_load, stats, error_flag_of(c));
+    MS_LAUNCH_CHECK("flow_check_kernel");
   }
-  flow_collect_kernel<<<collect_blocks, kSweepThreads, 0, st>>>(M, fs, expert_idx, cand, p.T, p.E, p.k, c->C, g, 0, 1, 32LL,
-                                                       expert_load, stats, error_flag_of(c), 0, nullptr);
-  MS_LAUNCH_CHECK("flow_collect_kernel(verify)");
+  // the last check pass has folded the internal-error flag into stats.status: start the next call clean
+  MS_CUDA(cudaMemsetAsync(error_flag_of(c), 0, sizeof(unsigned), st));
+  c->launches += 3 + 4 * kRounds;
   return MAXSCORE_OK;
 }
 
@@ -269,6 +295,7 @@ maxscore_status launch_index_build(maxscore_ctx* c, const int32_t* expert_idx, i
   index_fill_kernel<<<c->lay.n_idx_blocks, kIdxTok, 0, st>>>(expert_idx, bc, slot_idx, slot_token, expert_load, p.T,
                                                             p.E, p.k, c->C);
   MS_LAUNCH_CHECK("index_fill_kernel");
+  c->launches += 2;
   return MAXSCORE_OK;
 }
 
@@ -286,6 +313,7 @@ maxscore_status launch_zero_padding(maxscore_ctx* c, const int32_t* slot_token, 
   int blocks = (int)((n_slots + 7) / 8); if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
   zero_padding_kernel<<<blocks, 256, 0, st>>>(slot_token, (char*)dst, n_slots, (uint32_t)(c->p.d_model * elem_bytes(c)));
   MS_LAUNCH_CHECK("zero_padding_kernel");
+  c->launches += 1;
   return MAXSCORE_OK;
 }
 
@@ -329,15 +357,24 @@ maxscore_status maxscore_create(maxscore_ctx** out, const maxscore_params* param
     return MAXSCORE_ERR_CUDA;
   }
   MS_CUDA(cudaFuncSetAttribute(gate_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGateSmemBytes));
-  MS_CUDA(cudaFuncSetAttribute(flow_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kP2SmemMax));
+  MS_CUDA(cudaFuncSetAttribute(flow_exact_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRecSmemBytes));
   MS_CUDA(cudaFuncSetAttribute(gate_bwd_dh_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDhSmemMax));
   MS_CUDA(cudaFuncSetAttribute(gate_bwd_dw_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDwSmemMax));
+  int coop = 0, sweep_occ = 0;
+  MS_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+  MS_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&sweep_occ, flow_sweeps_kernel, kSwThreads, 0));
+  if (!coop || sweep_occ < 1) {
+    snprintf(g_last_error, sizeof(g_last_error), "the device cannot launch the cooperative sweeps kernel");
+    return MAXSCORE_ERR_CUDA;
+  }
   MS_CUDA(cudaMemsetAsync(workspace, 0, lay.cand, 0));
   MS_CUDA(cudaStreamSynchronize(0));
   maxscore_ctx* c = new (std::nothrow) maxscore_ctx();
   if (!c) return MAXSCORE_ERR_INVALID_ARG;
   c->p = *params; c->C = capacity_of(*params); c->lay = lay; c->ws = static_cast<char*>(workspace);
   c->encode = reinterpret_cast<EncodeTiledFn>(fn); c->sm_count = sms;
+  c->sweep_grid_max = sms * sweep_occ;
+  c->launches = 0;
   *out = c;
   return MAXSCORE_OK;
 }
@@ -367,6 +404,7 @@ maxscore_status maxscore_softtopk_bwd(maxscore_ctx* c, const float* logits, cons
   else
     softtopk_bwd_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, nullptr, dlogits, p.T, p.E, p.k, p.t);
   MS_LAUNCH_CHECK("softtopk_bwd_kernel");
+  c->launches += 1;
   return MAXSCORE_OK;
 }
 
@@ -381,6 +419,7 @@ maxscore_status maxscore_softtopk_bwd_aux(maxscore_ctx* c, const float* logits, 
   else
     softtopk_bwd_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, dscores_col, dlogits, p.T, p.E, p.k, p.t);
   MS_LAUNCH_CHECK("softtopk_bwd_kernel");
+  c->launches += 1;
   return MAXSCORE_OK;
 }
 
@@ -393,6 +432,7 @@ maxscore_status maxscore_aux_loss(maxscore_ctx* c, const float* scores, const in
   int blocks = (p.T + 7) / 8; if (blocks > c->sm_count * 4) blocks = c->sm_count * 4;
   aux_loss_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>(scores, expert_load, colsum, ticket, loss, dscores_col, p.T, p.E, lambda);
   MS_LAUNCH_CHECK("aux_loss_kernel");
+  c->launches += 1;
   return MAXSCORE_OK;
 }
 
@@ -431,6 +471,7 @@ maxscore_status maxscore_route_fwd(maxscore_ctx* c, const void* hidden, const vo
   int blocks = (int)((n + 255) / 256); if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
   gather_gate_w_kernel<<<blocks, 256, 0, st>>>(scores, expert_idx, gate_w, n, c->p.E, c->p.k);
   MS_LAUNCH_CHECK("gather_gate_w_kernel");
+  c->launches += 1;
   return MAXSCORE_OK;
 }
 
@@ -443,6 +484,7 @@ maxscore_status maxscore_dispatch(maxscore_ctx* c, const void* src, const int32_
   const uint32_t row_bytes = (uint32_t)(p.d_model * elem_bytes(c));
   dispatch_kernel<<<c->sm_count * 8, 256, 0, st>>>((const char*)src, expert_idx, slot_idx, (char*)dst, p.T, row_bytes, p.k, c->C);
   MS_LAUNCH_CHECK("dispatch_kernel");
+  c->launches += 1;
   return launch_zero_padding(c, slot_token, dst, st);
 }
 
@@ -460,6 +502,7 @@ maxscore_status maxscore_combine(maxscore_ctx* c, const void* src, const int32_t
     combine_kernel<float><<<blocks, 256, 0, (cudaStream_t)stream>>>((const float*)src, expert_idx, slot_idx, gate_w,
                                                                      (float*)dst, p.T, p.d_model, p.k, c->C, accumulate);
   MS_LAUNCH_CHECK("combine_kernel");
+  c->launches += 1;
   return MAXSCORE_OK;
 }
 
@@ -480,6 +523,7 @@ maxscore_status maxscore_combine_bwd(maxscore_ctx* c, const void* dY, const void
     combine_bwd_kernel<float><<<blocks, 256, 0, st>>>((const float*)dY, (const float*)yexp, expert_idx, slot_idx, gate_w,
                                                       (float*)dyexp, dgate_w, p.T, p.d_model, p.k, c->C);
   MS_LAUNCH_CHECK("combine_bwd_kernel");
+  c->launches += 1;
   return launch_zero_padding(c, slot_token, dyexp, st);
 }
 
@@ -530,11 +574,13 @@ maxscore_status maxscore_gate_bwd(maxscore_ctx* c, const void* hidden, const voi
     const long long nw = (long long)p.d_model * p.E;
     int rblocks = (int)((nw + 255) / 256); if (rblocks > c->sm_count * 8) rblocks = c->sm_count * 8;
     reduce_dw_kernel<<<rblocks, 256, 0, st>>>(part, dw_gate, nw, l.dw_splits);
+    c->launches += 5;
   } else {
     gate_bwd_dw_kernel<float><<<gw, 256, 0, st>>>((const float*)hidden, dlogits, dw_gate, p.T, p.d_model, p.E);
     MS_LAUNCH_CHECK("gate_bwd_dw_kernel");
     gate_bwd_dh_kernel<float><<<gh, 256, 0, st>>>(dlogits, (const float*)w_gate, (float*)dH, p.T, p.d_model, p.E,
                                                   p.w_gate_layout);
+    c->launches += 2;
   }
   MS_LAUNCH_CHECK("gate_bwd_dh_kernel");
   return MAXSCORE_OK;
@@ -551,6 +597,26 @@ maxscore_status maxscore_route_bwd(maxscore_ctx* c, const void* dY, const void* 
   s = maxscore_softtopk_bwd(c, logits, expert_idx, dgate_w, dlogits, stream);
   if (s) return s;
   return maxscore_gate_bwd(c, hidden, w_gate, dlogits, dw_gate, dH, stream);
+}
+
+long long maxscore_launch_count(const maxscore_ctx* c) { return c ? c->launches : -1; }
+
+maxscore_status maxscore_check_internal(maxscore_ctx* c, uint32_t* flag_out, void* stream) {
+  if (!c || !flag_out) return MAXSCORE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  unsigned v = 0;
+  MS_CUDA(cudaMemcpyAsync(&v, error_flag_of(c), sizeof(unsigned), cudaMemcpyDeviceToHost, st));
+  MS_CUDA(cudaMemsetAsync(error_flag_of(c), 0, sizeof(unsigned), st));
+  MS_CUDA(cudaStreamSynchronize(st));
+  *flag_out = v;
+  return MAXSCORE_OK;
+}
+
+maxscore_status maxscore_test_raise_internal(maxscore_ctx* c, void* stream) {
+  if (!c) return MAXSCORE_ERR_INVALID_ARG;
+  // every byte 1: any non-zero word reads as "a bounded wait gave up"
+  MS_CUDA(cudaMemsetAsync(error_flag_of(c), 1, sizeof(unsigned), (cudaStream_t)stream));
+  return MAXSCORE_OK;
 }
 
 maxscore_status maxscore_route_dispatch_host(maxscore_ctx* c, const void* hidden_host, const void* w_gate_host,

@@ -164,12 +164,12 @@ combine_kernel(const T* __restrict__ src, const int32_t* __restrict__ expert_idx
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   for (int tok = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; tok < Tn; tok += warps) {
-    long long my_off = 0; float my_w = 0.f;
+    long long my_off = -1; float my_w = 0.f;
     if (lane < k) {
       const int e = __ldg(expert_idx + (size_t)tok * k + lane);
       const int sl = __ldg(slot_idx + (size_t)tok * k + lane);
-      const bool valid = e >= 0 && sl >= 0 && sl < C;   // a malformed entry contributes nothing
-      my_off = valid ? ((long long)e * C + sl) * (long long)d : 0;
+      const bool valid = e >= 0 && sl >= 0 && sl < C;   // a malformed or surplus entry contributes nothing:
+      my_off = valid ? ((long long)e * C + sl) * (long long)d : -1;   // its row is neither read nor added
       my_w = !valid ? 0.f : gate_w ? __ldg(gate_w + (size_t)tok * k + lane) : 1.f;
     }
     long long rowoff[kMaxK]; float wgt[kMaxK];
@@ -187,10 +187,10 @@ combine_kernel(const T* __restrict__ src, const int32_t* __restrict__ expert_idx
       uint4 raw[kMaxK];
 #pragma unroll
       for (int c = 0; c < kMaxK; ++c)
-        if (c < k) raw[c] = ldg16(src + rowoff[c] + (size_t)v * N);
+        if (c < k && rowoff[c] >= 0) raw[c] = ldg16(src + rowoff[c] + (size_t)v * N);
 #pragma unroll
       for (int c = 0; c < kMaxK; ++c)
-        if (c < k) {
+        if (c < k && rowoff[c] >= 0) {
           float x[N];
           Vec16<T>::unpack(raw[c], x);
           const float w = wgt[c];

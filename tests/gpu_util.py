@@ -43,9 +43,6 @@ def assert_sum_close(got, ref, mag, tol, what=""):
 
 
 def float_keys(scores32: np.ndarray) -> np.ndarray:
-    """The keys the library documents for score_mode 0: rne(A * 2^40) plus the 12-bit position hash
-    ((i*E + j) * 2654435761 mod 2^32) >> 20, restated here from include/maxscore.h's description."""
-    T, E = scores32.shape
-    base = np.rint(scores32.astype(np.float64) * float(1 << 40)).astype(np.int64)
-    flat = (np.arange(T * E, dtype=np.uint64).reshape(T, E) * np.uint64(2654435761)) & np.uint64(0xFFFFFFFF)
-    return base + (flat >> np.uint64(20)).astype(np.int64)
+    """The keys the library documents for score_mode 0 (include/maxscore.h), computed by the oracle."""
+    import oracle
+    return oracle.keys_from_scores_hashed(np.asarray(scores32, dtype=np.float32).astype(np.float64))

@@ -293,3 +293,51 @@ def test_backward_chain_finite_differences(orc):
     assert (dyexp[slot_token < 0] == 0).all()
     np.testing.assert_allclose(dW, H.T @ dL, atol=1e-12)
     np.testing.assert_allclose(dH, dL @ W.T, atol=1e-12)
+
+
+def test_float_keys_round_to_nearest_even_on_the_2_pow_minus_40_grid(orc):
+    """mso_keys_from_scores against numpy's rint (an independent library routine), half-way cases included:
+    a plausible mistake (truncation, round-half-up, another scale) fails one of them."""
+    rng = np.random.default_rng(3)
+    A = rng.random((37, 11)) * 3.0
+    np.testing.assert_array_equal(orc.keys_from_scores(A), np.rint(A * 2.0 ** 40).astype(np.int64))
+    # exact half-way points (odd multiples of 2^-41) must go to the even neighbour, both signs
+    m = np.array([1, 3, 5, 7, 2 ** 20 + 1, 2 ** 30 + 3, -1, -3, -5], dtype=np.float64)
+    half = m * 2.0 ** -41
+    want = np.array([0, 2, 2, 4, 2 ** 19, 2 ** 29 + 2, 0, -2, -2], dtype=np.int64)
+    np.testing.assert_array_equal(orc.keys_from_scores(half.reshape(1, -1))[0], want)
+    # scale: one unit of the key is 2^-40 of score, so 1.0 -> 2^40 and 2^-40 -> 1
+    np.testing.assert_array_equal(orc.keys_from_scores(np.array([[1.0, 2.0 ** -40, 0.75]])),
+                                  np.array([[2 ** 40, 1, 3 * 2 ** 38]], dtype=np.int64))
+
+
+def test_hashed_float_keys_hand_values_and_bounds(orc):
+    """The position hash of the documented float-mode keys: hand-computed values of
+    ((i*E + j) * 2654435761 mod 2^32) >> 20 at a few positions, its range, that it depends on the position
+    only, and that it never changes which of two different float scores is larger."""
+    Z = np.zeros((3, 4))
+    h = orc.keys_from_scores_hashed(Z)
+    # position 0: 0; 1: 2654435761 >> 20 = 2531; 2: (5308871522 - 2^32 = 1013904226) >> 20 = 966;
+    # 3: (7963307283 - 2^32 = 3668339987) >> 20 = 3498; 5: (13272178805 - 3*2^32 = 387276917) >> 20 = 369
+    assert h[0, 0] == 0 and h[0, 1] == 2531 and h[0, 2] == 966 and h[0, 3] == 3498 and h[1, 1] == 369
+    rng = np.random.default_rng(5)
+    A = rng.random((64, 16)).astype(np.float32).astype(np.float64)
+    w0, w1 = orc.keys_from_scores(A), orc.keys_from_scores_hashed(A)
+    d = w1 - w0
+    assert d.min() >= 0 and d.max() < 4096
+    np.testing.assert_array_equal(d, orc.keys_from_scores_hashed(np.zeros_like(A)))      # position only
+    # the position is the row-major flat index i*E + j (a transposed index would give other values)
+    np.testing.assert_array_equal(d.reshape(-1), orc.keys_from_scores_hashed(np.zeros((1, 64 * 16)))[0])
+    assert not np.array_equal(d.T.reshape(-1), d.reshape(-1))
+    # two different fp32 scores differ by at least one ulp, which is >= 2^-24 relative, i.e. >= 2^16 key units
+    # for scores >= 2^-0: the 12-bit hash cannot reorder them
+    order0 = np.argsort(-w0, axis=1, kind="stable")
+    order1 = np.argsort(-w1, axis=1, kind="stable")
+    distinct = np.diff(np.sort(A, axis=1), axis=1).min() > 0
+    assert distinct and np.array_equal(order0, order1)
+    # and the optimum of a small problem moves by less than 4e-9 per chosen pair
+    T, E, k, C = 6, 4, 2, 3
+    S = rng.random((T, E)).astype(np.float32).astype(np.float64)
+    i0, _, _ = orc.flow_ssp(orc.keys_from_scores(S), k, C)
+    i1, _, _ = orc.flow_ssp(orc.keys_from_scores_hashed(S), k, C)
+    assert abs(orc.total_score(S, i0) - orc.total_score(S, i1)) < 4e-9 * T * k
