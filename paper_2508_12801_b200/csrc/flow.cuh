@@ -658,6 +658,9 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
     if (stall == 0) best_imb = sh.s_imb;
     done = (sh.s_imb == 0) || sweep >= a.n_sweeps || (stall >= kStallSweeps && sh.s_imb <= kStallImbalance);
     cumdrop += sh.s_drop;
+#ifdef MAXSCORE_TRACE
+    if (gtid == 0) printf("sweep %d imbalance %d stall %d eps %lld drop %lld\n", sweep, sh.s_imb, stall, eps, sh.s_drop);
+#endif
     { const long long ne = eps >> 1; eps = ne < a.eps_min ? a.eps_min : ne; }
   }
 
@@ -1097,6 +1100,7 @@ struct P2Shared {
   int flow[kMaxE];               // units on expert -> sink
   int estart[kMaxE + 2], efill[kMaxE + 1];   // entries grouped by expert: first position, fill counter
   int path_v[kMaxE + 2], path_u[kMaxE + 2], path_tok[kMaxE + 2], path_c[kMaxE + 2];
+  unsigned char failed[kMaxE + 4];   // deficit nodes whose walk came to a dead end in this search
   int npath, target, stop;
   long long dt, dtb;             // distance of the chosen target; best distance of any node with a deficit so far
 };
@@ -1253,7 +1257,8 @@ flow_exact_kernel(FlowState* st, int32_t* expert_idx, const int32_t* __restrict_
       }
       __syncthreads();
       bool changed = false;
-      const long long dtb = s.dtb;
+      // beyond the nearest deficit's distance plus theta no target can be used: its price update would leave the window
+      const long long dtb = (theta < kInf && s.dtb < kDistLimit - theta) ? s.dtb + theta + 1 : kDistLimit;
       {
         const int f = tid / kP2Group, sub = tid % kP2Group;      // every thread takes part in the group shuffles
         long long best = kInf;
@@ -1322,46 +1327,56 @@ flow_exact_kernel(FlowState* st, int32_t* expert_idx, const int32_t* __restrict_
       more = __syncthreads_or(changed);
       { long long* t = d0; d0 = dn; dn = t; }
     }
-    // ---- nearest node with a deficit (lowest index on ties); would the price update stay within theta? --
-    // Then the walk back from it, by one warp.  An arc u -> v is eligible when dist[u] + cost == dist[v] and
-    // u's distance was final before v's: such an arc exists for every reached node, and following them
-    // strictly lowers the level, so the walk ends at a node with excess without repeating a node.  Among the
-    // eligible arcs the Z arc wins, then the smallest token index, then the smallest tail: the choice does
-    // not depend on the order of the candidate list.  The offers of the last search round (which changed
-    // nothing) are still in place: an entry whose offer equals its node's distance is a tight arc from the
-    // expert its candidate is reached through; only if that expert's level does not fit are the candidate's
-    // other experts looked at.
+    // ---- augment along tight arcs, nearest deficit first, by one warp ------------------------------------
+    // With potentials lowered by min(dist, D), every arc u -> v with dist[u] + cost == dist[v] <= D has reduced
+    // cost zero, and so has its reverse: pushing a unit along ANY path of such arcs keeps all reduced costs
+    // non-negative.  One search therefore serves several augmentations: the deficit nodes are taken in order
+    // of distance (lowest index on ties) as long as the price update for D = their distance stays within theta.
+    // The walk back from a target: an arc u -> v is eligible when it is tight and u's distance was final before
+    // v's; such an arc exists for every reached node, and following them strictly lowers the level, so the walk
+    // ends at a node that had excess when the search began without repeating a node.  Among the eligible arcs
+    // the Z arc wins, then the smallest token index, then the smallest tail: the choice does not depend on the
+    // order of the candidate list.  The offers of the last search round (which changed nothing) are still in
+    // place: an entry whose offer equals its node's distance is a tight arc from the expert its candidate is
+    // reached through.  A token that has moved takes its offers off the table for the rest of this search.
     if (warp == 0) {
-      long long dt = kInf; int t = 0x7fffffff;
-      for (int v = lane; v <= E; v += 32)
-        if (s.imb[v] < 0 && d0[v] < dt) { dt = d0[v]; t = v; }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const long long od = __shfl_xor_sync(0xffffffffu, dt, o);
-        const int ot = __shfl_xor_sync(0xffffffffu, t, o);
-        if (od < dt || (od == dt && ot < t)) { dt = od; t = ot; }
-      }
-      int target = dt < kInf ? t : -1;
-      if (target >= 0) {
-        long long lo = kInf, hi = -kInf;
-        for (int e = lane; e < E; e += 32) {
-          const long long d = d0[e];
-          const long long chg = s.dp[e] - (d < dt ? d : dt);
-          lo = chg < lo ? chg : lo; hi = chg > hi ? chg : hi;
-        }
+      int napplied = 0, result = -1; long long dmax = 0;
+      for (int v = lane; v <= E; v += 32) s.failed[v] = 0;
+      __syncwarp();
+      const bool trusted = more == 0;                    // a search that never settled is not used
+      for (int attempt = 0; trusted && attempt < 4 * kMaxE; ++attempt) {
+        long long dt = kInf; int t = 0x7fffffff;
+        for (int v = lane; v <= E; v += 32)
+          if (s.imb[v] < 0 && !s.failed[v] && d0[v] < dt) { dt = d0[v]; t = v; }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
-          const long long ol = __shfl_xor_sync(0xffffffffu, lo, o), oh = __shfl_xor_sync(0xffffffffu, hi, o);
-          lo = ol < lo ? ol : lo; hi = oh > hi ? oh : hi;
+          const long long od = __shfl_xor_sync(0xffffffffu, dt, o);
+          const int ot = __shfl_xor_sync(0xffffffffu, t, o);
+          if (od < dt || (od == dt && ot < t)) { dt = od; t = ot; }
         }
-        if (theta < kInf && hi - lo > theta) {
-          target = -2;                                  // stop here; the next round lists more tokens:
-          if (lane == 0 && st->theta < 2 * (hi - lo)) st->theta = 2 * (hi - lo);   // enough of them for this price update
+        if (dt >= kInf) break;                           // no reachable deficit is left
+        {
+          long long lo = kInf, hi = -kInf;
+          for (int e = lane; e < E; e += 32) {
+            const long long d = d0[e];
+            const long long chg = s.dp[e] - (d < dt ? d : dt);
+            lo = chg < lo ? chg : lo; hi = chg > hi ? chg : hi;
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const long long ol = __shfl_xor_sync(0xffffffffu, lo, o), oh = __shfl_xor_sync(0xffffffffu, hi, o);
+            lo = ol < lo ? ol : lo; hi = oh > hi ? oh : hi;
+          }
+          if (theta < kInf && hi - lo > theta) {
+            if (napplied == 0) {
+              result = -2;                                // stop here; the next round lists more tokens:
+              if (lane == 0 && st->theta < 2 * (hi - lo)) st->theta = 2 * (hi - lo);   // enough of them for this price update
+            }
+            break;
+          }
         }
-      }
-      int len = 0; bool broken = more != 0;             // a search that never settled is not trusted
-      if (target >= 0 && !broken) {
-        int v = target;
+        // ---- walk back from t ----
+        int len = 0, v = t; bool dead = false;
         while (s.lvl[v] > 0 && len <= E + 1) {
           unsigned long long code = ~0ULL; int cc = -1;
           const long long dv = d0[v]; const int lv = s.lvl[v];
@@ -1421,46 +1436,57 @@ flow_exact_kernel(FlowState* st, int32_t* expert_idx, const int32_t* __restrict_
             const int occ = __shfl_xor_sync(0xffffffffu, cc, o);
             if (oc < code) { code = oc; cc = occ; }
           }
-          if (code == ~0ULL) { broken = true; break; }    // internal inconsistency: stop, the check pass will report it
+          if (code == ~0ULL) { dead = true; break; }      // every tight arc into v was used up earlier in this search
           const int u = (int)(code & 255ULL);
           if (lane == 0) { s.path_v[len] = v; s.path_u[len] = u; s.path_tok[len] = (int)(code >> 8) - 1; s.path_c[len] = cc; }
           ++len; v = u;
         }
-        if (!broken && (s.lvl[v] > 0 || s.imb[v] <= 0)) broken = true;
-        if (!broken && lane == 0) { s.imb[v] -= 1; s.imb[target] += 1; }
+        if (!dead && (s.lvl[v] > 0 || s.imb[v] <= 0)) dead = true;      // the walk must end at a node that still has excess
+        if (dead) {
+          if (napplied == 0 && attempt == 0 && s.lvl[v] > 0 && len > E + 1) { result = -3; break; }   // cannot happen
+          if (lane == 0) s.failed[t] = 1;
+          __syncwarp();
+          continue;
+        }
+        // ---- move one unit along the path ----
+        __syncwarp();
+        for (int a = lane; a < len; a += 32) {
+          const int pu = s.path_u[a], pv = s.path_v[a], tok = s.path_tok[a];
+          if (tok >= 0) {
+            const int c = s.path_c[a];
+            const int o = roff[c], m = rcnt[c];
+            for (int i = o; i < o + m; ++i) {
+              const int e = rmeta[i] & 255;
+              if (e == pu) rmeta[i] = (unsigned short)pu;             // given up
+              if (e == pv) rmeta[i] = (unsigned short)(pv | 256);     // taken
+              ndv[rpos[i]] = kInf;
+            }
+            for (int j = 0; j < k; ++j)
+              if (expert_idx[(size_t)tok * k + j] == pu) expert_idx[(size_t)tok * k + j] = pv;
+          } else if (pv == nZ) {
+            atomicAdd(&s.flow[pu], 1);
+          } else {
+            atomicAdd(&s.flow[pv], -1);
+          }
+        }
+        if (lane == 0) { s.imb[v] -= 1; s.imb[t] += 1; }
+        __syncwarp();
+        ++napplied; dmax = dt;
       }
-      if (lane == 0) { s.target = target; s.dt = dt; s.npath = len; if (broken) s.stop = 1; }
+      if (lane == 0) { s.target = napplied > 0 ? napplied : result; s.dt = dmax; if (!trusted || result == -3) s.stop = 1; }
     }
     __syncthreads();
     if (s.stop) { if (tid == 0) atomicOr(&st->status, 4u); break; }
-    if (s.target < 0) break;        // -1: no augmenting path inside the candidate graph
-    const long long dt = s.dt;
-    // ---- move one unit along the path ------------------------------------------------------------------
-    const int L = s.npath;
-    for (int v = tid; v <= E; v += blockDim.x) {
-      const long long d = d0[v];
-      const long long step = d < dt ? d : dt;
-      s.p[v] -= step; s.dp[v] -= step;
-    }
-    for (int a = tid; a < L; a += blockDim.x) {
-      const int u = s.path_u[a], v = s.path_v[a], tok = s.path_tok[a];
-      if (tok >= 0) {
-        const int c = s.path_c[a];
-        const int o = roff[c], m = rcnt[c];
-        for (int i = o; i < o + m; ++i) {
-          const int e = rmeta[i] & 255;
-          if (e == u) rmeta[i] = (unsigned short)u;             // given up
-          if (e == v) rmeta[i] = (unsigned short)(v | 256);     // taken
-        }
-        for (int j = 0; j < k; ++j)
-          if (expert_idx[(size_t)tok * k + j] == u) expert_idx[(size_t)tok * k + j] = v;
-      } else if (v == nZ) {
-        atomicAdd(&s.flow[u], 1);
-      } else {
-        atomicAdd(&s.flow[v], -1);
+    if (s.target < 0) break;        // -1: no augmenting path inside the candidate graph; -2: theta reached
+    {
+      const long long dt = s.dt;
+      for (int v = tid; v <= E; v += blockDim.x) {
+        const long long d = d0[v];
+        const long long step = d < dt ? d : dt;
+        s.p[v] -= step; s.dp[v] -= step;
       }
     }
-    ++naug;
+    naug += s.target;
     __syncthreads();
   }
   // ---- write back ---------------------------------------------------------------------------------

@@ -42,6 +42,31 @@ def assert_sum_close(got, ref, mag, tol, what=""):
     assert not bad.any(), f"{what}: {bad.sum()} entries off, worst {np.max(d / (mag + 1e-300)):.3e} > {tol}"
 
 
+def assert_row_rel(got, ref, tol, what=""):
+    """Row-relative bar for sums of signed products: per row max_i |d_i| <= tol * max_i |ref_i|.  Returns the
+    worst ratio seen, so that callers can report it."""
+    got = np.asarray(got, dtype=np.float64).reshape(-1, got.shape[-1])
+    ref = np.asarray(ref, dtype=np.float64).reshape(-1, ref.shape[-1])
+    rowmax = np.abs(ref).max(axis=1)
+    d = np.abs(got - ref).max(axis=1)
+    worst = float(np.max(d / (rowmax + 1e-300)))
+    assert (d <= tol * rowmax + 1e-300).all(), f"{what}: row-relative error {worst:.3e} > {tol}"
+    return worst
+
+
+def assert_rounded_sum_close(got, ref, mag, tol_acc, what=""):
+    """For outputs that are sums of signed products accumulated in fp32 and rounded ONCE to bf16:
+    |got - ref| <= 2^-8 |ref| + tol_acc * mag elementwise (one bf16 rounding of the result plus the
+    accumulation error, which scales with the sum of the absolute terms `mag`).  A dropped tile, expert
+    column or half of a split operand is far outside this bar."""
+    got = np.asarray(got, dtype=np.float64); ref = np.asarray(ref, dtype=np.float64)
+    mag = np.asarray(mag, dtype=np.float64)
+    d = np.abs(got - ref)
+    bar = 2.0 ** -8 * np.abs(ref) + tol_acc * mag
+    bad = d > bar
+    assert not bad.any(), f"{what}: {bad.sum()} entries off, worst {np.max(d / (bar + 1e-300)):.3f} x the bar"
+
+
 def float_keys(scores32: np.ndarray) -> np.ndarray:
     """The keys the library documents for score_mode 0 (include/maxscore.h), computed by the oracle."""
     import oracle

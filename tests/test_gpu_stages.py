@@ -3,13 +3,16 @@ CPU oracle on the same seeded inputs.  Downstream stages are fed the GPU's own u
 that a flipped near-tie upstream cannot pass for a downstream bug.
 
 Tolerances.  SoftTopk sums positive terms, so it is held to 1e-5 relative elementwise.  Outputs that
-are sums of signed products (gate, combine, the backward GEMMs) are held to tol * (the same sum over
-absolute values): 1e-5 for fp32 I/O, 2e-2 for bf16 I/O (one rounding to bf16 is 2^-9)."""
+are sums of signed products (gate, combine, the backward GEMMs) are held to
+  fp32 outputs:  1e-5 * (the same sum over absolute values), and per row max|d| <= 1e-5 * max|ref|;
+  bf16 outputs:  2^-8 * |ref| + 1e-5 * (the same sum over absolute values): one rounding of the result
+                 plus fp32 accumulation; and per row max|d| <= 2e-2 * max|ref| as the outer bar."""
 import numpy as np
 import pytest
 import torch
 
-from gpu_util import assert_rel, assert_sum_close, f64, float_keys, np32, raw16
+from gpu_util import (assert_rel, assert_rounded_sum_close, assert_row_rel, assert_sum_close, f64, float_keys, np32,
+                      raw16)
 
 pytestmark = pytest.mark.gpu
 
@@ -39,6 +42,16 @@ def _tol(dtype):
     return 2e-2 if dtype == "bf16" else 1e-5
 
 
+def _assert_out(got, ref, mag, dtype, what, rows=True):
+    """An output in the I/O dtype: fp32 accumulation error, plus one rounding when the output is bf16."""
+    if dtype == "bf16":
+        assert_rounded_sum_close(got, ref, mag, 1e-5, what)
+    else:
+        assert_sum_close(got, ref, mag, 1e-5, what)
+    if rows:
+        assert_row_rel(got, ref, _tol(dtype), what + " (row-relative)")
+
+
 # ------------------------------------------------------------------------------------------- gate
 @pytest.mark.parametrize("T,d,E,dtype,layout,bias", [
     (512, 256, 8, "f32", 0, False), (300, 100, 12, "f32", 1, True),
@@ -58,6 +71,7 @@ def test_gate(ms, orc, synth, T, d, E, dtype, layout, bias):
     ref = orc.gate(f64(H), f64(W), f64(b) if bias else None)
     mag = orc.gate(np.abs(f64(H)), np.abs(f64(W)), np.abs(f64(b)) if bias else None)
     assert_sum_close(np32(L), ref, mag, 1e-5, "gate")      # logits are fp32 in both I/O modes
+    assert_row_rel(np32(L), ref, 1e-5, "gate (row-relative)")
 
 
 # ------------------------------------------------------------------------------------------- SoftTopk
@@ -82,6 +96,50 @@ def test_softtopk_fwd_bwd(ms, orc, synth, T, E, k, t):
     got = np32(dL)
     rowmax = np.abs(refb).max(axis=1, keepdims=True)
     assert (np.abs(got - refb) <= 1e-5 * rowmax + 1e-9).all()
+
+
+def _softtopk_against_oracle(ms, orc, L, k, t):
+    T, E = L.shape
+    ctx = _ctx(ms, T, 64, E, k, cf=float(E), t=t)
+    Ld = L.to(DEV)
+    A = torch.empty_like(Ld)
+    ms.softtopk_fwd(ctx, Ld, A)
+    assert_rel(np32(A), orc.softtopk_fwd(f64(L), k, t), 1e-5, "SoftTopk fwd")
+    g = torch.Generator().manual_seed(5)
+    idx = torch.stack([torch.randperm(E, generator=g)[:k].sort().values for _ in range(T)]).to(torch.int32)
+    dg = torch.randn(T, k, generator=g)
+    dL = torch.empty_like(Ld)
+    ms.softtopk_bwd(ctx, Ld, idx.to(DEV), dg.to(DEV), dL)
+    G = np.zeros((T, E)); np.put_along_axis(G, idx.numpy().astype(np.int64), f64(dg), axis=1)
+    refb = orc.softtopk_bwd(f64(L), G, k, t)
+    scale = np.abs(G).max(axis=1, keepdims=True) * (k / t)          # |J^T g| <= k/t * max|g| per row
+    assert (np.abs(np32(dL) - refb) <= 1e-5 * scale + 1e-12).all()
+
+
+@pytest.mark.parametrize("E,k,t", [(8, 2, 1.0), (64, 8, 1.0), (128, 8, 0.25), (20, 3, 2.0)])
+def test_softtopk_tied_logits_take_the_lowest_index(ms, orc, synth, E, k, t):
+    """Logits on a 0.25 grid tie often, and some rows are all equal: which entry a level masks is then decided
+    by the lowest-expert-index rule, on both sides (Eq. 6's Topk is silent on ties)."""
+    T = 384
+    L = (synth.logits_like(T, E, seed=8) * 4).round() / 4
+    L[5] = 0.5; L[6] = -3.0; L[7, : E // 2] = 1.0; L[7, E // 2:] = 1.0      # all-equal rows
+    L[8] = 0.0; L[8, E - 1] = 2.0; L[8, 0] = 2.0                           # the maximum twice, far apart
+    _softtopk_against_oracle(ms, orc, L, k, t)
+
+
+@pytest.mark.parametrize("E,k,t", [(64, 8, 0.25), (128, 8, 0.25), (16, 4, 0.5)])
+def test_softtopk_rows_whose_levels_fall_far_below_the_row_maximum(ms, orc, synth, E, k, t):
+    """Widely spread logits (N(0,1) x 40 at a small temperature, and rows with one or two entries 100 t
+    above the rest): a later level's maximum then lies more than 60 t below the first one's, which makes
+    the kernel re-base its exponentials on that level's own maximum."""
+    T = 256
+    L = synth.logits_like(T, E, seed=9) * 40.0
+    L[3] = synth.logits_like(1, E, seed=10)[0]; L[3, 2] += 100.0 * t
+    L[4] = synth.logits_like(1, E, seed=11)[0]; L[4, 1] += 100.0 * t; L[4, E - 1] += 170.0 * t
+    # the spread must really exceed the re-base threshold on most rows
+    top = np.sort(f64(L), axis=1)[:, ::-1]
+    assert ((top[:, 0] - top[:, k - 1]) > 60.0 * t).mean() > 0.5
+    _softtopk_against_oracle(ms, orc, L, k, t)
 
 
 @pytest.mark.parametrize("T,E,k,lam", [(512, 8, 2, 1e-2), (1000, 16, 2, 1e-2), (4099, 64, 8, 3e-3), (777, 128, 8, 1.0),
@@ -300,21 +358,21 @@ def test_index_dispatch_combine_and_backward(ms, orc, synth, T, d, E, k, cf, dty
     ms.combine(ctx, yd, idx, slot_idx, gwd, Y)
     refY = orc.combine(f64(yexp), oidx, o_slot, f64(gw))
     magY = orc.combine(np.abs(f64(yexp)), oidx, o_slot, np.abs(f64(gw)))
-    assert_sum_close(f64(Y), refY, magY, _tol(dtype), "combine")
+    _assert_out(f64(Y), refY, magY, dtype, "combine")
     # unit weights + accumulate (dispatch backward into an existing gradient)
     base = torch.randn(T, d, generator=g).to(H.dtype)
     Y2 = base.clone().to(DEV)
     ms.combine(ctx, yd, idx, slot_idx, None, Y2, accumulate=1)
     ref2 = f64(base) + orc.combine(f64(yexp), oidx, o_slot, None)
     mag2 = np.abs(f64(base)) + orc.combine(np.abs(f64(yexp)), oidx, o_slot, None)
-    assert_sum_close(f64(Y2), ref2, mag2, _tol(dtype), "combine accumulate")
+    _assert_out(f64(Y2), ref2, mag2, dtype, "combine accumulate")
     # combine backward
     dY = synth.upstream_grad(wl, 2)
     dyexp = torch.full((E, C, d), 3.0, dtype=H.dtype, device=DEV)
     dgw = torch.empty(T, k, dtype=torch.float32, device=DEV)
     ms.combine_bwd(ctx, dY.to(DEV), yd, idx, slot_idx, gwd, slot_token, dyexp, dgw)
     r_dyexp, r_dgw = orc.combine_bwd(f64(dY), f64(yexp), oidx, o_slot, f64(gw))
-    assert_sum_close(f64(dyexp), r_dyexp, np.abs(r_dyexp), _tol(dtype), "dyexp")      # padding rows exactly zero
+    _assert_out(f64(dyexp), r_dyexp, np.abs(r_dyexp), dtype, "dyexp", rows=False)     # padding rows exactly zero
     _, m_dgw = orc.combine_bwd(np.abs(f64(dY)), np.abs(f64(yexp)), oidx, o_slot, np.abs(f64(gw)))
     assert_sum_close(np32(dgw), r_dgw, m_dgw, 1e-5, "dgate_w")                         # fp32 dot of exact products
 
@@ -333,7 +391,8 @@ def test_gate_bwd(ms, orc, synth, T, d, E, dtype, layout):
     r_dW, r_dH = orc.gate_bwd(f64(H), f64(W), f64(dL))
     m_dW, m_dH = orc.gate_bwd(np.abs(f64(H)), np.abs(f64(W)), np.abs(f64(dL)))
     assert_sum_close(np32(dW), r_dW, m_dW, 1e-5, "dW")
-    assert_sum_close(f64(dH), r_dH, m_dH, _tol(dtype), "dH")
+    _assert_out(f64(dH), r_dH, m_dH, dtype, "dH")
+    assert_row_rel(np32(dW), r_dW, 1e-5, "dW (row-relative)")
 
 
 # ------------------------------------------------------------------------------------------- whole path
@@ -415,3 +474,47 @@ def test_route_dispatch_from_host_buffers(ms, orc, synth, name, T, bias):
     np.testing.assert_array_equal(slot_h.numpy(), o_slot)
     ref = orc.dispatch(H.view(as_int).numpy(), o_tok)
     np.testing.assert_array_equal(xd2.cpu().view(as_int).numpy(), ref)
+
+@pytest.mark.parametrize("name", ["tiny", "k2e16"])
+def test_route_bwd_whole_call_at_the_small_configs(ms, orc, synth, name):
+    """maxscore_route_bwd as ONE call at the full shape of the two small workloads (fp32 I/O and bf16 I/O):
+    forward on the GPU with identity experts (yexp = xdisp), upstream gradients N(0,1) over the combine
+    output, then every output of the backward against the oracle's backward chain fed the GPU's own forward
+    outputs (all rows)."""
+    wl = synth.WORKLOADS[name]
+    T, d, E, k = wl.T, wl.d_model, wl.E, wl.k
+    H, W, dY = synth.hidden(wl), synth.w_gate(wl), synth.upstream_grad(wl)
+    ctx = _ctx(ms, T, d, E, k, cf=wl.capacity_factor, dtype=wl.dtype)
+    C = ctx.capacity
+    buf = ms.RouterBuffers(ctx)
+    Hd, Wd, dYd = H.to(DEV), W.to(DEV), dY.to(DEV)
+    ms.route_fwd(ctx, Hd, Wd, None, *buf.args())
+    xd = torch.empty(E, C, d, dtype=H.dtype, device=DEV)
+    ms.dispatch(ctx, Hd, buf.expert_idx, buf.slot_idx, buf.slot_token, xd)
+    dyexp = torch.full((E, C, d), 3.0, dtype=H.dtype, device=DEV)
+    dgw = torch.empty(T, k, dtype=torch.float32, device=DEV)
+    dL = torch.empty(T, E, dtype=torch.float32, device=DEV)
+    dW = torch.empty(d, E, dtype=torch.float32, device=DEV)
+    dH = torch.empty(T, d, dtype=H.dtype, device=DEV)
+    ms.route_bwd(ctx, dYd, xd, Hd, Wd, buf.logits, buf.expert_idx, buf.slot_idx, buf.gate_w, buf.slot_token,
+                 dyexp, dgw, dL, dW, dH)
+    torch.cuda.synchronize()
+    assert ms.read_stats(buf.stats).status == 0 and ms.check_internal(ctx) == 0
+    idx = buf.expert_idx.cpu().numpy(); slot = buf.slot_idx.cpu().numpy()
+    gw = np32(buf.gate_w).astype(np.float64); L = np32(buf.logits).astype(np.float64)
+    yexp = f64(xd)
+    r_dyexp, r_dgw = orc.combine_bwd(f64(dY), yexp, idx, slot, gw)
+    _, m_dgw = orc.combine_bwd(np.abs(f64(dY)), np.abs(yexp), idx, slot, np.abs(gw))
+    _assert_out(f64(dyexp), r_dyexp, np.abs(r_dyexp), wl.dtype, "dyexp", rows=False)
+    assert_sum_close(np32(dgw), r_dgw, m_dgw, 1e-5, "dgate_w")
+    # SoftTopk backward on the GPU's own dgate_w, gate backward on the GPU's own dlogits
+    G = np.zeros((T, E)); np.put_along_axis(G, idx.astype(np.int64), np32(dgw).astype(np.float64), axis=1)
+    r_dL = orc.softtopk_bwd(L, G, k, wl.temperature)
+    scale = np.abs(G).max(axis=1, keepdims=True) * (k / wl.temperature)
+    assert (np.abs(np32(dL) - r_dL) <= 1e-5 * scale + 1e-12).all()
+    dLf = np32(dL).astype(np.float64)
+    r_dW, r_dH = orc.gate_bwd(f64(H), f64(W), dLf)
+    m_dW, m_dH = orc.gate_bwd(np.abs(f64(H)), np.abs(f64(W)), np.abs(dLf))
+    assert_sum_close(np32(dW), r_dW, m_dW, 1e-5, "dW")
+    assert_row_rel(np32(dW), r_dW, 1e-5, "dW (row-relative)")
+    _assert_out(f64(dH), r_dH, m_dH, wl.dtype, "dH")

@@ -5,7 +5,8 @@ cudaMalloc would stall the GPU, as a plugin that may only touch tensors its host
 on top of a pool that is already fully carved up.  For them the library offers one entry point that
 needs no context and no workspace; its scratch sits in a fixed array inside the library.  This test
 calls it through the C ABI, twice in a row with different inputs (the scratch keeps the first call's
-contents), and checks every output against the regular maxscore_index_build, bit for bit.
+contents), and checks every output against the regular maxscore_index_build and against the CPU checker,
+bit for bit.
 It lives in a file that pytest collects last, so a run that stops at the first failure has already run
 every other test.
 """
@@ -36,7 +37,7 @@ def _regular(ms, idx, T, E, k, Cap):
     return slot_idx.cpu().numpy(), slot_token.cpu().numpy(), load.cpu().numpy()
 
 
-def test_index_build_noalloc_matches_regular_entry_point_twice():
+def test_index_build_noalloc_matches_regular_entry_point_twice(orc):
     from paper_2508_12801_b200 import binding as ms
     assert torch.cuda.is_available()
     # two calls in a row; the second is smaller, so stale scratch from the first would show
@@ -52,6 +53,11 @@ def test_index_build_noalloc_matches_regular_entry_point_twice():
         np.testing.assert_array_equal(slot_idx.cpu().numpy(), want[0])
         np.testing.assert_array_equal(slot_token.cpu().numpy(), want[1])
         np.testing.assert_array_equal(load.cpu().numpy(), want[2])
+        # and against the CPU checker's index build of the same assignment
+        o_slot, o_tok, o_load = orc.index_build(idx.cpu().numpy(), E, Cap)
+        np.testing.assert_array_equal(slot_idx.cpu().numpy(), o_slot)
+        np.testing.assert_array_equal(slot_token.cpu().numpy(), o_tok)
+        np.testing.assert_array_equal(load.cpu().numpy(), o_load)
 
 
 def test_index_build_noalloc_rejects_sizes_beyond_its_scratch():
