@@ -141,6 +141,26 @@ def softtopk_rankscale_bwd(L, G, k: int, t: float, beta: float, delta: int) -> n
     return dL
 
 
+def itertopk_fwd(L, k: int) -> np.ndarray:
+    """IterTopk of Table 2: y^(l) = y^(l-1) + g(x; 1 - y^(l-1)), g(x; w) = w e^x / sum(w e^x), y^(0) = 0."""
+    L = _f64(L)
+    T, E = L.shape
+    A = np.empty_like(L)
+    if lib().mso_itertopk_fwd(I64(T), I64(E), I64(k), _p(L), _p(A)):
+        raise ValueError("itertopk_fwd: bad arguments")
+    return A
+
+
+def itertopk_bwd(L, G, k: int) -> np.ndarray:
+    """dL = J^T G for IterTopk."""
+    L, G = _f64(L), _f64(G)
+    T, E = L.shape
+    dL = np.empty_like(L)
+    if lib().mso_itertopk_bwd(I64(T), I64(E), I64(k), _p(L), _p(G), _p(dL)):
+        raise ValueError("itertopk_bwd: bad arguments")
+    return dL
+
+
 def keys_from_scores(A) -> np.ndarray:
     """Fixed-point keys rne(A * 2^40) as int64."""
     A = _f64(A)

@@ -37,6 +37,7 @@
  * readings of Eq. 6 (pinned by the formula's own special cases only: the
  * paper prints no value that tells the readings of Eq. 6 apart).
  *   mso_softtopk_rankscale_fwd/bwd   Eq. 6 read literally (rank-scaled softmax)
+ *   mso_itertopk_fwd/bwd             IterTopk of Table 2 and its derivative
  *   mso_aux_loss_grad                derivative of Eq. 9 with respect to A
  */
 #include <math.h>
@@ -761,5 +762,72 @@ int mso_softtopk_rankscale_bwd(int64_t T, int64_t E, int64_t k, double t, double
     }
   }
   free(rank); free(p);
+  return MSO_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* IterTopk of Table 2: y^(0) = 0 and, for level l = 1..k,               */
+/*     y^(l) = y^(l-1) + g(x; 1 - y^(l-1)),   g(x; w)_j = w_j e^{x_j} / sum_i w_i e^{x_i}.  */
+/* Every level adds a distribution, so the result sums to k.  Table 2    */
+/* carries no temperature: the logits enter as they are.                 */
+int mso_itertopk_fwd(int64_t T, int64_t E, int64_t k, const double *L, double *A) {
+  if (k < 1 || k > E) return MSO_ERR_ARG;
+  for (int64_t r = 0; r < T; ++r) {
+    const double *x = L + r * E; double *y = A + r * E;
+    double m = x[0];
+    for (int64_t j = 1; j < E; ++j) if (x[j] > m) m = x[j];
+    for (int64_t j = 0; j < E; ++j) y[j] = 0.0;
+    for (int64_t l = 0; l < k; ++l) {
+      double s = 0.0;
+      for (int64_t j = 0; j < E; ++j) s += (1.0 - y[j]) * exp(x[j] - m);
+      /* all increments of a level come from the y of the level before */
+      for (int64_t j = 0; j < E; ++j) y[j] = y[j] + (1.0 - y[j]) * exp(x[j] - m) / s;
+    }
+  }
+  return MSO_OK;
+}
+
+/* Derivative of IterTopk: dL = J^T G, by reverse accumulation through   */
+/* the k levels.  With z_j = e^{x_j - m}, u_j = w_j z_j, s = sum u,      */
+/* r = u / s: given the gradient rb of r,                                */
+/*   ub_j = (rb_j - sum_i rb_i r_i) / s,  wb_j = ub_j z_j,  zb_j += ub_j w_j, */
+/* and since w = 1 - y^(l-1), the gradient of y^(l-1) is that of y^(l)   */
+/* minus wb.  Finally dx_j = zb_j z_j (the shift m drops out: IterTopk   */
+/* does not change when a constant is added to every logit).             */
+int mso_itertopk_bwd(int64_t T, int64_t E, int64_t k, const double *L, const double *G, double *dL) {
+  if (k < 1 || k > E) return MSO_ERR_ARG;
+  double *w = (double *)malloc(sizeof(double) * (size_t)(k * E));   /* w of every level */
+  double *z = (double *)malloc(sizeof(double) * (size_t)E);
+  double *yb = (double *)malloc(sizeof(double) * (size_t)E);
+  double *zb = (double *)malloc(sizeof(double) * (size_t)E);
+  double *ss = (double *)malloc(sizeof(double) * (size_t)k);
+  if (!w || !z || !yb || !zb || !ss) { free(w); free(z); free(yb); free(zb); free(ss); return MSO_ERR_ALLOC; }
+  for (int64_t r = 0; r < T; ++r) {
+    const double *x = L + r * E, *g = G + r * E;
+    double m = x[0];
+    for (int64_t j = 1; j < E; ++j) if (x[j] > m) m = x[j];
+    for (int64_t j = 0; j < E; ++j) { z[j] = exp(x[j] - m); yb[j] = g[j]; zb[j] = 0.0; }
+    /* forward, keeping each level's weights and normaliser */
+    for (int64_t j = 0; j < E; ++j) w[j] = 1.0;
+    for (int64_t l = 0; l < k; ++l) {
+      double s = 0.0;
+      for (int64_t j = 0; j < E; ++j) s += w[l * E + j] * z[j];
+      ss[l] = s;
+      if (l + 1 < k)
+        for (int64_t j = 0; j < E; ++j) w[(l + 1) * E + j] = w[l * E + j] - w[l * E + j] * z[j] / s;
+    }
+    for (int64_t l = k - 1; l >= 0; --l) {
+      const double s = ss[l];
+      double dot = 0.0;
+      for (int64_t j = 0; j < E; ++j) dot += yb[j] * (w[l * E + j] * z[j] / s);
+      for (int64_t j = 0; j < E; ++j) {
+        const double ub = (yb[j] - dot) / s;
+        zb[j] += ub * w[l * E + j];
+        yb[j] -= ub * z[j];              /* gradient of y^(l-1): through the sum and through w = 1 - y^(l-1) */
+      }
+    }
+    for (int64_t j = 0; j < E; ++j) dL[r * E + j] = zb[j] * z[j];
+  }
+  free(w); free(z); free(yb); free(zb); free(ss);
   return MSO_OK;
 }

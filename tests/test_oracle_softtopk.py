@@ -212,3 +212,50 @@ def test_rankscale_bwd_finite_differences(orc, beta, delta):
         assert abs(fd - got[r, l]) < 1e-7
     # a softmax Jacobian applied to anything sums to zero over the logits
     np.testing.assert_allclose(got.sum(1), 0.0, atol=1e-14)
+
+
+# ------------------------------------------------------------------------------------------- IterTopk (Table 2)
+def test_itertopk_special_cases_and_invariants(orc):
+    rng = np.random.default_rng(21)
+    L = rng.normal(size=(40, 12)) * 2.0
+    for k in (1, 2, 5, 12):
+        Y = orc.itertopk_fwd(L, k)
+        np.testing.assert_allclose(Y.sum(axis=1), k, rtol=0, atol=1e-12)          # every level adds a distribution
+        np.testing.assert_allclose(orc.itertopk_fwd(L + 3.25, k), Y, rtol=0, atol=1e-11 * np.abs(Y).max() ** 2)   # shift invariance
+        perm = rng.permutation(12)
+        # (at k = E the recursion overshoots 1 and amplifies rounding: the bar scales with the values)
+        np.testing.assert_allclose(orc.itertopk_fwd(L[:, perm], k), Y[:, perm], rtol=0, atol=1e-12 * np.abs(Y).max() ** 2)
+    from scipy.special import softmax
+    np.testing.assert_allclose(orc.itertopk_fwd(L, 1), softmax(L, axis=1), rtol=0, atol=1e-14)   # k = 1 is Softmax
+    # equal logits: every level is uniform over equal weights, so y = k / E
+    np.testing.assert_allclose(orc.itertopk_fwd(np.full((1, 8), 0.7), 3), np.full((1, 8), 3 / 8), atol=1e-15)
+
+
+def test_itertopk_two_experts_closed_form(orc):
+    """E = 2, k = 2 by hand: level 1 gives (p, 1-p) with p = softmax; level 2 weights are (1-p, p), and
+    (1-p) e^a and p e^b are equal (both are e^a e^b / (e^a + e^b)), so level 2 adds (1/2, 1/2)."""
+    for a, b in [(0.3, -1.1), (2.0, 2.0), (-4.0, 1.5)]:
+        p = np.exp(a) / (np.exp(a) + np.exp(b))
+        Y = orc.itertopk_fwd(np.array([[a, b]]), 2)
+        np.testing.assert_allclose(Y, [[p + 0.5, 1.5 - p]], rtol=0, atol=1e-14)
+    # E = 3, k = 2, worked with exact fractions for e^x = (4, 2, 2): level 1 = (1/2, 1/4, 1/4); weights (1/2, 3/4, 3/4);
+    # w e^x = (2, 3/2, 3/2), sum 5; level 2 = (2/5, 3/10, 3/10); total (9/10, 11/20, 11/20)
+    x = np.log(np.array([[4.0, 2.0, 2.0]]))
+    np.testing.assert_allclose(orc.itertopk_fwd(x, 2), [[0.9, 0.55, 0.55]], rtol=0, atol=1e-14)
+
+
+def test_itertopk_backward_against_finite_differences(orc):
+    rng = np.random.default_rng(22)
+    T, E = 6, 7
+    L = rng.normal(size=(T, E)) * 1.5
+    G = rng.normal(size=(T, E))
+    for k in (1, 2, 4, 7):
+        dL = orc.itertopk_bwd(L, G, k)
+        h = 1e-6
+        num = np.zeros_like(L)
+        for j in range(E):
+            Lp, Lm = L.copy(), L.copy()
+            Lp[:, j] += h; Lm[:, j] -= h
+            num[:, j] = ((orc.itertopk_fwd(Lp, k) - orc.itertopk_fwd(Lm, k)) * G).sum(axis=1) / (2 * h)
+        np.testing.assert_allclose(dL, num, rtol=1e-7, atol=2e-8)
+        np.testing.assert_allclose(dL.sum(axis=1), 0, atol=1e-10 * max(1.0, np.abs(dL).max()))   # shift invariance of the forward
