@@ -89,6 +89,9 @@ typedef struct {
                            /* 1: Eq. 6 read literally: y_i = p_i * (beta + t * min(rank_i - delta, */
                            /*    k)), p = Softmax over all experts, rank 1 = largest, ties: lowest */
                            /*    index first                                                       */
+                           /* 2: IterTopk of Table 2: y^(l) = y^(l-1) + g(x; 1 - y^(l-1)) for l = 1..k,  */
+                           /*    g(x; w) = w e^x / sum(w e^x), y^(0) = 0; Table 2 has no temperature,    */
+                           /*    so t is not used in this mode                                     */
   float rankscale_beta;    /* mode 1: 0 = the recursion starts from 0, 1 = it starts from Softmax  */
   int32_t rankscale_delta; /* mode 1: 0 = level j masks the j-1 largest, 1 = the j largest         */
 } maxscore_params;

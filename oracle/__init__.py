@@ -161,6 +161,19 @@ def itertopk_bwd(L, G, k: int) -> np.ndarray:
     return dL
 
 
+def iterative_reroute(A, k: int, Cap: int):
+    """Top-k with capacity, then greedy rerouting of the dropped pairs (Sec. 2.3).  Returns
+    (expert_idx [T,k] ascending with -1 last, load [E], pairs dropped in stage 1, slots left empty)."""
+    A = _f64(A)
+    T, E = A.shape
+    idx = np.empty((T, k), np.int32)
+    load = np.empty(E, np.int32)
+    counts = np.zeros(2, np.int64)
+    if lib().mso_iterative_reroute(I64(T), I64(E), I64(k), I64(Cap), _p(A), _p(idx), _p(load), _p(counts)):
+        raise ValueError("iterative_reroute: bad arguments")
+    return idx, load, int(counts[0]), int(counts[1])
+
+
 def keys_from_scores(A) -> np.ndarray:
     """Fixed-point keys rne(A * 2^40) as int64."""
     A = _f64(A)

@@ -38,6 +38,8 @@
  * paper prints no value that tells the readings of Eq. 6 apart).
  *   mso_softtopk_rankscale_fwd/bwd   Eq. 6 read literally (rank-scaled softmax)
  *   mso_itertopk_fwd/bwd             IterTopk of Table 2 and its derivative
+ *   mso_iterative_reroute            top-k with capacity, then greedy rerouting of the dropped pairs
+ *                                    (Sec. 2.3; the serving orders are this build's reading)
  *   mso_aux_loss_grad                derivative of Eq. 9 with respect to A
  */
 #include <math.h>
@@ -829,5 +831,69 @@ int mso_itertopk_bwd(int64_t T, int64_t E, int64_t k, const double *L, const dou
     for (int64_t j = 0; j < E; ++j) dL[r * E + j] = zb[j] * z[j];
   }
   free(w); free(z); free(yb); free(zb); free(ss);
+  return MSO_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* Iterative rerouting (Sec. 2.3, the Switch Transformers paragraph;     */
+/* the assignment step of "MaxScore-I", Sec. 4.1 Baselines).             */
+/* Stage 1: every token's k choices by descending affinity (ties: lowest */
+/* expert index); choice level 1 of all tokens is served first, then     */
+/* level 2, ..., within a level in ascending token index; a pair is      */
+/* accepted while its expert holds fewer than C tokens, else dropped.    */
+/* Stage 2: the dropped pairs, in ascending token index and within a     */
+/* token in level order, are each given to the expert of highest         */
+/* affinity among those that still have room and that the token does not */
+/* hold (ties: lowest index); if there is none the slot stays empty.     */
+/* The paper fixes neither order: both are this build's reading.         */
+/* Outputs: expert_idx [T,k] ascending with -1 (empty) last, load [E],   */
+/* counts[0] = pairs dropped in stage 1, counts[1] = slots left empty.   */
+int mso_iterative_reroute(int64_t T, int64_t E, int64_t k, int64_t C, const double *A,
+                          int32_t *expert_idx, int32_t *load, int64_t *counts) {
+  if (k < 1 || k > E || C < 0) return MSO_ERR_ARG;
+  int32_t *choice = (int32_t *)malloc(sizeof(int32_t) * (size_t)(T * k));   /* [T][k], level order */
+  unsigned char *held = (unsigned char *)calloc((size_t)(T * E), 1);
+  unsigned char *dropped = (unsigned char *)calloc((size_t)(T * k), 1);
+  if (!choice || !held || !dropped) { free(choice); free(held); free(dropped); return MSO_ERR_ALLOC; }
+  for (int64_t i = 0; i < T; ++i) {
+    const double *a = A + i * E;
+    for (int64_t r = 0; r < k; ++r) {
+      int64_t best = -1;
+      for (int64_t j = 0; j < E; ++j) {
+        int taken = 0;
+        for (int64_t q = 0; q < r; ++q) if (choice[i * k + q] == j) taken = 1;
+        if (taken) continue;
+        if (best < 0 || a[j] > a[best]) best = j;
+      }
+      choice[i * k + r] = (int32_t)best;
+    }
+  }
+  for (int64_t j = 0; j < E; ++j) load[j] = 0;
+  int64_t ndrop = 0, nempty = 0;
+  for (int64_t r = 0; r < k; ++r)
+    for (int64_t i = 0; i < T; ++i) {
+      const int32_t e = choice[i * k + r];
+      if (load[e] < C) { load[e] += 1; held[i * E + e] = 1; }
+      else { dropped[i * k + r] = 1; ++ndrop; }
+    }
+  for (int64_t i = 0; i < T; ++i)
+    for (int64_t r = 0; r < k; ++r) {
+      if (!dropped[i * k + r]) continue;
+      const double *a = A + i * E;
+      int64_t best = -1;
+      for (int64_t j = 0; j < E; ++j) {
+        if (load[j] >= C || held[i * E + j]) continue;
+        if (best < 0 || a[j] > a[best]) best = j;
+      }
+      if (best < 0) { ++nempty; continue; }
+      load[best] += 1; held[i * E + best] = 1;
+    }
+  for (int64_t i = 0; i < T; ++i) {
+    int64_t n = 0;
+    for (int64_t j = 0; j < E; ++j) if (held[i * E + j]) expert_idx[i * k + n++] = (int32_t)j;
+    while (n < k) expert_idx[i * k + n++] = -1;
+  }
+  counts[0] = ndrop; counts[1] = nempty;
+  free(choice); free(held); free(dropped);
   return MSO_OK;
 }

@@ -115,7 +115,7 @@ maxscore_status check_params(const maxscore_params* p) {
   if (p->capacity <= 0 && !(p->capacity_factor > 0.f)) return MAXSCORE_ERR_INVALID_ARG;
   if (p->score_mode == 1 && (p->quant_shift < 0 || p->quant_shift > 14)) return MAXSCORE_ERR_INVALID_ARG;
   if (p->max_sweeps < 0) return MAXSCORE_ERR_INVALID_ARG;
-  if (p->softtopk_mode != 0 && p->softtopk_mode != 1) return MAXSCORE_ERR_INVALID_ARG;
+  if (p->softtopk_mode < 0 || p->softtopk_mode > 2) return MAXSCORE_ERR_INVALID_ARG;
   if (p->softtopk_mode == 1 && (p->rankscale_delta < 0 || p->rankscale_delta > 1 || !isfinite(p->rankscale_beta)))
     return MAXSCORE_ERR_INVALID_ARG;
   if (p->k > p->E) return MAXSCORE_ERR_INFEASIBLE;
@@ -220,7 +220,9 @@ maxscore_status launch_gate(maxscore_ctx* c, const void* hidden, const void* w_g
 maxscore_status launch_softtopk_fwd(maxscore_ctx* c, const float* logits, float* scores, cudaStream_t st) {
   const maxscore_params& p = c->p;
   int blocks = (p.T + 7) / 8; if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
-  if (p.softtopk_mode == 1)
+  if (p.softtopk_mode == 2)
+    itertopk_kernel<false><<<blocks, 256, 0, st>>>(logits, nullptr, nullptr, nullptr, scores, p.T, p.E, p.k);
+  else if (p.softtopk_mode == 1)
     softtopk_rankscale_kernel<false><<<blocks, 256, 0, st>>>(logits, nullptr, nullptr, nullptr, scores, p.T, p.E, p.k, p.t,
                                                              p.rankscale_beta, p.rankscale_delta);
   else
@@ -398,7 +400,9 @@ maxscore_status maxscore_softtopk_bwd(maxscore_ctx* c, const float* logits, cons
   if (!c || !logits || !expert_idx || !dgate_w || !dlogits) return MAXSCORE_ERR_INVALID_ARG;
   const maxscore_params& p = c->p;
   int blocks = (p.T + 7) / 8; if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
-  if (p.softtopk_mode == 1)
+  if (p.softtopk_mode == 2)
+    itertopk_kernel<true><<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, nullptr, dlogits, p.T, p.E, p.k);
+  else if (p.softtopk_mode == 1)
     softtopk_rankscale_kernel<true><<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, nullptr, dlogits, p.T,
                                                                              p.E, p.k, p.t, p.rankscale_beta, p.rankscale_delta);
   else
@@ -413,7 +417,9 @@ maxscore_status maxscore_softtopk_bwd_aux(maxscore_ctx* c, const float* logits, 
   if (!c || !logits || !expert_idx || !dgate_w || !dscores_col || !dlogits) return MAXSCORE_ERR_INVALID_ARG;
   const maxscore_params& p = c->p;
   int blocks = (p.T + 7) / 8; if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
-  if (p.softtopk_mode == 1)
+  if (p.softtopk_mode == 2)
+    itertopk_kernel<true><<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, dscores_col, dlogits, p.T, p.E, p.k);
+  else if (p.softtopk_mode == 1)
     softtopk_rankscale_kernel<true><<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, dscores_col, dlogits,
                                                                              p.T, p.E, p.k, p.t, p.rankscale_beta, p.rankscale_delta);
   else

@@ -225,6 +225,88 @@ softtopk_rankscale_kernel(const float* __restrict__ logits, const int32_t* __res
   }
 }
 
+// IterTopk of Table 2: y^(0) = 0, y^(l) = y^(l-1) + g(x; 1 - y^(l-1)) with g(x; w) = w e^x / sum(w e^x), for
+// l = 1..k.  One warp per token, a lane holds experts lane, lane+32, ...; a level is one weighted sum.  The
+// backward pass (kBackward) keeps the weights of all k levels in registers and runs the recursion in reverse:
+// with z = e^{x - max}, u = w z, s = sum u, r = u / s and rb the gradient of r,
+//   ub = (rb - sum_i rb_i r_i) / s,   zb += ub w,   gradient of y^(l-1) = gradient of y^(l) - ub z,
+// and dx = zb z at the end.  Table 2 has no temperature: the logits enter as they are.
+template <bool kBackward>
+__global__ void __launch_bounds__(256)
+itertopk_kernel(const float* __restrict__ logits, const int32_t* __restrict__ expert_idx,
+                const float* __restrict__ dgate_w, const float* __restrict__ dscores_col,
+                float* __restrict__ out, int T, int E, int k) {
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  for (int tok = blockIdx.x * warps_per_block + (threadIdx.x >> 5); tok < T; tok += gridDim.x * warps_per_block) {
+    const float* row = logits + (size_t)tok * E;
+    float z[kEPL], w[kMaxK][kEPL], sl[kMaxK];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < kEPL; ++j) {
+      const int e = lane + 32 * j;
+      z[j] = e < E ? __ldg(row + e) : -INFINITY;
+      mx = fmaxf(mx, z[j]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+#pragma unroll
+    for (int j = 0; j < kEPL; ++j) z[j] = lane + 32 * j < E ? expf(z[j] - mx) : 0.f;
+    float y[kEPL];
+#pragma unroll
+    for (int j = 0; j < kEPL; ++j) y[j] = 0.f;
+#pragma unroll
+    for (int l = 0; l < kMaxK; ++l) {
+      if (l < k) {
+        float s = 0.f;
+#pragma unroll
+        for (int j = 0; j < kEPL; ++j) { w[l][j] = 1.f - y[j]; s += w[l][j] * z[j]; }
+        s = warp_sum(s);
+        sl[l] = s;
+        const float inv = 1.f / s;
+#pragma unroll
+        for (int j = 0; j < kEPL; ++j) y[j] = fmaf(w[l][j] * z[j], inv, y[j]);
+      }
+    }
+    float* o = out + (size_t)tok * E;
+    if (!kBackward) {
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j) { const int e = lane + 32 * j; if (e < E) o[e] = y[j]; }
+    } else {
+      float yb[kEPL], zb[kEPL];
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j) {
+        const int e = lane + 32 * j;
+        yb[j] = (e < E && dscores_col) ? __ldg(dscores_col + e) : 0.f; zb[j] = 0.f;
+      }
+      for (int c = 0; c < k; ++c) {
+        const int e = __ldg(expert_idx + (size_t)tok * k + c);
+        const float gv = __ldg(dgate_w + (size_t)tok * k + c);
+#pragma unroll
+        for (int j = 0; j < kEPL; ++j) if (lane + 32 * j == e) yb[j] += gv;
+      }
+#pragma unroll
+      for (int l = kMaxK - 1; l >= 0; --l) {
+        if (l < k) {
+          const float inv = 1.f / sl[l];
+          float dot = 0.f;
+#pragma unroll
+          for (int j = 0; j < kEPL; ++j) dot += yb[j] * (w[l][j] * z[j] * inv);
+          dot = warp_sum(dot);
+#pragma unroll
+          for (int j = 0; j < kEPL; ++j) {
+            const float ub = (yb[j] - dot) * inv;
+            zb[j] = fmaf(ub, w[l][j], zb[j]);
+            yb[j] = fmaf(-ub, z[j], yb[j]);
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < kEPL; ++j) { const int e = lane + 32 * j; if (e < E) o[e] = zb[j] * z[j]; }
+    }
+  }
+}
+
 // Auxiliary load-balance loss, Eq. 9: L = lambda / (E T^2) * sum_j (sum_i A_ij) * load_j, and its
 // gradient with respect to A (P is a constant): dL/dA_ij = lambda * load_j / (E T^2) for every token i.
 // Column sums are taken by warps over rows (lane l owns columns l, l+32, ...) in double precision and

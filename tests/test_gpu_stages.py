@@ -518,3 +518,27 @@ def test_route_bwd_whole_call_at_the_small_configs(ms, orc, synth, name):
     assert_sum_close(np32(dW), r_dW, m_dW, 1e-5, "dW")
     assert_row_rel(np32(dW), r_dW, 1e-5, "dW (row-relative)")
     _assert_out(f64(dH), r_dH, m_dH, wl.dtype, "dH")
+
+
+@pytest.mark.parametrize("T,E,k", [(512, 8, 2), (1000, 16, 2), (777, 64, 8), (515, 128, 8), (33, 5, 3), (64, 20, 1)])
+def test_itertopk_of_table_2_fwd_bwd(ms, orc, synth, T, E, k):
+    """softtopk_mode 2: IterTopk as Table 2 prints it, forward and backward, against the oracle."""
+    L = synth.logits_like(T, E, seed=12)
+    ctx = _ctx(ms, T, 64, E, k, cf=float(E), softtopk_mode=2)
+    Ld = L.to(DEV)
+    A = torch.empty_like(Ld)
+    ms.softtopk_fwd(ctx, Ld, A)
+    ref = orc.itertopk_fwd(f64(L), k)
+    assert_row_rel(np32(A), ref, 1e-5, "IterTopk fwd")          # later levels subtract: held to the row maximum
+    assert np.abs(np32(A).sum(axis=1) - k).max() <= 1e-4
+    g = torch.Generator().manual_seed(13)
+    idx = torch.stack([torch.randperm(E, generator=g)[:k].sort().values for _ in range(T)]).to(torch.int32)
+    dg = torch.randn(T, k, generator=g)
+    col = torch.randn(E, generator=g) * 0.1
+    dL = torch.empty_like(Ld)
+    ms.softtopk_bwd_aux(ctx, Ld, idx.to(DEV), dg.to(DEV), col.to(DEV), dL)
+    G = np.tile(f64(col), (T, 1))
+    G[np.arange(T)[:, None], idx.numpy().astype(np.int64)] += f64(dg)
+    refb = orc.itertopk_bwd(f64(L), G, k)
+    scale = np.abs(G).max(axis=1, keepdims=True) * k
+    assert (np.abs(np32(dL) - refb) <= 2e-5 * scale + 1e-12).all()

@@ -341,3 +341,72 @@ def test_hashed_float_keys_hand_values_and_bounds(orc):
     i0, _, _ = orc.flow_ssp(orc.keys_from_scores(S), k, C)
     i1, _, _ = orc.flow_ssp(orc.keys_from_scores_hashed(S), k, C)
     assert abs(orc.total_score(S, i0) - orc.total_score(S, i1)) < 4e-9 * T * k
+
+
+# ------------------------------------------------------------------------------------------- iterative rerouting
+def _reroute_by_hand(A, k, C):
+    """Independent restatement with Python lists and sorting (no shared code with the C routine)."""
+    T, E = A.shape
+    order = [sorted(range(E), key=lambda j: (-A[i, j], j))[:k] for i in range(T)]
+    load = [0] * E
+    held = [set() for _ in range(T)]
+    dropped = []
+    for r in range(k):
+        for i in range(T):
+            e = order[i][r]
+            if load[e] < C:
+                load[e] += 1; held[i].add(e)
+            else:
+                dropped.append((i, r))
+    empty = 0
+    for i, r in sorted(dropped):
+        free = [j for j in range(E) if load[j] < C and j not in held[i]]
+        if not free:
+            empty += 1
+            continue
+        e = min(free, key=lambda j: (-A[i, j], j))
+        load[e] += 1; held[i].add(e)
+    idx = np.full((T, k), -1, np.int32)
+    for i in range(T):
+        s = sorted(held[i])
+        idx[i, :len(s)] = s
+    return idx, np.array(load, np.int32), len(dropped), empty
+
+
+def test_iterative_reroute_small_cases_and_invariants(orc):
+    rng = np.random.default_rng(31)
+    for (T, E, k, C) in [(12, 4, 2, 6), (40, 8, 2, 10), (33, 5, 3, 20), (64, 16, 4, 16), (9, 3, 3, 9), (20, 4, 2, 7)]:
+        A = rng.random((T, E)).astype(np.float32).astype(np.float64)
+        idx, load, nd, ne = orc.iterative_reroute(A, k, C)
+        widx, wload, wnd, wne = _reroute_by_hand(A, k, C)
+        np.testing.assert_array_equal(idx, widx); np.testing.assert_array_equal(load, wload)
+        assert (nd, ne) == (wnd, wne)
+        assert (load <= C).all() and load.sum() == T * k - ne
+        filled = idx >= 0
+        assert np.array_equal(np.bincount(idx[filled], minlength=E), load)
+        for i in range(T):                                   # distinct experts, ascending, empty slots last
+            row = idx[i][idx[i] >= 0]
+            assert (np.diff(row) > 0).all() and (idx[i][len(row):] == -1).all()
+    # loose capacity: nothing is dropped and the result is plain top-k
+    A = rng.random((50, 8))
+    idx, load, nd, ne = orc.iterative_reroute(A, 3, 50)
+    assert nd == 0 and ne == 0
+    np.testing.assert_array_equal(idx, np.sort(np.argsort(-A, axis=1, kind="stable")[:, :3], axis=1))
+
+
+def test_iterative_reroute_hand_case_and_suboptimality(orc):
+    """Three tokens, two experts, k = 1, C = 2, affinities chosen so that level 1 overloads expert 0:
+    tokens 0 and 1 take it, token 2 is dropped and rerouted to expert 1.  The exact flow would instead move
+    the token that loses least (token 1): greedy rerouting is feasible but not optimal (Sec. 3.2's trade-off)."""
+    A = np.array([[0.9, 0.1], [0.6, 0.5], [0.8, 0.0]])
+    idx, load, nd, ne = orc.iterative_reroute(A, 1, 2)
+    np.testing.assert_array_equal(idx, [[0], [0], [1]])
+    np.testing.assert_array_equal(load, [2, 1])
+    assert (nd, ne) == (1, 0)
+    oidx, _, _ = orc.flow_ssp(orc.keys_from_scores(A), 1, 2)
+    np.testing.assert_array_equal(oidx, [[0], [1], [0]])
+    assert orc.total_score(A, oidx) > orc.total_score(A, idx)
+    # tied affinities go to the lowest expert index at both stages
+    A = np.array([[0.5, 0.5, 0.5], [0.5, 0.5, 0.5], [0.5, 0.5, 0.5]])
+    idx, load, nd, ne = orc.iterative_reroute(A, 1, 1)
+    np.testing.assert_array_equal(idx, [[0], [1], [2]])
