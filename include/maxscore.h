@@ -211,6 +211,20 @@ maxscore_status maxscore_softtopk_bwd_aux(maxscore_ctx* ctx, const float* logits
 maxscore_status maxscore_assign(maxscore_ctx* ctx, const float* matrix, int32_t* expert_idx,
                                 int32_t* expert_load, maxscore_stats* stats, void* cuda_stream);
 
+/* Iterative rerouting (Sec. 2.3, the Switch Transformers paragraph; the assignment of "MaxScore-I", Sec. 4.1):
+ * the fast, approximate alternative to the flow of Eq. 7-8 that Sec. 3.2 names for k > 2.
+ *   stage 1  top-k by affinity with capacity: choice level 1 of every token is served before level 2, ..., within
+ *            a level in ascending token index; a pair is accepted while its expert holds fewer than C tokens;
+ *   stage 2  the dropped pairs, in ascending token index and within a token in level order, go to the expert of
+ *            highest affinity among those with room that the token does not hold, or stay empty if there is none.
+ * Ties in affinity go to the lowest expert index.  The paper fixes neither serving order: both are this library's
+ * reading.  scores [T, E] fp32 (finite) in; expert_idx [T, k] out, ascending, empty slots = -1 and last (index build,
+ * dispatch and combine skip them); expert_load [E] out; counts [2] int32 DEVICE memory out: pairs dropped in stage 1,
+ * slots left empty after stage 2.  Uses the context's workspace.  The result is feasible but in general not the
+ * maximum of Eq. 8. */
+maxscore_status maxscore_assign_iterative(maxscore_ctx* ctx, const float* scores, int32_t* expert_idx,
+                                          int32_t* expert_load, int32_t* counts, void* cuda_stream);
+
 /* Slot indices of an assignment: slot_idx [T, k], slot_token [E, C], expert_load [E]. */
 maxscore_status maxscore_index_build(maxscore_ctx* ctx, const int32_t* expert_idx, int32_t* slot_idx,
                                      int32_t* slot_token, int32_t* expert_load, void* cuda_stream);

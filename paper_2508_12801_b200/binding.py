@@ -48,7 +48,7 @@ EXPORTS = ["maxscore_capacity", "maxscore_workspace_bytes", "maxscore_create", "
            "maxscore_assign", "maxscore_index_build", "maxscore_combine_bwd", "maxscore_gate_bwd",
            "maxscore_route_dispatch_host", "maxscore_index_build_noalloc", "maxscore_aux_loss",
            "maxscore_softtopk_bwd_aux", "maxscore_check_internal", "maxscore_launch_count",
-           "maxscore_test_raise_internal"]
+           "maxscore_test_raise_internal", "maxscore_assign_iterative"]
 
 
 def _load():
@@ -203,6 +203,12 @@ def aux_loss(ctx, scores, expert_load, lam, loss, dscores_col, stream=None):
 def assign(ctx, matrix, expert_idx, expert_load, stats, stream=None):
     _check(_lib.maxscore_assign(ctx.handle, _ptr(matrix), _ptr(expert_idx), _ptr(expert_load), _ptr(stats),
                                 _stream(stream)), "maxscore_assign")
+
+
+def assign_iterative(ctx, scores, expert_idx, expert_load, counts, stream=None):
+    """Top-k with capacity, then greedy rerouting of the dropped pairs; counts is an int32[2] device tensor."""
+    _check(_lib.maxscore_assign_iterative(ctx.handle, _ptr(scores), _ptr(expert_idx), _ptr(expert_load), _ptr(counts),
+                                          _stream(stream)), "maxscore_assign_iterative")
 
 
 def index_build(ctx, expert_idx, slot_idx, slot_token, expert_load, stream=None):

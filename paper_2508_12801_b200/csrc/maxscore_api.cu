@@ -15,6 +15,7 @@
 #include "gate.cuh"
 #include "move.cuh"
 #include "softtopk.cuh"
+#include "reroute.cuh"
 
 using namespace msr;
 
@@ -50,7 +51,7 @@ int32_t capacity_of(const maxscore_params& p) {
 }
 
 struct Layout {          // byte offsets inside the workspace
-  size_t state, aux, cand, rec_val, rec_meta, rec_pos, rec_bxc, rec_ndv, rec_off, rec_cnt, rec_aarg, cache_x, cache_id, cache_bound, cache_raw, block_counts, wt, error_flag, dls, wk, dwpart, total;
+  size_t state, aux, cand, rec_val, rec_meta, rec_pos, rec_bxc, rec_ndv, rec_off, rec_cnt, rec_aarg, rr_choice, rr_rank, rr_cnt, rr_base, rr_held, rr_dropped, cache_x, cache_id, cache_bound, cache_raw, block_counts, wt, error_flag, dls, wk, dwpart, total;
   int Npad, n_idx_blocks;
   int rec_cap;                                // entries of the exact phase's candidate records
   int Kpad, dw_splits, dw_tokens_per_split;   // tensor-core backward GEMMs (bf16 I/O)
@@ -79,6 +80,13 @@ Layout layout_of(const maxscore_params& p) {
   l.rec_off = off; off = align_up(off + sizeof(int32_t) * (size_t)p.T, 256);
   l.rec_cnt = off; off = align_up(off + sizeof(int32_t) * (size_t)p.T, 256);
   l.rec_aarg = off; off = align_up(off + sizeof(int32_t) * (size_t)p.T, 256);
+  // iterative rerouting (maxscore_assign_iterative)
+  l.rr_choice = off; off = align_up(off + sizeof(int32_t) * (size_t)p.k * p.T, 256);
+  l.rr_rank = off; off = align_up(off + sizeof(int32_t) * (size_t)p.k * p.T, 256);
+  l.rr_cnt = off; off = align_up(off + sizeof(int32_t) * (size_t)p.k * p.E, 256);
+  l.rr_base = off; off = align_up(off + sizeof(int32_t) * (size_t)(p.k + 1) * p.E, 256);
+  l.rr_held = off; off = align_up(off + sizeof(uint4) * (size_t)p.T, 256);
+  l.rr_dropped = off; off = align_up(off + (size_t)p.T, 256);
   l.cache_x = off; off = align_up(off + sizeof(float) * (size_t)kCacheN * p.T, 256);
   l.cache_id = off; off = align_up(off + (size_t)kCacheN * p.T, 256);
   l.cache_bound = off; off = align_up(off + sizeof(long long) * (size_t)p.T, 256);
@@ -603,6 +611,39 @@ maxscore_status maxscore_route_bwd(maxscore_ctx* c, const void* dY, const void* 
   s = maxscore_softtopk_bwd(c, logits, expert_idx, dgate_w, dlogits, stream);
   if (s) return s;
   return maxscore_gate_bwd(c, hidden, w_gate, dlogits, dw_gate, dH, stream);
+}
+
+maxscore_status maxscore_assign_iterative(maxscore_ctx* c, const float* scores, int32_t* expert_idx, int32_t* expert_load,
+                                          int32_t* counts, void* stream) {
+  if (!c || !scores || !expert_idx || !expert_load || !counts) return MAXSCORE_ERR_INVALID_ARG;
+  const maxscore_params& p = c->p;
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t* choice = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_choice);
+  int32_t* rank = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_rank);
+  int32_t* cnt = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_cnt);
+  int32_t* base = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_base);
+  uint4* held = reinterpret_cast<uint4*>(c->ws + c->lay.rr_held);
+  unsigned char* dropped = reinterpret_cast<unsigned char*>(c->ws + c->lay.rr_dropped);
+  int32_t* bc = reinterpret_cast<int32_t*>(c->ws + c->lay.block_counts);
+  MS_CUDA(cudaMemsetAsync(counts, 0, 2 * sizeof(int32_t), st));
+  const int warp_blocks = std::min((p.T + 7) / 8, c->sm_count * 8);
+  reroute_choices_kernel<<<warp_blocks, 256, 0, st>>>(scores, choice, p.T, p.E, p.k);
+  MS_LAUNCH_CHECK("reroute_choices_kernel");
+  for (int r = 0; r < p.k; ++r) {     // rank of every token among the tokens that chose the same expert at level r
+    index_count_kernel<<<c->lay.n_idx_blocks, kIdxTok, 0, st>>>(choice + (size_t)r * p.T, bc, p.T, p.E, 1);
+    index_fill_kernel<<<c->lay.n_idx_blocks, kIdxTok, 0, st>>>(choice + (size_t)r * p.T, bc, rank + (size_t)r * p.T, choice,
+                                                              cnt + (size_t)r * p.E, p.T, p.E, 1, 0);
+    MS_LAUNCH_CHECK("index_fill_kernel(level)");
+  }
+  reroute_base_kernel<<<1, 128, 0, st>>>(cnt, base, p.E, p.k, c->C);
+  const int tok_blocks = std::min((p.T + 255) / 256, c->sm_count * 8);
+  reroute_accept_kernel<<<tok_blocks, 256, 0, st>>>(choice, rank, base, held, dropped, counts, p.T, p.E, p.k, c->C);
+  reroute_place_kernel<<<1, kRerouteThreads, sizeof(RerouteShared), st>>>(scores, base, held, dropped, expert_load, counts,
+                                                                         p.T, p.E, p.k, c->C);
+  reroute_write_kernel<<<tok_blocks, 256, 0, st>>>(held, expert_idx, p.T, p.k);
+  MS_LAUNCH_CHECK("reroute kernels");
+  c->launches += 5 + 2 * p.k;
+  return MAXSCORE_OK;
 }
 
 long long maxscore_launch_count(const maxscore_ctx* c) { return c ? c->launches : -1; }

@@ -542,3 +542,38 @@ def test_itertopk_of_table_2_fwd_bwd(ms, orc, synth, T, E, k):
     refb = orc.itertopk_bwd(f64(L), G, k)
     scale = np.abs(G).max(axis=1, keepdims=True) * k
     assert (np.abs(np32(dL) - refb) <= 2e-5 * scale + 1e-12).all()
+
+
+@pytest.mark.parametrize("T,E,k,cf,skew", [(512, 8, 2, 1.0, False), (4096, 16, 2, 1.0, False), (1000, 16, 4, 1.0, False),
+                                            (2048, 64, 8, 1.0, False), (2048, 64, 8, 1.25, True), (300, 8, 2, 1.5, True),
+                                            (8192, 64, 8, 1.0, False), (129, 5, 5, 1.0, False), (3000, 128, 8, 1.0, True)])
+def test_iterative_rerouting_bit_exact(ms, orc, synth, T, E, k, cf, skew):
+    """maxscore_assign_iterative against the oracle's top-k-with-capacity + greedy rerouting: with both serving
+    orders fixed the result is unique, so everything is compared bit for bit.  Also: how far the greedy result
+    is from the exact flow's optimum on the same scores."""
+    wl = synth.Workload("a", T, 64, E, k, cf, "bf16", skew=skew)
+    L = synth.logits_like(T, E, seed=14, bias=synth.expert_bias(wl, 14))
+    A = torch.from_numpy(orc.softtopk_fwd(f64(L), k, 1.0).astype(np.float32))
+    ctx = _ctx(ms, T, 64, E, k, cf=cf)
+    C = ctx.capacity
+    idx = torch.empty(T, k, dtype=torch.int32, device=DEV)
+    load = torch.empty(E, dtype=torch.int32, device=DEV)
+    counts = torch.full((2,), -1, dtype=torch.int32, device=DEV)
+    for _ in range(2):                                    # twice: the workspace must come back usable
+        ms.assign_iterative(ctx, A.to(DEV), idx, load, counts)
+    torch.cuda.synchronize()
+    oidx, oload, ond, one = orc.iterative_reroute(f64(A), k, C)
+    np.testing.assert_array_equal(idx.cpu().numpy(), oidx)
+    np.testing.assert_array_equal(load.cpu().numpy(), oload)
+    assert counts.cpu().tolist() == [ond, one]
+    assert (oload <= C).all()
+    # the slots of the greedy assignment go through the same index build (empty slots are skipped)
+    slot_idx = torch.empty(T, k, dtype=torch.int32, device=DEV)
+    slot_token = torch.empty(E, C, dtype=torch.int32, device=DEV)
+    load2 = torch.empty(E, dtype=torch.int32, device=DEV)
+    ms.index_build(ctx, idx, slot_idx, slot_token, load2)
+    np.testing.assert_array_equal(load2.cpu().numpy(), oload)
+    # greedy is feasible, never better than the flow's optimum
+    if one == 0:
+        fidx, _, _ = orc.flow_condensed(orc.keys_from_scores(f64(A)), k, C)
+        assert orc.total_score(f64(A), oidx) <= orc.total_score(f64(A), fidx) * (1 + 1e-12)
