@@ -161,6 +161,22 @@ def itertopk_bwd(L, G, k: int) -> np.ndarray:
     return dL
 
 
+def alg1_top1_sinkhorn(A, Cap: int, eps: float, iters: int, want_plan: bool = False):
+    """Algorithm 1 (top-2): top-1, then capped Sinkhorn on the residual problem and argmax rounding.
+    Returns (first [T], second [T] with -1 = dropped, resid [E], top-1 pairs beyond Cap, seconds dropped[, plan])."""
+    A = _f64(A)
+    T, E = A.shape
+    first = np.empty(T, np.int32); second = np.empty(T, np.int32)
+    resid = np.empty(E, np.int64); counts = np.zeros(2, np.int64)
+    plan = np.empty((T, E), np.float64) if want_plan else None
+    rc = lib().mso_alg1_top1_sinkhorn(I64(T), I64(E), I64(Cap), _p(A), C.c_double(eps), I64(iters), _p(first), _p(second),
+                                      _p(plan) if want_plan else None, _p(resid), _p(counts))
+    if rc:
+        raise ValueError("alg1_top1_sinkhorn: bad arguments")
+    out = (first, second, resid, int(counts[0]), int(counts[1]))
+    return out + (plan,) if want_plan else out
+
+
 def iterative_reroute(A, k: int, Cap: int):
     """Top-k with capacity, then greedy rerouting of the dropped pairs (Sec. 2.3).  Returns
     (expert_idx [T,k] ascending with -1 last, load [E], pairs dropped in stage 1, slots left empty)."""

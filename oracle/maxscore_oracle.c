@@ -32,12 +32,19 @@
  * largest; ties go to the lowest expert index.
  *
  * Every function here is pinned by tests/test_oracle_*.py against closed
- * forms, library routines, brute force or invariants.  One pair is "parity
- * unpinned" against the paper: mso_softtopk_rankscale_fwd/bwd, the literal
- * readings of Eq. 6 (pinned by the formula's own special cases only: the
- * paper prints no value that tells the readings of Eq. 6 apart).
+ * forms, library routines, brute force or invariants.  "Parity unpinned"
+ * against the paper: mso_softtopk_rankscale_fwd/bwd, the literal readings of
+ * Eq. 6 (pinned by the formula's own special cases only: the paper prints no
+ * value that tells the readings of Eq. 6 apart), and the second stage of
+ * mso_alg1_top1_sinkhorn (the paper names Sinkhorn but gives neither its
+ * regulariser, nor its iteration count, nor how the plan is rounded; pinned by
+ * what the mathematics fixes: marginals, the LP optimum on tiny cases, plain
+ * top-2 under loose capacity).
  *   mso_softtopk_rankscale_fwd/bwd   Eq. 6 read literally (rank-scaled softmax)
  *   mso_itertopk_fwd/bwd             IterTopk of Table 2 and its derivative
+ *   mso_alg1_top1_sinkhorn           Algorithm 1: top-1, then Sinkhorn on the residual problem (k = 2);
+ *                                    Sinkhorn's regulariser, iteration count and rounding are this build's
+ *                                    reading: parity unpinned against the paper
  *   mso_iterative_reroute            top-k with capacity, then greedy rerouting of the dropped pairs
  *                                    (Sec. 2.3; the serving orders are this build's reading)
  *   mso_aux_loss_grad                derivative of Eq. 9 with respect to A
@@ -895,5 +902,97 @@ int mso_iterative_reroute(int64_t T, int64_t E, int64_t k, int64_t C, const doub
   }
   counts[0] = ndrop; counts[1] = nempty;
   free(choice); free(held); free(dropped);
+  return MSO_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* Algorithm 1: maximum score routing for top-2 (Sec. 3.2): top-1, then  */
+/* Sinkhorn on what is left.  Steps as the algorithm numbers them:       */
+/*   1  c_j = C                       (the caller's capacity, 2n/e in the paper)   */
+/*   2  a = the affinities A          (given)                            */
+/*   4  mask = one-hot of argmax_j a_ij (ties: lowest expert index)      */
+/*   5  the masked pair is removed from the second stage                 */
+/*   6  c_j = max(0, c_j - sum_i mask_ij)                                */
+/*   7  k_i = 1                                                          */
+/*   8-9  Sinkhorn for max sum P_ij a_ij over rows summing to 1 and      */
+/*        columns within c.                                              */
+/* What the paper leaves open, and the reading taken (all "parity        */
+/* unpinned against the paper"):                                         */
+/*   - Sinkhorn: entropic regularisation eps, kernel K_ij = exp((a_ij -  */
+/*     m_i) / eps) over the unmasked pairs (m_i the row maximum, which   */
+/*     the row scaling absorbs), `iters` rounds of                       */
+/*         u_i = 1 / sum_j K_ij v_j,  t_j = sum_i u_i K_ij,  v_j = min(1, c_j / t_j)  */
+/*     (columns are capped, not forced to equal c: the residual          */
+/*     capacities sum to at least n), then a last row scaling.  Its      */
+/*     fixed point has rows summing to 1 and every column either         */
+/*     uncapped (v = 1) or exactly full: the optimality conditions of    */
+/*     the entropic problem with capacity upper bounds.                  */
+/*   - rounding: token i takes argmax_j of its plan row (ties: lowest    */
+/*     index); per expert the first c_j such tokens in ascending token   */
+/*     index are kept, the rest lose their second expert (-1).           */
+/*   - top-1 pairs are never dropped here, even beyond C (step 6 clips   */
+/*     the residual at 0); the E x C buffers drop them downstream.       */
+/* Outputs: first/second [T] (second = -1: dropped), plan [T,E] (may be  */
+/* NULL), resid [E] residual capacities, counts[0] = top-1 pairs beyond  */
+/* C, counts[1] = second choices dropped.                                */
+int mso_alg1_top1_sinkhorn(int64_t T, int64_t E, int64_t C, const double *A, double eps, int64_t iters,
+                           int32_t *first, int32_t *second, double *plan, int64_t *resid, int64_t *counts) {
+  if (E < 2 || C < 0 || !(eps > 0.0) || iters < 0) return MSO_ERR_ARG;
+  double *K = (double *)malloc(sizeof(double) * (size_t)(T * E));
+  double *u = (double *)malloc(sizeof(double) * (size_t)T);
+  double *v = (double *)malloc(sizeof(double) * (size_t)E);
+  double *t = (double *)malloc(sizeof(double) * (size_t)E);
+  int64_t *cnt = (int64_t *)calloc((size_t)E, sizeof(int64_t));
+  if (!K || !u || !v || !t || !cnt) { free(K); free(u); free(v); free(t); free(cnt); return MSO_ERR_ALLOC; }
+  /* steps 4-6 */
+  for (int64_t i = 0; i < T; ++i) {
+    const double *a = A + i * E;
+    int64_t best = 0;
+    for (int64_t j = 1; j < E; ++j) if (a[j] > a[best]) best = j;
+    first[i] = (int32_t)best; cnt[best] += 1;
+  }
+  int64_t over = 0;
+  for (int64_t j = 0; j < E; ++j) {
+    resid[j] = C - cnt[j] > 0 ? C - cnt[j] : 0;
+    if (cnt[j] > C) over += cnt[j] - C;
+  }
+  /* steps 7-9 */
+  for (int64_t i = 0; i < T; ++i) {
+    const double *a = A + i * E;
+    double m = -INFINITY;
+    for (int64_t j = 0; j < E; ++j) if (j != first[i] && a[j] > m) m = a[j];
+    for (int64_t j = 0; j < E; ++j) K[i * E + j] = (j == first[i]) ? 0.0 : exp((a[j] - m) / eps);
+  }
+  for (int64_t j = 0; j < E; ++j) v[j] = resid[j] > 0 ? 1.0 : 0.0;
+  for (int64_t it = 0; it <= iters; ++it) {
+    for (int64_t i = 0; i < T; ++i) {
+      double s = 0.0;
+      for (int64_t j = 0; j < E; ++j) s += K[i * E + j] * v[j];
+      u[i] = s > 0.0 ? 1.0 / s : 0.0;
+    }
+    if (it == iters) break;                 /* the last row scaling */
+    for (int64_t j = 0; j < E; ++j) t[j] = 0.0;
+    for (int64_t i = 0; i < T; ++i)
+      for (int64_t j = 0; j < E; ++j) t[j] += u[i] * K[i * E + j];
+    for (int64_t j = 0; j < E; ++j) {
+      if (resid[j] <= 0) v[j] = 0.0;
+      else v[j] = (t[j] > (double)resid[j]) ? (double)resid[j] / t[j] : 1.0;
+    }
+  }
+  int64_t *taken = (int64_t *)calloc((size_t)E, sizeof(int64_t));
+  if (!taken) { free(K); free(u); free(v); free(t); free(cnt); return MSO_ERR_ALLOC; }
+  int64_t dropped = 0;
+  for (int64_t i = 0; i < T; ++i) {
+    int64_t best = -1; double pb = 0.0;
+    for (int64_t j = 0; j < E; ++j) {
+      const double p = u[i] * K[i * E + j] * v[j];
+      if (plan) plan[i * E + j] = p;
+      if (p > pb) { pb = p; best = j; }     /* strictly larger: ties keep the lowest index; zero mass is no choice */
+    }
+    if (best >= 0 && taken[best] < resid[best]) { taken[best] += 1; second[i] = (int32_t)best; }
+    else { second[i] = -1; ++dropped; }
+  }
+  counts[0] = over; counts[1] = dropped;
+  free(K); free(u); free(v); free(t); free(cnt); free(taken);
   return MSO_OK;
 }

@@ -410,3 +410,63 @@ def test_iterative_reroute_hand_case_and_suboptimality(orc):
     A = np.array([[0.5, 0.5, 0.5], [0.5, 0.5, 0.5], [0.5, 0.5, 0.5]])
     idx, load, nd, ne = orc.iterative_reroute(A, 1, 1)
     np.testing.assert_array_equal(idx, [[0], [1], [2]])
+
+
+# ------------------------------------------------------------------------------------------- Algorithm 1
+def test_alg1_first_stage_is_plain_top1_and_residuals(orc):
+    rng = np.random.default_rng(41)
+    T, E, C = 60, 6, 20
+    A = rng.random((T, E))
+    first, second, resid, over, dropped, plan = orc.alg1_top1_sinkhorn(A, C, 0.05, 2000, want_plan=True)
+    np.testing.assert_array_equal(first, A.argmax(axis=1))                       # step 4: one-hot of the arg-max
+    cnt = np.bincount(first, minlength=E)
+    np.testing.assert_array_equal(resid, np.maximum(0, C - cnt))                 # step 6
+    assert over == np.maximum(0, cnt - C).sum()
+    # the plan: masked pairs carry nothing, rows sum to one, capped columns stay within the residual capacity
+    assert (plan[np.arange(T), first] == 0).all()
+    np.testing.assert_allclose(plan.sum(axis=1), 1.0, atol=1e-12)
+    assert (plan.sum(axis=0) <= resid * (1 + 1e-3) + 1e-9).all()
+    # rounding: the second expert differs from the first, is the plan's arg-max unless dropped, and no expert
+    # gets more seconds than it has room for
+    keep = second >= 0
+    assert (second[keep] != first[keep]).all()
+    np.testing.assert_array_equal(second[keep], plan.argmax(axis=1)[keep])
+    assert (np.bincount(second[keep], minlength=E) <= resid).all()
+    assert dropped == (~keep).sum()
+    # ties in the first stage go to the lowest index
+    f2, *_ = orc.alg1_top1_sinkhorn(np.full((4, 3), 0.5), 4, 0.1, 3)
+    np.testing.assert_array_equal(f2, 0)
+
+
+def test_alg1_with_loose_capacity_is_plain_top2(orc):
+    rng = np.random.default_rng(42)
+    A = rng.random((80, 8))
+    first, second, resid, over, dropped = orc.alg1_top1_sinkhorn(A, 80, 0.07, 10)   # nobody is ever capped
+    order = np.argsort(-A, axis=1, kind="stable")
+    np.testing.assert_array_equal(first, order[:, 0])
+    np.testing.assert_array_equal(second, order[:, 1])
+    assert over == 0 and dropped == 0
+
+
+def test_alg1_second_stage_tends_to_the_lp_optimum(orc):
+    """Small regulariser, many iterations: the plan's value approaches the optimum of the residual transport
+    problem (rows = 1, columns <= residual capacity, masked pairs excluded), computed by scipy's LP solver."""
+    from scipy.optimize import linprog
+    rng = np.random.default_rng(43)
+    T, E, C = 10, 4, 5
+    A = rng.random((T, E))
+    first, second, resid, over, dropped, plan = orc.alg1_top1_sinkhorn(A, C, 0.01, 4000, want_plan=True)
+    cost = -A.copy(); cost[np.arange(T), first] = 0.0
+    bounds = [(0, 0) if j == first[i] else (0, None) for i in range(T) for j in range(E)]
+    A_eq = np.zeros((T, T * E)); A_ub = np.zeros((E, T * E))
+    for i in range(T):
+        A_eq[i, i * E:(i + 1) * E] = 1
+    for j in range(E):
+        A_ub[j, j::E] = 1
+    res = linprog(cost.reshape(-1), A_ub=A_ub, b_ub=resid.astype(float), A_eq=A_eq, b_eq=np.ones(T), bounds=bounds)
+    assert res.status == 0
+    got = (plan * A).sum()
+    # from above only by what the not yet fully converged column caps allow; from below by the entropic gap
+    # (at most eps * log E per token)
+    assert got <= -res.fun + 1e-3 and got >= -res.fun - 0.02 * T
+    np.testing.assert_allclose(plan.sum(axis=0), np.minimum(plan.sum(axis=0), resid), atol=1e-3)
