@@ -211,6 +211,26 @@ maxscore_status maxscore_softtopk_bwd_aux(maxscore_ctx* ctx, const float* logits
 maxscore_status maxscore_assign(maxscore_ctx* ctx, const float* matrix, int32_t* expert_idx,
                                 int32_t* expert_load, maxscore_stats* stats, void* cuda_stream);
 
+/* Algorithm 1 (Sec. 3.2): maximum score routing for top-2 the way the paper trains it.  Needs k = 2.
+ *   steps 1-2  c_j = C (the context's capacity; 2n/e in the paper); a = scores (SoftTopk affinities of the caller)
+ *   steps 4-6  every token's best expert (ties: lowest index) is fixed; the pair is removed from the second stage;
+ *              c_j = max(0, c_j - number of tokens whose best expert is j)
+ *   steps 7-9  one more expert per token by Sinkhorn on the residual problem.
+ * The paper names Sinkhorn and nothing else; this library's reading: entropic regularisation sinkhorn_eps (in units of
+ * score), K_ij = exp(a_ij / eps) over the pairs not fixed in step 4, sinkhorn_iters rounds of
+ *     u_i = 1 / sum_j K_ij v_j,   t_j = sum_i u_i K_ij,   v_j = min(1, c_j / t_j)
+ * (columns capped at the residual capacity rather than forced to meet it), a last row scaling, then every token takes
+ * the arg-max of its plan row (ties: lowest index) and per expert the first c_j such tokens in ascending token index keep
+ * it; the others end with one expert only.  Best-expert pairs are never dropped here, even beyond C: index build,
+ * dispatch and combine skip what does not fit.  All arithmetic is fp64.
+ *   scores [T, E] fp32 in; expert_idx [T, 2] out, ascending, -1 (dropped second expert) last; expert_load [E] out;
+ *   plan [T, E] fp64 out or NULL (the row-scaled plan u_i K_ij v_j); counts [2] int32 DEVICE memory out: best-expert
+ *   pairs beyond C, second experts dropped.  Uses the context's workspace.  The result approximates the maximum of
+ *   Eq. 8; maxscore_assign gives the exact one. */
+maxscore_status maxscore_assign_top2_sinkhorn(maxscore_ctx* ctx, const float* scores, float sinkhorn_eps,
+                                              int32_t sinkhorn_iters, int32_t* expert_idx, int32_t* expert_load,
+                                              double* plan, int32_t* counts, void* cuda_stream);
+
 /* Iterative rerouting (Sec. 2.3, the Switch Transformers paragraph; the assignment of "MaxScore-I", Sec. 4.1):
  * the fast, approximate alternative to the flow of Eq. 7-8 that Sec. 3.2 names for k > 2.
  *   stage 1  top-k by affinity with capacity: choice level 1 of every token is served before level 2, ..., within

@@ -48,7 +48,7 @@ EXPORTS = ["maxscore_capacity", "maxscore_workspace_bytes", "maxscore_create", "
            "maxscore_assign", "maxscore_index_build", "maxscore_combine_bwd", "maxscore_gate_bwd",
            "maxscore_route_dispatch_host", "maxscore_index_build_noalloc", "maxscore_aux_loss",
            "maxscore_softtopk_bwd_aux", "maxscore_check_internal", "maxscore_launch_count",
-           "maxscore_test_raise_internal", "maxscore_assign_iterative"]
+           "maxscore_test_raise_internal", "maxscore_assign_iterative", "maxscore_assign_top2_sinkhorn"]
 
 
 def _load():
@@ -203,6 +203,13 @@ def aux_loss(ctx, scores, expert_load, lam, loss, dscores_col, stream=None):
 def assign(ctx, matrix, expert_idx, expert_load, stats, stream=None):
     _check(_lib.maxscore_assign(ctx.handle, _ptr(matrix), _ptr(expert_idx), _ptr(expert_load), _ptr(stats),
                                 _stream(stream)), "maxscore_assign")
+
+
+def assign_top2_sinkhorn(ctx, scores, sinkhorn_eps, sinkhorn_iters, expert_idx, expert_load, plan, counts, stream=None):
+    """Algorithm 1 (k = 2): top-1, then capped Sinkhorn on the residual problem; plan may be None."""
+    _check(_lib.maxscore_assign_top2_sinkhorn(ctx.handle, _ptr(scores), C.c_float(sinkhorn_eps), C.c_int32(sinkhorn_iters),
+                                              _ptr(expert_idx), _ptr(expert_load), _ptr(plan), _ptr(counts),
+                                              _stream(stream)), "maxscore_assign_top2_sinkhorn")
 
 
 def assign_iterative(ctx, scores, expert_idx, expert_load, counts, stream=None):

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmaxscore.so")
 SOURCES = ["maxscore_api.cu"]
-HEADERS = ["common.cuh", "flow.cuh", "gate.cuh", "move.cuh", "softtopk.cuh", "reroute.cuh",
+HEADERS = ["common.cuh", "flow.cuh", "gate.cuh", "move.cuh", "softtopk.cuh", "reroute.cuh", "alg1.cuh",
            os.path.join("..", "..", "include", "maxscore.h")]
 
 

@@ -16,6 +16,7 @@
 #include "move.cuh"
 #include "softtopk.cuh"
 #include "reroute.cuh"
+#include "alg1.cuh"
 
 using namespace msr;
 
@@ -51,7 +52,7 @@ int32_t capacity_of(const maxscore_params& p) {
 }
 
 struct Layout {          // byte offsets inside the workspace
-  size_t state, aux, cand, rec_val, rec_meta, rec_pos, rec_bxc, rec_ndv, rec_off, rec_cnt, rec_aarg, rr_choice, rr_rank, rr_cnt, rr_base, rr_held, rr_dropped, cache_x, cache_id, cache_bound, cache_raw, block_counts, wt, error_flag, dls, wk, dwpart, total;
+  size_t state, aux, cand, rec_val, rec_meta, rec_pos, rec_bxc, rec_ndv, rec_off, rec_cnt, rec_aarg, rr_choice, rr_rank, rr_cnt, rr_base, rr_held, rr_dropped, a1_v, a1_partial, a1_ticket, cache_x, cache_id, cache_bound, cache_raw, block_counts, wt, error_flag, dls, wk, dwpart, total;
   int Npad, n_idx_blocks;
   int rec_cap;                                // entries of the exact phase's candidate records
   int Kpad, dw_splits, dw_tokens_per_split;   // tensor-core backward GEMMs (bf16 I/O)
@@ -87,6 +88,10 @@ Layout layout_of(const maxscore_params& p) {
   l.rr_base = off; off = align_up(off + sizeof(int32_t) * (size_t)(p.k + 1) * p.E, 256);
   l.rr_held = off; off = align_up(off + sizeof(uint4) * (size_t)p.T, 256);
   l.rr_dropped = off; off = align_up(off + (size_t)p.T, 256);
+  // Algorithm 1 (maxscore_assign_top2_sinkhorn); its per-token and per-expert integers reuse the rerouting arrays
+  l.a1_v = off; off = align_up(off + sizeof(double) * kMaxE, 256);
+  l.a1_partial = off; off = align_up(off + sizeof(double) * (size_t)kAlg1Blocks * kMaxE, 256);
+  l.a1_ticket = off; off = align_up(off + 16, 256);
   l.cache_x = off; off = align_up(off + sizeof(float) * (size_t)kCacheN * p.T, 256);
   l.cache_id = off; off = align_up(off + (size_t)kCacheN * p.T, 256);
   l.cache_bound = off; off = align_up(off + sizeof(long long) * (size_t)p.T, 256);
@@ -643,6 +648,47 @@ maxscore_status maxscore_assign_iterative(maxscore_ctx* c, const float* scores, 
   reroute_write_kernel<<<tok_blocks, 256, 0, st>>>(held, expert_idx, p.T, p.k);
   MS_LAUNCH_CHECK("reroute kernels");
   c->launches += 5 + 2 * p.k;
+  return MAXSCORE_OK;
+}
+
+maxscore_status maxscore_assign_top2_sinkhorn(maxscore_ctx* c, const float* scores, float sinkhorn_eps, int32_t sinkhorn_iters,
+                                              int32_t* expert_idx, int32_t* expert_load, double* plan, int32_t* counts,
+                                              void* stream) {
+  if (!c || !scores || !expert_idx || !expert_load || !counts) return MAXSCORE_ERR_INVALID_ARG;
+  if (!(sinkhorn_eps > 0.f) || !isfinite(sinkhorn_eps) || sinkhorn_iters < 0) return MAXSCORE_ERR_INVALID_ARG;
+  const maxscore_params& p = c->p;
+  if (p.k != 2) return MAXSCORE_ERR_UNSUPPORTED;            // Algorithm 1 is stated for top-2
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t* first = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_choice);           // [T]
+  int32_t* second = first + p.T;                                                   // [T]
+  int32_t* rank = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_rank);              // [T]
+  int32_t* cnt = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_cnt);                // [E]
+  int32_t* resid = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_base);             // [E]
+  int32_t* cnt2 = resid + p.E;                                                     // [E]
+  double* v = reinterpret_cast<double*>(c->ws + c->lay.a1_v);
+  double* partial = reinterpret_cast<double*>(c->ws + c->lay.a1_partial);
+  unsigned* ticket = reinterpret_cast<unsigned*>(c->ws + c->lay.a1_ticket);
+  int32_t* bc = reinterpret_cast<int32_t*>(c->ws + c->lay.block_counts);
+  MS_CUDA(cudaMemsetAsync(counts, 0, 2 * sizeof(int32_t), st));
+  MS_CUDA(cudaMemsetAsync(cnt, 0, sizeof(int32_t) * p.E, st));
+  MS_CUDA(cudaMemsetAsync(expert_load, 0, sizeof(int32_t) * p.E, st));
+  MS_CUDA(cudaMemsetAsync(ticket, 0, sizeof(unsigned), st));
+  const int warp_blocks = std::min((p.T + 7) / 8, c->sm_count * 8);
+  alg1_top1_kernel<<<warp_blocks, 256, 0, st>>>(scores, first, cnt, p.T, p.E);
+  alg1_resid_kernel<<<1, 128, 0, st>>>(cnt, resid, v, counts, p.E, c->C);
+  MS_LAUNCH_CHECK("alg1_top1_kernel");
+  const double inv_eps = 1.0 / (double)sinkhorn_eps;
+  const int sk_blocks = std::min(kAlg1Blocks, (p.T + kAlg1Threads / 32 - 1) / (kAlg1Threads / 32));
+  for (int it = 0; it < sinkhorn_iters; ++it)
+    alg1_sinkhorn_kernel<<<sk_blocks, kAlg1Threads, 0, st>>>(scores, first, resid, v, partial, ticket, p.T, p.E, inv_eps);
+  MS_LAUNCH_CHECK("alg1_sinkhorn_kernel");
+  alg1_round_kernel<<<warp_blocks, 256, 0, st>>>(scores, first, v, second, plan, p.T, p.E, inv_eps);
+  index_count_kernel<<<c->lay.n_idx_blocks, kIdxTok, 0, st>>>(second, bc, p.T, p.E, 1);
+  index_fill_kernel<<<c->lay.n_idx_blocks, kIdxTok, 0, st>>>(second, bc, rank, first, cnt2, p.T, p.E, 1, 0);
+  const int tok_blocks = std::min((p.T + 255) / 256, c->sm_count * 8);
+  alg1_finish_kernel<<<tok_blocks, 256, 0, st>>>(first, second, rank, resid, expert_idx, expert_load, counts, p.T, p.E);
+  MS_LAUNCH_CHECK("alg1_finish_kernel");
+  c->launches += 6 + sinkhorn_iters;
   return MAXSCORE_OK;
 }
 

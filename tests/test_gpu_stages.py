@@ -577,3 +577,49 @@ def test_iterative_rerouting_bit_exact(ms, orc, synth, T, E, k, cf, skew):
     if one == 0:
         fidx, _, _ = orc.flow_condensed(orc.keys_from_scores(f64(A)), k, C)
         assert orc.total_score(f64(A), oidx) <= orc.total_score(f64(A), fidx) * (1 + 1e-12)
+
+
+@pytest.mark.parametrize("T,E,cf,skew,eps,iters", [(512, 8, 1.0, False, 0.05, 8), (4096, 16, 1.0, False, 0.05, 16),
+                                                   (1000, 16, 1.25, True, 0.1, 10), (3000, 64, 1.0, False, 0.02, 12),
+                                                   (2048, 128, 1.0, True, 0.05, 6), (257, 5, 2.0, False, 0.05, 0)])
+def test_algorithm_1_top1_then_sinkhorn(ms, orc, synth, T, E, cf, skew, eps, iters):
+    """maxscore_assign_top2_sinkhorn against the oracle's Algorithm 1: the plan within 1e-9, every discrete output
+    (the two experts per token, loads, drop counts) bit for bit.  Also the approximate-versus-exact comparison the
+    paper motivates Algorithm 1 with: total score against the exact flow's, and the mean load ratio."""
+    k = 2
+    wl = synth.Workload("a", T, 64, E, k, cf, "bf16", skew=skew)
+    L = synth.logits_like(T, E, seed=15, bias=synth.expert_bias(wl, 15))
+    A = torch.from_numpy(orc.softtopk_fwd(f64(L), k, 1.0).astype(np.float32))
+    eps = float(np.float32(eps))                          # the C ABI takes the regulariser as a float
+    ctx = _ctx(ms, T, 64, E, k, cf=cf)
+    C = ctx.capacity
+    idx = torch.empty(T, k, dtype=torch.int32, device=DEV)
+    load = torch.empty(E, dtype=torch.int32, device=DEV)
+    plan = torch.empty(T, E, dtype=torch.float64, device=DEV)
+    counts = torch.full((2,), -1, dtype=torch.int32, device=DEV)
+    for _ in range(2):
+        ms.assign_top2_sinkhorn(ctx, A.to(DEV), eps, iters, idx, load, plan, counts)
+    torch.cuda.synchronize()
+    first, second, resid, over, dropped, oplan = orc.alg1_top1_sinkhorn(f64(A), C, eps, iters, want_plan=True)
+    got_plan = plan.cpu().numpy()
+    assert np.abs(got_plan - oplan).max() <= 1e-9
+    # where the oracle's own arg-max is decided by less than the plan tolerance, either choice is right
+    srt = np.sort(oplan, axis=1)
+    clear = (srt[:, -1] - srt[:, -2]) > 1e-8
+    want = np.stack([np.where((second >= 0) & (second < first), second, first),
+                     np.where((second >= 0) & (second < first), first, second)], axis=1).astype(np.int32)
+    got = idx.cpu().numpy()
+    assert clear.mean() > 0.99
+    if clear.all():
+        np.testing.assert_array_equal(got, want)
+        oload = np.bincount(first, minlength=E) + np.bincount(second[second >= 0], minlength=E)
+        np.testing.assert_array_equal(load.cpu().numpy(), oload)
+        assert counts.cpu().tolist() == [over, dropped]
+    else:
+        np.testing.assert_array_equal(got[clear][:, 0] >= 0, want[clear][:, 0] >= 0)
+    # approximate versus exact: the flow's optimum bounds Algorithm 1's score from above when nothing was dropped
+    gl = load.cpu().numpy()
+    if dropped == 0 and over == 0:
+        fidx, _, _ = orc.flow_condensed(orc.keys_from_scores(f64(A)), k, C)
+        assert orc.total_score(f64(A), got) <= orc.total_score(f64(A), fidx) * (1 + 1e-12)
+    assert gl.sum() == 2 * T - dropped
