@@ -29,7 +29,7 @@ def test_valid_params_give_a_workspace_size():
     (dict(t=0.0), INVALID), (dict(t=-1.0), INVALID), (dict(t=float("nan")), INVALID), (dict(t=float("inf")), INVALID),
     (dict(io_dtype=7), INVALID), (dict(score_mode=2), INVALID), (dict(w_gate_layout=3), INVALID),
     (dict(capacity_factor=0.0), INVALID), (dict(score_mode=1, quant_shift=15), INVALID), (dict(max_sweeps=-1), INVALID),
-    (dict(softtopk_mode=2), INVALID), (dict(softtopk_mode=1, rankscale_delta=2), INVALID),
+    (dict(softtopk_mode=3), INVALID), (dict(softtopk_mode=2), OK), (dict(softtopk_mode=1, rankscale_delta=2), INVALID),
     (dict(softtopk_mode=1, rankscale_beta=float("nan")), INVALID), (dict(softtopk_mode=1, rankscale_beta=1.0, rankscale_delta=1), OK),
     (dict(k=9, E=8), INFEASIBLE),                       # k > E
     (dict(capacity=100), INFEASIBLE),                   # 8 * 100 < 512 * 2
