@@ -323,6 +323,40 @@ def run_ours(args, wl):
     stats_s = ms.new_stats(dev)
     skew_ms = time_call(torch, lambda: ms.assign(ctx_s, As, idx_s, load_s, stats_s), reps=7, flush=flush)
     st_s = ms.read_stats(stats_s)
+
+    # ---- the paper's two approximate assignments beside the exact flow (Sec. 3.2): time, score reached, load ----
+    def pair_score(scores_t, idx_t):
+        ok = idx_t >= 0
+        return float(torch.where(ok, scores_t.gather(1, idx_t.clamp(min=0).long()), torch.zeros((), device=dev)).double().sum())
+    counts = torch.zeros(2, dtype=torch.int32, device=dev)
+    idx_i = torch.empty(T, k, dtype=torch.int32, device=dev)
+    load_i = torch.empty(E, dtype=torch.int32, device=dev)
+    it_ms = time_call(torch, lambda: ms.assign_iterative(ctx, buf.scores, idx_i, load_i, counts), flush=flush)
+    cnt_i = counts.cpu().tolist()
+    approx = {"iterative_reroute": {
+        "workload": wl.name, "ms": round(it_ms, 4), "pairs_dropped_in_stage_1": cnt_i[0], "slots_left_empty": cnt_i[1],
+        "score_over_exact": pair_score(buf.scores, idx_i) / st_a.total_score,
+        "mean_load_over_C": float(load_i.double().mean()) / C}}
+    k2 = synth.WORKLOADS["k2e16"]
+    ctx2 = ms.create(ms.make_params(k2.T, 64, k2.E, k2.k, k2.capacity_factor), dev)
+    L2 = synth.logits_like(k2.T, k2.E, 0).to(dev)
+    A2 = torch.empty_like(L2)
+    ms.softtopk_fwd(ctx2, L2, A2)
+    idx2 = torch.empty(k2.T, 2, dtype=torch.int32, device=dev)
+    load2 = torch.empty(k2.E, dtype=torch.int32, device=dev)
+    stats2 = ms.new_stats(dev)
+    ms.assign(ctx2, A2, idx2, load2, stats2)
+    exact2 = ms.read_stats(stats2).total_score
+    eps, iters = 0.05, 8
+    a1_ms = time_call(torch, lambda: ms.assign_top2_sinkhorn(ctx2, A2, eps, iters, idx2, load2, None, counts), flush=flush)
+    cnt_a = counts.cpu().tolist()
+    approx["algorithm_1_top1_sinkhorn"] = {
+        "workload": "k2e16 scores (T=4096, E=16, k=2, cf=1.0)", "sinkhorn_eps": eps, "sinkhorn_iters": iters,
+        "ms": round(a1_ms, 4), "top1_pairs_beyond_C": cnt_a[0], "second_experts_dropped": cnt_a[1],
+        "score_over_exact": pair_score(A2, idx2) / exact2,
+        "mean_load_over_C": float(torch.minimum(load2, torch.full_like(load2, ctx2.capacity)).double().mean()) / ctx2.capacity,
+        "paper_mean_load_over_C": 0.9996,       # Sec. 4.5, trained first layer, e=16, k=2: context, another workload
+    }
     del flush
 
     # ---- rooflines ----------------------------------------------------------------------------------------
@@ -406,6 +440,7 @@ def run_ours(args, wl):
                      "rule": "lowest fraction among the stages that take at least 5 % of the step",
                      "tensor_peak_TFLOPs": tpeak, "tensor_peak_source": tpeak_src},
         "roofline_span": roofline_span,
+        "approximate": approx,
         "cpu_baseline": cpu,
         "e2e": {"value": replicas.aggregate_tokens_per_s(info, T, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
