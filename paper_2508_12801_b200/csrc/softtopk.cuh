@@ -2,13 +2,11 @@
 //
 // Level j (1-based) of Eq. 6 adds a softmax with temperature t over the entries that are not among
 // the j-1 largest (ties: lowest expert index).  A lane holds experts lane, lane+32, ... so every
-// global access of a warp is one contiguous row segment.  The exponentials are taken once, relative to
-// the row maximum: a level's softmax is z_i / (sum of z over its unmasked entries) whatever the reference
-// point.  Only when a level's own maximum lies so far below the row maximum that z would leave the normal
-// fp32 range are they recomputed relative to that level's maximum.  A level costs one arg-max (two integer
-// warp reductions) and one broadcast: its sum is the previous level's sum minus the entry just masked, and
-// is only taken afresh (five shuffle rounds) after a re-base or once the running sum has dropped below an
-// eighth of the last fresh one, which keeps the cancellation error of the differences below 2e-6 relative.
+// global access of a warp is one contiguous row segment, and each level costs two shuffle
+// reductions (arg-max, sum).  The exponentials are taken once, relative to the row maximum: a level's
+// softmax is z_i / (sum of z over its unmasked entries) whatever the reference point.  Only when a
+// level's own maximum lies so far below the row maximum that z would leave the normal fp32 range are
+// they recomputed relative to that level's maximum.
 #pragma once
 #include "common.cuh"
 
@@ -47,34 +45,27 @@ softtopk_fwd_kernel(const float* __restrict__ logits, float* __restrict__ scores
     }
     float z[kEPL];
     float ref = 0.f;                                  // reference point of the current z
-    float zs = 0.f, zs_fresh = 0.f;                   // running sum of the unmasked z; the last sum taken afresh
     for (int level = 0; level < k; ++level) {
       float best = -INFINITY; int bidx = 0x7fffffff;
 #pragma unroll
       for (int j = 0; j < kEPL; ++j)
         if (live[j] && (a[j] > best || bidx == 0x7fffffff)) { best = a[j]; bidx = lane + 32 * j; }
       warp_argmax(best, bidx);
-      bool fresh = level == 0 || zs < 0.125f * zs_fresh;
       if (level == 0 || (ref - best) > 60.f * t) {    // (re)base the exponentials on this level's maximum
-        ref = best; fresh = true;
+        ref = best;
 #pragma unroll
         for (int j = 0; j < kEPL; ++j) z[j] = live[j] ? expf((a[j] - ref) / t) : 0.f;
       }
-      if (fresh) {
-        zs = 0.f;
+      float zs = 0.f;
 #pragma unroll
-        for (int j = 0; j < kEPL; ++j) zs += z[j];
-        zs = warp_sum(zs);
-        zs_fresh = zs;
-      }
+      for (int j = 0; j < kEPL; ++j) zs += z[j];
+      zs = warp_sum(zs);
       const float inv = 1.f / zs;
-      float zwin = 0.f;
 #pragma unroll
       for (int j = 0; j < kEPL; ++j) {
         y[j] = fmaf(z[j], inv, y[j]);
-        if (lane + 32 * j == bidx) { zwin = z[j]; live[j] = false; z[j] = 0.f; }   // masked from the next level on
+        if (lane + 32 * j == bidx) { live[j] = false; z[j] = 0.f; }   // masked from the next level on
       }
-      zs -= __shfl_sync(0xffffffffu, zwin, bidx & 31);
     }
     float* out = scores + (size_t)tok * E;
 #pragma unroll
@@ -116,37 +107,29 @@ softtopk_bwd_kernel(const float* __restrict__ logits, const int32_t* __restrict_
     float z[kEPL];
     float ref = 0.f;
     const float inv_t = 1.f / t;
-    float zs = 0.f, gz = 0.f, zs_fresh = 0.f;         // running sums over the unmasked entries: z and g z
     for (int level = 0; level < k; ++level) {
       float best = -INFINITY; int bidx = 0x7fffffff;
 #pragma unroll
       for (int j = 0; j < kEPL; ++j)
         if (live[j] && (a[j] > best || bidx == 0x7fffffff)) { best = a[j]; bidx = lane + 32 * j; }
       warp_argmax(best, bidx);
-      bool fresh = level == 0 || zs < 0.125f * zs_fresh;
       if (level == 0 || (ref - best) > 60.f * t) {
-        ref = best; fresh = true;
+        ref = best;
 #pragma unroll
         for (int j = 0; j < kEPL; ++j) z[j] = live[j] ? expf((a[j] - ref) / t) : 0.f;
       }
-      if (fresh) {
-        zs = 0.f; gz = 0.f;
+      float zs = 0.f, gz = 0.f;
 #pragma unroll
-        for (int j = 0; j < kEPL; ++j) { zs += z[j]; gz += g[j] * z[j]; }
-        zs = warp_sum(zs);
-        gz = warp_sum(gz);
-        zs_fresh = zs;
-      }
+      for (int j = 0; j < kEPL; ++j) { zs += z[j]; gz += g[j] * z[j]; }
+      zs = warp_sum(zs);
+      gz = warp_sum(gz);
       const float inv = 1.f / zs;
       const float gq = gz * inv;
-      float zwin = 0.f, gzwin = 0.f;
 #pragma unroll
       for (int j = 0; j < kEPL; ++j) {
         da[j] = fmaf(z[j] * inv, (g[j] - gq) * inv_t, da[j]);
-        if (lane + 32 * j == bidx) { zwin = z[j]; gzwin = g[j] * z[j]; live[j] = false; z[j] = 0.f; }
+        if (lane + 32 * j == bidx) { live[j] = false; z[j] = 0.f; }
       }
-      zs -= __shfl_sync(0xffffffffu, zwin, bidx & 31);
-      gz -= __shfl_sync(0xffffffffu, gzwin, bidx & 31);
     }
     float* out = dlogits + (size_t)tok * E;
 #pragma unroll
