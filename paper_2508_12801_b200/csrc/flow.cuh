@@ -989,7 +989,7 @@ flow_check_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, 
 // held is offered A - value(f).  Moving a token flips two flags of its record; nothing is rebuilt.
 constexpr int kP2Group = 4;                // threads that share one node of the graph in a search round
 constexpr int kP2Threads = kP2Group * kMaxE + 32;   // a group per expert node and one warp for node Z
-constexpr int kP2Own = 2;                  // candidates per thread whose records stay in registers during a search
+constexpr int kP2Own = 8;                  // candidates per thread whose experts and flags stay packed in registers during a search
 constexpr int kRecSmemBytes = 96 * 1024;   // records up to this size are mirrored in shared memory
 constexpr long long kDistLimit = 1LL << 58;  // distances stay below this, so that sums cannot overflow
 constexpr long long kExactCycleBudget = 4000000000LL;   // about two seconds: the exact phase gives up beyond this
@@ -1101,6 +1101,10 @@ struct P2Shared {
   int estart[kMaxE + 2], efill[kMaxE + 1];   // entries grouped by expert: first position, fill counter
   int path_v[kMaxE + 2], path_u[kMaxE + 2], path_tok[kMaxE + 2], path_c[kMaxE + 2];
   unsigned char failed[kMaxE + 4];   // deficit nodes whose walk came to a dead end in this search
+  unsigned char front[2][kMaxE + 4]; // nodes whose distance changed in the last search round / in the running one
+  unsigned char dirty[kMaxE + 4];    // nodes that were made a new offer in the running round
+  int nact;                          // candidates listed for the running round
+  int act[kP2Own * kP2Threads];      // their positions in the candidate list
   int npath, target, stop;
   long long dt, dtb;             // distance of the chosen target; best distance of any node with a deficit so far
 };
@@ -1186,83 +1190,127 @@ flow_exact_kernel(FlowState* st, int32_t* expert_idx, const int32_t* __restrict_
       if (s.stop) { if (tid == 0) atomicOr(&st->status, 4u); break; }
       if (!any || naug_before + naug >= max_aug) break;
     }
-    // ---- shortest paths from every node with excess: synchronous Bellman-Ford ---------------------------
-    // A round has two halves.  (A) One thread per candidate: A = the cheapest way to reach the token through
-    // an expert it holds; every entry it does not hold is offered A - value, written where the entry sits in
-    // the by-expert order.  (B) A group of threads per node: the best offer over the node's stretch of that
-    // order, and the arcs through Z.  No atomics on distances, and distances only ever come from the previous
-    // round's, so the round in which a node's distance became final orders the nodes.
-    // Offers that cannot beat the nearest node with a deficit found so far are dropped: all costs are
-    // non-negative, and beyond that distance the price update only needs to know "at least that far".
-    for (int v = tid; v <= E; v += blockDim.x) { d0[v] = s.imb[v] > 0 ? 0 : kInf; s.lvl[v] = 0; }
-    if (tid == 0) s.dtb = kDistLimit;
-    __syncthreads();
-    // this thread's candidates: entries, flags and current values in registers for the whole search
-    int om[kP2Own], oex[kP2Own][kRecUnroll], ops[kP2Own][kRecUnroll]; unsigned oheld[kP2Own]; long long ovc[kP2Own][kRecUnroll];
+    // ---- shortest paths from every node with excess: synchronous Bellman-Ford, frontier by frontier ------
+    // A candidate's offers only change when the distance of an expert it holds has changed, so a round
+    //   (0) lists the candidates that hold an expert of the frontier (the nodes whose distance changed in the
+    //       round before; at first the nodes with excess): one thread per candidate, from a packed copy of the
+    //       record's experts and flags that stays in registers;
+    //   (A) one thread per LISTED candidate: A = the cheapest way to reach the token through an expert it holds;
+    //       every entry it does not hold is offered A - value, written where the entry sits in the by-expert
+    //       order, and that expert is marked dirty;
+    //   (B) a group of threads per dirty node (and per node with a Z arc when Z moved): the best offer over the
+    //       node's stretch of the by-expert order, and the arcs through Z.
+    // Offers of candidates that were not listed are still those of their last evaluation, which used the same
+    // distances.  No atomics on distances, and distances only ever come from the previous round's, so the round
+    // in which a node's distance became final orders the nodes.  Offers that cannot beat the nearest node with a
+    // deficit found so far (plus theta) are dropped: all costs are non-negative, and beyond that distance the
+    // price update only needs to know "at least that far".
+    for (int v = tid; v <= E; v += blockDim.x) {
+      d0[v] = s.imb[v] > 0 ? 0 : kInf; s.lvl[v] = 0; s.dirty[v] = 0;
+      s.front[0][v] = s.imb[v] > 0 ? 1 : 0; s.front[1][v] = 0;
+    }
+    for (int i = tid; i < nent; i += blockDim.x) ndv[i] = kInf;        // no offers yet in this search
+    if (tid == 0) { s.dtb = kDistLimit; s.nact = 0; }
+    // packed copies of this thread's candidates: bytes 0..5 the experts of up to six entries, byte 6 their held
+    // flags, byte 7 the entry count (0xff: a record too long to pack, always evaluated)
+    unsigned long long own[kP2Own];
 #pragma unroll
     for (int r = 0; r < kP2Own; ++r) {
       const int c = tid + r * kP2Threads;
-      om[r] = c < n ? rcnt[c] : 0;
-      oheld[r] = 0;
-      if (om[r] > kRecUnroll) om[r] = -1;               // too long for registers: handled from memory below
-      const int o = c < n ? roff[c] : 0;
-#pragma unroll
-      for (int j = 0; j < kRecUnroll; ++j) {
-        const int i = j < om[r] ? o + j : o;
-        const int mt = om[r] > 0 ? rmeta[i] : 0;
-        oex[r][j] = mt & 255; ops[r][j] = om[r] > 0 ? rpos[i] : 0;
-        if (j < om[r] && (mt & 256)) oheld[r] |= 1u << j;
-        ovc[r][j] = om[r] > 0 ? rval[i] - s.dp[oex[r][j]] : 0;
+      unsigned long long pk = 0;
+      if (c < n) {
+        const int o = roff[c], m = rcnt[c];
+        if (m > kRecUnroll) pk = 0xffULL << 56;
+        else {
+          unsigned hb = 0;
+          for (int j = 0; j < m; ++j) {
+            const int mt = rmeta[o + j];
+            pk |= (unsigned long long)(mt & 255) << (8 * j);
+            if (mt & 256) hb |= 1u << j;
+          }
+          pk |= (unsigned long long)hb << 48 | (unsigned long long)m << 56;
+        }
       }
+      own[r] = pk;
     }
-    int more = 1;
+    __syncthreads();
+    int more = 1, cur = 0;
     for (int round = 1; round <= E + 2 && more; ++round) {
+      const unsigned char* fr = s.front[cur];
+      // (0) list the candidates touched by the frontier
 #pragma unroll
       for (int r = 0; r < kP2Own; ++r) {
-        if (om[r] <= 0) continue;
-        long long x[kRecUnroll];
+        const unsigned long long pk = own[r];
+        const int m = (int)(pk >> 56);
+        if (__all_sync(0xffffffffu, m == 0)) continue;               // nobody in the warp owns a candidate in this slot
+        bool hit = m == 0xff;
+        const unsigned hb = (unsigned)(pk >> 48) & 0xffu;
 #pragma unroll
-        for (int j = 0; j < kRecUnroll; ++j) {
-          const long long dv = d0[oex[r][j]];
-          x[j] = (j < om[r] && ((oheld[r] >> j) & 1u) && dv < kInf) ? dv + ovc[r][j] : kInf;
+        for (int j = 0; j < kRecUnroll; ++j)
+          if (j < m && ((hb >> j) & 1u)) hit |= fr[(pk >> (8 * j)) & 255u] != 0;
+        const unsigned hits = __ballot_sync(0xffffffffu, hit);        // one shared-memory atomic per warp, not per hit
+        if (hits) {
+          int base = 0;
+          if (lane == 0) base = atomicAdd(&s.nact, __popc(hits));
+          base = __shfl_sync(0xffffffffu, base, 0);
+          if (hit) s.act[base + __popc(hits & ((1u << lane) - 1u))] = tid + r * kP2Threads;
         }
-        long long A = kInf; int ae = 0;
-#pragma unroll
-        for (int j = 0; j < kRecUnroll; ++j)
-          if (x[j] < A || (x[j] == A && x[j] < kInf && oex[r][j] < ae)) { A = x[j]; ae = oex[r][j]; }
-#pragma unroll
-        for (int j = 0; j < kRecUnroll; ++j)
-          if (j < om[r]) ndv[ops[r][j]] = (!((oheld[r] >> j) & 1u) && A < kInf) ? A - ovc[r][j] : kInf;
-        aarg[tid + r * kP2Threads] = ae;
       }
-      for (int c = tid; c < n; c += blockDim.x) {
-        if (c < kP2Own * kP2Threads && rcnt[c] <= kRecUnroll) continue;      // done from registers above
+      __syncthreads();
+      // (A) offers of the listed candidates
+      const int nact = s.nact;
+      // (candidates beyond the packed copies are evaluated every round)
+      for (int ai = tid; ai < nact + max(0, n - kP2Own * kP2Threads); ai += blockDim.x) {
+        const int c = ai < nact ? s.act[ai] : kP2Own * kP2Threads + (ai - nact);
         const int o = roff[c], m = rcnt[c];
-        if (m == 0) continue;
         long long A = kInf; int ae = 0;
-        for (int i = o; i < o + m; ++i) {
-          const int mt = rmeta[i];
-          if (!(mt & 256)) continue;
-          const int e = mt & 255;
-          const long long du = d0[e];
-          if (du >= kInf) continue;
-          const long long x = du + (rval[i] - s.dp[e]);
-          if (x < A || (x == A && e < ae)) { A = x; ae = e; }
-        }
-        for (int i = o; i < o + m; ++i) {
-          const int mt = rmeta[i];
-          ndv[rpos[i]] = (!(mt & 256) && A < kInf) ? A - (rval[i] - s.dp[mt & 255]) : kInf;
+        if (m <= kRecUnroll) {
+          long long vc[kRecUnroll], x[kRecUnroll]; int ex[kRecUnroll], ps[kRecUnroll]; bool held[kRecUnroll];
+#pragma unroll
+          for (int j = 0; j < kRecUnroll; ++j) {
+            const int i = j < m ? o + j : o;
+            const int mt = rmeta[i];
+            ex[j] = mt & 255; held[j] = (mt & 256) != 0; ps[j] = rpos[i];
+            const long long dv = d0[ex[j]];
+            vc[j] = rval[i] - s.dp[ex[j]];
+            x[j] = (j < m && held[j] && dv < kInf) ? dv + vc[j] : kInf;
+          }
+#pragma unroll
+          for (int j = 0; j < kRecUnroll; ++j)
+            if (x[j] < A || (x[j] == A && x[j] < kInf && ex[j] < ae)) { A = x[j]; ae = ex[j]; }
+#pragma unroll
+          for (int j = 0; j < kRecUnroll; ++j)
+            if (j < m && !held[j]) { ndv[ps[j]] = A < kInf ? A - vc[j] : kInf; s.dirty[ex[j]] = 1; }
+        } else {
+          for (int i = o; i < o + m; ++i) {
+            const int mt = rmeta[i];
+            if (!(mt & 256)) continue;
+            const int e = mt & 255;
+            const long long du = d0[e];
+            if (du >= kInf) continue;
+            const long long x = du + (rval[i] - s.dp[e]);
+            if (x < A || (x == A && e < ae)) { A = x; ae = e; }
+          }
+          for (int i = o; i < o + m; ++i) {
+            const int mt = rmeta[i];
+            if (mt & 256) continue;
+            ndv[rpos[i]] = A < kInf ? A - (rval[i] - s.dp[mt & 255]) : kInf; s.dirty[mt & 255] = 1;
+          }
         }
         aarg[c] = ae;
       }
       __syncthreads();
+      // (B) nodes
       bool changed = false;
       // beyond the nearest deficit's distance plus theta no target can be used: its price update would leave the window
       const long long dtb = (theta < kInf && s.dtb < kDistLimit - theta) ? s.dtb + theta + 1 : kDistLimit;
+      unsigned char* fn = s.front[cur ^ 1];
+      const bool zmoved = fr[nZ] != 0;
       {
         const int f = tid / kP2Group, sub = tid % kP2Group;      // every thread takes part in the group shuffles
         long long best = kInf;
-        if (f < E) {
+        const bool work = f < E && (s.dirty[f] || (zmoved && s.flow[f] > 0));
+        if (work) {
           const int hi = s.estart[f + 1];
           for (int idx = s.estart[f] + sub; idx < hi; idx += 4 * kP2Group) {
             long long a[4];
@@ -1286,11 +1334,13 @@ flow_exact_kernel(FlowState* st, int32_t* expert_idx, const int32_t* __restrict_
         }
         if (f < E && sub == 0) {
           const long long old = d0[f];
-          if (best < old && best < dtb) {
-            dn[f] = best; s.lvl[f] = round; changed = true;
+          const bool better = work && best < old && best < dtb;
+          dn[f] = better ? best : old;
+          fn[f] = better ? 1 : 0;
+          s.dirty[f] = 0;
+          if (better) {
+            s.lvl[f] = round; changed = true;
             if (s.imb[f] < 0) atomicMin(&s.dtb, best);
-          } else {
-            dn[f] = old;
           }
         }
       }
@@ -1316,16 +1366,19 @@ flow_exact_kernel(FlowState* st, int32_t* expert_idx, const int32_t* __restrict_
         }
         if (lane == 0) {
           const long long old = d0[nZ];
-          if (best < old && best < dtb) {
-            dn[nZ] = best; s.lvl[nZ] = round; changed = true;
+          const bool better = best < old && best < dtb;
+          dn[nZ] = better ? best : old;
+          fn[nZ] = better ? 1 : 0;
+          if (better) {
+            s.lvl[nZ] = round; changed = true;
             if (s.imb[nZ] < 0) atomicMin(&s.dtb, best);
-          } else {
-            dn[nZ] = old;
           }
+          s.nact = 0;
         }
       }
       more = __syncthreads_or(changed);
       { long long* t = d0; d0 = dn; dn = t; }
+      cur ^= 1;
     }
     // ---- augment along tight arcs, nearest deficit first, by one warp ------------------------------------
     // With potentials lowered by min(dist, D), every arc u -> v with dist[u] + cost == dist[v] <= D has reduced
@@ -1430,11 +1483,13 @@ flow_exact_kernel(FlowState* st, int32_t* expert_idx, const int32_t* __restrict_
               }
             }
           }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            const unsigned long long oc = __shfl_xor_sync(0xffffffffu, code, o);
-            const int occ = __shfl_xor_sync(0xffffffffu, cc, o);
-            if (oc < code) { code = oc; cc = occ; }
+          {   // smallest code of the warp: its high word (token + 1), then its low byte (the tail) among the lanes that match
+            const unsigned hi = __reduce_min_sync(0xffffffffu, (unsigned)(code >> 8));
+            const unsigned lo = __reduce_min_sync(0xffffffffu, (unsigned)(code >> 8) == hi ? (unsigned)(code & 255ULL) : 0xffffffffu);
+            const unsigned who = __ballot_sync(0xffffffffu, (unsigned)(code >> 8) == hi && (unsigned)(code & 255ULL) == lo);
+            const bool none = hi == 0xffffffffu;
+            cc = __shfl_sync(0xffffffffu, cc, none ? 0 : __ffs(who) - 1);
+            code = none ? ~0ULL : (((unsigned long long)hi << 8) | lo);
           }
           if (code == ~0ULL) { dead = true; break; }      // every tight arc into v was used up earlier in this search
           const int u = (int)(code & 255ULL);
@@ -1461,8 +1516,12 @@ flow_exact_kernel(FlowState* st, int32_t* expert_idx, const int32_t* __restrict_
               if (e == pv) rmeta[i] = (unsigned short)(pv | 256);     // taken
               ndv[rpos[i]] = kInf;
             }
-            for (int j = 0; j < k; ++j)
-              if (expert_idx[(size_t)tok * k + j] == pu) expert_idx[(size_t)tok * k + j] = pv;
+            int rowv[kMaxK];                                   // all loads in flight before the one store
+#pragma unroll
+            for (int j = 0; j < kMaxK; ++j) rowv[j] = j < k ? expert_idx[(size_t)tok * k + j] : -1;
+#pragma unroll
+            for (int j = 0; j < kMaxK; ++j)
+              if (j < k && rowv[j] == pu) expert_idx[(size_t)tok * k + j] = pv;
           } else if (pv == nZ) {
             atomicAdd(&s.flow[pu], 1);
           } else {
