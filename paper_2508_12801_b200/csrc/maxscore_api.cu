@@ -246,6 +246,14 @@ maxscore_status launch_softtopk_fwd(maxscore_ctx* c, const float* logits, float*
 }
 
 constexpr int kSweeps = 24, kRounds = 6, kDefaultAug = 4096;
+// Dispatch through registers (dispatch_kernel, 0.91 of the copy peak on the stress shape) or through bulk copies
+// (dispatch_tma_kernel, 0.86: the 8-to-1 write-heavy stream is bound by the memory system's write path either way).
+// The bulk-copy variant is built with -DMAXSCORE_DISPATCH_TMA so that both can be profiled.
+#ifdef MAXSCORE_DISPATCH_TMA
+constexpr bool kDispatchByTma = true;
+#else
+constexpr bool kDispatchByTma = false;
+#endif
 
 maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_idx, int32_t* expert_load,
                               maxscore_stats* stats, cudaStream_t st) {
@@ -375,6 +383,7 @@ maxscore_status maxscore_create(maxscore_ctx** out, const maxscore_params* param
   MS_CUDA(cudaFuncSetAttribute(flow_exact_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRecSmemBytes));
   MS_CUDA(cudaFuncSetAttribute(gate_bwd_dh_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDhSmemMax));
   MS_CUDA(cudaFuncSetAttribute(gate_bwd_dw_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDwSmemMax));
+  MS_CUDA(cudaFuncSetAttribute(dispatch_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTmaWarps * kTmaStages * kTmaChunk));
   int coop = 0, sweep_occ = 0;
   MS_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
   MS_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&sweep_occ, flow_sweeps_kernel, kSwThreads, 0));
@@ -501,7 +510,14 @@ maxscore_status maxscore_dispatch(maxscore_ctx* c, const void* src, const int32_
   cudaStream_t st = (cudaStream_t)stream;
   const maxscore_params& p = c->p;
   const uint32_t row_bytes = (uint32_t)(p.d_model * elem_bytes(c));
-  dispatch_kernel<<<c->sm_count * 8, 256, 0, st>>>((const char*)src, expert_idx, slot_idx, (char*)dst, p.T, row_bytes, p.k, c->C);
+  if (kDispatchByTma) {
+    const uint32_t chunk = row_bytes < (uint32_t)kTmaChunk ? row_bytes : (uint32_t)kTmaChunk;      // multiples of 16 bytes
+    const size_t smem = (size_t)kTmaWarps * kTmaStages * chunk;
+    dispatch_tma_kernel<<<c->sm_count, kTmaWarps * 32, smem, st>>>((const char*)src, expert_idx, slot_idx, (char*)dst, p.T,
+                                                                  row_bytes, chunk, p.k, c->C, error_flag_of(c));
+  } else {
+    dispatch_kernel<<<c->sm_count * 8, 256, 0, st>>>((const char*)src, expert_idx, slot_idx, (char*)dst, p.T, row_bytes, p.k, c->C);
+  }
   MS_LAUNCH_CHECK("dispatch_kernel");
   c->launches += 1;
   return launch_zero_padding(c, slot_token, dst, st);

@@ -93,9 +93,9 @@ index_fill_kernel(const int32_t* __restrict__ expert_idx, const int32_t* __restr
 
 // ---------------------------------------------------------------------------------------------
 // Dispatch: xdisp[e, slot, :] = H[token, :] for the token's k (expert, slot) pairs.  Token-major, so
-// every row is read once and written k times.  (A variant that staged rows through a shared-memory
-// ring of 1-D bulk copies driven by one thread per CTA measured 0.86 of the HBM copy peak on the
-// write-heavy stress shape; this one measures 0.91.)
+// every row is read once and written k times.  (dispatch_tma_kernel below does the same through the copy
+// engine, every warp driving its own ring of bulk copies; it measures 0.86 of the HBM copy peak on the
+// write-heavy stress shape, this one 0.91, so this one is the default.)
 // One warp per token, a lane owns 16-byte column groups, kDispatchBatch groups are loaded (streaming
 // loads) before their copies are stored (streaming stores).
 constexpr int kDispatchBatch = 4;     // 16-byte groups a lane loads before it stores their copies
@@ -129,6 +129,73 @@ dispatch_kernel(const char* __restrict__ src, const int32_t* __restrict__ expert
       }
     }
   }
+}
+
+// Dispatch through the copy engine: every warp keeps a ring of kTmaStages row buffers in shared memory.  Lane 0
+// brings a token's row (or a piece of it, at most kTmaChunk bytes) in with one bulk copy global -> shared that
+// completes on an mbarrier; lanes 0..k-1 then each send it to one of the token's k slots with one bulk copy
+// shared -> global.  A buffer is reused once the copies out of it have finished reading it
+// (cp.async.bulk.wait_group.read).  No register or LSU traffic for the data: the load/store units only carry
+// the indices.  Every mbarrier wait is bounded; a wait that runs out raises the error flag and the warp stops.
+constexpr int kTmaStages = 4, kTmaWarps = 4, kTmaChunk = 8192;
+__global__ void __launch_bounds__(kTmaWarps * 32)
+dispatch_tma_kernel(const char* __restrict__ src, const int32_t* __restrict__ expert_idx,
+                    const int32_t* __restrict__ slot_idx, char* __restrict__ dst, int Tn, uint32_t row_bytes,
+                    uint32_t chunk, int k, int C, unsigned* error_flag) {
+  extern __shared__ __align__(128) unsigned char tma_smem[];
+  __shared__ __align__(8) uint64_t bars[kTmaWarps][kTmaStages];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned char* ring = tma_smem + (size_t)warp * kTmaStages * chunk;
+  if (lane == 0)
+    for (int s = 0; s < kTmaStages; ++s) mbar_init(&bars[warp][s], 1);
+  fence_barrier_init();
+  __syncwarp();
+  const uint32_t pieces = (row_bytes + chunk - 1) / chunk;
+  const long long units = (long long)Tn * pieces;
+  const long long first = (long long)blockIdx.x * kTmaWarps + warp, stride = (long long)gridDim.x * kTmaWarps;
+  auto issue_load = [&](long long u, int s) {            // lane 0 only
+    const long long tok = u / pieces; const uint32_t pc = (uint32_t)(u - tok * pieces);
+    const uint32_t off = pc * chunk, bytes = min(chunk, row_bytes - off);
+    mbar_expect_tx(&bars[warp][s], bytes);
+    bulk_g2s(ring + (size_t)s * chunk, src + (size_t)tok * row_bytes + off, bytes, &bars[warp][s]);
+  };
+  // Two loads run ahead of the unit being sent out.  With four buffers that leaves one for the unit in hand and
+  // one whose outgoing copies (committed one iteration ago) may still be reading it.
+  constexpr int kAhead = kTmaStages - 2;
+  if (lane == 0)
+    for (int s = 0; s < kAhead; ++s)
+      if (first + s * stride < units) issue_load(first + s * stride, s);
+  int it = 0; bool failed = false;
+  for (long long u = first; u < units; u += stride, ++it) {
+    const int s = it % kTmaStages;
+    const long long tok = u / pieces; const uint32_t pc = (uint32_t)(u - tok * pieces);
+    const uint32_t off = pc * chunk, bytes = min(chunk, row_bytes - off);
+    long long my_off = -1;
+    if (lane < k) {
+      const int e = __ldg(expert_idx + (size_t)tok * k + lane), sl = __ldg(slot_idx + (size_t)tok * k + lane);
+      if (e >= 0 && sl >= 0 && sl < C) my_off = ((long long)e * C + sl) * (long long)row_bytes + off;
+    }
+    // the buffer the next load lands in was last read by the copies committed two iterations ago: every lane
+    // waits until at most its latest group is still reading, then the warp agrees before lane 0 overwrites it
+    bulk_wait_read<1>();
+    __syncwarp();
+    if (lane == 0 && u + kAhead * stride < units) issue_load(u + kAhead * stride, (it + kAhead) % kTmaStages);
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait_bounded(&bars[warp][s], (it / kTmaStages) & 1) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    __syncwarp();
+    if (!ok) { failed = true; break; }
+    if (my_off >= 0) bulk_s2g(dst + my_off, ring + (size_t)s * chunk, bytes);
+    bulk_commit();
+  }
+  if (failed) {
+    // a load never arrived: report it, give the loads still in flight a bounded chance to land, and leave
+    if (lane == 0) {
+      atomicExch(error_flag, 1u);
+      for (int a = 1; a <= kAhead; ++a) mbar_wait_bounded(&bars[warp][(it + a) % kTmaStages], ((it + a) / kTmaStages) & 1, 1u << 16);
+    }
+  }
+  bulk_wait_all<0>();
 }
 
 // Zero the rows of padding slots (slot_token < 0) of an [E*C, row] buffer.
