@@ -269,7 +269,10 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   a.balanced = ((long long)p.E * c->C == (long long)p.T * p.k) ? 1 : 0;
   a.eps0 = 1LL << (scale_bits - 10);
   a.eps_min = p.score_mode == 0 ? (1LL << 20) : (1LL << 12);
-  a.theta0 = 1LL << (scale_bits - 15);
+  // first candidate threshold: 2^-14 of a unit of score.  Half of it lists fewer tokens but on the stress workload
+  // often needs a second round (records, exact phase and check pass again); twice as much makes every search
+  // round of the exact phase walk over twice as many records
+  a.theta0 = 1LL << (scale_bits - 14);
   int max_aug = budget - a.n_sweeps;
 
   flow_init_kernel<<<32, 256, 0, st>>>(fs, kCapLogMax, a.theta0, a.balanced, p.E);
