@@ -654,8 +654,11 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
     ++sweep;
     // a small imbalance that has stopped shrinking is a price war between a few experts: the exact phase
     // ends it faster than more sweeps would
-    stall = sh.s_imb < best_imb ? 0 : stall + 1;
-    if (stall == 0) best_imb = sh.s_imb;
+    // (progress = the imbalance fell below 7/8 of the best one seen so far: slower than that, an augmentation of the
+    // exact phase costs about as much as the sweep and removes more)
+    const bool progress = (long long)sh.s_imb * 8 < (long long)best_imb * 7 || best_imb == 0x7fffffff;
+    stall = progress ? 0 : stall + 1;
+    if (sh.s_imb < best_imb) best_imb = sh.s_imb;
     done = (sh.s_imb == 0) || sweep >= a.n_sweeps || (stall >= kStallSweeps && sh.s_imb <= kStallImbalance);
     cumdrop += sh.s_drop;
 #ifdef MAXSCORE_TRACE

@@ -245,7 +245,9 @@ maxscore_status launch_softtopk_fwd(maxscore_ctx* c, const float* logits, float*
   return MAXSCORE_OK;
 }
 
-constexpr int kSweeps = 24, kRounds = 6, kDefaultAug = 4096;
+// rounds of (records, exact phase, check): candidate thresholds theta0, then two wider ones (four times the last, or twice
+// the price spread that stopped the exact phase), then every token.  The documented workloads need one to three.
+constexpr int kSweeps = 24, kRounds = 4, kDefaultAug = 4096;
 // Dispatch through registers (dispatch_kernel, 0.91 of the copy peak on the stress shape) or through bulk copies
 // (dispatch_tma_kernel, 0.86: the 8-to-1 write-heavy stream is bound by the memory system's write path either way).
 // The bulk-copy variant is built with -DMAXSCORE_DISPATCH_TMA so that both can be profiled.
