@@ -12,8 +12,8 @@
 // with base[r][e] = min(C, base[r-1][e] + cnt[r-1][e]) tokens and accepts the first C - base[r][e] of them
 // in token order, so a pair is accepted iff base + (its rank among that level's choosers) < C.  The ranks
 // come from the index-build kernels.  Stage 2 is sequential by definition (every placement changes what the
-// next pair may take); it runs in one CTA that stages the rows of the next 64 dropped tokens in shared memory
-// while one warp places them.
+// next pair may take); it runs in one CTA that stages the rows, held masks and dropped bits of the next 64 dropped
+// tokens in shared memory, after which one warp places them without touching global memory.
 #pragma once
 #include "common.cuh"
 #include "softtopk.cuh"
@@ -80,6 +80,8 @@ struct RerouteShared {
   int nlist, nempty;
   int wcount[kRerouteThreads / 32];
   float rows[kRerouteBatch][kMaxE];
+  uint4 hrow[kRerouteBatch];       // held masks and dropped-level bits of the staged tokens
+  unsigned drow[kRerouteBatch];
 };
 
 // Stage 2, one CTA.  Tokens are scanned in chunks of kRerouteThreads; the chunk's tokens with a dropped pair are
@@ -116,13 +118,14 @@ reroute_place_kernel(const float* __restrict__ A, const int32_t* __restrict__ ba
         const int q = i / E, e = i - q * E;
         s.rows[q][e] = __ldg(A + (size_t)s.list[b0 + q] * E + e);
       }
+      if (tid < nb) { s.hrow[tid] = held[s.list[b0 + tid]]; s.drow[tid] = dropped[s.list[b0 + tid]]; }
       __syncthreads();
       if (warp == 0) {
         for (int q = 0; q < nb; ++q) {
           const int t2 = s.list[b0 + q];
-          uint4 hv = held[t2];
+          const uint4 hv = s.hrow[q];
           unsigned hm[4] = {hv.x, hv.y, hv.z, hv.w};
-          const unsigned db = dropped[t2];
+          const unsigned db = s.drow[q];
           for (int r = 0; r < k; ++r) {
             if (!((db >> r) & 1u)) continue;
             float best = -INFINITY; int bidx = 0x7fffffff;
