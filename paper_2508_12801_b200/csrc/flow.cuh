@@ -811,19 +811,34 @@ flow_check_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, 
           slow = true;                                    // only the bound on the uncached experts is in the way
         }
       }
-      // statistics: the score of the held pairs and how many of them are not among the token's k best raw keys
+      // statistics: the score of the held pairs and how many of them are not among the token's k best raw keys.
+      // A cache built at zero prices lists its entries by descending raw value, so its first k entries are the
+      // raw top-k as soon as each of them beats every later entry and the bound on the uncached ones exactly;
+      // otherwise (a near-tie, or a cache rebuilt at other prices) the held entries are counted one by one.
       if (!slow) {
         int rer = 0; double sc = 0.0;
+        long long lo_first = kInf, hi_rest = -kInf;
 #pragma unroll
         for (int j = 0; j < kCacheN; ++j) {
-          if (!((heldbits >> j) & 1u)) continue;
-          int above = 0;
-#pragma unroll
-          for (int i = 0; i < kCacheN; ++i) above += key[i] > key[j] ? 1 : 0;
-          if (above >= k) ++rer;
-          else if (bound > -kInf && (!raw || key[j] <= bound)) slow = true;   // an uncached raw key might be larger
-          sc += g.mode == 0 ? (double)x[j] : (double)key[j];
+          if (j < k) lo_first = key[j] < lo_first ? key[j] : lo_first;
+          else hi_rest = key[j] > hi_rest ? key[j] : hi_rest;
         }
+        if (raw && lo_first > hi_rest && (bound <= -kInf || lo_first > bound)) {
+          rer = __popc(heldbits >> k);                    // held entries listed after the raw top-k
+        } else {
+#pragma unroll
+          for (int j = 0; j < kCacheN; ++j) {
+            if (!((heldbits >> j) & 1u)) continue;
+            int above = 0;
+#pragma unroll
+            for (int i = 0; i < kCacheN; ++i) above += key[i] > key[j] ? 1 : 0;
+            if (above >= k) ++rer;
+            else if (bound > -kInf && (!raw || key[j] <= bound)) slow = true;   // an uncached raw key might be larger
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < kCacheN; ++j)
+          if ((heldbits >> j) & 1u) sc += g.mode == 0 ? (double)x[j] : (double)key[j];
         if (!slow) { t_rer += rer; t_score += sc; }
       }
       if (!slow) {
