@@ -52,7 +52,7 @@ int32_t capacity_of(const maxscore_params& p) {
 }
 
 struct Layout {          // byte offsets inside the workspace
-  size_t state, aux, cand, rec_val, rec_meta, rec_pos, rec_bxc, rec_ndv, rec_off, rec_cnt, rec_aarg, rr_choice, rr_rank, rr_cnt, rr_base, rr_held, rr_dropped, a1_v, a1_partial, a1_ticket, cache_x, cache_id, cache_bound, cache_raw, block_counts, wt, error_flag, dls, wk, dwpart, total;
+  size_t state, aux, cand, rec_val, rec_meta, rec_pos, rec_bxc, rec_ndv, rec_off, rec_cnt, rec_aarg, rr_choice, rr_rank, rr_cnt, rr_base, rr_held, rr_dropped, rr_bc, rr_blk, rr_dtok, rr_order, rr_dnum, a1_v, a1_partial, a1_ticket, cache_x, cache_id, cache_bound, cache_raw, block_counts, wt, error_flag, dls, wk, dwpart, total;
   int Npad, n_idx_blocks;
   int rec_cap;                                // entries of the exact phase's candidate records
   int Kpad, dw_splits, dw_tokens_per_split;   // tensor-core backward GEMMs (bf16 I/O)
@@ -88,6 +88,11 @@ Layout layout_of(const maxscore_params& p) {
   l.rr_base = off; off = align_up(off + sizeof(int32_t) * (size_t)(p.k + 1) * p.E, 256);
   l.rr_held = off; off = align_up(off + sizeof(uint4) * (size_t)p.T, 256);
   l.rr_dropped = off; off = align_up(off + (size_t)p.T, 256);
+  l.rr_bc = off; off = align_up(off + sizeof(int32_t) * (((size_t)p.k * p.T + kIdxTok - 1) / kIdxTok) * p.E, 256);
+  l.rr_blk = off; off = align_up(off + sizeof(int32_t) * (2 * (((size_t)p.T + kRrTokBlock - 1) / kRrTokBlock) + 1), 256);
+  l.rr_dtok = off; off = align_up(off + sizeof(int32_t) * (size_t)p.T, 256);
+  l.rr_order = off; off = align_up(off + (size_t)kRrRow * p.T, 256);
+  l.rr_dnum = off; off = align_up(off + (size_t)p.T, 256);
   // Algorithm 1 (maxscore_assign_top2_sinkhorn); its per-token and per-expert integers reuse the rerouting arrays
   l.a1_v = off; off = align_up(off + sizeof(double) * kMaxE, 256);
   l.a1_partial = off; off = align_up(off + sizeof(double) * (size_t)kAlg1Blocks * kMaxE, 256);
@@ -644,31 +649,37 @@ maxscore_status maxscore_assign_iterative(maxscore_ctx* c, const float* scores, 
   if (!c || !scores || !expert_idx || !expert_load || !counts) return MAXSCORE_ERR_INVALID_ARG;
   const maxscore_params& p = c->p;
   cudaStream_t st = (cudaStream_t)stream;
-  int32_t* choice = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_choice);
-  int32_t* rank = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_rank);
-  int32_t* cnt = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_cnt);
-  int32_t* base = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_base);
+  int32_t* choice = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_choice);      // [k][T], level-major
+  int32_t* rank = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_rank);          // [k][T]
+  int32_t* total = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_cnt);          // [E] pairs that chose the expert
   uint4* held = reinterpret_cast<uint4*>(c->ws + c->lay.rr_held);
   unsigned char* dropped = reinterpret_cast<unsigned char*>(c->ws + c->lay.rr_dropped);
-  int32_t* bc = reinterpret_cast<int32_t*>(c->ws + c->lay.block_counts);
+  int32_t* bc = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_bc);
+  const int nblk = (p.T + kRrTokBlock - 1) / kRrTokBlock;
+  int32_t* blk_cnt = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_blk);        // [nblk]
+  int32_t* blk_off = blk_cnt + nblk;                                           // [nblk + 1]
+  int32_t* dtok = reinterpret_cast<int32_t*>(c->ws + c->lay.rr_dtok);
+  unsigned char* order = reinterpret_cast<unsigned char*>(c->ws + c->lay.rr_order);     // [T][kRrRow]
+  unsigned char* dnum = reinterpret_cast<unsigned char*>(c->ws + c->lay.rr_dnum);
   MS_CUDA(cudaMemsetAsync(counts, 0, 2 * sizeof(int32_t), st));
   const int warp_blocks = std::min((p.T + 7) / 8, c->sm_count * 8);
   reroute_choices_kernel<<<warp_blocks, 256, 0, st>>>(scores, choice, p.T, p.E, p.k);
   MS_LAUNCH_CHECK("reroute_choices_kernel");
-  for (int r = 0; r < p.k; ++r) {     // rank of every token among the tokens that chose the same expert at level r
-    index_count_kernel<<<c->lay.n_idx_blocks, kIdxTok, 0, st>>>(choice + (size_t)r * p.T, bc, p.T, p.E, 1);
-    index_fill_kernel<<<c->lay.n_idx_blocks, kIdxTok, 0, st>>>(choice + (size_t)r * p.T, bc, rank + (size_t)r * p.T, choice,
-                                                              cnt + (size_t)r * p.E, p.T, p.E, 1, 0);
-    MS_LAUNCH_CHECK("index_fill_kernel(level)");
-  }
-  reroute_base_kernel<<<1, 128, 0, st>>>(cnt, base, p.E, p.k, c->C);
+  // rank of every pair among the pairs of its expert in level-major order: the choice array as k*T tokens of one expert each
+  const int flat = p.T * p.k;
+  const int flat_blocks = (flat + kIdxTok - 1) / kIdxTok;
+  index_count_kernel<<<flat_blocks, kIdxTok, 0, st>>>(choice, bc, flat, p.E, 1);
+  index_fill_kernel<<<flat_blocks, kIdxTok, 0, st>>>(choice, bc, rank, choice, total, flat, p.E, 1, 0);
+  MS_LAUNCH_CHECK("index_fill_kernel(levels)");
+  reroute_accept_kernel<<<nblk, kRrTokBlock, 0, st>>>(choice, rank, held, dropped, blk_cnt, counts, p.T, p.E, p.k, c->C);
+  reroute_scan_kernel<<<1, 1024, 0, st>>>(blk_cnt, blk_off, nblk);
+  reroute_compact_kernel<<<nblk, kRrTokBlock, 0, st>>>(dropped, blk_off, dtok, dnum, p.T);
+  reroute_order_kernel<<<c->sm_count * 4, 256, 0, st>>>(scores, total, held, blk_off + nblk, dtok, order, p.E, c->C);
+  reroute_place_kernel<<<1, kRrThreads, 0, st>>>(total, held, blk_off + nblk, dtok, dnum, order, expert_load, counts, p.E, c->C);
   const int tok_blocks = std::min((p.T + 255) / 256, c->sm_count * 8);
-  reroute_accept_kernel<<<tok_blocks, 256, 0, st>>>(choice, rank, base, held, dropped, counts, p.T, p.E, p.k, c->C);
-  reroute_place_kernel<<<1, kRerouteThreads, sizeof(RerouteShared), st>>>(scores, base, held, dropped, expert_load, counts,
-                                                                         p.T, p.E, p.k, c->C);
   reroute_write_kernel<<<tok_blocks, 256, 0, st>>>(held, expert_idx, p.T, p.k);
   MS_LAUNCH_CHECK("reroute kernels");
-  c->launches += 5 + 2 * p.k;
+  c->launches += 9;
   return MAXSCORE_OK;
 }
 

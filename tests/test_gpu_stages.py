@@ -546,7 +546,8 @@ def test_itertopk_of_table_2_fwd_bwd(ms, orc, synth, T, E, k):
 
 @pytest.mark.parametrize("T,E,k,cf,skew", [(512, 8, 2, 1.0, False), (4096, 16, 2, 1.0, False), (1000, 16, 4, 1.0, False),
                                             (2048, 64, 8, 1.0, False), (2048, 64, 8, 1.25, True), (300, 8, 2, 1.5, True),
-                                            (8192, 64, 8, 1.0, False), (129, 5, 5, 1.0, False), (3000, 128, 8, 1.0, True)])
+                                            (8192, 64, 8, 1.0, False), (129, 5, 5, 1.0, False), (3000, 128, 8, 1.0, True),
+                                            (16384, 64, 8, 1.0, True), (20000, 32, 4, 1.0, True), (40000, 128, 8, 1.0, False)])
 def test_iterative_rerouting_bit_exact(ms, orc, synth, T, E, k, cf, skew):
     """maxscore_assign_iterative against the oracle's top-k-with-capacity + greedy rerouting: with both serving
     orders fixed the result is unique, so everything is compared bit for bit.  Also: how far the greedy result
@@ -573,8 +574,8 @@ def test_iterative_rerouting_bit_exact(ms, orc, synth, T, E, k, cf, skew):
     load2 = torch.empty(E, dtype=torch.int32, device=DEV)
     ms.index_build(ctx, idx, slot_idx, slot_token, load2)
     np.testing.assert_array_equal(load2.cpu().numpy(), oload)
-    # greedy is feasible, never better than the flow's optimum
-    if one == 0:
+    # greedy is feasible, never better than the flow's optimum (checked where the exact solver on the CPU takes seconds)
+    if one == 0 and T <= 8192:
         fidx, _, _ = orc.flow_condensed(orc.keys_from_scores(f64(A)), k, C)
         assert orc.total_score(f64(A), oidx) <= orc.total_score(f64(A), fidx) * (1 + 1e-12)
 
