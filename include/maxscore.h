@@ -279,7 +279,13 @@ maxscore_status maxscore_test_raise_internal(maxscore_ctx* ctx, void* cuda_strea
  * Copies hidden_host (and w_gate_host, expert_bias_host) to the device buffers given in `dev`,
  * runs maxscore_route_fwd and maxscore_dispatch, copies expert_idx, slot_idx, gate_w and stats back
  * to the *_host outputs and synchronises the stream before returning.  xdisp stays on the device
- * (dev->xdisp) for the experts to consume. */
+ * (dev->xdisp) for the experts to consume.
+ * The rows of hidden_host go up in as many as eight blocks on a second stream that the context creates on
+ * the first call (and maxscore_destroy releases); the gate GEMM and SoftTopk of a block run as soon as it has
+ * landed, and the index arrays come back on that stream while the rows are dispatched.  The assignment
+ * itself needs every row's scores, so it starts when the last block is in.  Both streams are ordered after
+ * what was queued on cuda_stream before the call, and the results are the same as those of
+ * maxscore_route_fwd + maxscore_dispatch on the same inputs.  Every dev buffer must be 16-byte aligned. */
 typedef struct {
   void* hidden; void* w_gate; float* expert_bias; float* logits; float* scores; int32_t* expert_idx;
   int32_t* slot_idx; float* gate_w; int32_t* slot_token; int32_t* expert_load; maxscore_stats* stats;

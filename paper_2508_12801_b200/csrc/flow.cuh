@@ -89,6 +89,7 @@ struct FlowState {
   double total_score;
   int load[kMaxE];           // accumulated by the running pass, consumed by its price step / last CTA
   int load_cur[kMaxE];       // loads of the assignment currently written in expert_idx
+  int load0[kMaxE];          // loads of the first sweep (every price zero): how popular each expert is
   alignas(16) unsigned hist_up[2][kMaxE * kNB];   // [sweep parity]; read and cleared with 16-byte accesses
   alignas(16) unsigned hist_dn[2][kMaxE * kNB];
   long long min_up[kMaxE], min_dn[kMaxE];   // smallest margin recorded by the running sweep (reset by the price step)
@@ -418,11 +419,20 @@ struct SweepShared {
   int nflag, nslow, s_imb;
   long long s_drop, s_pmin;
   int slow[kSwThreads];
+  int trim[kMaxE];                           // room the sweeps leave unused on purpose (see SweepArgs::slack)
+  int l0[kMaxE], srt[kMaxE], s_nb, s_level, s_rem;
 };
 
 struct SweepArgs {
   int T, E, k, C, n_sweeps, balanced;
   long long eps0, eps_min, theta0;
+  // E*C - T*k when that is positive but small (else 0).  Prices that may not fall below zero make the sweeps crawl
+  // when almost every expert ends up full: the few experts that keep room pin the price floor and everyone else has
+  // to climb away from it one sweep at a time.  So the sweeps then solve the problem with the spare room taken away
+  // from the least popular experts (as much from each as brings them level), where prices are free to move both ways
+  // as when nothing is spare; the pick anchors the lowest price at zero and the exact phase repairs what the guess
+  // of who keeps the room got wrong.
+  int slack;
 };
 
 struct TokCache {          // one token's cache entries in registers
@@ -538,6 +548,10 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gtid = blockIdx.x * blockDim.x + tid, gsize = gridDim.x * blockDim.x;
   const bool resident = T <= gsize;
+  bool hiding = a.slack > 0;                               // spare room is hidden from the sweeps (see SweepArgs::slack)
+  bool free_prices = a.balanced || hiding;                 // prices may go below zero until they are anchored
+  bool pending = false; long long pend_anchor = 0;         // an anchoring that the next price step still has to apply
+  for (int e = tid; e < kMaxE; e += blockDim.x) sh.trim[e] = 0;
   unsigned epoch = 0;
   long long cumdrop = 0, eps = a.eps0;
   int best_imb = 0x7fffffff, stall = 0, sweep = 0;
@@ -597,6 +611,34 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
     __syncthreads();
   };
 
+  // Anchoring (every CTA does the same to its copy of the prices).
+  auto anchor_prices = [&]() -> long long {
+      // Prices are only defined up to a shift when every expert must be full: anchor the minimum at 0.  A uniform shift
+      // moves every value of a token alike, the bound on its uncached experts included.
+      // With spare room hidden, the experts that gave up room are the ones that will keep it, so they belong at price
+      // zero: the anchor is the highest price among them, and whoever is cheaper still is lifted to zero as well (these
+      // fell less than the anchor, which therefore still bounds every expert's fall).
+      __syncthreads();
+      if (tid == 0) {
+        long long m = kInf;
+        if (a.slack > 0) {
+          m = -kInf;
+          for (int e = 0; e < E; ++e) if (sh.trim[e] > 0 && sh.sp[e] > m) m = sh.sp[e];
+        }
+        if (m >= kInf || m <= -kInf) { m = sh.sp[0]; for (int e = 1; e < E; ++e) m = sh.sp[e] < m ? sh.sp[e] : m; }
+        sh.s_pmin = m;
+      }
+      __syncthreads();
+      const long long pmin = sh.s_pmin;
+      for (int e = tid; e < E; e += blockDim.x) {
+        const long long pe = sh.sp[e] - pmin;
+        sh.sp[e] = pe < 0 ? 0 : pe; sh.spf[e] = (float)sh.sp[e];
+      }
+      cumdrop += pmin;
+      __syncthreads();
+    return pmin;
+  };
+
   load_state();
   while (!done) {
     const int par = sweep & 1;
@@ -616,14 +658,16 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
 
     // ---- price step: one warp per expert, every input fetched in one round trip -------------------------
     for (int e = blockIdx.x + warp * gridDim.x; e < E; e += gridDim.x * (kSwThreads / 32)) {
-      const int xs = __ldcg(&st->load[e]) - C;
-      const long long ps = __ldcg(&st->p[e]);
+      const int load_e = __ldcg(&st->load[e]);
+      const int xs = load_e - (C - sh.trim[e]);
+      long long ps = __ldcg(&st->p[e]);
+      if (pending) { ps -= pend_anchor; if (ps < 0) ps = 0; }
       const int cup = __ldcg(&st->cap_up[e]), cdn = __ldcg(&st->cap_dn[e]);
       const long long mu = __ldcg(&st->min_up[e]), md = __ldcg(&st->min_dn[e]);
       const uint4* hu = reinterpret_cast<const uint4*>(hup + e * kNB) + 2 * lane;
       const uint4* hd = reinterpret_cast<const uint4*>(hdn + e * kNB) + 2 * lane;
       const uint4 hau = __ldcg(hu), hbu = __ldcg(hu + 1), had = __ldcg(hd), hbd = __ldcg(hd + 1);
-      const bool up = xs > 0, dn = xs < 0 && (a.balanced || ps > 0);
+      const bool up = xs > 0, dn = xs < 0 && (free_prices || ps > 0);
       long long p = ps; int flag = 0, imb = 0;
       if (up) {
         int cl = cup; bool shortw;
@@ -633,7 +677,7 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
       } else if (dn) {
         int cl = cdn; bool shortw;
         p -= price_step_warp(had, hbd, -xs, eps, cl, shortw, kCapLogMax, md);
-        if (!a.balanced && p < 0) p = 0;
+        if (!free_prices && p < 0) p = 0;
         if (lane == 0) st->cap_dn[e] = cl;
         flag = shortw ? 1 : 0;
         imb = -xs;
@@ -645,12 +689,41 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
         st->flag_dn[e] = flag; st->load[e] = 0; st->min_up[e] = kInf; st->min_dn[e] = kInf;
         st->imb_e[e] = imb; st->drop_e[e] = ps - p > 0 ? ps - p : 0;
         st->p[e] = p;
+        if (sweep == 0) st->load0[e] = load_e;
       }
     }
+    pending = false;
     if (!grid_barrier(st, epoch)) return;
 
     // ---- every CTA draws the same conclusions from the same numbers ----------------------------------
     load_state();
+    if (a.slack > 0 && sweep == 0) {
+      // who gives up room: raise a water level under the first sweep's loads until the room below it is the spare room
+      for (int e = tid; e < E; e += blockDim.x) sh.l0[e] = __ldcg(&st->load0[e]);
+      __syncthreads();
+      for (int e = tid; e < E; e += blockDim.x) {
+        int rank = 0;
+        for (int x = 0; x < E; ++x) rank += (sh.l0[x] < sh.l0[e] || (sh.l0[x] == sh.l0[e] && x < e)) ? 1 : 0;
+        sh.srt[rank] = sh.l0[e]; sh.trim[e] = rank;
+      }
+      __syncthreads();
+      if (tid == 0) {
+        long long rem = a.slack; int j = 1;               // the j least popular experts are below the level srt[j - 1]
+        while (j < E) {
+          const long long need = (long long)j * (sh.srt[j] - sh.srt[j - 1]);
+          if (need > rem) break;
+          rem -= need; ++j;
+        }
+        sh.s_nb = j; sh.s_level = sh.srt[j - 1] + (int)(rem / j); sh.s_rem = (int)(rem % j);
+      }
+      __syncthreads();
+      for (int e = tid; e < E; e += blockDim.x) {
+        const int rank = sh.trim[e];
+        const int t = rank < sh.s_nb ? sh.s_level - sh.l0[e] + (rank < sh.s_rem ? 1 : 0) : 0;
+        sh.trim[e] = t < C ? t : C;
+      }
+      __syncthreads();
+    }
     ++sweep;
     // a small imbalance that has stopped shrinking is a price war between a few experts: the exact phase
     // ends it faster than more sweeps would
@@ -660,6 +733,15 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
     stall = progress ? 0 : stall + 1;
     if (sh.s_imb < best_imb) best_imb = sh.s_imb;
     done = (sh.s_imb == 0) || sweep >= a.n_sweeps || (stall >= kStallSweeps && sh.s_imb <= kStallImbalance);
+    if (done && hiding && sweep < a.n_sweeps) {
+      // the problem without the spare room is as good as solved: put the experts that gave up room at price zero, hand
+      // the room back and let the sweeps go on under the real rules (no price below zero, room allowed at price zero)
+      pend_anchor = anchor_prices(); pending = true;
+      for (int e = tid; e < kMaxE; e += blockDim.x) sh.trim[e] = 0;
+      hiding = false; free_prices = a.balanced != 0;
+      best_imb = 0x7fffffff; stall = 0; done = false;
+      __syncthreads();
+    }
     cumdrop += sh.s_drop;
 #ifdef MAXSCORE_TRACE
     if (gtid == 0) printf("sweep %d imbalance %d stall %d eps %lld drop %lld\n", sweep, sh.s_imb, stall, eps, sh.s_drop);
@@ -668,17 +750,7 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
   }
 
   // ---- first pick: every token's top-k under the final prices, candidates listed ----------------------
-  if (a.balanced) {
-    // prices are only defined up to a shift when every expert must be full; anchor the minimum at 0.
-    // A uniform shift moves every value of a token alike, the bound on its uncached experts included.
-    __syncthreads();
-    if (tid == 0) { long long m = sh.sp[0]; for (int e = 1; e < E; ++e) m = sh.sp[e] < m ? sh.sp[e] : m; sh.s_pmin = m; }
-    __syncthreads();
-    const long long pmin = sh.s_pmin;
-    for (int e = tid; e < E; e += blockDim.x) { sh.sp[e] -= pmin; sh.spf[e] = (float)sh.sp[e]; }
-    cumdrop += pmin;
-    __syncthreads();
-  }
+  if (free_prices) anchor_prices();
   token_pass(std::true_type{}, nullptr, nullptr);
   for (int e = tid; e < E; e += blockDim.x)
     if (sh.sload[e]) atomicAdd(&st->load[e], sh.sload[e]);
@@ -961,6 +1033,9 @@ flow_check_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache, 
   if (tid == 0) {
     const int viol = *(volatile int*)&st->violations;
     const bool ok = viol == 0 && s_badload == 0;
+#ifdef MAXSCORE_TRACE
+    printf("check round %d: violations %d experts off %d listed %d theta %lld\n", st->round, viol, s_badload, st->ncand, theta);
+#endif
     st->violations = 0;
     st->ticket = 0;
     if (ok || final_pass) {
@@ -1568,6 +1643,14 @@ flow_exact_kernel(FlowState* st, int32_t* expert_idx, const int32_t* __restrict_
   }
   // ---- write back ---------------------------------------------------------------------------------
   __syncthreads();
+#ifdef MAXSCORE_TRACE
+  if (tid == 0) {
+    int ex = 0, de = 0;
+    for (int e = 0; e < E; ++e) { if (s.imb[e] > 0) ex += s.imb[e]; if (s.imb[e] < 0) de -= s.imb[e]; }
+    printf("exact round %d: cand %d entries %d aug %d last %d excess %d deficit %d z %d theta %lld\n", st->round, n, nent, naug,
+           s.target, ex, de, s.imb[nZ], theta);
+  }
+#endif
   if (tid == 0) s.dt = 0;
   __syncthreads();
   for (int e = tid; e < E; e += blockDim.x) {

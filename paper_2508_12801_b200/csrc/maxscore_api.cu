@@ -166,6 +166,9 @@ struct maxscore_ctx {
   int sm_count;
   int sweep_grid_max;   // CTAs of the sweeps kernel that are resident at once
   long long launches;   // kernels launched through this context so far
+  // host path (maxscore_route_dispatch_host): a copy stream and its events, made on the first call
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_routed = nullptr, ev_copied = nullptr, ev_chunk[8] = {};
 };
 
 namespace {
@@ -203,51 +206,74 @@ maxscore_status make_tmap_bf16(const maxscore_ctx* c, CUtensorMap* tm, const voi
 unsigned* error_flag_of(const maxscore_ctx* c) { return reinterpret_cast<unsigned*>(c->ws + c->lay.error_flag); }
 size_t elem_bytes(const maxscore_ctx* c) { return c->p.io_dtype == MAXSCORE_BF16 ? 2 : 4; }
 
-maxscore_status launch_gate(maxscore_ctx* c, const void* hidden, const void* w_gate, const float* bias,
-                            float* logits, cudaStream_t st) {
+// The gate GEMM of Eq. 2 in two steps, so that the host path can run it over row blocks as they arrive:
+// the weight in the tile layout of the tensor-core kernel (bf16 only), then the rows [row0, row0 + rows).
+maxscore_status launch_gate_prepare(maxscore_ctx* c, const void* w_gate, cudaStream_t st) {
   const maxscore_params& p = c->p;
+  if (p.io_dtype == MAXSCORE_F32) return MAXSCORE_OK;
+  __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(c->ws + c->lay.wt);
+  const int Npad = c->lay.Npad;
+  const long long n = (long long)Npad * p.d_model;
+  int blocks = (int)((n + 255) / 256); if (blocks > 1184) blocks = 1184;
+  wgate_prepare_kernel<<<blocks, 256, 0, st>>>((const __nv_bfloat16*)w_gate, wt, p.d_model, p.E, Npad, p.w_gate_layout);
+  MS_LAUNCH_CHECK("wgate_prepare_kernel");
+  c->launches += 1;
+  return MAXSCORE_OK;
+}
+
+maxscore_status launch_gate_rows(maxscore_ctx* c, const void* hidden, const void* w_gate, const float* bias, float* logits,
+                                 int row0, int rows, cudaStream_t st) {
+  const maxscore_params& p = c->p;
+  float* out = logits + (size_t)row0 * p.E;
   if (p.io_dtype == MAXSCORE_F32) {
-    dim3 grid((p.T + 15) / 16, (p.E + 15) / 16);
-    gate_gemm_simt_kernel<float><<<grid, 256, 0, st>>>((const float*)hidden, (const float*)w_gate, bias, logits,
-                                                        p.T, p.d_model, p.E, p.w_gate_layout);
+    dim3 grid((rows + 15) / 16, (p.E + 15) / 16);
+    gate_gemm_simt_kernel<float><<<grid, 256, 0, st>>>((const float*)hidden + (size_t)row0 * p.d_model, (const float*)w_gate,
+                                                        bias, out, rows, p.d_model, p.E, p.w_gate_layout);
     MS_LAUNCH_CHECK("gate_gemm_simt_kernel");
     c->launches += 1;
     return MAXSCORE_OK;
   }
   __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(c->ws + c->lay.wt);
   const int Npad = c->lay.Npad;
-  {
-    const long long n = (long long)Npad * p.d_model;
-    int blocks = (int)((n + 255) / 256); if (blocks > 1184) blocks = 1184;
-    wgate_prepare_kernel<<<blocks, 256, 0, st>>>((const __nv_bfloat16*)w_gate, wt, p.d_model, p.E, Npad, p.w_gate_layout);
-    MS_LAUNCH_CHECK("wgate_prepare_kernel");
-  }
   CUtensorMap tmH, tmW;
-  maxscore_status s = make_tmap_bf16(c, &tmH, hidden, (uint64_t)p.d_model, (uint64_t)p.T, kGateBK, kGateBM);
+  maxscore_status s = make_tmap_bf16(c, &tmH, (const __nv_bfloat16*)hidden + (size_t)row0 * p.d_model, (uint64_t)p.d_model,
+                                     (uint64_t)rows, kGateBK, kGateBM);
   if (s) return s;
   s = make_tmap_bf16(c, &tmW, wt, (uint64_t)p.d_model, (uint64_t)Npad, kGateBK, (uint32_t)Npad);
   if (s) return s;
   const int num_kb = (p.d_model + kGateBK - 1) / kGateBK;
-  gate_gemm_tc_kernel<<<(p.T + kGateBM - 1) / kGateBM, 128, kGateSmemBytes, st>>>(tmH, tmW, bias, logits, p.T, p.E,
-                                                                                   Npad, num_kb, error_flag_of(c));
+  gate_gemm_tc_kernel<<<(rows + kGateBM - 1) / kGateBM, 128, kGateSmemBytes, st>>>(tmH, tmW, bias, out, rows, p.E, Npad, num_kb,
+                                                                                  error_flag_of(c));
   MS_LAUNCH_CHECK("gate_gemm_tc_kernel");
-  c->launches += 2;
+  c->launches += 1;
+  return MAXSCORE_OK;
+}
+
+maxscore_status launch_gate(maxscore_ctx* c, const void* hidden, const void* w_gate, const float* bias,
+                            float* logits, cudaStream_t st) {
+  maxscore_status s = launch_gate_prepare(c, w_gate, st);
+  if (s) return s;
+  return launch_gate_rows(c, hidden, w_gate, bias, logits, 0, c->p.T, st);
+}
+
+// SoftTopk (Eq. 6) or one of its variants over `rows` rows (every row is on its own).
+maxscore_status launch_softtopk_rows(maxscore_ctx* c, const float* logits, float* scores, int rows, cudaStream_t st) {
+  const maxscore_params& p = c->p;
+  int blocks = (rows + 7) / 8; if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
+  if (p.softtopk_mode == 2)
+    itertopk_kernel<false><<<blocks, 256, 0, st>>>(logits, nullptr, nullptr, nullptr, scores, rows, p.E, p.k);
+  else if (p.softtopk_mode == 1)
+    softtopk_rankscale_kernel<false><<<blocks, 256, 0, st>>>(logits, nullptr, nullptr, nullptr, scores, rows, p.E, p.k, p.t,
+                                                             p.rankscale_beta, p.rankscale_delta);
+  else
+    softtopk_fwd_kernel<<<blocks, 256, 0, st>>>(logits, scores, rows, p.E, p.k, p.t);
+  MS_LAUNCH_CHECK("softtopk_fwd_kernel");
+  c->launches += 1;
   return MAXSCORE_OK;
 }
 
 maxscore_status launch_softtopk_fwd(maxscore_ctx* c, const float* logits, float* scores, cudaStream_t st) {
-  const maxscore_params& p = c->p;
-  int blocks = (p.T + 7) / 8; if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
-  if (p.softtopk_mode == 2)
-    itertopk_kernel<false><<<blocks, 256, 0, st>>>(logits, nullptr, nullptr, nullptr, scores, p.T, p.E, p.k);
-  else if (p.softtopk_mode == 1)
-    softtopk_rankscale_kernel<false><<<blocks, 256, 0, st>>>(logits, nullptr, nullptr, nullptr, scores, p.T, p.E, p.k, p.t,
-                                                             p.rankscale_beta, p.rankscale_delta);
-  else
-    softtopk_fwd_kernel<<<blocks, 256, 0, st>>>(logits, scores, p.T, p.E, p.k, p.t);
-  MS_LAUNCH_CHECK("softtopk_fwd_kernel");
-  c->launches += 1;
-  return MAXSCORE_OK;
+  return launch_softtopk_rows(c, logits, scores, c->p.T, st);
 }
 
 // rounds of (records, exact phase, check): candidate thresholds theta0, then two wider ones (four times the last, or twice
@@ -274,6 +300,11 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   a.T = p.T; a.E = p.E; a.k = p.k; a.C = c->C;
   a.n_sweeps = budget < kSweeps ? budget : kSweeps;
   a.balanced = ((long long)p.E * c->C == (long long)p.T * p.k) ? 1 : 0;
+  {   // a few units of spare room per expert at most: the sweeps hide them at first (see SweepArgs::slack).  With more
+      // spare room than that the guess of who keeps it costs more repairs than the slow start it avoids.
+    const long long spare = (long long)p.E * c->C - (long long)p.T * p.k;
+    a.slack = (spare > 0 && spare <= 4LL * p.E) ? (int)spare : 0;
+  }
   a.eps0 = 1LL << (scale_bits - 10);
   a.eps_min = p.score_mode == 0 ? (1LL << 20) : (1LL << 12);
   // first candidate threshold: 2^-14 of a unit of score.  Half of it lists fewer tokens but on the stress workload
@@ -339,6 +370,34 @@ __global__ void gather_gate_w_kernel(const float* __restrict__ scores, const int
     const int e = expert_idx[i];
     gate_w[i] = (e >= 0 && e < E) ? scores[tok * E + e] : 0.f;
   }
+}
+
+constexpr int kHostChunks = 8, kHostChunkMinRows = 1024;     // row blocks of the host path, and the smallest worth a copy
+maxscore_status host_path_streams(maxscore_ctx* c) {
+  static_assert(sizeof(c->ev_chunk) / sizeof(c->ev_chunk[0]) == kHostChunks, "one event per row block");
+  if (c->copy_stream) return MAXSCORE_OK;
+  MS_CUDA(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+  MS_CUDA(cudaEventCreateWithFlags(&c->ev_start, cudaEventDisableTiming));
+  MS_CUDA(cudaEventCreateWithFlags(&c->ev_routed, cudaEventDisableTiming));
+  MS_CUDA(cudaEventCreateWithFlags(&c->ev_copied, cudaEventDisableTiming));
+  for (int i = 0; i < kHostChunks; ++i) MS_CUDA(cudaEventCreateWithFlags(&c->ev_chunk[i], cudaEventDisableTiming));
+  return MAXSCORE_OK;
+}
+
+// The part of the forward route that needs every token's scores: assignment, slots, gate weights.
+maxscore_status route_after_scores(maxscore_ctx* c, const float* logits, const float* scores, int32_t* expert_idx,
+                                   int32_t* slot_idx, float* gate_w, int32_t* slot_token, int32_t* expert_load,
+                                   maxscore_stats* stats, cudaStream_t st) {
+  maxscore_status s = launch_assign(c, c->p.score_mode == 0 ? scores : logits, expert_idx, expert_load, stats, st);
+  if (s) return s;
+  s = launch_index_build(c, expert_idx, slot_idx, slot_token, expert_load, st);
+  if (s) return s;
+  const long long n = (long long)c->p.T * c->p.k;
+  int blocks = (int)((n + 255) / 256); if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
+  gather_gate_w_kernel<<<blocks, 256, 0, st>>>(scores, expert_idx, gate_w, n, c->p.E, c->p.k);
+  MS_LAUNCH_CHECK("gather_gate_w_kernel");
+  c->launches += 1;
+  return MAXSCORE_OK;
 }
 
 maxscore_status launch_zero_padding(maxscore_ctx* c, const int32_t* slot_token, void* dst, cudaStream_t st) {
@@ -413,7 +472,15 @@ maxscore_status maxscore_create(maxscore_ctx** out, const maxscore_params* param
   return MAXSCORE_OK;
 }
 
-void maxscore_destroy(maxscore_ctx* ctx) { delete ctx; }
+void maxscore_destroy(maxscore_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  if (ctx->ev_start) cudaEventDestroy(ctx->ev_start);
+  if (ctx->ev_routed) cudaEventDestroy(ctx->ev_routed);
+  if (ctx->ev_copied) cudaEventDestroy(ctx->ev_copied);
+  for (cudaEvent_t e : ctx->ev_chunk) if (e) cudaEventDestroy(e);
+  delete ctx;
+}
 
 maxscore_status maxscore_gate(maxscore_ctx* c, const void* hidden, const void* w_gate, const float* bias,
                               float* logits, void* stream) {
@@ -501,16 +568,7 @@ maxscore_status maxscore_route_fwd(maxscore_ctx* c, const void* hidden, const vo
   if (s) return s;
   s = launch_softtopk_fwd(c, logits, scores, st);
   if (s) return s;
-  s = launch_assign(c, c->p.score_mode == 0 ? scores : logits, expert_idx, expert_load, stats, st);
-  if (s) return s;
-  s = launch_index_build(c, expert_idx, slot_idx, slot_token, expert_load, st);
-  if (s) return s;
-  const long long n = (long long)c->p.T * c->p.k;
-  int blocks = (int)((n + 255) / 256); if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
-  gather_gate_w_kernel<<<blocks, 256, 0, st>>>(scores, expert_idx, gate_w, n, c->p.E, c->p.k);
-  MS_LAUNCH_CHECK("gather_gate_w_kernel");
-  c->launches += 1;
-  return MAXSCORE_OK;
+  return route_after_scores(c, logits, scores, expert_idx, slot_idx, gate_w, slot_token, expert_load, stats, st);
 }
 
 maxscore_status maxscore_dispatch(maxscore_ctx* c, const void* src, const int32_t* expert_idx,
@@ -751,23 +809,54 @@ maxscore_status maxscore_route_dispatch_host(maxscore_ctx* c, const void* hidden
   if (!c || !hidden_host || !w_gate_host || !dev || !expert_idx_host || !slot_idx_host || !gate_w_host || !stats_host)
     return MAXSCORE_ERR_INVALID_ARG;
   if (!dev->hidden || !dev->w_gate || !dev->xdisp || (bias_host && !dev->expert_bias)) return MAXSCORE_ERR_INVALID_ARG;
+  if (!aligned16(dev->hidden) || !aligned16(dev->w_gate) || !aligned16(dev->logits) || !aligned16(dev->scores) ||
+      !aligned16(dev->xdisp))
+    return MAXSCORE_ERR_INVALID_ARG;
   const maxscore_params& p = c->p;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t eb = elem_bytes(c);
-  MS_CUDA(cudaMemcpyAsync(dev->hidden, hidden_host, eb * (size_t)p.T * p.d_model, cudaMemcpyHostToDevice, st));
+  maxscore_status s = host_path_streams(c);
+  if (s) return s;
+  cudaStream_t cs = c->copy_stream;
+  // The token rows go up in blocks on a second stream; the gate GEMM and SoftTopk of a block start when it has
+  // landed, so only the last block's share of them is left when the copy ends.  The assignment needs every row.
   MS_CUDA(cudaMemcpyAsync(dev->w_gate, w_gate_host, eb * (size_t)p.d_model * p.E, cudaMemcpyHostToDevice, st));
   if (bias_host) MS_CUDA(cudaMemcpyAsync(dev->expert_bias, bias_host, sizeof(float) * p.E, cudaMemcpyHostToDevice, st));
-  maxscore_status s = maxscore_route_fwd(c, dev->hidden, dev->w_gate, bias_host ? dev->expert_bias : nullptr, dev->logits,
-                                         dev->scores, dev->expert_idx, dev->slot_idx, dev->gate_w, dev->slot_token,
-                                         dev->expert_load, dev->stats, stream);
+  s = launch_gate_prepare(c, dev->w_gate, st);
   if (s) return s;
+  MS_CUDA(cudaEventRecord(c->ev_start, st));          // what ran before on the caller's stream may still read dev->hidden
+  MS_CUDA(cudaStreamWaitEvent(cs, c->ev_start, 0));
+  int nchunks = p.T / kHostChunkMinRows < kHostChunks ? p.T / kHostChunkMinRows : kHostChunks;
+  if (nchunks < 1) nchunks = 1;
+  const int rows_per = (int)align_up((size_t)((p.T + nchunks - 1) / nchunks), 128);
+  const float* bias_dev = bias_host ? dev->expert_bias : nullptr;
+  for (int i = 0, row0 = 0; row0 < p.T; ++i, row0 += rows_per) {
+    const int rows = p.T - row0 < rows_per ? p.T - row0 : rows_per;
+    const size_t off = eb * (size_t)row0 * p.d_model;
+    MS_CUDA(cudaMemcpyAsync((char*)dev->hidden + off, (const char*)hidden_host + off, eb * (size_t)rows * p.d_model,
+                            cudaMemcpyHostToDevice, cs));
+    MS_CUDA(cudaEventRecord(c->ev_chunk[i], cs));
+    MS_CUDA(cudaStreamWaitEvent(st, c->ev_chunk[i], 0));
+    s = launch_gate_rows(c, dev->hidden, dev->w_gate, bias_dev, dev->logits, row0, rows, st);
+    if (s) return s;
+    s = launch_softtopk_rows(c, dev->logits + (size_t)row0 * p.E, dev->scores + (size_t)row0 * p.E, rows, st);
+    if (s) return s;
+  }
+  s = route_after_scores(c, dev->logits, dev->scores, dev->expert_idx, dev->slot_idx, dev->gate_w, dev->slot_token,
+                         dev->expert_load, dev->stats, st);
+  if (s) return s;
+  // the indices go back on the copy stream while the rows are dispatched
+  MS_CUDA(cudaEventRecord(c->ev_routed, st));
+  MS_CUDA(cudaStreamWaitEvent(cs, c->ev_routed, 0));
+  const size_t nk = (size_t)p.T * p.k;
+  MS_CUDA(cudaMemcpyAsync(expert_idx_host, dev->expert_idx, sizeof(int32_t) * nk, cudaMemcpyDeviceToHost, cs));
+  MS_CUDA(cudaMemcpyAsync(slot_idx_host, dev->slot_idx, sizeof(int32_t) * nk, cudaMemcpyDeviceToHost, cs));
+  MS_CUDA(cudaMemcpyAsync(gate_w_host, dev->gate_w, sizeof(float) * nk, cudaMemcpyDeviceToHost, cs));
+  MS_CUDA(cudaMemcpyAsync(stats_host, dev->stats, sizeof(maxscore_stats), cudaMemcpyDeviceToHost, cs));
+  MS_CUDA(cudaEventRecord(c->ev_copied, cs));
   s = maxscore_dispatch(c, dev->hidden, dev->expert_idx, dev->slot_idx, dev->slot_token, dev->xdisp, stream);
   if (s) return s;
-  const size_t nk = (size_t)p.T * p.k;
-  MS_CUDA(cudaMemcpyAsync(expert_idx_host, dev->expert_idx, sizeof(int32_t) * nk, cudaMemcpyDeviceToHost, st));
-  MS_CUDA(cudaMemcpyAsync(slot_idx_host, dev->slot_idx, sizeof(int32_t) * nk, cudaMemcpyDeviceToHost, st));
-  MS_CUDA(cudaMemcpyAsync(gate_w_host, dev->gate_w, sizeof(float) * nk, cudaMemcpyDeviceToHost, st));
-  MS_CUDA(cudaMemcpyAsync(stats_host, dev->stats, sizeof(maxscore_stats), cudaMemcpyDeviceToHost, st));
+  MS_CUDA(cudaStreamWaitEvent(st, c->ev_copied, 0));   // later work on the caller's stream may overwrite the indices
   MS_CUDA(cudaStreamSynchronize(st));
   return MAXSCORE_OK;
 }

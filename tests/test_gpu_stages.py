@@ -250,7 +250,9 @@ def _check_feasible(idx, load, T, E, k, C, st=None):
                                             (1000, 16, 4, 1.0, False), (2048, 64, 8, 1.0, False),
                                             (2048, 64, 8, 1.25, True), (300, 8, 2, 1.5, True),
                                             (8192, 64, 8, 1.0, False), (129, 5, 5, 1.0, False),
-                                            (257, 12, 1, 1.0, True)])
+                                            (257, 12, 1, 1.0, True),
+                                            # a few units of spare room (T*k not a multiple of E): the sweeps hide them at first
+                                            (4097, 16, 2, 1.0, False), (2051, 64, 8, 1.0, False), (8269, 128, 8, 1.0, False)])
 def test_assign_float_scores(ms, orc, synth, T, E, k, cf, skew):
     wl = synth.Workload("a", T, 64, E, k, cf, "bf16", skew=skew)
     L = synth.logits_like(T, E, seed=7, bias=synth.expert_bias(wl, 7))
@@ -281,7 +283,8 @@ def test_assign_float_scores(ms, orc, synth, T, E, k, cf, skew):
 
 @pytest.mark.parametrize("T,E,k,cf,skew,seed", [(512, 8, 2, 1.0, False, 0), (2048, 64, 8, 1.0, False, 0),
                                                  (2048, 64, 8, 1.25, True, 1), (8192, 64, 8, 1.0, False, 0),
-                                                 (1000, 16, 3, 1.0, False, 2)])
+                                                 (1000, 16, 3, 1.0, False, 2), (4097, 16, 2, 1.0, False, 0),
+                                                 (2051, 64, 8, 1.0, False, 3)])
 def test_assign_integer_keys_bit_exact(ms, orc, synth, T, E, k, cf, skew, seed):
     wl = synth.Workload("a", T, 64, E, k, cf, "bf16", skew=skew)
     L = synth.logits_like(T, E, seed=11, bias=synth.expert_bias(wl, 11))
@@ -430,11 +433,13 @@ def test_route_fwd_end_to_end(ms, orc, synth, name, T):
     np.testing.assert_array_equal(np32(buf.gate_w), np.take_along_axis(A, idx.astype(np.int64), axis=1))
 
 
-@pytest.mark.parametrize("name,T,bias", [("tiny", None, False), ("k2e16", 1000, False), ("skew", 2048, True)])
+@pytest.mark.parametrize("name,T,bias", [("tiny", None, False), ("k2e16", 1000, False), ("skew", 2048, True),
+                                         ("skew", 9000, True), ("stress", 8269, False)])
 def test_route_dispatch_from_host_buffers(ms, orc, synth, name, T, bias):
     """The end-to-end entry point: batch in host memory in, indices and combine weights back in host memory,
     dispatched rows on the device.  Same kernels as route_fwd + dispatch, so the results are bit-identical to
-    that path, and the dispatched rows are checked against the oracle."""
+    that path, and the dispatched rows are checked against the oracle.  The larger cases go up in eight row
+    blocks with a ragged last one."""
     wl = synth.WORKLOADS[name]
     wl = synth.scaled(wl, T=T, d_model=min(wl.d_model, 512)) if T else wl
     T, d, E, k = wl.T, wl.d_model, wl.E, wl.k
