@@ -310,7 +310,9 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
   // first candidate threshold: 2^-14 of a unit of score.  Half of it lists fewer tokens but on the stress workload
   // often needs a second round (records, exact phase and check pass again); twice as much makes every search
   // round of the exact phase walk over twice as many records
-  a.theta0 = 1LL << (scale_bits - 14);
+  // (integer keys are logits, whose k-th and (k+1)-th values lie some twenty times further apart than those of the
+  // scores, and whose ties the fp32 sweeps cannot tell apart: 2^-11 of a unit lists about as many tokens there)
+  a.theta0 = 1LL << (scale_bits - (p.score_mode == 0 ? 14 : 11));
   int max_aug = budget - a.n_sweeps;
 
   flow_init_kernel<<<32, 256, 0, st>>>(fs, kCapLogMax, a.theta0, a.balanced, p.E);
