@@ -265,8 +265,14 @@ maxscore_status launch_softtopk_rows(maxscore_ctx* c, const float* logits, float
   else if (p.softtopk_mode == 1)
     softtopk_rankscale_kernel<false><<<blocks, 256, 0, st>>>(logits, nullptr, nullptr, nullptr, scores, rows, p.E, p.k, p.t,
                                                              p.rankscale_beta, p.rankscale_delta);
-  else
-    softtopk_fwd_kernel<<<blocks, 256, 0, st>>>(logits, scores, rows, p.E, p.k, p.t);
+  else {
+    const int tiles = (rows + kStTok - 1) / kStTok;
+    const int grid = tiles < c->sm_count * 6 ? tiles : c->sm_count * 6;
+    const size_t smem = sizeof(float) * (size_t)kStTok * st_stride(p.E);
+    if (p.k <= 2) softtopk_fwd_kernel<2><<<grid, kStThreads, smem, st>>>(logits, scores, rows, p.E, p.k, p.t);
+    else if (p.k <= 4) softtopk_fwd_kernel<4><<<grid, kStThreads, smem, st>>>(logits, scores, rows, p.E, p.k, p.t);
+    else softtopk_fwd_kernel<8><<<grid, kStThreads, smem, st>>>(logits, scores, rows, p.E, p.k, p.t);
+  }
   MS_LAUNCH_CHECK("softtopk_fwd_kernel");
   c->launches += 1;
   return MAXSCORE_OK;
@@ -274,6 +280,20 @@ maxscore_status launch_softtopk_rows(maxscore_ctx* c, const float* logits, float
 
 maxscore_status launch_softtopk_fwd(maxscore_ctx* c, const float* logits, float* scores, cudaStream_t st) {
   return launch_softtopk_rows(c, logits, scores, c->p.T, st);
+}
+
+void launch_softtopk_bwd_tiles(maxscore_ctx* c, const float* logits, const int32_t* expert_idx, const float* dgate_w,
+                               const float* dscores_col, float* dlogits, cudaStream_t st) {
+  const maxscore_params& p = c->p;
+  const int tiles = (p.T + kStTok - 1) / kStTok;
+  const int grid = tiles < c->sm_count * 6 ? tiles : c->sm_count * 6;
+  const size_t smem = sizeof(float) * ((size_t)kStTok * st_stride(p.E) + p.E);
+  if (p.k <= 2)
+    softtopk_bwd_kernel<2><<<grid, kStThreads, smem, st>>>(logits, expert_idx, dgate_w, dscores_col, dlogits, p.T, p.E, p.k, p.t);
+  else if (p.k <= 4)
+    softtopk_bwd_kernel<4><<<grid, kStThreads, smem, st>>>(logits, expert_idx, dgate_w, dscores_col, dlogits, p.T, p.E, p.k, p.t);
+  else
+    softtopk_bwd_kernel<8><<<grid, kStThreads, smem, st>>>(logits, expert_idx, dgate_w, dscores_col, dlogits, p.T, p.E, p.k, p.t);
 }
 
 // rounds of (records, exact phase, check): candidate thresholds theta0, then two wider ones (four times the last, or twice
@@ -451,6 +471,15 @@ maxscore_status maxscore_create(maxscore_ctx** out, const maxscore_params* param
     return MAXSCORE_ERR_CUDA;
   }
   MS_CUDA(cudaFuncSetAttribute(gate_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGateSmemBytes));
+  {
+    const int st_smem = (int)(sizeof(float) * ((size_t)kStTok * st_stride(kMaxE) + kMaxE));
+    MS_CUDA(cudaFuncSetAttribute(softtopk_fwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, st_smem));
+    MS_CUDA(cudaFuncSetAttribute(softtopk_fwd_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, st_smem));
+    MS_CUDA(cudaFuncSetAttribute(softtopk_fwd_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, st_smem));
+    MS_CUDA(cudaFuncSetAttribute(softtopk_bwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, st_smem));
+    MS_CUDA(cudaFuncSetAttribute(softtopk_bwd_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, st_smem));
+    MS_CUDA(cudaFuncSetAttribute(softtopk_bwd_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, st_smem));
+  }
   MS_CUDA(cudaFuncSetAttribute(flow_exact_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRecSmemBytes));
   MS_CUDA(cudaFuncSetAttribute(gate_bwd_dh_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDhSmemMax));
   MS_CUDA(cudaFuncSetAttribute(gate_bwd_dw_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDwSmemMax));
@@ -507,7 +536,7 @@ maxscore_status maxscore_softtopk_bwd(maxscore_ctx* c, const float* logits, cons
     softtopk_rankscale_kernel<true><<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, nullptr, dlogits, p.T,
                                                                              p.E, p.k, p.t, p.rankscale_beta, p.rankscale_delta);
   else
-    softtopk_bwd_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, nullptr, dlogits, p.T, p.E, p.k, p.t);
+    launch_softtopk_bwd_tiles(c, logits, expert_idx, dgate_w, nullptr, dlogits, (cudaStream_t)stream);
   MS_LAUNCH_CHECK("softtopk_bwd_kernel");
   c->launches += 1;
   return MAXSCORE_OK;
@@ -524,7 +553,7 @@ maxscore_status maxscore_softtopk_bwd_aux(maxscore_ctx* c, const float* logits, 
     softtopk_rankscale_kernel<true><<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, dscores_col, dlogits,
                                                                              p.T, p.E, p.k, p.t, p.rankscale_beta, p.rankscale_delta);
   else
-    softtopk_bwd_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>(logits, expert_idx, dgate_w, dscores_col, dlogits, p.T, p.E, p.k, p.t);
+    launch_softtopk_bwd_tiles(c, logits, expert_idx, dgate_w, dscores_col, dlogits, (cudaStream_t)stream);
   MS_LAUNCH_CHECK("softtopk_bwd_kernel");
   c->launches += 1;
   return MAXSCORE_OK;
