@@ -396,7 +396,7 @@ def run_ours(args, wl):
     if d == 4096 and k == 8 and eb == 2 and dom_name in ncu_bytes_per_token:
         traffic = ncu_bytes_per_token[dom_name] * T
     elif dom_name == "assign" and (T, E, k) == (65536, 128, 8) and wl.capacity_factor == 1.0:
-        # the 19 launches of one solver call at this very size (profiles/ncu_solver_T65536_stress.md): the score matrix
+        # the 19 launches of one solver call at this very size (ncu capture summarised under profiles/): the score matrix
         # once (33.6 MB), then caches, histograms and records; far below the algorithmic bytes, which count a full
         # pass over the matrix for the scan, every sweep and every check
         traffic = 49.2e6
