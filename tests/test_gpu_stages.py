@@ -76,7 +76,10 @@ def test_gate(ms, orc, synth, T, d, E, dtype, layout, bias):
 
 # ------------------------------------------------------------------------------------------- SoftTopk
 @pytest.mark.parametrize("T,E,k,t", [(512, 8, 2, 1.0), (512, 8, 2, 4.0), (1000, 16, 2, 1.0), (777, 64, 8, 1.0),
-                                      (515, 128, 8, 0.25), (64, 20, 3, 2.0), (33, 5, 5, 1.0), (40, 128, 1, 1.0)])
+                                      (515, 128, 8, 0.25), (64, 20, 3, 2.0), (33, 5, 5, 1.0), (40, 128, 1, 1.0),
+                                      # odd expert counts (the two lanes of a token get unequal shares), k = E (no tail),
+                                      # several tiles with a ragged last one, every list width (k <= 2, <= 4, <= 8)
+                                      (300, 77, 5, 1.0), (130, 8, 8, 0.5), (4133, 101, 4, 1.0), (257, 3, 1, 1.0), (1, 128, 8, 1.0)])
 def test_softtopk_fwd_bwd(ms, orc, synth, T, E, k, t):
     L = synth.logits_like(T, E, seed=3)
     ctx = _ctx(ms, T, 64, E, k, cf=float(E), t=t)       # capacity irrelevant here
