@@ -548,8 +548,8 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gtid = blockIdx.x * blockDim.x + tid, gsize = gridDim.x * blockDim.x;
   const bool resident = T <= gsize;
-  bool hiding = a.slack > 0;                               // spare room is hidden from the sweeps (see SweepArgs::slack)
-  bool free_prices = a.balanced || hiding;                 // prices may go below zero until they are anchored
+  bool hiding = false;                                     // spare room is hidden from the sweeps (see SweepArgs::slack)
+  bool free_prices = a.balanced != 0;                      // prices may go below zero until they are anchored
   bool pending = false; long long pend_anchor = 0;         // an anchoring that the next price step still has to apply
   for (int e = tid; e < kMaxE; e += blockDim.x) sh.trim[e] = 0;
   unsigned epoch = 0;
@@ -697,32 +697,47 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
 
     // ---- every CTA draws the same conclusions from the same numbers ----------------------------------
     load_state();
-    if (a.slack > 0 && sweep == 0) {
-      // who gives up room: raise a water level under the first sweep's loads until the room below it is the spare room
+    if (sweep == 0 && (a.slack > 0 || a.balanced)) {
+      // The first sweep (every price zero) tells how lopsided the router is.  Free prices pay off when the loads are
+      // roughly even: experts short of tokens then hear from enough tokens that rank them next to cut their price by
+      // the right amount.  With most pairs on a few experts they hear from hardly anyone, cut blindly and overshoot,
+      // and the prices swing ever wider; there the prices keep their floor at zero and only the crowded experts move.
       for (int e = tid; e < E; e += blockDim.x) sh.l0[e] = __ldcg(&st->load0[e]);
+      if (tid == 0) sh.s_nb = 0;
       __syncthreads();
-      for (int e = tid; e < E; e += blockDim.x) {
-        int rank = 0;
-        for (int x = 0; x < E; ++x) rank += (sh.l0[x] < sh.l0[e] || (sh.l0[x] == sh.l0[e] && x < e)) ? 1 : 0;
-        sh.srt[rank] = sh.l0[e]; sh.trim[e] = rank;
-      }
+      for (int e = tid; e < E; e += blockDim.x) if (sh.l0[e] > C) atomicAdd(&sh.s_nb, sh.l0[e] - C);
       __syncthreads();
-      if (tid == 0) {
-        long long rem = a.slack; int j = 1;               // the j least popular experts are below the level srt[j - 1]
-        while (j < E) {
-          const long long need = (long long)j * (sh.srt[j] - sh.srt[j - 1]);
-          if (need > rem) break;
-          rem -= need; ++j;
+      const bool even = (long long)sh.s_nb * 8 <= (long long)T * a.k;
+      __syncthreads();
+      if (a.slack > 0 && even) {
+        // who gives up room: raise a water level under the first sweep's loads until the room below it is the spare room
+        for (int e = tid; e < E; e += blockDim.x) {
+          int rank = 0;
+          for (int x = 0; x < E; ++x) rank += (sh.l0[x] < sh.l0[e] || (sh.l0[x] == sh.l0[e] && x < e)) ? 1 : 0;
+          sh.srt[rank] = sh.l0[e]; sh.trim[e] = rank;
         }
-        sh.s_nb = j; sh.s_level = sh.srt[j - 1] + (int)(rem / j); sh.s_rem = (int)(rem % j);
+        __syncthreads();
+        if (tid == 0) {
+          long long rem = a.slack; int j = 1;               // the j least popular experts are below the level srt[j - 1]
+          while (j < E) {
+            const long long need = (long long)j * (sh.srt[j] - sh.srt[j - 1]);
+            if (need > rem) break;
+            rem -= need; ++j;
+          }
+          sh.s_nb = j; sh.s_level = sh.srt[j - 1] + (int)(rem / j); sh.s_rem = (int)(rem % j);
+        }
+        __syncthreads();
+        for (int e = tid; e < E; e += blockDim.x) {
+          const int rank = sh.trim[e];
+          const int t = rank < sh.s_nb ? sh.s_level - sh.l0[e] + (rank < sh.s_rem ? 1 : 0) : 0;
+          sh.trim[e] = t < C ? t : C;
+        }
+        hiding = true; free_prices = true;
+        __syncthreads();
+      } else if (a.balanced && !even) {
+        pend_anchor = anchor_prices(); pending = true;      // lowest price to zero, and from here on none below it
+        free_prices = false;
       }
-      __syncthreads();
-      for (int e = tid; e < E; e += blockDim.x) {
-        const int rank = sh.trim[e];
-        const int t = rank < sh.s_nb ? sh.s_level - sh.l0[e] + (rank < sh.s_rem ? 1 : 0) : 0;
-        sh.trim[e] = t < C ? t : C;
-      }
-      __syncthreads();
     }
     ++sweep;
     // a small imbalance that has stopped shrinking is a price war between a few experts: the exact phase
