@@ -415,8 +415,8 @@ struct SweepShared {
   float spf[kMaxE];
   unsigned smin_up[kMaxE], smin_dn[kMaxE];   // smallest margins of the pass, as float bit patterns
   float capu[kMaxE], capd[kMaxE];            // margins at or above these are not recorded
-  int sload[kMaxE], sflag[kMaxE];
-  int nflag, nslow, s_imb;
+  int sload[kMaxE], sflag[kMaxE], sdeaf[kMaxE];   // sdeaf: flagged experts that heard from no token at all
+  int nflag, ndeaf, nslow, s_imb;
   long long s_drop, s_pmin;
   int slow[kSwThreads];
   int trim[kMaxE];                           // room the sweeps leave unused on purpose (see SweepArgs::slack)
@@ -450,7 +450,7 @@ __device__ __forceinline__ void load_tok_cache(TokCache& c, const SweepCache& ca
 // do (what they leave undone the exact phase repairs, and the first pick and the check pass are exact).
 // Returns false when the cache cannot vouch for the token's k+2 best experts any more (the caller then has
 // the row rescanned and calls again).
-__device__ __forceinline__ bool sweep_token(int tok, const TokCache& c, SweepShared& sh, const SweepArgs& a,
+__device__ __forceinline__ bool sweep_token(const float* __restrict__ M, int tok, const TokCache& c, SweepShared& sh, const SweepArgs& a,
                                             const KeyGen& g, float cumdropf, unsigned* hup, unsigned* hdn) {
   const int E = a.E, k = a.k;
   const int need = min(k + 2, E);                       // sorted values a token has to know
@@ -490,6 +490,24 @@ __device__ __forceinline__ bool sweep_token(int tok, const TokCache& c, SweepSha
       // its best alternatives
       for (int q = 0; q < nflag; ++q) rec |= sh.sflag[q] == e;
       if (rec) emit_margin(hdn, sh.smin_dn, sh.capd, e, vk - v[j]);
+    }
+  }
+  // An expert that heard from no token at all (with a lopsided router the unpopular experts are in nobody's cache)
+  // could never find the price at which anyone joins it: for those, one score per token is read from the matrix.
+  const int ndeaf = sh.ndeaf;
+  if (ndeaf) {
+    unsigned cached[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int j = 0; j < kCacheN; ++j) {
+      const int e = (int)((c.idws[j >> 2] >> (8 * (j & 3))) & 255u);
+#pragma unroll
+      for (int w = 0; w < 4; ++w) if ((e >> 5) == w) cached[w] |= 1u << (e & 31);
+    }
+    for (int q = 0; q < ndeaf; ++q) {
+      const int e = sh.sdeaf[q];
+      const unsigned word = (e & 64) ? ((e & 32) ? cached[3] : cached[2]) : ((e & 32) ? cached[1] : cached[0]);
+      if ((word >> (e & 31)) & 1u) continue;
+      emit_margin(hdn, sh.smin_dn, sh.capd, e, vk - (approx_key(g, __ldg(M + (size_t)tok * E + e)) - sh.spf[e]));
     }
   }
   return true;
@@ -571,7 +589,7 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
       if (tok < T) {
         if (!resident) load_tok_cache(mine, cache, tok, T);
         const bool ok = kPick ? pick_token(tok, mine, st, sh, a, g, cumdrop, expert_idx, cand)
-                              : sweep_token(tok, mine, sh, a, g, (float)cumdrop, hup, hdn);
+                              : sweep_token(M, tok, mine, sh, a, g, (float)cumdrop, hup, hdn);
         if (!ok) { sh.slow[atomicAdd(&sh.nslow, 1)] = tok; was_slow = true; }
       }
       __syncthreads();
@@ -586,7 +604,7 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
             TokCache fresh;
             load_tok_cache(fresh, cache, t2, T);
             if (kPick) pick_token(t2, fresh, st, sh, a, g, cumdrop, expert_idx, cand);
-            else sweep_token(t2, fresh, sh, a, g, (float)cumdrop, hup, hdn);
+            else sweep_token(M, t2, fresh, sh, a, g, (float)cumdrop, hup, hdn);
           }
         }
         __syncthreads();
@@ -596,7 +614,7 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
   };
   // prices, caps and flags for the next pass; on the way, what the last price step left behind
   auto load_state = [&]() {
-    if (tid == 0) { sh.nflag = 0; sh.s_imb = 0; sh.s_drop = 0; }
+    if (tid == 0) { sh.nflag = 0; sh.ndeaf = 0; sh.s_imb = 0; sh.s_drop = 0; }
     __syncthreads();
     for (int e = tid; e < E; e += blockDim.x) {
       const long long pe = __ldcg(&st->p[e]);
@@ -605,6 +623,7 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
       sh.sp[e] = pe; sh.spf[e] = (float)pe; sh.sload[e] = 0; sh.capu[e] = ldexpf(1.f, cu); sh.capd[e] = ldexpf(1.f, cd);
       sh.smin_up[e] = 0x7f800000u; sh.smin_dn[e] = 0x7f800000u;
       if (fl) sh.sflag[atomicAdd(&sh.nflag, 1)] = e;
+      if (fl == 2) sh.sdeaf[atomicAdd(&sh.ndeaf, 1)] = e;
       if (im) atomicAdd(&sh.s_imb, im);
       if (dr > 0) atomicMax(&sh.s_drop, dr);
     }
@@ -676,10 +695,13 @@ flow_sweeps_kernel(const float* __restrict__ M, FlowState* st, SweepCache cache,
         imb = xs;
       } else if (dn) {
         int cl = cdn; bool shortw;
-        p -= price_step_warp(had, hbd, -xs, eps, cl, shortw, kCapLogMax, md);
+        const long long cutby = price_step_warp(had, hbd, -xs, eps, cl, shortw, kCapLogMax, md);
+        p -= cutby;
         if (!free_prices && p < 0) p = 0;
         if (lane == 0) st->cap_dn[e] = cl;
-        flag = shortw ? 1 : 0;
+        // 2: nothing recorded at all and the price could not move.  When every expert has to end up full such an
+        // expert must be heard sooner or later; when there is room to spare it may simply be one that stays short.
+        flag = shortw ? ((cutby == 0 && a.balanced) ? 2 : 1) : 0;
         imb = -xs;
       }
       p = p > kPriceLimit ? kPriceLimit : (p < -kPriceLimit ? -kPriceLimit : p);

@@ -284,6 +284,27 @@ def test_assign_float_scores(ms, orc, synth, T, E, k, cf, skew):
     assert st.rerouted == int((~inside).sum())
 
 
+@pytest.mark.parametrize("T,E,k", [(4096, 64, 8), (16000, 64, 8), (6000, 100, 4)])
+def test_assign_lopsided_router_with_every_expert_full(ms, orc, synth, T, E, k):
+    """Zipf-biased router at capacity factor 1 with T*k a multiple of E: most pairs start on a few experts and every
+    expert has to end up full, the unpopular ones included, which no token keeps among its cached experts.  The
+    oracle's solver would take minutes here, so optimality is certified instead: the oracle's certificate of the
+    GPU's assignment (complementary slackness on the documented keys) and exact duality."""
+    wl = synth.Workload("a", T, 64, E, k, 1.0, "bf16", skew=True)
+    L = synth.logits_like(T, E, seed=21, bias=synth.expert_bias(wl, 21))
+    A = torch.from_numpy(orc.softtopk_fwd(f64(L), k, 1.0).astype(np.float32))
+    ctx, idx, load, st = _run_assign(ms, A, T, E, k, 1.0)
+    C = ctx.capacity
+    assert E * C == T * k
+    _check_feasible(idx, load, T, E, k, C, st)
+    assert st.status == 0, _describe(st)
+    assert (load == C).all()
+    keys = float_keys(A.numpy())
+    res, prices = orc.flow_certificate(keys, idx, C)
+    assert res >= 1, _describe(st)
+    assert orc.dual_value(keys, prices, k, C) == orc.primal_value(keys, idx)
+
+
 @pytest.mark.parametrize("T,E,k,cf,skew,seed", [(512, 8, 2, 1.0, False, 0), (2048, 64, 8, 1.0, False, 0),
                                                  (2048, 64, 8, 1.25, True, 1), (8192, 64, 8, 1.0, False, 0),
                                                  (1000, 16, 3, 1.0, False, 2), (4097, 16, 2, 1.0, False, 0),
