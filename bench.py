@@ -225,15 +225,15 @@ def run_ours(args, wl):
     gw_host = torch.empty(T, k, dtype=torch.float32).pin_memory()
     stats_host = torch.zeros(40, dtype=torch.uint8).pin_memory()
     devbuf = buf.device_buffers(Hd, Wd, bd, xd)
-    stage_names = ["route_fwd", "dispatch", "combine", "combine_bwd", "softtopk_bwd", "gate_bwd", "dispatch_bwd"]
+    stage_names = ["route_fwd", "dispatch", "combine", "route_bwd", "dispatch_bwd"]
 
     def rest_of_step(ev=None):
         mark = (lambda i: ev[i].record()) if ev else (lambda i: None)
         ms.combine(ctx, xd, buf.expert_idx, buf.slot_idx, buf.gate_w, Y); mark(3)
-        ms.combine_bwd(ctx, dY, xd, buf.expert_idx, buf.slot_idx, buf.gate_w, buf.slot_token, dyexp, dgw); mark(4)
-        ms.softtopk_bwd(ctx, buf.logits, buf.expert_idx, dgw, dL); mark(5)
-        ms.gate_bwd(ctx, Hd, Wd, dL, dW, dH); mark(6)
-        ms.combine(ctx, dyexp, buf.expert_idx, buf.slot_idx, None, dH, accumulate=1); mark(7)
+        # combine backward, SoftTopk backward and gate backward as the one call the header exports for them
+        ms.route_bwd(ctx, dY, xd, Hd, Wd, buf.logits, buf.expert_idx, buf.slot_idx, buf.gate_w, buf.slot_token, dyexp, dgw,
+                     dL, dW, dH); mark(4)
+        ms.combine(ctx, dyexp, buf.expert_idx, buf.slot_idx, None, dH, accumulate=1); mark(5)
 
     def step(ev=None):
         if ev:
@@ -262,7 +262,7 @@ def run_ours(args, wl):
     if rank == 0:
         sampler.start()
         time.sleep(0.2)
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(8)] for _ in range(args.steps)]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sync_all()
     launches0 = ms.launch_count(ctx)
@@ -274,7 +274,7 @@ def run_ours(args, wl):
     launches = ms.launch_count(ctx) - launches0           # counted by the library at every launch site
     clocks = sampler.stop() if rank == 0 else None
     ms_total = e0.elapsed_time(e1)
-    stage_ms = [sum(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(args.steps)) / args.steps for j in range(7)]
+    stage_ms = [sum(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(args.steps)) / args.steps for j in range(5)]
     ms_step = replicas.max_over_ranks(info, ms_total, dev) / args.steps
     st2 = ms.read_stats(buf.stats)
 
@@ -302,8 +302,8 @@ def run_ours(args, wl):
         replicas.shutdown(info)
         return
 
-    # ---- the stages of route_fwd one by one (the same kernels through the single-stage entry points), each
-    # timed after an L2 flush; and the solver on the skewed workload's shape, where it has to reroute heavily
+    # ---- the stages of route_fwd and route_bwd one by one (the same kernels through the single-stage entry points),
+    # each timed after an L2 flush; and the solver on the skewed workload's shape, where it has to reroute heavily
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     sub_ms = {
         "gate": time_call(torch, lambda: ms.gate(ctx, Hd, Wd, bd, buf.logits), flush=flush),
@@ -313,6 +313,12 @@ def run_ours(args, wl):
                                                                 buf.expert_load), flush=flush),
     }
     st_a = ms.read_stats(buf.stats)
+    sub_ms.update({
+        "combine_bwd": time_call(torch, lambda: ms.combine_bwd(ctx, dY, xd, buf.expert_idx, buf.slot_idx, buf.gate_w,
+                                                                buf.slot_token, dyexp, dgw), flush=flush),
+        "softtopk_bwd": time_call(torch, lambda: ms.softtopk_bwd(ctx, buf.logits, buf.expert_idx, dgw, dL), flush=flush),
+        "gate_bwd": time_call(torch, lambda: ms.gate_bwd(ctx, Hd, Wd, dL, dW, dH), flush=flush),
+    })
     skew = synth.WORKLOADS["skew"]
     ctx_s = ms.create(ms.make_params(skew.T, 64, skew.E, skew.k, skew.capacity_factor), dev)
     Ls = synth.logits_like(skew.T, skew.E, 0, bias=synth.expert_bias(skew, 0)).to(dev)
@@ -377,6 +383,7 @@ def run_ours(args, wl):
         "gate_bwd": 2 * T * row + T * E * 4,                       # read H (dW) and dL, write dH
         "dispatch_bwd": T * k * row + 2 * T * row,                 # read k rows, read-modify-write dH
     }
+    alg_bytes["route_bwd"] = alg_bytes["combine_bwd"] + alg_bytes["softtopk_bwd"] + alg_bytes["gate_bwd"]
     all_ms = dict(zip(stage_names, stage_ms))
     all_ms.update(sub_ms)
     def frac_of(n):

@@ -282,18 +282,19 @@ maxscore_status launch_softtopk_fwd(maxscore_ctx* c, const float* logits, float*
   return launch_softtopk_rows(c, logits, scores, c->p.T, st);
 }
 
+// dl_split (may be null): the gradient also as hi + lo bf16 halves, in the layout the tensor-core gate backward reads
 void launch_softtopk_bwd_tiles(maxscore_ctx* c, const float* logits, const int32_t* expert_idx, const float* dgate_w,
-                               const float* dscores_col, float* dlogits, cudaStream_t st) {
+                               const float* dscores_col, float* dlogits, cudaStream_t st, __nv_bfloat16* dl_split = nullptr) {
   const maxscore_params& p = c->p;
   const int tiles = (p.T + kStTok - 1) / kStTok;
   const int grid = tiles < c->sm_count * 6 ? tiles : c->sm_count * 6;
   const size_t smem = sizeof(float) * ((size_t)kStTok * st_stride(p.E) + p.E);
   if (p.k <= 2)
-    softtopk_bwd_kernel<2><<<grid, kStThreads, smem, st>>>(logits, expert_idx, dgate_w, dscores_col, dlogits, p.T, p.E, p.k, p.t);
+    softtopk_bwd_kernel<2><<<grid, kStThreads, smem, st>>>(logits, expert_idx, dgate_w, dscores_col, dlogits, dl_split, c->lay.Kpad, p.T, p.E, p.k, p.t);
   else if (p.k <= 4)
-    softtopk_bwd_kernel<4><<<grid, kStThreads, smem, st>>>(logits, expert_idx, dgate_w, dscores_col, dlogits, p.T, p.E, p.k, p.t);
+    softtopk_bwd_kernel<4><<<grid, kStThreads, smem, st>>>(logits, expert_idx, dgate_w, dscores_col, dlogits, dl_split, c->lay.Kpad, p.T, p.E, p.k, p.t);
   else
-    softtopk_bwd_kernel<8><<<grid, kStThreads, smem, st>>>(logits, expert_idx, dgate_w, dscores_col, dlogits, p.T, p.E, p.k, p.t);
+    softtopk_bwd_kernel<8><<<grid, kStThreads, smem, st>>>(logits, expert_idx, dgate_w, dscores_col, dlogits, dl_split, c->lay.Kpad, p.T, p.E, p.k, p.t);
 }
 
 // rounds of (records, exact phase, check): candidate thresholds theta0, then two wider ones (four times the last, or twice
@@ -661,8 +662,17 @@ maxscore_status maxscore_combine_bwd(maxscore_ctx* c, const void* dY, const void
   return launch_zero_padding(c, slot_token, dyexp, st);
 }
 
+static maxscore_status gate_bwd_impl(maxscore_ctx* c, const void* hidden, const void* w_gate, const float* dlogits,
+                                     float* dw_gate, void* dH, void* stream, bool split_ready);
+
 maxscore_status maxscore_gate_bwd(maxscore_ctx* c, const void* hidden, const void* w_gate, const float* dlogits,
                                   float* dw_gate, void* dH, void* stream) {
+  return gate_bwd_impl(c, hidden, w_gate, dlogits, dw_gate, dH, stream, false);
+}
+
+// split_ready: the hi/lo bf16 halves of dlogits are already in the workspace (written by the SoftTopk backward)
+static maxscore_status gate_bwd_impl(maxscore_ctx* c, const void* hidden, const void* w_gate, const float* dlogits,
+                                     float* dw_gate, void* dH, void* stream, bool split_ready) {
   if (!c || !hidden || !w_gate || !dlogits || !dw_gate || !dH) return MAXSCORE_ERR_INVALID_ARG;
   if (!aligned16(hidden) || !aligned16(w_gate) || !aligned16(dlogits) || !aligned16(dw_gate) || !aligned16(dH))
     return MAXSCORE_ERR_INVALID_ARG;
@@ -680,8 +690,11 @@ maxscore_status maxscore_gate_bwd(maxscore_ctx* c, const void* hidden, const voi
     {
       long long n = (long long)p.T * Kpad;
       int blocks = (int)((n + 255) / 256); if (blocks > c->sm_count * 16) blocks = c->sm_count * 16;
-      split_dlogits_kernel<<<blocks, 256, 0, st>>>(dlogits, dls, p.T, p.E, Kpad);
-      MS_LAUNCH_CHECK("split_dlogits_kernel");
+      if (!split_ready) {
+        split_dlogits_kernel<<<blocks, 256, 0, st>>>(dlogits, dls, p.T, p.E, Kpad);
+        MS_LAUNCH_CHECK("split_dlogits_kernel");
+        c->launches += 1;
+      }
       n = (long long)p.d_model * Kpad;
       blocks = (int)((n + 255) / 256); if (blocks > c->sm_count * 16) blocks = c->sm_count * 16;
       wgate_kmajor_kernel<<<blocks, 256, 0, st>>>((const __nv_bfloat16*)w_gate, wk, p.d_model, p.E, Kpad, p.w_gate_layout);
@@ -708,7 +721,7 @@ maxscore_status maxscore_gate_bwd(maxscore_ctx* c, const void* hidden, const voi
     const long long nw = (long long)p.d_model * p.E;
     int rblocks = (int)((nw + 255) / 256); if (rblocks > c->sm_count * 8) rblocks = c->sm_count * 8;
     reduce_dw_kernel<<<rblocks, 256, 0, st>>>(part, dw_gate, nw, l.dw_splits);
-    c->launches += 5;
+    c->launches += 4;
   } else {
     gate_bwd_dw_kernel<float><<<gw, 256, 0, st>>>((const float*)hidden, dlogits, dw_gate, p.T, p.d_model, p.E);
     MS_LAUNCH_CHECK("gate_bwd_dw_kernel");
@@ -728,6 +741,15 @@ maxscore_status maxscore_route_bwd(maxscore_ctx* c, const void* dY, const void* 
   if (!logits || !dlogits) return MAXSCORE_ERR_INVALID_ARG;
   maxscore_status s = maxscore_combine_bwd(c, dY, yexp, expert_idx, slot_idx, gate_w, slot_token, dyexp, dgate_w, stream);
   if (s) return s;
+  if (c->p.io_dtype == MAXSCORE_BF16 && c->p.softtopk_mode == 0) {
+    // the SoftTopk backward also leaves its result as the hi/lo bf16 halves that the tensor-core gate backward reads
+    if (!expert_idx || !dgate_w) return MAXSCORE_ERR_INVALID_ARG;
+    launch_softtopk_bwd_tiles(c, logits, expert_idx, dgate_w, nullptr, dlogits, (cudaStream_t)stream,
+                              reinterpret_cast<__nv_bfloat16*>(c->ws + c->lay.dls));
+    MS_LAUNCH_CHECK("softtopk_bwd_kernel");
+    c->launches += 1;
+    return gate_bwd_impl(c, hidden, w_gate, dlogits, dw_gate, dH, stream, true);
+  }
   s = maxscore_softtopk_bwd(c, logits, expert_idx, dgate_w, dlogits, stream);
   if (s) return s;
   return maxscore_gate_bwd(c, hidden, w_gate, dlogits, dw_gate, dH, stream);

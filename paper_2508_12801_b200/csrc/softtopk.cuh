@@ -102,6 +102,23 @@ __device__ __forceinline__ void st_insert(float (&tv)[K], int (&ti)[K], float v,
   ti[0] = above[0] ? e : ti[0];
 }
 
+// The rows of a tile as two bf16 halves, value = hi + lo (what the tensor-core gate backward reads): row t of `split`
+// holds hi in columns [0, Kpad) and lo in [Kpad, 2 Kpad), zeros from column E on.  Two columns per lane and step.
+__device__ __forceinline__ void st_store_split(__nv_bfloat16* __restrict__ split, const float* sm, int rows, int E,
+                                               int stride, int Kpad) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int r = warp; r < rows; r += kStThreads / 32) {
+    __nv_bfloat16* out = split + (size_t)r * 2 * Kpad;
+    for (int c = 2 * lane; c < Kpad; c += 64) {
+      const float x0 = c < E ? sm[r * stride + c] : 0.f, x1 = c + 1 < E ? sm[r * stride + c + 1] : 0.f;
+      const __nv_bfloat16 h0 = __float2bfloat16(x0), h1 = __float2bfloat16(x1);
+      const __nv_bfloat16 l0 = __float2bfloat16(x0 - __bfloat162float(h0)), l1 = __float2bfloat16(x1 - __bfloat162float(h1));
+      *reinterpret_cast<__nv_bfloat162*>(out + c) = __halves2bfloat162(h0, h1);
+      *reinterpret_cast<__nv_bfloat162*>(out + Kpad + c) = __halves2bfloat162(l0, l1);
+    }
+  }
+}
+
 // The K largest entries of a row (lane q scans experts q, q + 2, ...; then the lanes' lists are merged), the same
 // in every lane of the token.  Slots that no entry reached keep index -1.
 template <int K>
@@ -215,7 +232,7 @@ template <int K>
 __global__ void __launch_bounds__(kStThreads, 5)
 softtopk_bwd_kernel(const float* __restrict__ logits, const int32_t* __restrict__ expert_idx,
                     const float* __restrict__ dgate_w, const float* __restrict__ dscores_col,
-                    float* __restrict__ dlogits, int T, int E, int k, float t) {
+                    float* __restrict__ dlogits, __nv_bfloat16* __restrict__ dl_split, int Kpad, int T, int E, int k, float t) {
   extern __shared__ float st_sm[];
   const int stride = st_stride(E);
   float* col = st_sm + kStTok * stride;                  // the shared per-expert term (zeros if none)
@@ -283,6 +300,7 @@ softtopk_bwd_kernel(const float* __restrict__ logits, const int32_t* __restrict_
     }
     __syncthreads();
     st_store_tile(dlogits + (size_t)row0 * E, st_sm, rows, E, stride);
+    if (dl_split) st_store_split(dl_split + (size_t)row0 * 2 * Kpad, st_sm, rows, E, stride, Kpad);
     __syncthreads();
   }
 }
