@@ -16,7 +16,10 @@
 //             margin at a time.  This is an epsilon-scaled simultaneous price adjustment (auction-style);
 //             it ends a few dozen token moves away from the optimum and stops early once a small imbalance
 //             has stopped shrinking.  A token whose cache can no longer vouch for its top-(k+2) (the bound
-//             on the uncached experts has come too close) is rescanned by a warp.  The kernel ends by
+//             on the uncached experts has come too close) is rescanned by a warp.  Whether prices may
+//             fall below zero on the way (anchored afterwards) or keep their floor at zero, and whether a few
+//             units of spare room are hidden at first, is decided from the loads of the first sweep (see
+//             SweepArgs::slack and the comments at that decision).  The kernel ends by
 //             writing every token's top-k under the final prices and listing the tokens whose k-th and
 //             (k+1)-th values differ by at most theta as candidates.
 //   records   per candidate, the experts it could give up or take within the arc window (whole GPU).

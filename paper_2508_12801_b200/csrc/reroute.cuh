@@ -18,9 +18,9 @@
 // and the first token whose proposal finds its expert used up by earlier proposals marks the end of the prefix
 // that is final.  Everything before it is placed, the expert that ran out is closed, and the next round starts
 // at that token.  A round therefore places everything up to the next expert that fills up.
-// A token's candidate list holds its 16 best experts among those it does not hold and that had room when the
-// list was made (by descending affinity, ties by ascending index); a list that runs out of experts with room
-// before the token is served is rebuilt from the token's row.
+// A token's candidate order holds every expert that it does not hold and that has room after stage 1, by descending
+// affinity (ties by ascending index), a byte each; it is made once, by one warp per listed token across the whole GPU,
+// and a thread reads its token's order 16 experts at a time as far as it has to.
 #pragma once
 #include "common.cuh"
 #include "softtopk.cuh"
