@@ -1701,7 +1701,18 @@ flow_exact_kernel(FlowState* st, int32_t* expert_idx, const int32_t* __restrict_
   }
   __syncthreads();
   // the caches' bounds on uncached experts must keep up with prices that fell during this round
-  if (tid == 0) { st->cumdrop += s.dt; st->naug += naug; st->ncand_last = n; st->ncand = 0; st->nrec = 0; }
+  if (tid == 0) {
+    st->cumdrop += s.dt; st->naug += naug; st->ncand_last = n; st->ncand = 0; st->nrec = 0;
+    // Excess left and no path to a deficit among the listed tokens at all: the list is far too short (a price spread
+    // that stopped the round tells how far to look; this tells nothing), so the next listing looks four times further
+    // than it would have.
+    if (s.target == -1 && theta < (kInf >> 8)) {
+      bool left = false;
+      for (int e = 0; e <= E; ++e) left |= s.imb[e] > 0;
+      const long long th = st->theta;
+      if (left && th < (kInf >> 8)) st->theta = th * 4;
+    }
+  }
 }
 
 }  // namespace msr
