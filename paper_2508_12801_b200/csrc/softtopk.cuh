@@ -3,6 +3,7 @@
 // Level j (1-based) of Eq. 6 adds a softmax with temperature t over the entries that are not among
 // the j-1 largest (ties: lowest expert index).
 #pragma once
+#include <cuda_pipeline.h>
 #include "common.cuh"
 
 namespace msr {
@@ -47,10 +48,21 @@ constexpr int kStThreads = kStTok * kStSplit;
 
 __host__ __device__ constexpr int st_stride(int E) { return (E + 31) / 32 * 32 + kStSplit; }
 
-// Eight rows at a time per warp, so that up to 32 loads per lane are in flight before the first is used.
+// With an even expert count every row starts on an 8-byte boundary in global and in shared memory (the stride is
+// even), and the whole tile goes through asynchronous 8-byte copies: all of a warp's rows are in flight at once and no
+// register holds them.  Otherwise eight rows at a time per warp through registers (up to 32 loads per lane in flight).
 __device__ __forceinline__ void st_load_tile(const float* __restrict__ g, float* sm, int rows, int E, int stride) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   constexpr int kWarps = kStThreads / 32, kBatch = 8;
+  if ((E & 1) == 0) {
+    const int pairs = E >> 1;
+    for (int r = warp; r < rows; r += kWarps)
+      for (int c = lane; c < pairs; c += 32)
+        __pipeline_memcpy_async(sm + r * stride + 2 * c, g + (size_t)r * E + 2 * c, 8);
+    __pipeline_commit();
+    __pipeline_wait_prior(0);
+    return;
+  }
   for (int r0 = warp; r0 < rows; r0 += kWarps * kBatch) {
     float v[kBatch][kEPL];
 #pragma unroll
