@@ -373,26 +373,18 @@ maxscore_status launch_assign(maxscore_ctx* c, const float* M, int32_t* expert_i
 }
 
 maxscore_status launch_index_build(maxscore_ctx* c, const int32_t* expert_idx, int32_t* slot_idx, int32_t* slot_token,
-                                   int32_t* expert_load, cudaStream_t st) {
+                                   int32_t* expert_load, cudaStream_t st, const float* scores = nullptr,
+                                   float* gate_w = nullptr) {
   const maxscore_params& p = c->p;
   int32_t* bc = reinterpret_cast<int32_t*>(c->ws + c->lay.block_counts);
   MS_CUDA(cudaMemsetAsync(slot_token, 0xFF, sizeof(int32_t) * (size_t)p.E * c->C, st));
   index_count_kernel<<<c->lay.n_idx_blocks, kIdxTok, 0, st>>>(expert_idx, bc, p.T, p.E, p.k);
   MS_LAUNCH_CHECK("index_count_kernel");
   index_fill_kernel<<<c->lay.n_idx_blocks, kIdxTok, 0, st>>>(expert_idx, bc, slot_idx, slot_token, expert_load, p.T,
-                                                            p.E, p.k, c->C);
+                                                            p.E, p.k, c->C, scores, gate_w);
   MS_LAUNCH_CHECK("index_fill_kernel");
   c->launches += 2;
   return MAXSCORE_OK;
-}
-
-__global__ void gather_gate_w_kernel(const float* __restrict__ scores, const int32_t* __restrict__ expert_idx,
-                                     float* __restrict__ gate_w, long long n, int E, int k) {
-  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
-    const long long tok = i / k;
-    const int e = expert_idx[i];
-    gate_w[i] = (e >= 0 && e < E) ? scores[tok * E + e] : 0.f;
-  }
 }
 
 constexpr int kHostChunks = 8, kHostChunkMinRows = 1024;     // row blocks of the host path, and the smallest worth a copy
@@ -413,13 +405,9 @@ maxscore_status route_after_scores(maxscore_ctx* c, const float* logits, const f
                                    maxscore_stats* stats, cudaStream_t st) {
   maxscore_status s = launch_assign(c, c->p.score_mode == 0 ? scores : logits, expert_idx, expert_load, stats, st);
   if (s) return s;
-  s = launch_index_build(c, expert_idx, slot_idx, slot_token, expert_load, st);
+  // slots and, in the same pass over expert_idx, the combine weights gate_w[i, c] = scores[i, expert_idx[i, c]]
+  s = launch_index_build(c, expert_idx, slot_idx, slot_token, expert_load, st, scores, gate_w);
   if (s) return s;
-  const long long n = (long long)c->p.T * c->p.k;
-  int blocks = (int)((n + 255) / 256); if (blocks > c->sm_count * 8) blocks = c->sm_count * 8;
-  gather_gate_w_kernel<<<blocks, 256, 0, st>>>(scores, expert_idx, gate_w, n, c->p.E, c->p.k);
-  MS_LAUNCH_CHECK("gather_gate_w_kernel");
-  c->launches += 1;
   return MAXSCORE_OK;
 }
 

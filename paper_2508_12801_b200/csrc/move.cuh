@@ -32,7 +32,8 @@ index_count_kernel(const int32_t* __restrict__ expert_idx, int32_t* __restrict__
 __global__ void __launch_bounds__(kIdxTok)
 index_fill_kernel(const int32_t* __restrict__ expert_idx, const int32_t* __restrict__ block_counts,
                   int32_t* __restrict__ slot_idx, int32_t* __restrict__ slot_token,
-                  int32_t* __restrict__ expert_load, int T, int E, int k, int C) {
+                  int32_t* __restrict__ expert_load, int T, int E, int k, int C,
+                  const float* __restrict__ scores = nullptr, float* __restrict__ gate_w = nullptr) {
   __shared__ int base[kMaxE];                       // first slot of this block per expert
   __shared__ int wcnt[kIdxTok / 32][kMaxE + 1];     // per-warp counts, then exclusive offsets
   __shared__ unsigned bits[kIdxTok / 32][kMaxE];    // lanes of the warp that hold the expert
@@ -70,6 +71,8 @@ index_fill_kernel(const int32_t* __restrict__ expert_idx, const int32_t* __restr
     if (c < k && tok < T) {
       int e = __ldg(expert_idx + (size_t)tok * k + c);
       if (e >= 0 && e < E) { mine[c] = e; atomicOr(&bits[warp][e], 1u << lane); }
+      // on the way, if asked for: the combine weight of the pair, i.e. the token's score for that expert (Eq. 1)
+      if (gate_w) gate_w[(size_t)tok * k + c] = (e >= 0 && e < E) ? __ldg(scores + (size_t)tok * E + e) : 0.f;
     }
   }
   __syncthreads();
