@@ -65,14 +65,16 @@ index_fill_kernel(const int32_t* __restrict__ expert_idx, const int32_t* __restr
     for (int e = threadIdx.x; e < E; e += blockDim.x) expert_load[e] = total[e];
   const int tok = blockIdx.x * kIdxTok + threadIdx.x;
   int mine[kMaxK];
+  float gw[kMaxK];
 #pragma unroll
   for (int c = 0; c < kMaxK; ++c) {
     mine[c] = -1;
     if (c < k && tok < T) {
       int e = __ldg(expert_idx + (size_t)tok * k + c);
       if (e >= 0 && e < E) { mine[c] = e; atomicOr(&bits[warp][e], 1u << lane); }
-      // on the way, if asked for: the combine weight of the pair, i.e. the token's score for that expert (Eq. 1)
-      if (gate_w) gate_w[(size_t)tok * k + c] = (e >= 0 && e < E) ? __ldg(scores + (size_t)tok * E + e) : 0.f;
+      // on the way, if asked for: the combine weight of the pair, i.e. the token's score for that expert (Eq. 1);
+      // all k loads are issued before the first is stored
+      if (gate_w) gw[c] = (e >= 0 && e < E) ? __ldg(scores + (size_t)tok * E + e) : 0.f;
     }
   }
   __syncthreads();
@@ -91,6 +93,10 @@ index_fill_kernel(const int32_t* __restrict__ expert_idx, const int32_t* __restr
       slot_idx[(size_t)tok * k + c] = slot;
       if (slot < C) slot_token[(size_t)e * C + slot] = tok;
     }
+  }
+  if (gate_w && tok < T) {
+#pragma unroll
+    for (int c = 0; c < kMaxK; ++c) if (c < k) gate_w[(size_t)tok * k + c] = gw[c];
   }
 }
 
